@@ -1,0 +1,193 @@
+/*
+ * sparseffn.h — C ABI of libsparseffn.so: the sparsified Transformer-FFN training step on
+ * NVIDIA B200 (sm_100a).
+ *
+ * The step (paper: Algorithms 1 and 2, Sections 2.1-2.3, 3) re-prunes the FFN weights to 2:4
+ * every iteration, computes SquaredReLU(X W1^T), sparsifies the activation into the V:N:M
+ * (Venom) format and runs the forward/backward products with exactly one sparse operand each.
+ *
+ * Conventions for every entry point
+ *   - Tensors are row-major bf16 (16-bit patterns) unless stated. T = tokens, D = d_model,
+ *     F = d_ffn.  X [T,D], W1 [F,D], W2 [D,F], Y/dY [T,D]  (the paper writes the weights
+ *     transposed, W1 [D,F], W2 [F,D]; the mathematics is the same).
+ *   - Pointers are DEVICE pointers owned by the caller unless the name says "host". The
+ *     library never allocates or frees device memory and never synchronises, except where an
+ *     entry point says so. Work is enqueued on the caller's stream (`stream` is a
+ *     cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - Return value: SF_OK (0) or a negative sf_status. No exceptions cross the boundary. On a
+ *     non-zero return nothing has been launched.
+ *   - Base pointers must be 16-byte aligned and leading dimensions multiples of 8 elements.
+ *   - Canonical 2:4 metadata: one nibble per group of four, `pos0 | pos1 << 2` with
+ *     pos0 < pos1 the kept positions; four consecutive groups of a row are packed
+ *     little-endian into one uint16.
+ */
+#ifndef SPARSEFFN_H_
+#define SPARSEFFN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SF_API __attribute__((visibility("default")))
+#else
+#define SF_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum sf_status {
+  SF_OK = 0,
+  SF_ERR_NULL = -1,      /* a required pointer is NULL */
+  SF_ERR_SHAPE = -2,     /* a size violates the divisibility rules stated per call */
+  SF_ERR_ALIGN = -3,     /* base pointer not 16-byte aligned or ld not a multiple of 8 */
+  SF_ERR_WORKSPACE = -4, /* workspace / context too small */
+  SF_ERR_ARCH = -5,      /* current device is not compute capability 10.x */
+  SF_ERR_CUDA = -6,      /* a CUDA call failed; see sf_last_cuda_error() */
+  SF_ERR_TIMEOUT = -7,   /* a bounded device-side wait expired (reported by sf_check_status) */
+  SF_ERR_UNSUPPORTED = -8 /* legal per the paper but not built (e.g. N != 2) */
+} sf_status;
+
+/* Problem descriptor of one FFN layer step. Ragged shapes are rejected, never padded:
+ * T % 128 == 0, T % V == 0, D % 128 == 0, F % 128 == 0, F % (4*M) == 0, V in {64,128},
+ * N == 2, M in {4,8,16,32}. */
+typedef struct sf_ffn_desc {
+  int64_t T, D, F;
+  int32_t V, N, M;
+  int32_t prune_mode;  /* 0: hard magnitude top-2-of-4; 1: soft-thresholding (Section 2.2) */
+  int32_t flags;       /* bit0: also store the full bf16 pre-activation y1 in the context */
+} sf_ffn_desc;
+
+SF_API const char* sf_status_string(int status);
+/* cudaError_t value of the most recent failed CUDA call made by this library (per process). */
+SF_API int sf_last_cuda_error(void);
+
+/* ---------------------------------------------------------------------------------------
+ * 2:4 weight sparsification (Section 2.2; Section 3.2.1 "packed format along with sparsity
+ * metadata"; Algorithm 1 line 4, Algorithm 2 line 2).
+ *
+ * Per group of four consecutive elements along the chosen dimension keep the two largest
+ * magnitudes (ties to the lower index); prune_mode 1 additionally subtracts the group's
+ * second-smallest magnitude from the kept magnitudes (soft-thresholding).
+ *
+ *   W          [rows, cols] bf16, leading dimension ld (elements)
+ *   group_dim  1: groups along a row (contiguous);   R = rows, K = cols
+ *              0: groups along a column (strided);   R = cols, K = rows; outputs are written
+ *                 K-major, i.e. as for the transposed matrix
+ *   vals       out, bf16 [R, K/2]   kept values in position order
+ *   meta       out, uint16 [R, K/16] canonical metadata
+ *   dense_out  optional out (may be NULL): the pruned matrix in the input's own layout
+ *              [rows, cols] with leading dimension cols, dropped entries +0
+ * Shape rules: K % 16 == 0; group_dim 0 additionally needs cols % 8 == 0.
+ * sf_prune24_sizes reports the byte sizes of vals and meta.
+ */
+SF_API int sf_prune24_sizes(int64_t rows, int64_t cols, int group_dim, size_t* vals_bytes, size_t* meta_bytes);
+SF_API int sf_prune24_compress(const void* W, int64_t rows, int64_t cols, int64_t ld, int group_dim,
+                        int prune_mode, void* vals, void* meta, void* dense_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * SquaredReLU + V:N:M activation sparsification (Eq. 2; Section 2.3; Table 5; Algorithm 1
+ * lines 5-6 with magnitude selection in place of the learned router).
+ *
+ * The [T,F] input is cut into blocks of V rows x M columns. Per block the four columns with
+ * the largest score stay, where score = sum over the block's rows (first to last, float32) of
+ * |h|, h = bf16(max(p,0)^2) when apply_sqrelu != 0, else h = p; ties to the lower column.
+ * Per row the two largest magnitudes among those four columns stay (ties to the lower one).
+ *
+ *   preact     [T, F] bf16, leading dimension ld
+ *   vals       out, bf16 [T, 2F/M]        kept h values, position order
+ *   meta       out, uint16 [T, F/(4M)]    canonical nibbles over the condensed [T, 4F/M] matrix
+ *   colidx     out, uint8 [T/V, F/M, 4]   kept columns per block, ascending, each < M
+ *   relu_vals  optional out, bf16 [T, 2F/M]: max(p,0) at the kept positions (needed by the
+ *              backward pass; ignored when apply_sqrelu == 0)
+ *   dense_out  optional out, bf16 [T, F]: h on the mask, +0 elsewhere
+ * Shape rules: N == 2; M in {4,8,16,32,64}; T % V == 0; V in [1,128]; F % (4*M) == 0; F % 64 == 0.
+ */
+SF_API int sf_vnm_sizes(int64_t T, int64_t F, int V, int N, int M,
+                 size_t* vals_bytes, size_t* meta_bytes, size_t* colidx_bytes);
+SF_API int sf_vnm_sparsify_act(const void* preact, int64_t T, int64_t F, int64_t ld, int V, int N, int M,
+                        int apply_sqrelu, void* vals, void* meta, void* colidx, void* relu_vals,
+                        void* dense_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Single products on the tensor cores (the building blocks of Algorithms 1 and 2, exposed for
+ * parity tests and for the 2:4 / Venom micro-benchmarks of Section 5.2.3).
+ *
+ * sf_gemm_dense:  C[Mr,Nc] = op(A) op(B)^T, fp32 accumulate, bf16 out.
+ *     a_kmajor = 1: A is [Mr,K] row-major;  0: A is stored [K,Mr] row-major (M contiguous)
+ *     b_kmajor = 1: B is [Nc,K] row-major;  0: B is stored [K,Nc] row-major (N contiguous)
+ *     Mr % 128 == 0, Nc % 128 == 0, K % 64 == 0.
+ * sf_gemm_sparse24:  Ct[Nc,Mr] (transposed output!) with C[Mr,Nc] = A_s[Mr,K] B[Nc,K]^T where
+ *     A_s is given packed: a_vals bf16 [Mr,K/2], a_meta canonical uint16 [Mr,K/16].
+ *     This is y1 = X W1s^T with A_s = W1s, B = X, output y1 [T,F].  Mr,Nc % 128, K % 128.
+ * sf_gemm_venom:  C[T,Nc] = A_vnm[T,F] Bt[F,Nc] with A_vnm in V:N:M packed form (vals, meta,
+ *     colidx as produced by sf_vnm_sparsify_act) and Bt row-major [F,Nc] (rows are gathered by
+ *     colidx).  T % 128, V in {64,128}, Nc % 128, (4F/M) % 128 == 0.
+ * `workspace` needs sf_gemm_workspace_size() bytes (hardware-ordered metadata copy + status).
+ */
+SF_API int sf_gemm_workspace_size(int64_t Mr, int64_t K, size_t* bytes);
+SF_API int sf_gemm_dense(const void* A, int a_kmajor, const void* B, int b_kmajor, void* C,
+                  int64_t Mr, int64_t Nc, int64_t K, void* workspace, void* stream);
+SF_API int sf_gemm_sparse24(const void* a_vals, const void* a_meta, const void* B, void* Ct,
+                     int64_t Mr, int64_t Nc, int64_t K, void* workspace, void* stream);
+SF_API int sf_gemm_venom(const void* a_vals, const void* a_meta, const void* colidx, const void* Bt,
+                  void* C, int64_t T, int64_t F, int64_t Nc, int V, int M,
+                  void* workspace, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * The FFN step (Algorithm 1 = forward, Algorithm 2 = backward; Eqs. 1-8 for the dense phase).
+ *
+ * sf_ffn_workspace_size: bytes of the forward context (saved for backward) and of the scratch
+ * workspace for `desc`. Both buffers are caller-allocated device memory, 256-byte aligned.
+ *
+ * sf_sparse_ffn_fwd:  W1s = prune24(W1 along D);  y1 = X W1s^T;  y2 = V:N:M(ReLU(y1)^2);
+ *                     Y = y2 W2^T  (W2 dense).  Saves packed y2, packed ReLU(y1), metadata,
+ *                     column indices (and y1 if flags bit0) in fwd_ctx.
+ * sf_sparse_ffn_bwd:  W2s = prune24(W2 along D);  dy2 = dY W2s;  dy1 = 2 dy2 ReLU(y1) on y2's
+ *                     mask;  dX = dy1 W1 (W1 dense);  dW1 = dy1^T X [F,D];  dW2 = dY^T y2 [D,F].
+ * sf_dense_ffn_fwd/bwd: the same equations with no pruning; fwd_ctx holds y1 (bf16 [T,F]).
+ */
+SF_API int sf_ffn_workspace_size(const sf_ffn_desc* desc, size_t* fwd_ctx_bytes, size_t* workspace_bytes);
+SF_API int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, const void* W2,
+                      void* Y, void* fwd_ctx, void* workspace, void* stream);
+SF_API int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, const void* W1,
+                      const void* W2, const void* fwd_ctx, void* dX, void* dW1, void* dW2,
+                      void* workspace, void* stream);
+SF_API int sf_dense_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, const void* W2,
+                     void* Y, void* fwd_ctx, void* workspace, void* stream);
+SF_API int sf_dense_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, const void* W1,
+                     const void* W2, const void* fwd_ctx, void* dX, void* dW1, void* dW2,
+                     void* workspace, void* stream);
+
+/* Views into a sparse forward context (device pointers into fwd_ctx; nothing is copied). */
+typedef enum sf_ctx_field {
+  SF_CTX_Y2_VALS = 0,   /* bf16 [T, 2F/M] */
+  SF_CTX_RELU_VALS = 1, /* bf16 [T, 2F/M] */
+  SF_CTX_META = 2,      /* uint16 [T, F/(4M)] canonical */
+  SF_CTX_COLIDX = 3,    /* uint8 [T/V, F/M, 4] */
+  SF_CTX_Y1 = 4,        /* bf16 [T, F] (only with flags bit0) */
+  SF_CTX_DY1_VALS = 5   /* bf16 [T, 2F/M], lives in the WORKSPACE after sf_sparse_ffn_bwd */
+} sf_ctx_field;
+SF_API int sf_ctx_view(const sf_ffn_desc* desc, const void* fwd_ctx_or_workspace, int field,
+                const void** ptr, size_t* bytes);
+
+/* One whole training step from HOST buffers (pinned memory recommended): copies X, W1, W2, dY
+ * to the device staging area inside `workspace`, runs sf_sparse_ffn_fwd + sf_sparse_ffn_bwd
+ * (dense != 0: the dense pair), copies Y, dX, dW1, dW2 back, all on `stream`. Does not
+ * synchronise. host_* pointers are HOST pointers; `device_staging` is a DEVICE buffer of
+ * sf_ffn_host_staging_size() bytes. */
+SF_API int sf_ffn_host_staging_size(const sf_ffn_desc* desc, size_t* bytes);
+SF_API int sf_ffn_step_host(const sf_ffn_desc* desc, int dense, const void* host_X, const void* host_W1,
+                     const void* host_W2, const void* host_dY, void* host_Y, void* host_dX,
+                     void* host_dW1, void* host_dW2, void* device_staging, void* fwd_ctx,
+                     void* workspace, void* stream);
+
+/* Synchronises `stream` and reads the device status word kept at the start of `workspace`:
+ * SF_OK, or SF_ERR_TIMEOUT if a bounded wait inside a tensor-core kernel expired. */
+SF_API int sf_check_status(void* workspace, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSEFFN_H_ */

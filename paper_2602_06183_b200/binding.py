@@ -1,0 +1,279 @@
+"""ctypes binding of libsparseffn.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (see include/sparseffn.h) and takes
+torch tensors (device memory, streams) or raw integers; no step of the method runs in Python.
+The shared library must have been built (``python -m paper_2602_06183_b200.build``); loading
+fails loudly otherwise and there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsparseffn.so")
+
+SF_OK = 0
+SF_ERR_NULL, SF_ERR_SHAPE, SF_ERR_ALIGN, SF_ERR_WORKSPACE = -1, -2, -3, -4
+SF_ERR_ARCH, SF_ERR_CUDA, SF_ERR_TIMEOUT, SF_ERR_UNSUPPORTED = -5, -6, -7, -8
+
+SF_CTX_Y2_VALS, SF_CTX_RELU_VALS, SF_CTX_META, SF_CTX_COLIDX, SF_CTX_Y1, SF_CTX_DY1_VALS = range(6)
+
+
+class sf_ffn_desc(C.Structure):
+    _fields_ = [("T", C.c_int64), ("D", C.c_int64), ("F", C.c_int64),
+                ("V", C.c_int32), ("N", C.c_int32), ("M", C.c_int32),
+                ("prune_mode", C.c_int32), ("flags", C.c_int32)]
+
+
+class SparseFFNError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (cuda error {last_cuda_error()})")
+
+
+_lib = None
+
+_vp, _i64, _i32, _sz = C.c_void_p, C.c_int64, C.c_int, C.c_size_t
+_SIGNATURES = {
+    "sf_status_string": (C.c_char_p, [_i32]),
+    "sf_last_cuda_error": (_i32, []),
+    "sf_prune24_sizes": (_i32, [_i64, _i64, _i32, C.POINTER(_sz), C.POINTER(_sz)]),
+    "sf_prune24_compress": (_i32, [_vp, _i64, _i64, _i64, _i32, _i32, _vp, _vp, _vp, _vp]),
+    "sf_vnm_sizes": (_i32, [_i64, _i64, _i32, _i32, _i32, C.POINTER(_sz), C.POINTER(_sz), C.POINTER(_sz)]),
+    "sf_vnm_sparsify_act": (_i32, [_vp, _i64, _i64, _i64, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_gemm_workspace_size": (_i32, [_i64, _i64, C.POINTER(_sz)]),
+    "sf_gemm_dense": (_i32, [_vp, _i32, _vp, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
+    "sf_gemm_sparse24": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
+    "sf_gemm_venom": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp, _vp]),
+    "sf_ffn_workspace_size": (_i32, [C.POINTER(sf_ffn_desc), C.POINTER(_sz), C.POINTER(_sz)]),
+    "sf_sparse_ffn_fwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_sparse_ffn_bwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_dense_ffn_fwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_dense_ffn_bwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_ctx_view": (_i32, [C.POINTER(sf_ffn_desc), _vp, _i32, C.POINTER(_vp), C.POINTER(_sz)]),
+    "sf_ffn_host_staging_size": (_i32, [C.POINTER(sf_ffn_desc), C.POINTER(_sz)]),
+    "sf_ffn_step_host": (_i32, [C.POINTER(sf_ffn_desc), _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_check_status": (_i32, [_vp, _vp]),
+}
+
+EXPORTED_SYMBOLS = tuple(_SIGNATURES)
+
+
+def lib() -> C.CDLL:
+    """Load the shared library (once). Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2602_06183_b200.build` "
+                "(there is no fallback implementation)")
+        _lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(_lib, name)
+            fn.restype, fn.argtypes = res, args
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().sf_status_string(status).decode()
+
+
+def last_cuda_error() -> int:
+    return lib().sf_last_cuda_error()
+
+
+def _check(status: int, where: str) -> None:
+    if status != SF_OK:
+        raise SparseFFNError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream: Optional[torch.cuda.Stream] = None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def make_desc(T, D, F, V, M, N=2, prune_mode=0, flags=0) -> sf_ffn_desc:
+    return sf_ffn_desc(T, D, F, V, N, M, prune_mode, flags)
+
+
+# ---- 2:4 pruning -----------------------------------------------------------------------------
+
+def sf_prune24_sizes(rows: int, cols: int, group_dim: int):
+    a, b = _sz(), _sz()
+    _check(lib().sf_prune24_sizes(rows, cols, group_dim, C.byref(a), C.byref(b)), "sf_prune24_sizes")
+    return a.value, b.value
+
+
+def sf_prune24_compress(W: torch.Tensor, group_dim: int = 1, prune_mode: int = 0, want_dense: bool = False,
+                        out=None, stream=None):
+    """W: [rows, cols] 16-bit tensor on the device. Returns (vals, meta, dense_or_None)."""
+    rows, cols = W.shape
+    R, K = (rows, cols) if group_dim == 1 else (cols, rows)
+    sf_prune24_sizes(rows, cols, group_dim)
+    if out is None:
+        vals = torch.empty((R, K // 2), dtype=W.dtype, device=W.device)
+        meta = torch.empty((R, K // 16), dtype=torch.int16, device=W.device)
+        dense = torch.empty((rows, cols), dtype=W.dtype, device=W.device) if want_dense else None
+    else:
+        vals, meta, dense = out
+    st = lib().sf_prune24_compress(_ptr(W), rows, cols, W.stride(0), group_dim, prune_mode,
+                                   _ptr(vals), _ptr(meta), _ptr(dense), _stream(stream))
+    _check(st, "sf_prune24_compress")
+    return vals, meta, dense
+
+
+# ---- V:N:M activation sparsification ------------------------------------------------------------
+
+def sf_vnm_sizes(T, F, V, N, M):
+    a, b, c = _sz(), _sz(), _sz()
+    _check(lib().sf_vnm_sizes(T, F, V, N, M, C.byref(a), C.byref(b), C.byref(c)), "sf_vnm_sizes")
+    return a.value, b.value, c.value
+
+
+def sf_vnm_sparsify_act(P: torch.Tensor, V: int, M: int, N: int = 2, apply_sqrelu: bool = True,
+                        want_relu: bool = True, want_dense: bool = False, out=None, stream=None):
+    """P: [T, F] 16-bit tensor. Returns (vals, meta, colidx, relu_vals_or_None, dense_or_None)."""
+    T, F = P.shape
+    sf_vnm_sizes(T, F, V, N, M)
+    if out is None:
+        G = F // M
+        vals = torch.empty((T, 2 * G), dtype=P.dtype, device=P.device)
+        meta = torch.empty((T, G // 4), dtype=torch.int16, device=P.device)
+        colidx = torch.empty((T // V, G, 4), dtype=torch.uint8, device=P.device)
+        relu = torch.empty((T, 2 * G), dtype=P.dtype, device=P.device) if (want_relu and apply_sqrelu) else None
+        dense = torch.empty((T, F), dtype=P.dtype, device=P.device) if want_dense else None
+    else:
+        vals, meta, colidx, relu, dense = out
+    st = lib().sf_vnm_sparsify_act(_ptr(P), T, F, P.stride(0), V, N, M, int(apply_sqrelu), _ptr(vals), _ptr(meta),
+                                   _ptr(colidx), _ptr(relu), _ptr(dense), _stream(stream))
+    _check(st, "sf_vnm_sparsify_act")
+    return vals, meta, colidx, relu, dense
+
+
+# ---- single products -----------------------------------------------------------------------------
+
+def sf_gemm_workspace_size(Mr: int, K: int) -> int:
+    a = _sz()
+    _check(lib().sf_gemm_workspace_size(Mr, K, C.byref(a)), "sf_gemm_workspace_size")
+    return a.value
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.zeros((max(nbytes, 256),), dtype=torch.uint8, device=device)
+
+
+def sf_gemm_dense(A: torch.Tensor, a_kmajor: bool, B: torch.Tensor, b_kmajor: bool, C_out=None,
+                  workspace=None, stream=None):
+    """C[Mr,Nc] = op(A) op(B)^T. A is [Mr,K] (a_kmajor) or [K,Mr]; B is [Nc,K] (b_kmajor) or [K,Nc]."""
+    Mr, K = A.shape if a_kmajor else (A.shape[1], A.shape[0])
+    Nc = B.shape[0] if b_kmajor else B.shape[1]
+    if C_out is None:
+        C_out = torch.empty((Mr, Nc), dtype=A.dtype, device=A.device)
+    if workspace is None:
+        workspace = _workspace(sf_gemm_workspace_size(Mr, K), A.device)
+    st = lib().sf_gemm_dense(_ptr(A), int(a_kmajor), _ptr(B), int(b_kmajor), _ptr(C_out), Mr, Nc, K,
+                             _ptr(workspace), _stream(stream))
+    _check(st, "sf_gemm_dense")
+    return C_out, workspace
+
+
+def sf_gemm_sparse24(a_vals, a_meta, B, Ct_out=None, workspace=None, stream=None):
+    """Ct[Nc,Mr] = (A_s[Mr,K] B[Nc,K]^T)^T with A_s packed (vals [Mr,K/2], meta [Mr,K/16])."""
+    Mr, K = a_vals.shape[0], a_vals.shape[1] * 2
+    Nc = B.shape[0]
+    if Ct_out is None:
+        Ct_out = torch.empty((Nc, Mr), dtype=B.dtype, device=B.device)
+    if workspace is None:
+        workspace = _workspace(sf_gemm_workspace_size(Mr, K), B.device)
+    st = lib().sf_gemm_sparse24(_ptr(a_vals), _ptr(a_meta), _ptr(B), _ptr(Ct_out), Mr, Nc, K,
+                                _ptr(workspace), _stream(stream))
+    _check(st, "sf_gemm_sparse24")
+    return Ct_out, workspace
+
+
+def sf_gemm_venom(a_vals, a_meta, colidx, Bt, V: int, M: int, C_out=None, workspace=None, stream=None):
+    """C[T,Nc] = A_vnm[T,F] Bt[F,Nc] with A_vnm in packed V:N:M form."""
+    T = a_vals.shape[0]
+    F, Nc = Bt.shape
+    if C_out is None:
+        C_out = torch.empty((T, Nc), dtype=Bt.dtype, device=Bt.device)
+    if workspace is None:
+        workspace = _workspace(sf_gemm_workspace_size(T, 4 * F // M), Bt.device)
+    st = lib().sf_gemm_venom(_ptr(a_vals), _ptr(a_meta), _ptr(colidx), _ptr(Bt), _ptr(C_out), T, F, Nc, V, M,
+                             _ptr(workspace), _stream(stream))
+    _check(st, "sf_gemm_venom")
+    return C_out, workspace
+
+
+# ---- FFN step --------------------------------------------------------------------------------------
+
+def sf_ffn_workspace_size(desc: sf_ffn_desc):
+    a, b = _sz(), _sz()
+    _check(lib().sf_ffn_workspace_size(C.byref(desc), C.byref(a), C.byref(b)), "sf_ffn_workspace_size")
+    return a.value, b.value
+
+
+def alloc_ffn_buffers(desc: sf_ffn_desc, device="cuda"):
+    """(fwd_ctx, workspace) as zero-initialised uint8 tensors of the sizes the library asks for."""
+    c, w = sf_ffn_workspace_size(desc)
+    return _workspace(c, device), _workspace(w, device)
+
+
+def sf_sparse_ffn_fwd(desc, X, W1, W2, Y, fwd_ctx, workspace, stream=None):
+    _check(lib().sf_sparse_ffn_fwd(C.byref(desc), _ptr(X), _ptr(W1), _ptr(W2), _ptr(Y), _ptr(fwd_ctx),
+                                   _ptr(workspace), _stream(stream)), "sf_sparse_ffn_fwd")
+
+
+def sf_sparse_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stream=None):
+    _check(lib().sf_sparse_ffn_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(W1), _ptr(W2), _ptr(fwd_ctx),
+                                   _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace), _stream(stream)),
+           "sf_sparse_ffn_bwd")
+
+
+def sf_dense_ffn_fwd(desc, X, W1, W2, Y, fwd_ctx, workspace, stream=None):
+    _check(lib().sf_dense_ffn_fwd(C.byref(desc), _ptr(X), _ptr(W1), _ptr(W2), _ptr(Y), _ptr(fwd_ctx),
+                                  _ptr(workspace), _stream(stream)), "sf_dense_ffn_fwd")
+
+
+def sf_dense_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stream=None):
+    _check(lib().sf_dense_ffn_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(W1), _ptr(W2), _ptr(fwd_ctx),
+                                  _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace), _stream(stream)),
+           "sf_dense_ffn_bwd")
+
+
+_CTX_DTYPES = {SF_CTX_Y2_VALS: torch.bfloat16, SF_CTX_RELU_VALS: torch.bfloat16, SF_CTX_META: torch.int16,
+               SF_CTX_COLIDX: torch.uint8, SF_CTX_Y1: torch.bfloat16, SF_CTX_DY1_VALS: torch.bfloat16}
+
+
+def sf_ctx_view(desc, buf: torch.Tensor, field: int) -> torch.Tensor:
+    """A flat tensor aliasing one field of the forward context (or workspace for DY1_VALS)."""
+    p, n = _vp(), _sz()
+    _check(lib().sf_ctx_view(C.byref(desc), _ptr(buf), field, C.byref(p), C.byref(n)), "sf_ctx_view")
+    off = p.value - buf.data_ptr()
+    return buf[off:off + n.value].view(_CTX_DTYPES[field])
+
+
+def sf_ffn_host_staging_size(desc) -> int:
+    a = _sz()
+    _check(lib().sf_ffn_host_staging_size(C.byref(desc), C.byref(a)), "sf_ffn_host_staging_size")
+    return a.value
+
+
+def sf_ffn_step_host(desc, dense: bool, hX, hW1, hW2, hdY, hY, hdX, hdW1, hdW2, staging, fwd_ctx, workspace,
+                     stream=None):
+    """Host tensors in, host tensors out (pinned memory recommended); does not synchronise."""
+    _check(lib().sf_ffn_step_host(C.byref(desc), int(dense), _ptr(hX), _ptr(hW1), _ptr(hW2), _ptr(hdY), _ptr(hY),
+                                  _ptr(hdX), _ptr(hdW1), _ptr(hdW2), _ptr(staging), _ptr(fwd_ctx), _ptr(workspace),
+                                  _stream(stream)), "sf_ffn_step_host")
+
+
+def sf_check_status(workspace, stream=None) -> int:
+    return lib().sf_check_status(_ptr(workspace), _stream(stream))

@@ -1,0 +1,233 @@
+// 2:4 weight sparsification + packing (Section 2.2 and Section 3.2.1 of the paper).
+//
+// Streaming, HBM-bound kernels: 2 B read + 1 B packed values + 1/8 B metadata per element.
+//   * contiguous groups: one thread owns 16 consecutive elements of a row (four groups, one
+//     metadata word): two 128-bit loads, one 128-bit store of packed values, one 16-bit store.
+//   * strided groups (groups along dim 0, output K-major): a CTA stages a [128 x 64] panel in
+//     shared memory, selects per column, and writes the transposed packed panel with 128-bit
+//     stores through a padded staging buffer.
+#include "sf_common.cuh"
+
+namespace sf {
+
+namespace {
+
+// Selection for one group given the four raw bf16 patterns; returns nibble, writes the two
+// packed output patterns (hard: kept bits; soft: shrunk by the third-ranked magnitude).
+template <bool kSoft>
+__device__ __forceinline__ uint32_t prune_group(uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                uint32_t& o0, uint32_t& o1) {
+  const uint32_t a[4] = {a0, a1, a2, a3};
+  uint32_t third;
+  const uint32_t nib = top2of4(a0 & 0x7FFFu, a1 & 0x7FFFu, a2 & 0x7FFFu, a3 & 0x7FFFu, &third);
+  const uint32_t p0 = nib & 3u, p1 = nib >> 2;
+  // register-only selects (no dynamic indexing into local memory)
+  uint32_t v0 = p0 == 0 ? a[0] : p0 == 1 ? a[1] : a[2];
+  uint32_t v1 = p1 == 1 ? a[1] : p1 == 2 ? a[2] : a[3];
+  if (kSoft) {
+    const uint32_t tk = (third == 0 ? a[0] : third == 1 ? a[1] : third == 2 ? a[2] : a[3]) & 0x7FFFu;
+    const float t = bf16_bits_to_float(tk);
+    const float f0 = bf16_bits_to_float(v0), f1 = bf16_bits_to_float(v1);
+    const float s0 = f0 > 0.f ? __fsub_rn(f0, t) : (f0 < 0.f ? __fadd_rn(f0, t) : 0.f);
+    const float s1 = f1 > 0.f ? __fsub_rn(f1, t) : (f1 < 0.f ? __fadd_rn(f1, t) : 0.f);
+    v0 = float_to_bf16_bits(s0);
+    v1 = float_to_bf16_bits(s1);
+  }
+  o0 = v0;
+  o1 = v1;
+  return nib;
+}
+
+// Expand (nibble, two values) to the four dense patterns of a group.
+__device__ __forceinline__ void expand_group(uint32_t nib, uint32_t v0, uint32_t v1, uint32_t d[4]) {
+  const uint32_t p0 = nib & 3u, p1 = nib >> 2;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) d[i] = (p0 == (uint32_t)i) ? v0 : (p1 == (uint32_t)i) ? v1 : 0u;
+}
+
+template <bool kSoft>
+__global__ void __launch_bounds__(256)
+prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int64_t cols, int64_t ld,
+                    uint4* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
+                    uint4* __restrict__ dense_out) {
+  const int64_t words_per_row = cols >> 4;                       // 16-element chunks per row
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * words_per_row) return;
+  const int64_t r = idx / words_per_row, kw = idx - r * words_per_row;
+
+  const uint4* src = W + ((r * ld) >> 3) + (kw << 1);
+  const uint4 q0 = __ldg(src), q1 = __ldg(src + 1);
+  const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+
+  uint32_t packed[4], m = 0, dense[8];
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const uint32_t lo = w[2 * g], hi = w[2 * g + 1];
+    uint32_t o0, o1;
+    const uint32_t nib = prune_group<kSoft>(lo & 0xFFFFu, lo >> 16, hi & 0xFFFFu, hi >> 16, o0, o1);
+    packed[g] = o0 | (o1 << 16);
+    m |= nib << (4 * g);
+    if (dense_out) {
+      uint32_t d[4];
+      expand_group(nib, o0, o1, d);
+      dense[2 * g] = d[0] | (d[1] << 16);
+      dense[2 * g + 1] = d[2] | (d[3] << 16);
+    }
+  }
+  vals[idx] = make_uint4(packed[0], packed[1], packed[2], packed[3]);       // [R, K/2] bf16: 8 per chunk
+  meta[idx] = (uint16_t)m;
+  if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(r, kw, cols)) = (uint16_t)m;
+  if (dense_out) {
+    uint4* dst = dense_out + ((r * cols) >> 3) + (kw << 1);
+    dst[0] = make_uint4(dense[0], dense[1], dense[2], dense[3]);
+    dst[1] = make_uint4(dense[4], dense[5], dense[6], dense[7]);
+  }
+}
+
+// Strided groups. W is [Kd, Rc] row-major (Kd = rows = reduction dim, Rc = cols); outputs are
+// vals [Rc, Kd/2], meta [Rc, Kd/16]. Panel: 128 reduction rows x 64 columns per CTA.
+constexpr int kPanelK = 128, kPanelC = 64;
+constexpr int kStageRow = (kPanelK / 2) * 2 + 16;   // packed bytes per column + 16 B pad
+
+template <bool kSoft>
+__global__ void __launch_bounds__(256)
+prune24_cols_kernel(const uint16_t* __restrict__ W, int64_t Kd, int64_t Rc, int64_t ld,
+                    uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
+                    uint16_t* __restrict__ dense_out) {
+  __shared__ __align__(16) uint16_t tile[kPanelK][kPanelC + 8];          // +8: 16 B pad per row
+  __shared__ __align__(16) uint8_t stage[kPanelC][kStageRow];
+  __shared__ uint16_t mstage[kPanelC][kPanelK / 16];
+
+  const int64_t c0 = (int64_t)blockIdx.x * kPanelC;
+  const int64_t k0 = (int64_t)blockIdx.y * kPanelK;
+  const int tid = threadIdx.x;
+  const int kvalid = (int)min((int64_t)kPanelK, Kd - k0);               // multiple of 16
+  const int cvalid = (int)min((int64_t)kPanelC, Rc - c0);               // multiple of 8
+
+  // load: 8 threads x 16 B per row of 64 columns
+  for (int i = tid; i < kPanelK * (kPanelC / 8); i += 256) {
+    const int kr = i >> 3, cc = (i & 7) << 3;
+    if (kr < kvalid && cc < cvalid) {
+      const uint4 q = __ldg(reinterpret_cast<const uint4*>(W + (k0 + kr) * ld + c0 + cc));
+      *reinterpret_cast<uint4*>(&tile[kr][cc]) = q;
+    }
+  }
+  __syncthreads();
+
+  // select: lanes along columns (conflict-free), one thread per (column, 16-row chunk)
+  for (int i = tid; i < kPanelC * (kPanelK / 16); i += 256) {
+    const int c = i & (kPanelC - 1), ch = i >> 6;                        // ch: chunk of 16 rows
+    if (c >= cvalid || ch * 16 >= kvalid) continue;
+    uint32_t packed[4], m = 0;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const int kr = ch * 16 + g * 4;
+      uint32_t o0, o1;
+      const uint32_t nib = prune_group<kSoft>(tile[kr][c], tile[kr + 1][c], tile[kr + 2][c], tile[kr + 3][c], o0, o1);
+      packed[g] = o0 | (o1 << 16);
+      m |= nib << (4 * g);
+      if (dense_out) {
+        uint32_t d[4];
+        expand_group(nib, o0, o1, d);
+        tile[kr][c] = (uint16_t)d[0];
+        tile[kr + 1][c] = (uint16_t)d[1];
+        tile[kr + 2][c] = (uint16_t)d[2];
+        tile[kr + 3][c] = (uint16_t)d[3];
+      }
+    }
+    *reinterpret_cast<uint4*>(&stage[c][ch * 16]) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    mstage[c][ch] = (uint16_t)m;
+  }
+  __syncthreads();
+
+  // store packed values: per column kvalid/2 elements = kvalid bytes, 16 B per thread
+  const int chunks = kvalid >> 4;
+  for (int i = tid; i < kPanelC * chunks; i += 256) {
+    const int c = i / chunks, ch = i - c * chunks;
+    if (c >= cvalid) continue;
+    const uint4 q = *reinterpret_cast<const uint4*>(&stage[c][ch * 16]);
+    *reinterpret_cast<uint4*>(vals + (c0 + c) * (Kd >> 1) + (k0 >> 1) + ch * 8) = q;
+    const uint16_t mw = mstage[c][ch];
+    const int64_t kw = (k0 >> 4) + ch;
+    meta[(c0 + c) * (Kd >> 4) + kw] = mw;
+    if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(c0 + c, kw, Kd)) = mw;
+  }
+  if (dense_out) {
+    for (int i = tid; i < kPanelK * (kPanelC / 8); i += 256) {
+      const int kr = i >> 3, cc = (i & 7) << 3;
+      if (kr < kvalid && cc < cvalid)
+        *reinterpret_cast<uint4*>(dense_out + (k0 + kr) * Rc + c0 + cc) = *reinterpret_cast<const uint4*>(&tile[kr][cc]);
+    }
+  }
+}
+
+// Plain tiled transpose of a bf16 matrix: out[c][r] = in[r][c].
+__global__ void __launch_bounds__(256)
+transpose_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, int64_t rows, int64_t cols) {
+  __shared__ uint16_t t[64][64 + 2];
+  const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;                // 32 x 8
+  for (int i = ty; i < 64; i += 8) {
+    const int64_t r = r0 + i;
+    if (r < rows) {
+      const int64_t c = c0 + 2 * tx;
+      if (c + 1 < cols) {
+        const uint32_t v = *reinterpret_cast<const uint32_t*>(in + r * cols + c);
+        t[i][2 * tx] = (uint16_t)v;
+        t[i][2 * tx + 1] = (uint16_t)(v >> 16);
+      } else if (c < cols) {
+        t[i][2 * tx] = in[r * cols + c];
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = ty; i < 64; i += 8) {
+    const int64_t c = c0 + i;                                            // output row
+    if (c < cols) {
+      const int64_t r = r0 + 2 * tx;
+      if (r + 1 < rows) {
+        const uint32_t v = (uint32_t)t[2 * tx][i] | ((uint32_t)t[2 * tx + 1][i] << 16);
+        *reinterpret_cast<uint32_t*>(out + c * rows + r) = v;
+      } else if (r < rows) {
+        out[c * rows + r] = t[2 * tx][i];
+      }
+    }
+  }
+}
+
+}  // namespace
+
+int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int group_dim, int prune_mode,
+                   void* vals, void* meta, void* meta_hw, void* dense_out, cudaStream_t s) {
+  if (rows == 0 || cols == 0) return SF_OK;
+  if (group_dim == 1) {
+    const int64_t n = rows * (cols >> 4);
+    const unsigned grid = (unsigned)((n + 255) / 256);
+    if (prune_mode == 0)
+      prune24_rows_kernel<false><<<grid, 256, 0, s>>>((const uint4*)W, rows, cols, ld, (uint4*)vals,
+                                                      (uint16_t*)meta, (uint8_t*)meta_hw, (uint4*)dense_out);
+    else
+      prune24_rows_kernel<true><<<grid, 256, 0, s>>>((const uint4*)W, rows, cols, ld, (uint4*)vals,
+                                                     (uint16_t*)meta, (uint8_t*)meta_hw, (uint4*)dense_out);
+  } else {
+    dim3 grid((unsigned)((cols + kPanelC - 1) / kPanelC), (unsigned)((rows + kPanelK - 1) / kPanelK));
+    if (prune_mode == 0)
+      prune24_cols_kernel<false><<<grid, 256, 0, s>>>((const uint16_t*)W, rows, cols, ld, (uint16_t*)vals,
+                                                      (uint16_t*)meta, (uint8_t*)meta_hw, (uint16_t*)dense_out);
+    else
+      prune24_cols_kernel<true><<<grid, 256, 0, s>>>((const uint16_t*)W, rows, cols, ld, (uint16_t*)vals,
+                                                     (uint16_t*)meta, (uint8_t*)meta_hw, (uint16_t*)dense_out);
+  }
+  SF_LAUNCH_CHECK();
+  return SF_OK;
+}
+
+int launch_transpose(const void* in, void* out, int64_t rows, int64_t cols, cudaStream_t s) {
+  if (rows == 0 || cols == 0) return SF_OK;
+  dim3 grid((unsigned)((cols + 63) / 64), (unsigned)((rows + 63) / 64));
+  transpose_kernel<<<grid, 256, 0, s>>>((const uint16_t*)in, (uint16_t*)out, rows, cols);
+  SF_LAUNCH_CHECK();
+  return SF_OK;
+}
+
+}  // namespace sf

@@ -1,0 +1,84 @@
+// Shared host/device helpers of libsparseffn (private to csrc/).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/sparseffn.h"
+
+namespace sf {
+
+// Most recent failing cudaError_t (process-wide, informational).
+extern int g_last_cuda_error;
+
+inline int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = static_cast<int>(e);
+  return SF_ERR_CUDA;
+}
+
+#define SF_CUDA_TRY(expr)                               \
+  do {                                                  \
+    cudaError_t _e = (expr);                            \
+    if (_e != cudaSuccess) return ::sf::cuda_fail(_e);  \
+  } while (0)
+
+#define SF_LAUNCH_CHECK()                               \
+  do {                                                  \
+    cudaError_t _e = cudaGetLastError();                \
+    if (_e != cudaSuccess) return ::sf::cuda_fail(_e);  \
+  } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Returns SF_OK when the current device is compute capability 10.x.
+int check_arch();
+
+// ---- bf16 bit helpers (device) ---------------------------------------------------------
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+
+// round-to-nearest-even float -> bf16 bits (finite inputs; NaN stays NaN)
+__device__ __forceinline__ uint32_t float_to_bf16_bits(float f) {
+  return static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(f)));
+}
+
+// Top-2-of-4 by key (larger first, ties to the lower index). Returns the nibble
+// pos0 | pos1 << 2 with pos0 < pos1; *third receives the index of the element ranked third.
+__device__ __forceinline__ uint32_t top2of4(uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3,
+                                            uint32_t* third = nullptr) {
+  // c_ij (i < j) is 1 when element i precedes element j in (key desc, index asc)
+  const uint32_t c01 = k0 >= k1, c02 = k0 >= k2, c03 = k0 >= k3;
+  const uint32_t c12 = k1 >= k2, c13 = k1 >= k3, c23 = k2 >= k3;
+  const uint32_t r0 = (1 - c01) + (1 - c02) + (1 - c03);
+  const uint32_t r1 = c01 + (1 - c12) + (1 - c13);
+  const uint32_t r2 = c02 + c12 + (1 - c23);
+  const uint32_t r3 = c03 + c13 + c23;
+  const uint32_t keep = (r0 < 2 ? 1u : 0u) | (r1 < 2 ? 2u : 0u) | (r2 < 2 ? 4u : 0u) | (r3 < 2 ? 8u : 0u);
+  const uint32_t pos0 = __ffs(keep) - 1;
+  const uint32_t pos1 = 31 - __clz(keep);
+  if (third) *third = (r0 == 2) ? 0u : (r1 == 2) ? 1u : (r2 == 2) ? 2u : 3u;
+  return pos0 | (pos1 << 2);
+}
+
+// ---- internal launchers (defined in the .cu files) ---------------------------------------
+// meta_hw (optional) receives the same metadata words in the order the sparse tensor-core
+// instruction reads them (see gemm_sparse.cu); requires R % 128 == 0 and K % 128 == 0.
+int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int group_dim, int prune_mode,
+                   void* vals, void* meta, void* meta_hw, void* dense_out, cudaStream_t s);
+int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
+               void* vals, void* meta, void* meta_hw, void* colidx, void* relu_vals, void* dense_out,
+               cudaStream_t s);
+int launch_transpose(const void* in, void* out, int64_t rows, int64_t cols, cudaStream_t s);
+
+// Byte offset of the metadata word (row m, 16-column word kw) inside the hardware-ordered
+// metadata tensor of a [R, K] 2:4 operand: 2 KB atoms of 128 rows x 128 columns, atoms of one
+// row block stored consecutively along K.
+__host__ __device__ __forceinline__ size_t meta_hw_offset(int64_t m, int64_t kw, int64_t K) {
+  const int64_t atoms_per_rowblock = K >> 7;
+  const int64_t atom = (m >> 7) * atoms_per_rowblock + (kw >> 3);
+  const int mi = static_cast<int>(m & 127), kwi = static_cast<int>(kw & 7);
+  return static_cast<size_t>(atom) * 2048 + (mi >> 4) * 256 + (kwi & 1) * 128 + (mi & 7) * 16 +
+         (kwi >> 1) * 4 + ((mi >> 3) & 1) * 2;
+}
+
+}  // namespace sf

@@ -1,0 +1,171 @@
+// SquaredReLU + V:N:M (Venom) activation sparsification (Eq. 2, Section 2.3, Table 5).
+//
+// One CTA owns a strip of V rows x kCW columns (kCW / M blocks of V x M). The strip is staged in
+// shared memory once, so every input element is read from HBM exactly once:
+//   pass A  one thread per column: float32 score = sum over the V rows, first to last, of the
+//           magnitude of the stored activation; the four best columns of each M-column group
+//           stay (ties to the lower index) and are recorded in ascending order;
+//   pass B  one thread per (row, group): 2:4 among the four kept columns, emit two values, the
+//           two matching ReLU values, one metadata nibble (four neighbours form a uint16).
+// The accumulation order of pass A is part of the format: it is what makes the mask unique.
+#include "sf_common.cuh"
+
+namespace sf {
+
+namespace {
+
+constexpr int kCW = 256;          // columns per CTA strip
+constexpr int kPad = 8;           // 16 B row padding (bank spread)
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ void sqrelu_bits(uint32_t x, bool apply, uint32_t& h, uint32_t& relu) {
+  if (!apply) { h = x; relu = 0; return; }
+  const float y = bf16_bits_to_float(x);
+  const float r = y > 0.f ? y : 0.f;
+  relu = y > 0.f ? x : 0u;
+  h = float_to_bf16_bits(__fmul_rn(r, r));
+}
+
+__global__ void __launch_bounds__(kThreads)
+vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply,
+           uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
+           uint8_t* __restrict__ colidx, uint16_t* __restrict__ relu_vals, uint16_t* __restrict__ dense_out) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  uint16_t* tile = reinterpret_cast<uint16_t*>(smem_raw);                        // [V][kCW + kPad]
+  uint32_t* score = reinterpret_cast<uint32_t*>(tile + (size_t)V * (kCW + kPad)); // [kCW] float bits
+  uint8_t* keepf = reinterpret_cast<uint8_t*>(score + kCW);                       // [kCW]
+  uint8_t* cidx = keepf + kCW;                                                    // [kCW / 4][4]
+  constexpr int kRow = kCW + kPad;
+
+  const int tid = threadIdx.x;
+  const int64_t c0 = (int64_t)blockIdx.x * kCW;
+  const int64_t blk = blockIdx.y;
+  const int64_t t0 = blk * V;
+  const int cvalid = (int)min((int64_t)kCW, F - c0);
+  const int64_t G = F / M;
+
+  // ---- stage the strip
+  for (int i = tid; i < V * (kCW / 8); i += kThreads) {
+    const int r = i / (kCW / 8), cc = (i % (kCW / 8)) * 8;
+    if (cc < cvalid) {
+      const uint4 q = __ldg(reinterpret_cast<const uint4*>(P + (t0 + r) * ld + c0 + cc));
+      *reinterpret_cast<uint4*>(tile + r * kRow + cc) = q;
+    }
+  }
+  __syncthreads();
+
+  // ---- pass A: column scores (sequential float32 adds, rows in ascending order)
+  {
+    const int j = tid;
+    float s = 0.f;
+    if (j < cvalid) {
+      for (int r = 0; r < V; ++r) {
+        uint32_t h, relu;
+        sqrelu_bits(tile[r * kRow + j], apply, h, relu);
+        s = __fadd_rn(s, bf16_bits_to_float(h & 0x7FFFu));
+      }
+    }
+    score[j] = __float_as_uint(s);
+  }
+  __syncthreads();
+  {
+    const int j = tid, jm = j % M, base = j - jm;
+    const uint32_t s = score[j];
+    int rank = 0;
+    for (int i = 0; i < M; ++i) {
+      const uint32_t si = score[base + i];
+      rank += (si > s) || (si == s && i < jm);
+    }
+    keepf[j] = rank < 4;
+  }
+  __syncthreads();
+  {
+    const int j = tid, jm = j % M, base = j - jm;
+    if (keepf[j] && j < cvalid) {
+      int pos = 0;
+      for (int i = 0; i < jm; ++i) pos += keepf[base + i];
+      cidx[(j / M) * 4 + pos] = (uint8_t)jm;
+    }
+  }
+  __syncthreads();
+  const int ng = cvalid / M;                                  // groups in this strip (multiple of 4)
+  if (tid < ng) {
+    const uint32_t c4 = *reinterpret_cast<const uint32_t*>(cidx + tid * 4);
+    *reinterpret_cast<uint32_t*>(colidx + (blk * G + c0 / M + tid) * 4) = c4;
+  }
+
+  // ---- pass B: 2:4 inside the kept columns, one (row, group) item per thread
+  const int items = V * ng;
+  const int items_pad = (items + 31) & ~31;
+  const int64_t g0 = c0 / M;
+  for (int i = tid; i < items_pad; i += kThreads) {
+    const bool valid = i < items;
+    const int r = valid ? i / ng : 0, g = valid ? i - r * ng : 0;
+    const uint32_t c4 = *reinterpret_cast<const uint32_t*>(cidx + g * 4);
+    const uint16_t* row = tile + r * kRow + g * M;
+    uint32_t h[4], rl[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) sqrelu_bits(row[(c4 >> (8 * k)) & 0xFFu], apply, h[k], rl[k]);
+    const uint32_t nib = top2of4(h[0] & 0x7FFFu, h[1] & 0x7FFFu, h[2] & 0x7FFFu, h[3] & 0x7FFFu);
+    const uint32_t p0 = nib & 3u, p1 = nib >> 2;
+    const uint32_t v0 = p0 == 0 ? h[0] : p0 == 1 ? h[1] : h[2];
+    const uint32_t v1 = p1 == 1 ? h[1] : p1 == 2 ? h[2] : h[3];
+    const int64_t t = t0 + r;
+    if (valid) {
+      *reinterpret_cast<uint32_t*>(vals + t * (2 * G) + 2 * (g0 + g)) = v0 | (v1 << 16);
+      if (relu_vals && apply) {
+        const uint32_t r0 = p0 == 0 ? rl[0] : p0 == 1 ? rl[1] : rl[2];
+        const uint32_t r1 = p1 == 1 ? rl[1] : p1 == 2 ? rl[2] : rl[3];
+        *reinterpret_cast<uint32_t*>(relu_vals + t * (2 * G) + 2 * (g0 + g)) = r0 | (r1 << 16);
+      }
+      if (dense_out) {
+        const uint32_t ca = (c4 >> (8 * p0)) & 0xFFu, cb = (c4 >> (8 * p1)) & 0xFFu;
+        uint16_t* drow = dense_out + t * F + c0 + g * M;
+        for (int m8 = 0; m8 < M; m8 += 8) {
+          uint32_t w[4] = {0, 0, 0, 0};
+          if (ca >= (uint32_t)m8 && ca < (uint32_t)m8 + 8) w[(ca - m8) >> 1] |= v0 << (16 * ((ca - m8) & 1));
+          if (cb >= (uint32_t)m8 && cb < (uint32_t)m8 + 8) w[(cb - m8) >> 1] |= v1 << (16 * ((cb - m8) & 1));
+          if (M >= 8) {
+            *reinterpret_cast<uint4*>(drow + m8) = make_uint4(w[0], w[1], w[2], w[3]);
+          } else {                                              // M == 4: 8-byte group
+            *reinterpret_cast<uint2*>(drow) = make_uint2(w[0], w[1]);
+          }
+        }
+      }
+    }
+    // four neighbouring groups of a row -> one metadata word (ng is a multiple of 4)
+    uint32_t word = valid ? nib : 0u;
+    word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 4;
+    word |= __shfl_down_sync(0xFFFFFFFFu, word, 2) << 8;
+    if (valid && (g & 3) == 0) {
+      const int64_t kw = (g0 + g) >> 2;
+      meta[t * (G >> 2) + kw] = (uint16_t)word;
+      if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(t, kw, 4 * G)) = (uint16_t)word;
+    }
+  }
+}
+
+}  // namespace
+
+int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
+               void* vals, void* meta, void* meta_hw, void* colidx, void* relu_vals, void* dense_out,
+               cudaStream_t s) {
+  if (T == 0 || F == 0) return SF_OK;
+  const size_t smem = (size_t)V * (kCW + kPad) * 2 + kCW * 4 + kCW + kCW;
+  static bool attr_set[64] = {false};                         // per device
+  int dev = 0;
+  SF_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    SF_CUDA_TRY(cudaFuncSetAttribute(vnm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     128 * (kCW + kPad) * 2 + kCW * 6));
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  dim3 grid((unsigned)((F + kCW - 1) / kCW), (unsigned)(T / V));
+  vnm_kernel<<<grid, kThreads, smem, s>>>((const uint16_t*)P, T, F, ld, V, M, apply_sqrelu, (uint16_t*)vals,
+                                          (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
+                                          (uint16_t*)relu_vals, (uint16_t*)dense_out);
+  SF_LAUNCH_CHECK();
+  return SF_OK;
+}
+
+}  // namespace sf

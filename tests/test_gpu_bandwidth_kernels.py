@@ -1,0 +1,93 @@
+"""Bit-exact parity of prune24_compress and vnm_sparsify_act (CUDA, through the C ABI) with the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_06183_b200 import binding, synth
+from util import to_dev, bits
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("rows,cols", [(128, 256), (96, 1040), (1, 16), (513, 4112)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_prune24_rows_bit_exact(rows, cols, mode):
+    w = synth.prune_sweep_matrix(rows, cols, seed=1000 + rows + mode, tie_frac=0.1)
+    ref = oracle.prune24(w, group_dim=1, mode=mode)
+    vals, meta, dense = binding.sf_prune24_compress(to_dev(w), 1, mode, want_dense=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(meta), ref.meta)
+    assert np.array_equal(bits(vals), ref.vals)
+    assert np.array_equal(bits(dense), ref.dense)
+
+
+@pytest.mark.parametrize("rows,cols", [(128, 64), (256, 1000), (16, 8), (4112, 520)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_prune24_cols_bit_exact(rows, cols, mode):
+    w = synth.prune_sweep_matrix(rows, cols, seed=2000 + rows + mode, tie_frac=0.1, axis=0)
+    ref = oracle.prune24(w, group_dim=0, mode=mode)
+    vals, meta, dense = binding.sf_prune24_compress(to_dev(w), 0, mode, want_dense=True)
+    torch.cuda.synchronize()
+    assert vals.shape == (cols, rows // 2)
+    assert np.array_equal(bits(meta), ref.meta)
+    assert np.array_equal(bits(vals), ref.vals)
+    assert np.array_equal(bits(dense), ref.dense)
+
+
+def test_prune24_strided_input_and_special_values():
+    w = synth.prune_sweep_matrix(64, 512, seed=5, tie_frac=0.5)
+    w[:, :16] = 0                       # all-zero groups
+    w[0, 16:32] = 0x8000                # negative zeros
+    big = to_dev(np.concatenate([w, w], axis=1))        # ld = 1024, logical cols = 512
+    view = big[:, :512]
+    ref = oracle.prune24(w, 1, 0)
+    vals, meta, _ = binding.sf_prune24_compress(view, 1, 0)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(meta), ref.meta) and np.array_equal(bits(vals), ref.vals)
+
+
+@pytest.mark.parametrize("T,F,V,M", [(128, 512, 64, 8), (256, 1024, 128, 16), (128, 320, 64, 4),
+                                     (64, 256, 32, 32), (128, 256, 64, 64), (192, 832, 64, 8)])
+def test_vnm_bit_exact(T, F, V, M):
+    p = synth.act_sweep_matrix(T, F, seed=3000 + T + M)
+    ref = oracle.vnm_sparsify(p, V=V, M=M)
+    vals, meta, colidx, relu, dense = binding.sf_vnm_sparsify_act(to_dev(p), V, M, want_dense=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(colidx.cpu().numpy(), ref.colidx)
+    assert np.array_equal(bits(meta), ref.meta)
+    assert np.array_equal(bits(vals), ref.vals)
+    assert np.array_equal(bits(relu), ref.relu_vals)
+    assert np.array_equal(bits(dense), ref.dense)
+
+
+def test_vnm_no_activation_and_ties():
+    # raw magnitudes with many exact ties, negative values, apply_sqrelu = 0
+    p = synth.prune_sweep_matrix(128, 512, seed=9, tie_frac=0.5)
+    p[:64, :64] = 0
+    ref = oracle.vnm_sparsify(p, V=64, M=8, apply_sqrelu=False)
+    vals, meta, colidx, relu, dense = binding.sf_vnm_sparsify_act(to_dev(p), 64, 8, apply_sqrelu=False, want_dense=True)
+    torch.cuda.synchronize()
+    assert relu is None
+    assert np.array_equal(colidx.cpu().numpy(), ref.colidx)
+    assert np.array_equal(bits(meta), ref.meta) and np.array_equal(bits(vals), ref.vals)
+    assert np.array_equal(bits(dense), ref.dense)
+
+
+def test_vnm_accumulation_order_case():
+    y = np.zeros((128, 256), dtype=np.float32)
+    y[0, 0] = 2.0 ** 24
+    y[1:, 0] = 1.0
+    y[0, 1] = 2.0 ** 24
+    y[1, 1] = 64.0
+    y[:, 2:5] = 2.0 ** 25
+    p = synth.f32_to_bf16_bits(y)
+    ref = oracle.vnm_sparsify(p, V=128, M=8, apply_sqrelu=False)
+    _, _, colidx, _, _ = binding.sf_vnm_sparsify_act(to_dev(p), 128, 8, apply_sqrelu=False)
+    assert tuple(colidx.cpu().numpy()[0, 0]) == (1, 2, 3, 4) == tuple(ref.colidx[0, 0])
+
+
+def test_empty_inputs_are_noops():
+    w = torch.empty((0, 256), dtype=torch.bfloat16, device="cuda")
+    vals, meta, _ = binding.sf_prune24_compress(w, 1, 0)
+    assert vals.numel() == 0 and meta.numel() == 0
