@@ -50,8 +50,8 @@ typedef enum sf_status {
 } sf_status;
 
 /* Problem descriptor of one FFN layer step. Ragged shapes are rejected, never padded:
- * T % 128 == 0, T % V == 0, D % 128 == 0, F % 128 == 0, F % (4*M) == 0, V in {64,128},
- * N == 2, M in {4,8,16,32}. */
+ * T, D, F multiples of 256, T % V == 0, (4F/M) % 128 == 0, V in {64,128}, N == 2,
+ * M in {4,8,16,32}. */
 typedef struct sf_ffn_desc {
   int64_t T, D, F;
   int32_t V, N, M;
@@ -117,13 +117,13 @@ SF_API int sf_vnm_sparsify_act(const void* preact, int64_t T, int64_t F, int64_t
  * sf_gemm_dense:  C[Mr,Nc] = op(A) op(B)^T, fp32 accumulate, bf16 out.
  *     a_kmajor = 1: A is [Mr,K] row-major;  0: A is stored [K,Mr] row-major (M contiguous)
  *     b_kmajor = 1: B is [Nc,K] row-major;  0: B is stored [K,Nc] row-major (N contiguous)
- *     Mr % 128 == 0, Nc % 128 == 0, K % 64 == 0.
+ *     Mr % 128 == 0, Nc % 256 == 0, K % 64 == 0.
  * sf_gemm_sparse24:  Ct[Nc,Mr] (transposed output!) with C[Mr,Nc] = A_s[Mr,K] B[Nc,K]^T where
  *     A_s is given packed: a_vals bf16 [Mr,K/2], a_meta canonical uint16 [Mr,K/16].
- *     This is y1 = X W1s^T with A_s = W1s, B = X, output y1 [T,F].  Mr,Nc % 128, K % 128.
+ *     This is y1 = X W1s^T with A_s = W1s, B = X, output y1 [T,F].  Mr % 128, Nc % 256, K % 128.
  * sf_gemm_venom:  C[T,Nc] = A_vnm[T,F] Bt[F,Nc] with A_vnm in V:N:M packed form (vals, meta,
  *     colidx as produced by sf_vnm_sparsify_act) and Bt row-major [F,Nc] (rows are gathered by
- *     colidx).  T % 128, V in {64,128}, Nc % 128, (4F/M) % 128 == 0.
+ *     colidx).  T % 128, V in {64,128}, Nc % 256, (4F/M) % 128 == 0.
  * `workspace` needs sf_gemm_workspace_size() bytes (hardware-ordered metadata copy + status).
  */
 SF_API int sf_gemm_workspace_size(int64_t Mr, int64_t K, size_t* bytes);
@@ -139,7 +139,8 @@ SF_API int sf_gemm_venom(const void* a_vals, const void* a_meta, const void* col
  * The FFN step (Algorithm 1 = forward, Algorithm 2 = backward; Eqs. 1-8 for the dense phase).
  *
  * sf_ffn_workspace_size: bytes of the forward context (saved for backward) and of the scratch
- * workspace for `desc`. Both buffers are caller-allocated device memory, 256-byte aligned.
+ * workspace for `desc`. Both buffers are caller-allocated device memory, 256-byte aligned. The
+ * first 256 bytes of a workspace hold the device status word: zero them once before first use.
  *
  * sf_sparse_ffn_fwd:  W1s = prune24(W1 along D);  y1 = X W1s^T;  y2 = V:N:M(ReLU(y1)^2);
  *                     Y = y2 W2^T  (W2 dense).  Saves packed y2, packed ReLU(y1), metadata,

@@ -1,0 +1,478 @@
+// Tensor-core products of the FFN step on sm_100a: tcgen05.mma with TMEM accumulators, operands
+// staged in shared memory by TMA, warp-specialised roles.
+//
+//   mode DENSE     D[M,N] = A[M,K] B[N,K]^T                       (Eqs. 1-8; weight-gradient products)
+//   mode SPARSE24  A is 2:4-compressed (values [M,K/2] + metadata) (Algorithm 1 line 4, Algorithm 2 line 2)
+//   mode VENOM     A is V:N:M-compressed; B rows are gathered by the block's kept columns
+//                  (Algorithm 1 line 7, Algorithm 2 line 5)
+//
+// CTA = 6 warps: warp 0 TMA producer, warp 1 MMA issuer (+ TMEM owner), warps 2-5 epilogue (each
+// owns the 32 TMEM lanes of its quadrant). Tile 128 x 256, persistent over tiles (m fastest).
+// A stage holds A (<= 16 KB), B (32 KB) and, for sparse modes, one 2 KB metadata atom covering
+// 128 rows x 128 logical K (copied smem -> TMEM by tcgen05.cp every second stage).
+// Dense mode double-buffers the 256-column accumulator so the epilogue of tile i overlaps the main
+// loop of tile i+1; sparse modes keep one accumulator plus the metadata columns.
+// Every mbarrier wait is bounded; on expiry the CTA raises a flag in the status word and leaves.
+#include "sf_common.cuh"
+#include "tc_ptx.cuh"
+#include "gemm_tc.cuh"
+
+namespace sf {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128, BN = 256;
+constexpr int kStages = 4;
+constexpr int kAStageBytes = 16384, kBStageBytes = 32768, kMetaStageBytes = 2048;
+constexpr int kStageBytes = kAStageBytes + kBStageBytes + kMetaStageBytes;          // 51200 (1024-aligned)
+constexpr int kEpiStageRow = 80;                                                      // bytes: 32 bf16 + 16 pad
+constexpr int kEpiStageBytes = 4 * 32 * kEpiStageRow;                                 // 4 warps
+constexpr int kSmemBytes = 1024 /*align slack*/ + kStages * kStageBytes + kEpiStageBytes + 256 /*barriers*/;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kMetaTmemCol = 256;
+
+struct SmemCtl {
+  uint64_t full[kStages];
+  uint64_t empty[kStages];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  return float_to_bf16_bits(lo) | (float_to_bf16_bits(hi) << 16);
+}
+
+template <int kMode, bool kAMN, bool kBMN, int kEpi>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+               const GemmArgs args) {
+  extern __shared__ uint8_t smem_dyn[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  uint8_t* epi_stage = smem + kStages * kStageBytes;
+  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(epi_stage + kEpiStageBytes);
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr bool kSparse = kMode != MODE_DENSE;
+  constexpr int kAccBufs = kSparse ? 1 : 2;
+  constexpr int kMmaPerStage = kSparse ? 2 : 4;      // dense: K=16 x4 = 64; sparse: logical K=32 x2 = 64
+
+  const int num_m_tiles = args.num_m_tiles, num_n_tiles = args.num_n_tiles;
+  const int num_tiles = num_m_tiles * num_n_tiles;
+  const int nkb = args.num_k_blocks;                 // 64-wide (logical) k blocks per sweep
+  const int sweeps = (kMode == MODE_VENOM && args.V == 64) ? 2 : 1;
+  const int iters = nkb * sweeps;
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&tmapA);
+    prefetch_tmap(&tmapB);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&ctl->full[s], 1);
+      mbar_init(&ctl->empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&ctl->tmem_full[b], 1);
+      mbar_init(&ctl->tmem_empty[b], 4);
+    }
+    ctl->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&ctl->tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+
+  if (warp == 0) {
+    // =========================== TMA producer ===========================
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      const int m0 = mt * BM, n0 = nt * BN;
+      for (int it = 0; it < iters; ++it) {
+        const int sweep = it / nkb, kb = it - sweep * nkb;
+        if (!mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+        uint8_t* sA = smem + stage * kStageBytes;
+        uint8_t* sB = sA + kAStageBytes;
+        uint8_t* sM = sB + kBStageBytes;
+        uint64_t* bar = &ctl->full[stage];
+        const bool load_meta = kSparse && ((kb & 1) == 0);
+        if (lane == 0) {
+          uint32_t bytes = kBStageBytes + (kSparse ? 8192u : 16384u) + (load_meta ? (uint32_t)kMetaStageBytes : 0u);
+          mbar_arrive_expect_tx(bar, bytes);
+          // ---- A
+          if (kMode == MODE_DENSE) {
+            if (!kAMN) {
+              tma_load_2d(sA, &tmapA, bar, kb * 64, m0);                       // box {64 k, 128 m}
+            } else {
+              tma_load_2d(sA, &tmapA, bar, m0, kb * 64);                       // box {64 m, 64 k}
+              tma_load_2d(sA + 8192, &tmapA, bar, m0 + 64, kb * 64);
+            }
+          } else if (kMode == MODE_SPARSE24 || sweeps == 1) {
+            tma_load_2d(sA, &tmapA, bar, kb * 32, m0);                         // stored: box {32, 128}
+          } else {
+            // V = 64: this sweep owns one 64-row half of the tile; the other half reads the zero
+            // fill of an out-of-range row coordinate. (box {32, 64})
+            const int oob = (int)args.M + 64;
+            tma_load_2d(sA, &tmapA, bar, kb * 32, sweep == 0 ? m0 : oob);
+            tma_load_2d(sA + 4096, &tmapA, bar, kb * 32, sweep == 1 ? m0 + 64 : oob);
+          }
+          // ---- metadata atom (2 KB, contiguous in the hardware-ordered tensor)
+          if (load_meta) {
+            const uint8_t* src = args.meta_hw + ((size_t)mt * (size_t)(nkb >> 1) + (size_t)(kb >> 1)) * 2048;
+            bulk_load(sM, src, kMetaStageBytes, bar);
+          }
+          // ---- B (non-gathered)
+          if (kMode != MODE_VENOM) {
+            if (!kBMN) {
+              tma_load_2d(sB, &tmapB, bar, kb * 64, n0);                       // box {64 k, 256 n}
+            } else {
+#pragma unroll
+              for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * 8192, &tmapB, bar, n0 + c * 64, kb * 64);
+            }
+          }
+        }
+        if (kMode == MODE_VENOM) {
+          // gathered B: 16 groups x 4 rows per stage; lane = (group, half of the 4 column chunks)
+          __syncwarp();
+          const int grp = lane >> 1, half = lane & 1;
+          const int blk = (args.V == 64) ? (2 * mt + sweep) : mt;
+          const int64_t g = (int64_t)kb * 16 + grp;                             // group index in the row
+          const uint32_t c4 = *reinterpret_cast<const uint32_t*>(args.colidx + ((int64_t)blk * args.G + g) * 4);
+          const int base = (int)(g * args.Mv);
+          const int r0 = base + (c4 & 0xFF), r1 = base + ((c4 >> 8) & 0xFF), r2 = base + ((c4 >> 16) & 0xFF),
+                    r3 = base + (c4 >> 24);
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            const int c = half * 2 + cc;
+            tma_gather4_2d(sB + c * 8192 + grp * 4 * 128, &tmapB, bar, n0 + c * 64, r0, r1, r2, r3);
+          }
+        }
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    // =========================== MMA issuer ===========================
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16(BM, BN, kAMN, kBMN || kMode == MODE_VENOM, kSparse);
+      uint32_t stage = 0, phase = 0;
+      uint32_t acc = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        if (!mbar_wait(&ctl->tmem_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + acc * BN;
+        for (int it = 0; it < iters; ++it) {
+          const int kb = it % nkb;
+          if (!mbar_wait(&ctl->full[stage], phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sA = smem_u32(smem + stage * kStageBytes);
+          const uint32_t sB = sA + kAStageBytes;
+          const uint32_t sM = sB + kBStageBytes;
+          if (kSparse && (kb & 1) == 0) {
+            // 128 rows x 16 B, no swizzle: 8-row core matrices 128 B apart
+            tmem_cp_128x128b(tmem_base + kMetaTmemCol, smem_desc(sM, 128, 128, kSwizzleNone));
+          }
+#pragma unroll
+          for (int k = 0; k < kMmaPerStage; ++k) {
+            uint64_t adesc, bdesc;
+            if (kMode == MODE_DENSE) {
+              adesc = kAMN ? smem_desc(sA + k * 2048, 8192, 1024, kSwizzle128B)
+                           : smem_desc(sA + k * 32, 16, 1024, kSwizzle128B);
+            } else {
+              adesc = smem_desc(sA + k * 32, 16, 512, 4 /* 64 B swizzle */);
+            }
+            if (kMode == MODE_VENOM || kBMN) {
+              // MN-major: 16 (dense) or 32 (sparse) k rows of 128 B per instruction
+              bdesc = smem_desc(sB + k * (kSparse ? 4096 : 2048), 8192, 1024, kSwizzle128B);
+            } else {
+              bdesc = smem_desc(sB + k * (kSparse ? 64 : 32), 16, 1024, kSwizzle128B);
+            }
+            const uint32_t accum = (it > 0 || k > 0) ? 1u : 0u;
+            if (kSparse) {
+              const uint32_t col = (uint32_t)((kb & 1) * 2 + k);              // metadata column of this k step
+              mma_sp_f16(tmem_d, adesc, bdesc, tmem_base + kMetaTmemCol + (col & ~1u), idesc | (col & 1u), accum);
+            } else {
+              mma_f16(tmem_d, adesc, bdesc, idesc, accum);
+            }
+          }
+          mma_commit(&ctl->empty[stage]);                                      // frees the smem stage
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        mma_commit(&ctl->tmem_full[acc]);                                      // accumulator ready
+        if (++acc == (uint32_t)kAccBufs) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else {
+    // =========================== epilogue (warps 2..5) ===========================
+    const int q = warp & 3;                                                    // TMEM lane quadrant
+    uint8_t* my_stage = epi_stage + q * 32 * kEpiStageRow;
+    uint32_t acc = 0, acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      const int64_t m0 = (int64_t)mt * BM, n0 = (int64_t)nt * BN;
+      if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
+      const int64_t row = m0 + q * 32 + lane;                                  // this thread's D row
+#pragma unroll 1
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        uint32_t v[32];
+        tmem_ld_32x32b_x32(taddr + ch * 32, v);
+        tmem_ld_wait();
+        const int64_t col0 = n0 + ch * 32;
+        if (kEpi == EPI_STORE || kEpi == EPI_SQRELU || kEpi == EPI_DRELU) {
+          uint16_t* crow = reinterpret_cast<uint16_t*>(args.C) + row * args.ldc + col0;
+          if (kEpi == EPI_STORE) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint4 o;
+              o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
+              o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
+              o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
+              o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+              reinterpret_cast<uint4*>(crow)[j] = o;
+            }
+          } else if (kEpi == EPI_SQRELU) {
+            uint16_t* hrow = reinterpret_cast<uint16_t*>(args.C2) + row * args.ldc2 + col0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t y[4], h[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const uint32_t y0 = float_to_bf16_bits(__uint_as_float(v[8 * j + 2 * e]));
+                const uint32_t y1 = float_to_bf16_bits(__uint_as_float(v[8 * j + 2 * e + 1]));
+                const float f0 = fmaxf(bf16_bits_to_float(y0), 0.f), f1 = fmaxf(bf16_bits_to_float(y1), 0.f);
+                y[e] = y0 | (y1 << 16);
+                h[e] = pack_bf16x2(__fmul_rn(f0, f0), __fmul_rn(f1, f1));
+              }
+              reinterpret_cast<uint4*>(crow)[j] = make_uint4(y[0], y[1], y[2], y[3]);
+              reinterpret_cast<uint4*>(hrow)[j] = make_uint4(h[0], h[1], h[2], h[3]);
+            }
+          } else {  // EPI_DRELU: C = bf16(2 * acc * relu(aux))
+            const uint16_t* arow = reinterpret_cast<const uint16_t*>(args.aux) + row * args.ldaux + col0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint4 a = __ldg(reinterpret_cast<const uint4*>(arow) + j);
+              const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
+              uint32_t o[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float r0 = fmaxf(bf16_bits_to_float(aw[e] & 0xFFFFu), 0.f);
+                const float r1 = fmaxf(bf16_bits_to_float(aw[e] >> 16), 0.f);
+                const float d0 = __fmul_rn(__fmul_rn(2.f, __uint_as_float(v[8 * j + 2 * e])), r0);
+                const float d1 = __fmul_rn(__fmul_rn(2.f, __uint_as_float(v[8 * j + 2 * e + 1])), r1);
+                o[e] = pack_bf16x2(d0, d1);
+              }
+              reinterpret_cast<uint4*>(crow)[j] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+          }
+        } else {
+          // Transposed output: D row = feature (lane), D column = token. C is [N, M] row-major.
+          float r[32];
+          if (kEpi == EPI_DRELU_T) {
+            // aux[token, feature] chunk -> staging -> one column per lane
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int t = i * 8 + (lane >> 2), seg = lane & 3;
+              const uint4 a = __ldg(reinterpret_cast<const uint4*>(
+                  reinterpret_cast<const uint16_t*>(args.aux) + (col0 + t) * args.ldaux + m0 + q * 32 + seg * 8));
+              *reinterpret_cast<uint4*>(my_stage + t * kEpiStageRow + seg * 16) = a;
+            }
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              r[j] = bf16_bits_to_float(*reinterpret_cast<const uint16_t*>(my_stage + j * kEpiStageRow + lane * 2));
+          }
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float x = __uint_as_float(v[j]);
+            uint32_t b;
+            if (kEpi == EPI_DRELU_T) {
+              // aux holds ReLU(y1) on the activation mask and +0 elsewhere: off-mask entries become +0
+              b = (r[j] == 0.f) ? 0u : float_to_bf16_bits(__fmul_rn(__fmul_rn(2.f, x), r[j]));
+            } else {
+              b = float_to_bf16_bits(x);
+            }
+            *reinterpret_cast<uint16_t*>(my_stage + j * kEpiStageRow + lane * 2) = (uint16_t)b;
+          }
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int t = i * 8 + (lane >> 2), seg = lane & 3;
+            const uint4 o = *reinterpret_cast<const uint4*>(my_stage + t * kEpiStageRow + seg * 16);
+            *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.C) + (col0 + t) * args.ldc + m0 + q * 32 + seg * 8) = o;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctl->tmem_empty[acc]);
+      if (++acc == (uint32_t)kAccBufs) { acc = 0; acc_phase ^= 1; }
+    }
+  }
+
+  // =========================== teardown ===========================
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && ctl->abort_flag) atomicExch(args.status, 1);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---- host side -----------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2D bf16 tensor map over a row-major [rows, cols] matrix; box = {box_cols, box_rows}.
+int make_tmap(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
+              uint32_t box_rows, CUtensorMapSwizzle swz) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return cuda_fail(cudaErrorUnknown);
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda_error = (int)r;
+    return SF_ERR_CUDA;
+  }
+  return SF_OK;
+}
+
+int sm_count() {
+  static int n[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (n[dev] == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    n[dev] = v;
+  }
+  return n[dev];
+}
+
+template <int kMode, bool kAMN, bool kBMN, int kEpi>
+int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& a, cudaStream_t s) {
+  auto kern = gemm_tc_kernel<kMode, kAMN, kBMN, kEpi>;
+  static bool attr_done[64] = {false};
+  int dev = 0;
+  SF_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+    SF_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    if (dev >= 0 && dev < 64) attr_done[dev] = true;
+  }
+  const int tiles = a.num_m_tiles * a.num_n_tiles;
+  const int grid = tiles < sm_count() ? tiles : sm_count();
+  kern<<<grid, kThreads, kSmemBytes, s>>>(ta, tb, a);
+  SF_LAUNCH_CHECK();
+  return SF_OK;
+}
+
+}  // namespace
+
+int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64_t M, int64_t N, int64_t K, int epi,
+               void* C, int64_t ldc, void* C2, int64_t ldc2, const void* aux, int64_t ldaux, int* status,
+               cudaStream_t s) {
+  if (M % BM || N % BN || K % 64) return SF_ERR_SHAPE;
+  if (M == 0 || N == 0) return SF_OK;
+  CUtensorMap ta, tb;
+  int st;
+  if (a_kmajor) st = make_tmap(&ta, A, M, K, K, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  else          st = make_tmap(&ta, A, K, M, M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  if (b_kmajor) st = make_tmap(&tb, B, N, K, K, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+  else          st = make_tmap(&tb, B, K, N, N, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = M; a.N = N; a.K = K;
+  a.C = C; a.ldc = ldc; a.C2 = C2; a.ldc2 = ldc2; a.aux = aux; a.ldaux = ldaux;
+  a.status = status;
+  a.num_m_tiles = (int)(M / BM); a.num_n_tiles = (int)(N / BN); a.num_k_blocks = (int)(K / 64);
+#define SF_DENSE_CASE(AMN, BMN, EPI) return launch_one<MODE_DENSE, AMN, BMN, EPI>(ta, tb, a, s)
+  const bool amn = !a_kmajor, bmn = !b_kmajor;
+  if (epi == EPI_STORE) {
+    if (!amn && !bmn) SF_DENSE_CASE(false, false, EPI_STORE);
+    if (!amn && bmn) SF_DENSE_CASE(false, true, EPI_STORE);
+    if (amn && !bmn) SF_DENSE_CASE(true, false, EPI_STORE);
+    SF_DENSE_CASE(true, true, EPI_STORE);
+  } else if (epi == EPI_SQRELU) {
+    if (!amn && !bmn) SF_DENSE_CASE(false, false, EPI_SQRELU);
+  } else if (epi == EPI_DRELU) {
+    if (!amn && bmn) SF_DENSE_CASE(false, true, EPI_DRELU);
+  }
+#undef SF_DENSE_CASE
+  return SF_ERR_UNSUPPORTED;
+}
+
+int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, int64_t M, int64_t N, int64_t K,
+                  int epi, void* Ct, int64_t ldc, const void* aux, int64_t ldaux, int* status, cudaStream_t s) {
+  if (M % BM || N % BN || K % 128) return SF_ERR_SHAPE;
+  if (M == 0 || N == 0) return SF_OK;
+  CUtensorMap ta, tb;
+  int st = make_tmap(&ta, a_vals, M, K / 2, K / 2, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tb, B, N, K, K, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = M; a.N = N; a.K = K;
+  a.C = Ct; a.ldc = ldc; a.aux = aux; a.ldaux = ldaux; a.meta_hw = meta_hw; a.status = status;
+  a.num_m_tiles = (int)(M / BM); a.num_n_tiles = (int)(N / BN); a.num_k_blocks = (int)(K / 64);
+  if (epi == EPI_STORE_T) return launch_one<MODE_SPARSE24, false, false, EPI_STORE_T>(ta, tb, a, s);
+  if (epi == EPI_DRELU_T) return launch_one<MODE_SPARSE24, false, false, EPI_DRELU_T>(ta, tb, a, s);
+  return SF_ERR_UNSUPPORTED;
+}
+
+int gemm_venom(const void* a_vals, const uint8_t* meta_hw, const uint8_t* colidx, const void* Bt, int64_t T,
+               int64_t F, int64_t N, int V, int Mv, void* C, int64_t ldc, int* status, cudaStream_t s) {
+  const int64_t Kc = 4 * F / Mv;                                               // condensed reduction length
+  if (T % BM || N % BN || Kc % 128 || (V != 64 && V != 128)) return SF_ERR_SHAPE;
+  if (T == 0 || N == 0) return SF_OK;
+  CUtensorMap ta, tb;
+  int st = make_tmap(&ta, a_vals, T, Kc / 2, Kc / 2, 32, V == 64 ? 64 : 128, CU_TENSOR_MAP_SWIZZLE_64B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tb, Bt, F, N, N, 64, 1, CU_TENSOR_MAP_SWIZZLE_128B);        // row gather: one row per box
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = T; a.N = N; a.K = Kc;
+  a.C = C; a.ldc = ldc; a.meta_hw = meta_hw; a.colidx = colidx; a.V = V; a.Mv = Mv; a.G = F / Mv;
+  a.status = status;
+  a.num_m_tiles = (int)(T / BM); a.num_n_tiles = (int)(N / BN); a.num_k_blocks = (int)(Kc / 64);
+  return launch_one<MODE_VENOM, false, true, EPI_STORE>(ta, tb, a, s);
+}
+
+}  // namespace sf

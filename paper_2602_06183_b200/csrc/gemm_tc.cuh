@@ -1,0 +1,52 @@
+// Internal interface of the tensor-core products (gemm_tc.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sf {
+
+enum GemmMode { MODE_DENSE = 0, MODE_SPARSE24 = 1, MODE_VENOM = 2 };
+
+enum GemmEpilogue {
+  EPI_STORE = 0,    // C[m, n] = bf16(acc)
+  EPI_SQRELU = 1,   // C = y = bf16(acc);  C2 = bf16(max(y, 0)^2)                     (Eq. 2)
+  EPI_DRELU = 2,    // C = bf16(2 * acc * max(aux[m, n], 0))                           (Eq. 6)
+  EPI_STORE_T = 3,  // C[n, m] = bf16(acc)          (accumulator rows are output columns)
+  EPI_DRELU_T = 4   // C[n, m] = bf16(2 * acc * aux[n, m]), +0 where aux is zero       (Eq. 6 on the mask)
+};
+
+struct GemmArgs {
+  int64_t M, N, K;
+  void* C;
+  int64_t ldc;
+  void* C2;
+  int64_t ldc2;
+  const void* aux;
+  int64_t ldaux;
+  const uint8_t* meta_hw;   // sparse modes: hardware-ordered metadata atoms
+  const uint8_t* colidx;    // Venom: [T/V, G, 4]
+  int64_t G;                // Venom: groups per row (F / Mv)
+  int V, Mv;                // Venom block height and group width
+  int* status;              // device status word (set to 1 when a bounded wait expires)
+  int num_m_tiles, num_n_tiles, num_k_blocks;
+};
+
+// D[M,N] = op(A) op(B)^T, tiles 128 x 256, K % 64 == 0.
+int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64_t M, int64_t N, int64_t K, int epi,
+               void* C, int64_t ldc, void* C2, int64_t ldc2, const void* aux, int64_t ldaux, int* status,
+               cudaStream_t s);
+// Ct[N,M] = (A_s[M,K] B[N,K]^T)^T with A_s 2:4-packed; epi in {EPI_STORE_T, EPI_DRELU_T}.
+int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, int64_t M, int64_t N, int64_t K,
+                  int epi, void* Ct, int64_t ldc, const void* aux, int64_t ldaux, int* status, cudaStream_t s);
+// C[T,N] = A_vnm[T,F] Bt[F,N]; A_vnm packed (vals [T, 2F/Mv], hardware-ordered metadata, colidx).
+int gemm_venom(const void* a_vals, const uint8_t* meta_hw, const uint8_t* colidx, const void* Bt, int64_t T,
+               int64_t F, int64_t N, int V, int Mv, void* C, int64_t ldc, int* status, cudaStream_t s);
+
+// canonical [R, K/16] metadata words -> hardware-ordered atoms (R % 128 == 0, K % 128 == 0)
+int launch_meta_reorder(const void* meta, void* meta_hw, int64_t R, int64_t K, cudaStream_t s);
+// dy1 packing: gather a dense [T, F] matrix at the positions recorded by (colidx, meta)
+int launch_pack_like(const void* dense, const void* meta, const void* colidx, void* vals, int64_t T, int64_t F,
+                     int V, int Mv, cudaStream_t s);
+
+}  // namespace sf

@@ -26,10 +26,31 @@ __device__ __forceinline__ void sqrelu_bits(uint32_t x, bool apply, uint32_t& h,
   h = float_to_bf16_bits(__fmul_rn(r, r));
 }
 
+// One group of M columns of a dense row: values va, vb at columns ca < cb, +0 elsewhere.
+__device__ __forceinline__ void write_group_dense(uint16_t* drow, int M, uint32_t ca, uint32_t cb, uint32_t va,
+                                                  uint32_t vb) {
+  for (int m8 = 0; m8 < M; m8 += 8) {
+    uint32_t w0 = 0, w1 = 0, w2 = 0, w3 = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const uint32_t col = (uint32_t)(m8 + e);
+      const uint32_t val = (col == ca) ? va : (col == cb) ? vb : 0u;
+      const uint32_t sh = val << (16 * (e & 1));
+      if (e < 2) w0 |= sh; else if (e < 4) w1 |= sh; else if (e < 6) w2 |= sh; else w3 |= sh;
+    }
+    if (M >= 8) {
+      *reinterpret_cast<uint4*>(drow + m8) = make_uint4(w0, w1, w2, w3);
+    } else {                                              // M == 4: one 8-byte group
+      *reinterpret_cast<uint2*>(drow) = make_uint2(w0, w1);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreads)
 vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply,
            uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
-           uint8_t* __restrict__ colidx, uint16_t* __restrict__ relu_vals, uint16_t* __restrict__ dense_out) {
+           uint8_t* __restrict__ colidx, uint16_t* __restrict__ relu_vals, uint16_t* __restrict__ dense_out,
+           uint16_t* __restrict__ relu_dense_out) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   uint16_t* tile = reinterpret_cast<uint16_t*>(smem_raw);                        // [V][kCW + kPad]
   uint32_t* score = reinterpret_cast<uint32_t*>(tile + (size_t)V * (kCW + kPad)); // [kCW] float bits
@@ -113,25 +134,12 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
     const int64_t t = t0 + r;
     if (valid) {
       *reinterpret_cast<uint32_t*>(vals + t * (2 * G) + 2 * (g0 + g)) = v0 | (v1 << 16);
-      if (relu_vals && apply) {
-        const uint32_t r0 = p0 == 0 ? rl[0] : p0 == 1 ? rl[1] : rl[2];
-        const uint32_t r1 = p1 == 1 ? rl[1] : p1 == 2 ? rl[2] : rl[3];
-        *reinterpret_cast<uint32_t*>(relu_vals + t * (2 * G) + 2 * (g0 + g)) = r0 | (r1 << 16);
-      }
-      if (dense_out) {
-        const uint32_t ca = (c4 >> (8 * p0)) & 0xFFu, cb = (c4 >> (8 * p1)) & 0xFFu;
-        uint16_t* drow = dense_out + t * F + c0 + g * M;
-        for (int m8 = 0; m8 < M; m8 += 8) {
-          uint32_t w[4] = {0, 0, 0, 0};
-          if (ca >= (uint32_t)m8 && ca < (uint32_t)m8 + 8) w[(ca - m8) >> 1] |= v0 << (16 * ((ca - m8) & 1));
-          if (cb >= (uint32_t)m8 && cb < (uint32_t)m8 + 8) w[(cb - m8) >> 1] |= v1 << (16 * ((cb - m8) & 1));
-          if (M >= 8) {
-            *reinterpret_cast<uint4*>(drow + m8) = make_uint4(w[0], w[1], w[2], w[3]);
-          } else {                                              // M == 4: 8-byte group
-            *reinterpret_cast<uint2*>(drow) = make_uint2(w[0], w[1]);
-          }
-        }
-      }
+      const uint32_t r0 = p0 == 0 ? rl[0] : p0 == 1 ? rl[1] : rl[2];
+      const uint32_t r1 = p1 == 1 ? rl[1] : p1 == 2 ? rl[2] : rl[3];
+      if (relu_vals && apply) *reinterpret_cast<uint32_t*>(relu_vals + t * (2 * G) + 2 * (g0 + g)) = r0 | (r1 << 16);
+      const uint32_t ca = (c4 >> (8 * p0)) & 0xFFu, cb = (c4 >> (8 * p1)) & 0xFFu;
+      if (dense_out) write_group_dense(dense_out + t * F + c0 + g * M, M, ca, cb, v0, v1);
+      if (relu_dense_out) write_group_dense(relu_dense_out + t * F + c0 + g * M, M, ca, cb, r0, r1);
     }
     // four neighbouring groups of a row -> one metadata word (ng is a multiple of 4)
     uint32_t word = valid ? nib : 0u;
@@ -149,7 +157,7 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
 
 int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
                void* vals, void* meta, void* meta_hw, void* colidx, void* relu_vals, void* dense_out,
-               cudaStream_t s) {
+               void* relu_dense_out, cudaStream_t s) {
   if (T == 0 || F == 0) return SF_OK;
   const size_t smem = (size_t)V * (kCW + kPad) * 2 + kCW * 4 + kCW + kCW;
   static bool attr_set[64] = {false};                         // per device
@@ -163,7 +171,7 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
   dim3 grid((unsigned)((F + kCW - 1) / kCW), (unsigned)(T / V));
   vnm_kernel<<<grid, kThreads, smem, s>>>((const uint16_t*)P, T, F, ld, V, M, apply_sqrelu, (uint16_t*)vals,
                                           (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
-                                          (uint16_t*)relu_vals, (uint16_t*)dense_out);
+                                          (uint16_t*)relu_vals, (uint16_t*)dense_out, (uint16_t*)relu_dense_out);
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
