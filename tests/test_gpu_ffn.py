@@ -1,0 +1,132 @@
+"""Parity of the sparse and dense FFN step (CUDA, through the C ABI) with the oracle.
+
+Protocol: stage-wise, teacher-forced. The oracle re-runs the selection on the GPU's own bf16
+pre-activations (a one-ulp difference in y1 may legitimately flip a near-tie), so masks, metadata
+and packed values must be bit-identical; products are compared in relative Frobenius norm against
+float64-accumulated references evaluated with those masks. The free-running oracle is compared too.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_06183_b200 import binding, synth
+from util import to_dev, bits, f32, rel_fro
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+def _run_sparse(cfg, prune_mode=0, act_shift=0.0):
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"], act_shift=act_shift)
+    desc = binding.make_desc(T, D, F, V, M, prune_mode=prune_mode, flags=1)
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
+    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+    gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
+    binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    binding.sf_sparse_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    G = F // M
+    out = dict(
+        y1=bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y1)).reshape(T, F),
+        y2_vals=bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y2_VALS)).reshape(T, 2 * G),
+        relu_vals=bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_RELU_VALS)).reshape(T, 2 * G),
+        meta=bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_META)).reshape(T, G // 4),
+        colidx=binding.sf_ctx_view(desc, ctx, binding.SF_CTX_COLIDX).cpu().numpy().reshape(T // V, G, 4),
+        dy1_vals=bits(binding.sf_ctx_view(desc, ws, binding.SF_CTX_DY1_VALS)).reshape(T, 2 * G),
+        Y=f32(Y), dX=f32(gX), dW1=f32(gW1), dW2=f32(gW2))
+    return (X, W1, W2, dY), out
+
+
+@pytest.mark.parametrize("prune_mode,act_shift", [(0, 0.0), (1, 0.0), (0, -1.3)])
+def test_sparse_ffn_c1_teacher_forced(prune_mode, act_shift):
+    cfg = synth.FFN_CONFIGS["c1_small"]
+    (X, W1, W2, dY), g = _run_sparse(cfg, prune_mode, act_shift)
+    V, M = cfg["V"], cfg["M"]
+    # stage 1: the GPU's y1 against the oracle's own product with the pruned W1
+    free = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, prune_mode=prune_mode)
+    assert rel_fro(oracle.bf16_to_f32(g["y1"]), oracle.bf16_to_f32(free.y1b)) < TOL
+    # stage 2: selection on the GPU's y1 must agree bit for bit
+    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, prune_mode=prune_mode, forced_y1b=g["y1"])
+    assert np.array_equal(g["colidx"], fwd.act.colidx)
+    assert np.array_equal(g["meta"], fwd.act.meta)
+    assert np.array_equal(g["y2_vals"], fwd.act.vals)
+    assert np.array_equal(g["relu_vals"], fwd.act.relu_vals)
+    # stage 3: products with those masks
+    assert rel_fro(g["Y"], fwd.y3) < TOL
+    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd, prune_mode=prune_mode)
+    assert rel_fro(oracle.bf16_to_f32(g["dy1_vals"]), oracle.bf16_to_f32(bwd.dy1_vals)) < TOL
+    assert rel_fro(g["dX"], bwd.dX) < TOL
+    assert rel_fro(g["dW1"], bwd.dW1) < TOL
+    assert rel_fro(g["dW2"], bwd.dW2) < TOL
+    # free-running comparison: masks may differ in a few near-tie blocks only
+    disagree = float((free.act.colidx != g["colidx"]).any(axis=-1).mean())
+    assert disagree < 0.05
+    assert rel_fro(g["Y"], free.y3) < 5e-2
+
+
+def test_sparse_ffn_v128_m16():
+    cfg = dict(T=512, D=256, F=2048, V=128, N=2, M=16, sigma_w=0.05, seed=17)
+    (X, W1, W2, dY), g = _run_sparse(cfg)
+    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=128, M=16, forced_y1b=g["y1"])
+    assert np.array_equal(g["colidx"], fwd.act.colidx) and np.array_equal(g["meta"], fwd.act.meta)
+    assert np.array_equal(g["y2_vals"], fwd.act.vals)
+    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd)
+    for k, ref in (("Y", fwd.y3), ("dX", bwd.dX), ("dW1", bwd.dW1), ("dW2", bwd.dW2)):
+        assert rel_fro(g[k], ref) < TOL, k
+
+
+def test_dense_ffn_c1():
+    cfg = synth.FFN_CONFIGS["c1_small"]
+    T, D, F = cfg["T"], cfg["D"], cfg["F"]
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
+    desc = binding.make_desc(T, D, F, cfg["V"], cfg["M"])
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
+    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+    gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
+    binding.sf_dense_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
+    binding.sf_dense_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    y1 = bits(ctx[: T * F * 2].view(torch.bfloat16)).reshape(T, F)
+    free = oracle.dense_ffn_fwd(X, W1, W2)
+    assert rel_fro(oracle.bf16_to_f32(y1), oracle.bf16_to_f32(free.y1b)) < TOL
+    fwd = oracle.dense_ffn_fwd(X, W1, W2, forced_y1b=y1)
+    bwd = oracle.dense_ffn_bwd(dY, X, W1, W2, fwd)
+    assert rel_fro(f32(Y), fwd.y3) < TOL
+    assert rel_fro(f32(gX), bwd.dX) < TOL
+    assert rel_fro(f32(gW1), bwd.dW1) < TOL
+    assert rel_fro(f32(gW2), bwd.dW2) < TOL
+
+
+def test_step_from_host_buffers_matches_device_path():
+    cfg = synth.FFN_CONFIGS["c1_small"]
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
+    desc = binding.make_desc(T, D, F, V, M)
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    staging = torch.empty((binding.sf_ffn_host_staging_size(desc),), dtype=torch.uint8, device="cuda")
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
+    hX, hW1, hW2, hdY = pin(X), pin(W1), pin(W2), pin(dY)
+    hY, hdX = torch.empty_like(hX), torch.empty_like(hX)
+    hdW1, hdW2 = torch.empty_like(hW1), torch.empty_like(hW2)
+    binding.sf_ffn_step_host(desc, False, hX, hW1, hW2, hdY, hY, hdX, hdW1, hdW2, staging, ctx, ws)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    (_, _, _, _), g = _run_sparse(cfg)
+    as_f32 = lambda t: t.view(torch.bfloat16).float().numpy()
+    assert np.array_equal(as_f32(hY), g["Y"]) and np.array_equal(as_f32(hdX), g["dX"])
+    assert np.array_equal(as_f32(hdW1), g["dW1"]) and np.array_equal(as_f32(hdW2), g["dW2"])
+
+
+def test_ffn_rejects_ragged_shapes():
+    desc = binding.make_desc(1000, 256, 1024, 64, 8)
+    with pytest.raises(binding.SparseFFNError) as e:
+        binding.sf_ffn_workspace_size(desc)
+    assert e.value.status == binding.SF_ERR_SHAPE
+    desc = binding.make_desc(1024, 256, 1024, 64, 8, N=1)
+    with pytest.raises(binding.SparseFFNError) as e:
+        binding.sf_ffn_workspace_size(desc)
+    assert e.value.status == binding.SF_ERR_UNSUPPORTED
