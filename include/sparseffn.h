@@ -184,6 +184,17 @@ SF_API int sf_ffn_step_host(const sf_ffn_desc* desc, int dense, const void* host
                      void* host_dW1, void* host_dW2, void* device_staging, void* fwd_ctx,
                      void* workspace, void* stream);
 
+/* Stage tracing, a measurement aid (the paper has no counterpart). `events` is a caller-owned HOST
+ * array of `capacity` cudaEvent_t handles (created with timing enabled) that must stay valid until
+ * tracing is switched off with capacity 0. While set, every FFN step call records one event
+ * before its first kernel and one after each kernel, in launch order, on the call's stream:
+ *   sparse fwd: 6 events (prune W1 | y1 product | V:N:M | W2 transpose | y3 product)
+ *   sparse bwd: 7 events (prune W2 | dy1 product | pack | dX product | dW2 product | dW1 product)
+ *   dense fwd: 3 events, dense bwd: 5 events.
+ * sf_trace_count returns how many events have been recorded since sf_trace_set. Not thread-safe. */
+SF_API int sf_trace_set(void** events, int capacity);
+SF_API int sf_trace_count(void);
+
 /* Synchronises `stream` and reads the device status word kept at the start of `workspace`:
  * SF_OK, or SF_ERR_TIMEOUT if a bounded wait inside a tensor-core kernel expired. */
 SF_API int sf_check_status(void* workspace, void* stream);

@@ -57,6 +57,8 @@ _SIGNATURES = {
     "sf_ctx_view": (_i32, [C.POINTER(sf_ffn_desc), _vp, _i32, C.POINTER(_vp), C.POINTER(_sz)]),
     "sf_ffn_host_staging_size": (_i32, [C.POINTER(sf_ffn_desc), C.POINTER(_sz)]),
     "sf_ffn_step_host": (_i32, [C.POINTER(sf_ffn_desc), _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_trace_set": (_i32, [C.POINTER(_vp), _i32]),
+    "sf_trace_count": (_i32, []),
     "sf_check_status": (_i32, [_vp, _vp]),
 }
 
@@ -277,3 +279,31 @@ def sf_ffn_step_host(desc, dense: bool, hX, hW1, hW2, hdY, hY, hdX, hdW1, hdW2, 
 
 def sf_check_status(workspace, stream=None) -> int:
     return lib().sf_check_status(_ptr(workspace), _stream(stream))
+
+
+class StageTrace:
+    """Records CUDA events between the kernels of the FFN step calls made inside the `with` block.
+
+    After the block, ``durations_ms()`` returns the time between consecutive events (the caller
+    knows the stage order of the calls it made; see sf_trace_set in the header)."""
+
+    def __init__(self, capacity: int):
+        self.events = [torch.cuda.Event(enable_timing=True) for _ in range(capacity)]
+        for e in self.events:          # torch creates the CUDA event lazily on first record
+            e.record()
+        torch.cuda.synchronize()
+        self._arr = (C.c_void_p * capacity)(*[C.c_void_p(e.cuda_event) for e in self.events])
+        self.count = 0
+
+    def __enter__(self):
+        _check(lib().sf_trace_set(self._arr, len(self.events)), "sf_trace_set")
+        return self
+
+    def __exit__(self, *exc):
+        self.count = lib().sf_trace_count()
+        lib().sf_trace_set(None, 0)
+        return False
+
+    def durations_ms(self):
+        torch.cuda.synchronize()
+        return [self.events[i].elapsed_time(self.events[i + 1]) for i in range(self.count - 1)]

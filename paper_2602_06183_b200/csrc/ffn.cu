@@ -15,6 +15,14 @@ constexpr size_t kStatusBytes = 256;       // status word lives at the start of 
 
 inline size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
+// Optional stage tracing: caller-owned CUDA events recorded between the kernels of a step.
+cudaEvent_t* g_trace_events = nullptr;
+int g_trace_cap = 0, g_trace_n = 0;
+
+inline void trace_mark(cudaStream_t s) {
+  if (g_trace_events && g_trace_n < g_trace_cap) cudaEventRecord(g_trace_events[g_trace_n++], s);
+}
+
 // ---- small helper kernels -------------------------------------------------------------------
 
 __global__ void meta_reorder_kernel(const uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw, int64_t R,
@@ -229,18 +237,24 @@ int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, co
   void* y1 = (d.flags & 1) ? (void*)at(fwd_ctx, L.y1) : (void*)at(workspace, L.ws_y1);
 
   // Algorithm 1 line 4: W1s = sparsify24(W1) along d_model, then y1 = X W1s^T
+  trace_mark(s);
   SF_TRY(launch_prune24(W1, d.F, d.D, d.D, 1, d.prune_mode, at(workspace, L.w1_vals), at(workspace, L.w1_meta),
                         at(workspace, L.w1_meta_hw), nullptr, s));
+  trace_mark(s);
   SF_TRY(gemm_sparse24(at(workspace, L.w1_vals), at(workspace, L.w1_meta_hw), X, d.F, d.T, d.D, EPI_STORE_T, y1,
                        d.F, nullptr, 0, status, s));
+  trace_mark(s);
   // lines 5-6: y2 = ReLU(y1)^2 in V:N:M form (+ what the backward pass needs)
   SF_TRY(launch_vnm(y1, d.T, d.F, d.F, d.V, d.M, 1, at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta),
                     at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), at(fwd_ctx, L.relu_vals),
                     at(fwd_ctx, L.y2_dense), at(fwd_ctx, L.relu_dense), s));
+  trace_mark(s);
   // line 7: y3 = y2 W2^T with W2 dense; rows of W2^T are gathered by the kept columns
   SF_TRY(launch_transpose(W2, at(fwd_ctx, L.w2t), d.D, d.F, s));
+  trace_mark(s);
   SF_TRY(gemm_venom(at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), at(fwd_ctx, L.w2t), d.T,
                     d.F, d.D, d.V, d.M, Y, d.D, status, s));
+  trace_mark(s);
   return SF_OK;
 }
 
@@ -256,20 +270,27 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
 
   // Algorithm 2 line 2: W2s = sparsify24(W2^T) along d_model (contiguous in the saved W2^T copy),
   // dy2 = dY W2s;  line 4: dy1 = 2 dy2 ReLU(y1) on y2's mask (fused into the product's epilogue)
+  trace_mark(s);
   SF_TRY(launch_prune24(at(fwd_ctx, L.w2t), d.F, d.D, d.D, 1, d.prune_mode, at(workspace, L.w2_vals),
                         at(workspace, L.w2_meta), at(workspace, L.w2_meta_hw), nullptr, s));
+  trace_mark(s);
   SF_TRY(gemm_sparse24(at(workspace, L.w2_vals), at(workspace, L.w2_meta_hw), dY, d.F, d.T, d.D, EPI_DRELU_T,
                        at(workspace, L.dy1_dense), d.F, at(fwd_ctx, L.relu_dense), d.F, status, s));
+  trace_mark(s);
   SF_TRY(launch_pack_like(at(workspace, L.dy1_dense), at(fwd_ctx, L.meta), at(fwd_ctx, L.colidx),
                           at(workspace, L.dy1_vals), d.T, d.F, d.V, d.M, s));
+  trace_mark(s);
   // line 5: dX = dy1 W1 with W1 dense (rows gathered by the kept columns)
   SF_TRY(gemm_venom(at(workspace, L.dy1_vals), at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), W1, d.T, d.F, d.D, d.V,
                     d.M, dX, d.D, status, s));
+  trace_mark(s);
   // line 3: dW2 = dY^T y2 [D, F];  line 6: dW1 = dy1^T X [F, D]  (reduction over tokens)
   SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.y2_dense), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0,
                     nullptr, 0, status, s));
+  trace_mark(s);
   SF_TRY(gemm_dense(at(workspace, L.dy1_dense), false, X, false, d.F, d.D, d.T, EPI_STORE, dW1, d.D, nullptr, 0,
                     nullptr, 0, status, s));
+  trace_mark(s);
   return SF_OK;
 }
 
@@ -283,10 +304,13 @@ int sf_dense_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, con
   cudaStream_t s = (cudaStream_t)stream;
   int* status = (int*)workspace;
   // Eq. 1-2: y1 = X W1^T, h = ReLU(y1)^2 (fused);  Eq. 3: Y = h W2^T
+  trace_mark(s);
   SF_TRY(gemm_dense(X, true, W1, true, d.T, d.F, d.D, EPI_SQRELU, at(fwd_ctx, L.y1), d.F, at(fwd_ctx, L.h), d.F,
                     nullptr, 0, status, s));
+  trace_mark(s);
   SF_TRY(gemm_dense(at(fwd_ctx, L.h), true, W2, true, d.T, d.D, d.F, EPI_STORE, Y, d.D, nullptr, 0, nullptr, 0,
                     status, s));
+  trace_mark(s);
   return SF_OK;
 }
 
@@ -301,14 +325,19 @@ int sf_dense_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, con
   int* status = (int*)workspace;
   void* dy1 = at(workspace, L.dy1);
   // Eq. 4 + 6: dy1 = 2 (dY W2) ReLU(y1)
+  trace_mark(s);
   SF_TRY(gemm_dense(dY, true, W2, false, d.T, d.F, d.D, EPI_DRELU, dy1, d.F, nullptr, 0, at(fwd_ctx, L.y1), d.F,
                     status, s));
+  trace_mark(s);
   // Eq. 7: dX = dy1 W1
   SF_TRY(gemm_dense(dy1, true, W1, false, d.T, d.D, d.F, EPI_STORE, dX, d.D, nullptr, 0, nullptr, 0, status, s));
+  trace_mark(s);
   // Eq. 5: dW2 = dY^T h [D, F];  Eq. 8: dW1 = dy1^T X [F, D]
   SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.h), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0, nullptr, 0,
                     status, s));
+  trace_mark(s);
   SF_TRY(gemm_dense(dy1, false, X, false, d.F, d.D, d.T, EPI_STORE, dW1, d.D, nullptr, 0, nullptr, 0, status, s));
+  trace_mark(s);
   return SF_OK;
 }
 
@@ -376,6 +405,16 @@ int sf_ffn_step_host(const sf_ffn_desc* desc, int dense, const void* host_X, con
   SF_CUDA_TRY(cudaMemcpyAsync(host_dW2, ddW2, F * D * 2, cudaMemcpyDeviceToHost, s));
   return SF_OK;
 }
+
+int sf_trace_set(void** events, int capacity) {
+  if (capacity < 0 || (capacity > 0 && !events)) return SF_ERR_NULL;
+  g_trace_events = capacity > 0 ? reinterpret_cast<cudaEvent_t*>(events) : nullptr;
+  g_trace_cap = capacity;
+  g_trace_n = 0;
+  return SF_OK;
+}
+
+int sf_trace_count(void) { return g_trace_n; }
 
 int sf_check_status(void* workspace, void* stream) {
   if (!workspace) return SF_ERR_NULL;
