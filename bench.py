@@ -182,7 +182,7 @@ def run_ours(args, cfg):
             ms = float(t.item())
         return ms
 
-    for _ in range(max(W, 3)):
+    for _ in range(W if args.quick else max(W, 3)):
         sparse_step()
     if binding.sf_check_status(ws) != binding.SF_OK:
         raise SystemExit("device status: a bounded wait expired during warm-up")
@@ -193,6 +193,11 @@ def run_ours(args, cfg):
     flop_step = 12.0 * T * D * F
     value = world * flop_step * K / (ms / 1e3) / 1e12
 
+    if args.quick:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+                              "ms_per_step": ms / K, "config": {"workload": args.workload}, "quick": True}))
+        return
     for _ in range(2):
         dense_step()
     ms_dense = timed(dense_step, K)
@@ -299,6 +304,8 @@ def main():
     ap.add_argument("--workload", default="c4_d4096")
     ap.add_argument("--prune-mode", type=int, default=0)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="sparse step only (no dense step, trace, e2e, CPU baseline): for profiler captures")
     args = ap.parse_args()
     from paper_2602_06183_b200 import synth
     cfg = synth.FFN_CONFIGS[args.workload]

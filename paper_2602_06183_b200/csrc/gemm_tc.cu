@@ -8,14 +8,19 @@
 //
 // CTA = 6 warps: warp 0 TMA producer, warp 1 MMA issuer (+ TMEM owner), warps 2-5 epilogue (each
 // owns the 32 TMEM lanes of its quadrant). Tile 128 x 256, persistent over tiles (m fastest).
-// A stage holds A (<= 16 KB), B (32 KB) and, for sparse modes, one 2 KB metadata atom covering
-// 128 rows x 128 logical K (copied smem -> TMEM by tcgen05.cp every second stage).
+// Venom mode adds warps 6-17, which gather the kept rows of B into the 128B-swizzled MN-major
+// layout the MMA reads: 8 warps issue TMA row gathers, 4 warps issue 16-byte cp.async copies.
+// A stage holds A (16 KB dense, 8 KB compressed), B (32 KB) and, for sparse modes, one 2 KB metadata
+// atom covering 128 rows x 128 logical K (copied smem -> TMEM by tcgen05.cp every second stage);
+// 4 stages dense, 5 stages sparse.
 // Dense mode double-buffers the 256-column accumulator so the epilogue of tile i overlaps the main
 // loop of tile i+1; sparse modes keep one accumulator plus the metadata columns.
 // Every mbarrier wait is bounded; on expiry the CTA raises a flag in the status word and leaves.
 #include "sf_common.cuh"
 #include "tc_ptx.cuh"
 #include "gemm_tc.cuh"
+
+#include <cstdlib>
 
 namespace sf {
 
@@ -24,19 +29,27 @@ namespace {
 using namespace ptx;
 
 constexpr int BM = 128, BN = 256;
-constexpr int kStages = 4;
-constexpr int kAStageBytes = 16384, kBStageBytes = 32768, kMetaStageBytes = 2048;
-constexpr int kStageBytes = kAStageBytes + kBStageBytes + kMetaStageBytes;          // 51200 (1024-aligned)
+constexpr int kMaxStages = 5;
+constexpr int kBStageBytes = 32768, kMetaStageBytes = 2048;
+// dense: A 16 KB + B 32 KB, 4 stages; sparse modes: A 8 KB (stored half) + B 32 KB + metadata 2 KB, 5 stages
+__host__ __device__ constexpr int a_stage_bytes(bool sparse) { return sparse ? 8192 : 16384; }
+__host__ __device__ constexpr int stage_bytes(bool sparse) {
+  return a_stage_bytes(sparse) + kBStageBytes + (sparse ? kMetaStageBytes : 0);
+}
+__host__ __device__ constexpr int num_stages(bool sparse) { return sparse ? 5 : 4; }
 constexpr int kEpiStageRow = 80;                                                      // bytes: 32 bf16 + 16 pad
 constexpr int kEpiStageBytes = 4 * 32 * kEpiStageRow;                                 // 4 warps
-constexpr int kSmemBytes = 1024 /*align slack*/ + kStages * kStageBytes + kEpiStageBytes + 256 /*barriers*/;
-constexpr int kThreads = 192;
+__host__ __device__ constexpr int smem_bytes(bool sparse) {
+  return 1024 /*align slack*/ + num_stages(sparse) * stage_bytes(sparse) + kEpiStageBytes + 256 /*barriers*/;
+}
+constexpr int kThreads = 192;                 // dense / 2:4 modes: producer, MMA, 4 epilogue warps
+constexpr int kThreadsVenom = 576;            // + 8 TMA-gather warps and 4 cp.async-gather warps
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kMetaTmemCol = 256;
 
 struct SmemCtl {
-  uint64_t full[kStages];
-  uint64_t empty[kStages];
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint32_t tmem_base;
@@ -48,17 +61,20 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 
 template <int kMode, bool kAMN, bool kBMN, int kEpi>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kMode == MODE_VENOM ? kThreadsVenom : kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                const GemmArgs args) {
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  constexpr bool kSparse = kMode != MODE_DENSE;
+  constexpr int kStages = num_stages(kSparse);
+  constexpr int kAStageBytes = a_stage_bytes(kSparse);
+  constexpr int kStageBytes = stage_bytes(kSparse);
   uint8_t* epi_stage = smem + kStages * kStageBytes;
   SmemCtl* ctl = reinterpret_cast<SmemCtl*>(epi_stage + kEpiStageBytes);
   volatile int* abort_flag = &ctl->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr bool kSparse = kMode != MODE_DENSE;
   constexpr int kAccBufs = kSparse ? 1 : 2;
   constexpr int kMmaPerStage = kSparse ? 2 : 4;      // dense: K=16 x4 = 64; sparse: logical K=32 x2 = 64
 
@@ -72,7 +88,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     prefetch_tmap(&tmapA);
     prefetch_tmap(&tmapB);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&ctl->full[s], 1);
+      mbar_init(&ctl->full[s], kMode == MODE_VENOM ? 1 + 128 : 1);   // Venom: + every cp.async gather thread
       mbar_init(&ctl->empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -107,7 +123,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         uint64_t* bar = &ctl->full[stage];
         const bool load_meta = kSparse && ((kb & 1) == 0);
         if (lane == 0) {
-          uint32_t bytes = kBStageBytes + (kSparse ? 8192u : 16384u) + (load_meta ? (uint32_t)kMetaStageBytes : 0u);
+          const uint32_t b_tx = (kMode != MODE_VENOM) ? (uint32_t)kBStageBytes
+                                                      : (uint32_t)args.gather_tma_groups * 2048u;  // TMA-gathered part
+          uint32_t bytes = b_tx + (kSparse ? 8192u : 16384u) + (load_meta ? (uint32_t)kMetaStageBytes : 0u);
           mbar_arrive_expect_tx(bar, bytes);
           // ---- A
           if (kMode == MODE_DENSE) {
@@ -139,22 +157,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 #pragma unroll
               for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * 8192, &tmapB, bar, n0 + c * 64, kb * 64);
             }
-          }
-        }
-        if (kMode == MODE_VENOM) {
-          // gathered B: 16 groups x 4 rows per stage; lane = (group, half of the 4 column chunks)
-          __syncwarp();
-          const int grp = lane >> 1, half = lane & 1;
-          const int blk = (args.V == 64) ? (2 * mt + sweep) : mt;
-          const int64_t g = (int64_t)kb * 16 + grp;                             // group index in the row
-          const uint32_t c4 = *reinterpret_cast<const uint32_t*>(args.colidx + ((int64_t)blk * args.G + g) * 4);
-          const int base = (int)(g * args.Mv);
-          const int r0 = base + (c4 & 0xFF), r1 = base + ((c4 >> 8) & 0xFF), r2 = base + ((c4 >> 16) & 0xFF),
-                    r3 = base + (c4 >> 24);
-#pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            const int c = half * 2 + cc;
-            tma_gather4_2d(sB + c * 8192 + grp * 4 * 128, &tmapB, bar, n0 + c * 64, r0, r1, r2, r3);
           }
         }
         if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -213,6 +215,58 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         if (++acc == (uint32_t)kAccBufs) { acc = 0; acc_phase ^= 1; }
       }
     }
+  } else if (kMode == MODE_VENOM && warp >= 6) {
+    // =========================== B gather (warps 6..17, Venom only) ===========================
+    // Stage rows are the kept feature rows of Bt in condensed-k order: row r of the stage is
+    // feature g*Mv + colidx[blk][g][r & 3] with g = kb*16 + r/4. Two engines work side by side:
+    //   warps 6..13  TMA row gather (4 rows x 128 B per instruction) for the first `ntma` groups,
+    //   warps 14..17 16-byte cp.async (one warp-wide copy = 512 B of one row) for the others.
+    // Neither path alone keeps up with the tensor core; their in-flight limits are independent.
+    const int gw = warp - 6;
+    const int ntma = args.gather_tma_groups;
+    const uint16_t* Bt = reinterpret_cast<const uint16_t*>(args.aux);
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      const int64_t n0 = (int64_t)nt * BN;
+      for (int it = 0; it < iters; ++it) {
+        const int sweep = it / nkb, kb = it - sweep * nkb;
+        if (!mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+        const uint32_t sB = smem_u32(smem + stage * kStageBytes + kAStageBytes);
+        const int blk = (args.V == 64) ? (2 * mt + sweep) : mt;
+        const uint8_t* cbase = args.colidx + ((int64_t)blk * args.G + (int64_t)kb * 16) * 4;
+        if (gw < 8) {
+          const int grp = gw + 8 * (lane >> 2), c = lane & 3;             // lanes 0..7: two groups x 4 chunks
+          if (lane < 8 && grp < ntma) {
+            const uint32_t cg = *reinterpret_cast<const uint32_t*>(cbase + grp * 4);
+            const int base = (int)(((int64_t)kb * 16 + grp) * args.Mv);
+            tma_gather4_2d(sB + c * 8192 + grp * 4 * 128, &tmapB, &ctl->full[stage], (int)n0 + c * 64,
+                           base + (int)(cg & 0xFF), base + (int)((cg >> 8) & 0xFF), base + (int)((cg >> 16) & 0xFF),
+                           base + (int)(cg >> 24));
+          }
+        } else {
+          const int cw = gw - 8;                                          // 0..3
+          for (int grp = ntma + cw; grp < 16; grp += 4) {
+            const uint32_t cg = *reinterpret_cast<const uint32_t*>(cbase + grp * 4);
+            const int64_t fbase = ((int64_t)kb * 16 + grp) * args.Mv;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int row = grp * 4 + i;
+              const uint16_t* src = Bt + (fbase + ((cg >> (8 * i)) & 0xFFu)) * args.ldaux + n0 + lane * 8;
+              const uint32_t dst = sB + (lane >> 3) * 8192 + row * 128 + (((lane & 7) ^ (row & 7)) << 4);
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+            }
+          }
+          // The barrier's pending count is raised now and lowered when this thread's copies have
+          // landed; the plain arrive accounts for the thread itself. No blocking wait.
+          asm volatile("cp.async.mbarrier.arrive.shared::cta.b64 [%0];" ::"r"(smem_u32(&ctl->full[stage])) : "memory");
+          mbar_arrive(&ctl->full[stage]);
+        }
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
+    }
+    if (gw >= 8) asm volatile("cp.async.wait_all;" ::: "memory");
   } else {
     // =========================== epilogue (warps 2..5) ===========================
     const int q = warp & 3;                                                    // TMEM lane quadrant
@@ -393,12 +447,12 @@ int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& a, 
   int dev = 0;
   SF_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-    SF_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    SF_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(kMode != MODE_DENSE)));
     if (dev >= 0 && dev < 64) attr_done[dev] = true;
   }
   const int tiles = a.num_m_tiles * a.num_n_tiles;
   const int grid = tiles < sm_count() ? tiles : sm_count();
-  kern<<<grid, kThreads, kSmemBytes, s>>>(ta, tb, a);
+  kern<<<grid, kMode == MODE_VENOM ? kThreadsVenom : kThreads, smem_bytes(kMode != MODE_DENSE), s>>>(ta, tb, a);
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
@@ -468,7 +522,14 @@ int gemm_venom(const void* a_vals, const uint8_t* meta_hw, const uint8_t* colidx
   st = make_tmap(&tb, Bt, F, N, N, 64, 1, CU_TENSOR_MAP_SWIZZLE_128B);        // row gather: one row per box
   if (st != SF_OK) return st;
   GemmArgs a{};
+  {
+    const char* e = getenv("SF_GATHER_TMA_GROUPS");
+    a.gather_tma_groups = e ? atoi(e) : 12;
+    if (a.gather_tma_groups < 0) a.gather_tma_groups = 0;
+    if (a.gather_tma_groups > 16) a.gather_tma_groups = 16;
+  }
   a.M = T; a.N = N; a.K = Kc;
+  a.aux = Bt; a.ldaux = N;
   a.C = C; a.ldc = ldc; a.meta_hw = meta_hw; a.colidx = colidx; a.V = V; a.Mv = Mv; a.G = F / Mv;
   a.status = status;
   a.num_m_tiles = (int)(T / BM); a.num_n_tiles = (int)(N / BN); a.num_k_blocks = (int)(Kc / 64);

@@ -30,6 +30,7 @@ struct GemmArgs {
   int V, Mv;                // Venom block height and group width
   int* status;              // device status word (set to 1 when a bounded wait expires)
   int num_m_tiles, num_n_tiles, num_k_blocks;
+  int gather_tma_groups;    // Venom: groups (of 16 per stage) fetched by TMA row gather; the rest by cp.async
 };
 
 // D[M,N] = op(A) op(B)^T, tiles 128 x 256, K % 64 == 0.

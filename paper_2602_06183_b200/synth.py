@@ -30,6 +30,9 @@ __all__ = [
 FFN_CONFIGS = {
     "c1_small": dict(T=1024, D=256, F=1024, V=64, N=2, M=8, sigma_w=0.02, seed=0),
     "c4_d4096": dict(T=8192, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
+    # one eighth of c4's tokens with the full-size layer: weights (134 MB each) still exceed the
+    # L2, device footprint ~1.5 GB; used for profiler captures that must stay small
+    "c4_slice": dict(T=1024, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
     "c5_d8192": dict(T=16384, D=8192, F=28672, V=128, N=2, M=8, sigma_w=0.015, seed=5),
 }
 
