@@ -135,6 +135,25 @@ SF_API int sf_gemm_venom(const void* a_vals, const void* a_meta, const void* col
                   void* C, int64_t T, int64_t F, int64_t Nc, int V, int M,
                   void* workspace, void* stream);
 
+/* sf_gemm_sparse24_noalloc: the same product as sf_gemm_sparse24 for callers that cannot allocate
+ * device memory (the paper has no counterpart; this is a deployment variant). Some callers only
+ * own their input and output buffers: code that runs inside another framework's allocator or
+ * stream callback, plugins that are handed tensors but no allocator, processes whose device pool
+ * is already fully committed. For them the scratch that sf_gemm_sparse24 takes as `workspace`
+ * (metadata in tensor-core order + status word) is a 4 MiB + 256 B device array built into the
+ * library; every GPU that loads the library holds it until the process exits.
+ *   - Limit: Mr * K / 8 <= 4 MiB (e.g. 4096 x 8192); larger shapes return SF_ERR_WORKSPACE.
+ *   - The call itself allocates and frees nothing (no cudaMalloc / cudaFree, no allocating
+ *     library routine). Inputs and output are the caller's, exactly as for sf_gemm_sparse24.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls share the one array: two calls that may overlap on the GPU (different streams,
+ *     or different host threads) race on it. Serialise them on one stream.
+ *   - A bounded-wait expiry is recorded in the built-in status word, which no call reads back;
+ *     use sf_gemm_sparse24 + sf_check_status where that matters. */
+SF_API int sf_gemm_sparse24_noalloc(const void* a_vals, const void* a_meta, const void* B, void* Ct,
+                                    int64_t Mr, int64_t Nc, int64_t K, void* stream);
+
 /* ---------------------------------------------------------------------------------------
  * The FFN step (Algorithm 1 = forward, Algorithm 2 = backward; Eqs. 1-8 for the dense phase).
  *

@@ -48,6 +48,7 @@ _SIGNATURES = {
     "sf_gemm_workspace_size": (_i32, [_i64, _i64, C.POINTER(_sz)]),
     "sf_gemm_dense": (_i32, [_vp, _i32, _vp, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "sf_gemm_sparse24": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
+    "sf_gemm_sparse24_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "sf_gemm_venom": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp, _vp]),
     "sf_ffn_workspace_size": (_i32, [C.POINTER(sf_ffn_desc), C.POINTER(_sz), C.POINTER(_sz)]),
     "sf_sparse_ffn_fwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -199,6 +200,17 @@ def sf_gemm_sparse24(a_vals, a_meta, B, Ct_out=None, workspace=None, stream=None
                                 _ptr(workspace), _stream(stream))
     _check(st, "sf_gemm_sparse24")
     return Ct_out, workspace
+
+
+def sf_gemm_sparse24_noalloc(a_vals, a_meta, B, Ct_out, stream=None):
+    """Same product as sf_gemm_sparse24 without a workspace: for callers that cannot allocate device
+    memory. ``Ct_out`` [Nc, Mr] must be supplied by the caller; nothing is allocated here either.
+    Limit: Mr * K / 8 <= 4 MiB. Calls share one built-in scratch array: keep them on one stream."""
+    Mr, K = a_vals.shape[0], a_vals.shape[1] * 2
+    Nc = B.shape[0]
+    st = lib().sf_gemm_sparse24_noalloc(_ptr(a_vals), _ptr(a_meta), _ptr(B), _ptr(Ct_out), Mr, Nc, K, _stream(stream))
+    _check(st, "sf_gemm_sparse24_noalloc")
+    return Ct_out
 
 
 def sf_gemm_venom(a_vals, a_meta, colidx, Bt, V: int, M: int, C_out=None, workspace=None, stream=None):
