@@ -276,12 +276,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
       const int64_t m0 = (int64_t)mt * BM, n0 = (int64_t)nt * BN;
+      // The dy1 epilogue multiplies by a [token, feature] tile of the saved activations; its loads do
+      // not depend on the accumulator, so they are issued before the wait and land during the main loop.
+      uint4 ax[kEpi == EPI_DRELU_T ? BN / 32 : 1][4];
+      if (kEpi == EPI_DRELU_T) {
+#pragma unroll
+        for (int ch = 0; ch < BN / 32; ++ch)
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            ax[ch][i] = __ldg(reinterpret_cast<const uint4*>(
+                reinterpret_cast<const uint16_t*>(args.aux) + (n0 + ch * 32 + i * 8 + (lane >> 2)) * args.ldaux + m0 +
+                q * 32 + (lane & 3) * 8));
+      }
       if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
       const int64_t row = m0 + q * 32 + lane;                                  // this thread's D row
-#pragma unroll 1
-      for (int ch = 0; ch < BN / 32; ++ch) {
+      auto chunk = [&](int ch, const uint4 (&a4)[4]) {
         uint32_t v[32];
         tmem_ld_32x32b_x32(taddr + ch * 32, v);
         tmem_ld_wait();
@@ -339,12 +350,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             // aux[token, feature] chunk -> staging -> one column per lane
             __syncwarp();
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int t = i * 8 + (lane >> 2), seg = lane & 3;
-              const uint4 a = __ldg(reinterpret_cast<const uint4*>(
-                  reinterpret_cast<const uint16_t*>(args.aux) + (col0 + t) * args.ldaux + m0 + q * 32 + seg * 8));
-              *reinterpret_cast<uint4*>(my_stage + t * kEpiStageRow + seg * 16) = a;
-            }
+            for (int i = 0; i < 4; ++i)
+              *reinterpret_cast<uint4*>(my_stage + (i * 8 + (lane >> 2)) * kEpiStageRow + (lane & 3) * 16) = a4[i];
             __syncwarp();
 #pragma unroll
             for (int j = 0; j < 32; ++j)
@@ -371,6 +378,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.C) + (col0 + t) * args.ldc + m0 + q * 32 + seg * 8) = o;
           }
         }
+            };
+      if (kEpi == EPI_DRELU_T) {
+#pragma unroll
+        for (int ch = 0; ch < BN / 32; ++ch) chunk(ch, ax[ch]);
+      } else {
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) chunk(ch, ax[0]);
       }
       tc_fence_before();
       __syncwarp();

@@ -38,6 +38,23 @@ __device__ __forceinline__ uint32_t prune_group(uint32_t a0, uint32_t a1, uint32
   return nib;
 }
 
+// Packed variant for the row kernel: lo/hi hold the group's four patterns; returns the nibble and
+// the two kept (hard) or shrunk (soft) values packed into one word.
+template <bool kSoft>
+__device__ __forceinline__ uint32_t prune_group_packed(uint32_t lo, uint32_t hi, uint32_t& packed) {
+  uint32_t third;
+  const uint32_t nib = top2of4_packed(lo, hi, &packed, kSoft ? &third : nullptr);
+  if (kSoft) {
+    const uint32_t tw = (third & 2u) ? hi : lo;
+    const float t = bf16_bits_to_float(((third & 1u) ? (tw >> 16) : tw) & 0x7FFFu);
+    const float f0 = bf16_bits_to_float(packed & 0xFFFFu), f1 = bf16_bits_to_float(packed >> 16);
+    const float s0 = f0 > 0.f ? __fsub_rn(f0, t) : (f0 < 0.f ? __fadd_rn(f0, t) : 0.f);
+    const float s1 = f1 > 0.f ? __fsub_rn(f1, t) : (f1 < 0.f ? __fadd_rn(f1, t) : 0.f);
+    packed = float_to_bf16_bits(s0) | (float_to_bf16_bits(s1) << 16);
+  }
+  return nib;
+}
+
 // Expand (nibble, two values) to the four dense patterns of a group.
 __device__ __forceinline__ void expand_group(uint32_t nib, uint32_t v0, uint32_t v1, uint32_t d[4]) {
   const uint32_t p0 = nib & 3u, p1 = nib >> 2;
@@ -62,14 +79,11 @@ prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int64_t cols, int
   uint32_t packed[4], m = 0, dense[8];
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
-    const uint32_t lo = w[2 * g], hi = w[2 * g + 1];
-    uint32_t o0, o1;
-    const uint32_t nib = prune_group<kSoft>(lo & 0xFFFFu, lo >> 16, hi & 0xFFFFu, hi >> 16, o0, o1);
-    packed[g] = o0 | (o1 << 16);
+    const uint32_t nib = prune_group_packed<kSoft>(w[2 * g], w[2 * g + 1], packed[g]);
     m |= nib << (4 * g);
     if (dense_out) {
       uint32_t d[4];
-      expand_group(nib, o0, o1, d);
+      expand_group(nib, packed[g] & 0xFFFFu, packed[g] >> 16, d);
       dense[2 * g] = d[0] | (d[1] << 16);
       dense[2 * g + 1] = d[2] | (d[3] << 16);
     }

@@ -60,6 +60,32 @@ __device__ __forceinline__ uint32_t top2of4(uint32_t k0, uint32_t k1, uint32_t k
   return pos0 | (pos1 << 2);
 }
 
+// Same selection on a packed group (lo = elements 0,1; hi = elements 2,3; bf16 patterns), built for
+// few instructions: each 15-bit magnitude is widened to magnitude*4 + (3 - index), which makes all
+// four keys distinct and orders ties towards the lower index; a five-comparator network then
+// yields the first, second and third key, whose low two bits name their positions.
+// Returns the nibble; *packed = kept values (pos0 low half, pos1 high half); *third_idx = index of
+// the third-ranked element.
+__device__ __forceinline__ uint32_t top2of4_packed(uint32_t lo, uint32_t hi, uint32_t* packed,
+                                                   uint32_t* third_idx = nullptr) {
+  const uint32_t c0 = ((lo << 2) & 0x1FFFCu) | 3u, c1 = ((lo >> 14) & 0x1FFFCu) | 2u;
+  const uint32_t c2 = ((hi << 2) & 0x1FFFCu) | 1u, c3 = ((hi >> 14) & 0x1FFFCu);
+  const uint32_t h01 = max(c0, c1), l01 = min(c0, c1), h23 = max(c2, c3), l23 = min(c2, c3);
+  const uint32_t top1 = max(h01, h23), mid = min(h01, h23);
+  const bool first_pair_wins = h01 > h23;
+  const uint32_t under = first_pair_wins ? l01 : l23;        // partner of the winner
+  const uint32_t top2 = max(mid, under);
+  const uint32_t ia = 3u - (top1 & 3u), ib = 3u - (top2 & 3u);
+  const uint32_t p0 = min(ia, ib), p1 = max(ia, ib);
+  // byte permute: bytes (2p0, 2p0+1) then (2p1, 2p1+1) out of the 8 bytes {lo, hi}
+  *packed = __byte_perm(lo, hi, 0x1010u + p0 * 0x22u + p1 * 0x2200u);
+  if (third_idx) {
+    const uint32_t other_low = first_pair_wins ? l23 : l01;
+    *third_idx = 3u - (max(min(mid, under), other_low) & 3u);
+  }
+  return p0 | (p1 << 2);
+}
+
 // ---- internal launchers (defined in the .cu files) ---------------------------------------
 // meta_hw (optional) receives the same metadata words in the order the sparse tensor-core
 // instruction reads them (see gemm_sparse.cu); requires R % 128 == 0 and K % 128 == 0.

@@ -153,6 +153,161 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
   }
 }
 
+
+// ---- M = 8 fast path ---------------------------------------------------------------------------
+// Same computation as vnm_kernel for groups of eight columns, written for a low instruction count:
+// packed bf16x2 arithmetic (max with zero, then one correctly rounded bf16 multiply, which equals
+// rounding the exact float32 square), whole 16-byte groups from shared memory, byte permutes with
+// selectors that depend only on the block's kept columns (constant per thread: a thread always
+// serves the same group of the strip), and mask words for the dense copies.
+__device__ __forceinline__ uint32_t relu2(uint32_t w) {
+  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&w);
+  __nv_bfloat162 z = __hmax2(x, __float2bfloat162_rn(0.f));
+  return *reinterpret_cast<uint32_t*>(&z);
+}
+__device__ __forceinline__ uint32_t sq2(uint32_t r) {
+  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&r);
+  __nv_bfloat162 z = __hmul2(x, x);
+  return *reinterpret_cast<uint32_t*>(&z);
+}
+
+__global__ void __launch_bounds__(kThreads)
+vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int V, int apply,
+            uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
+            uint8_t* __restrict__ colidx, uint16_t* __restrict__ relu_vals, uint16_t* __restrict__ dense_out,
+            uint16_t* __restrict__ relu_dense_out) {
+  constexpr int M = 8;
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  uint16_t* tile = reinterpret_cast<uint16_t*>(smem_raw);                        // [V][kCW + kPad]
+  uint32_t* score = reinterpret_cast<uint32_t*>(tile + (size_t)V * (kCW + kPad));
+  uint8_t* keepf = reinterpret_cast<uint8_t*>(score + kCW);
+  uint8_t* cidx = keepf + kCW;
+  constexpr int kRow = kCW + kPad;
+
+  const int tid = threadIdx.x;
+  const int64_t c0 = (int64_t)blockIdx.x * kCW;
+  const int64_t blk = blockIdx.y;
+  const int64_t t0 = blk * V;
+  const int cvalid = (int)min((int64_t)kCW, F - c0);
+  const int64_t G = F / M;
+
+  for (int i = tid; i < V * (kCW / 8); i += kThreads) {
+    const int r = i / (kCW / 8), cc = (i % (kCW / 8)) * 8;
+    if (cc < cvalid) {
+      const uint4 q = __ldg(reinterpret_cast<const uint4*>(P + (t0 + r) * ld + c0 + cc));
+      *reinterpret_cast<uint4*>(tile + r * kRow + cc) = q;
+    }
+  }
+  __syncthreads();
+
+  // pass A: two columns per thread, rows first to last, one float32 add per element
+  if (tid < kCW / 2) {
+    float s0 = 0.f, s1 = 0.f;
+    if (2 * tid < cvalid) {
+      const uint32_t* col = reinterpret_cast<const uint32_t*>(tile) + tid;
+      for (int r = 0; r < V; ++r) {
+        const uint32_t w = col[r * (kRow / 2)];
+        const uint32_t h = apply ? sq2(relu2(w)) : (w & 0x7FFF7FFFu);
+        s0 = __fadd_rn(s0, __uint_as_float(h << 16));
+        s1 = __fadd_rn(s1, __uint_as_float(h & 0xFFFF0000u));
+      }
+    }
+    score[2 * tid] = __float_as_uint(s0);
+    score[2 * tid + 1] = __float_as_uint(s1);
+  }
+  __syncthreads();
+  {
+    const int j = tid, jm = j & 7, base = j - jm;
+    const uint32_t s = score[j];
+    int rank = 0;
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+      const uint32_t si = score[base + i];
+      rank += (si > s) || (si == s && i < jm);
+    }
+    keepf[j] = rank < 4;
+  }
+  __syncthreads();
+  {
+    const int j = tid, jm = j & 7, base = j - jm;
+    if (keepf[j] && j < cvalid) {
+      int pos = 0;
+      for (int i = 0; i < jm; ++i) pos += keepf[base + i];
+      cidx[(j >> 3) * 4 + pos] = (uint8_t)jm;
+    }
+  }
+  __syncthreads();
+  const int ng = cvalid / M;                                  // multiple of 4; kThreads % ng == 0
+  if (tid < ng) {
+    const uint32_t c4 = *reinterpret_cast<const uint32_t*>(cidx + tid * 4);
+    *reinterpret_cast<uint32_t*>(colidx + (blk * G + c0 / M + tid) * 4) = c4;
+  }
+
+  // pass B: a thread serves one group g = tid % ng for rows tid / ng, tid / ng + kThreads / ng, ...
+  const int g = tid % ng, rstep = kThreads / ng;
+  const int64_t g0 = c0 / M;
+  const uint32_t c4 = *reinterpret_cast<const uint32_t*>(cidx + g * 4);
+  // per-thread constants: permute selectors / half masks that pick the kept columns out of a group
+  uint32_t selp[2], mhi[2];
+#pragma unroll
+  for (int pr = 0; pr < 2; ++pr) {
+    const uint32_t ca = (c4 >> (16 * pr)) & 0xFFu, cb = (c4 >> (16 * pr + 8)) & 0xFFu;
+    const uint32_t sa = 2u * (ca & 3u), sb = 2u * (cb & 3u);
+    selp[pr] = sa | ((sa + 1u) << 4) | (sb << 8) | ((sb + 1u) << 12);
+    mhi[pr] = ((ca & 4u) ? 0x0000FFFFu : 0u) | ((cb & 4u) ? 0xFFFF0000u : 0u);   // take from columns 4..7
+  }
+  const bool lead = (g & 3) == 0;
+  for (int r = tid / ng; r < V; r += rstep) {
+    const uint4 q = *reinterpret_cast<const uint4*>(tile + r * kRow + g * M);
+    uint32_t rw[4] = {q.x, q.y, q.z, q.w}, hw[4];
+    if (apply) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { rw[j] = relu2(rw[j]); hw[j] = sq2(rw[j]); }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) hw[j] = rw[j];
+    }
+    // kept columns c0 < c1 | c2 < c3 as two packed pairs
+    uint32_t hk[2], rk[2];
+#pragma unroll
+    for (int pr = 0; pr < 2; ++pr) {
+      const uint32_t a = __byte_perm(hw[0], hw[1], selp[pr]), b = __byte_perm(hw[2], hw[3], selp[pr]);
+      hk[pr] = (a & ~mhi[pr]) | (b & mhi[pr]);
+      const uint32_t ra = __byte_perm(rw[0], rw[1], selp[pr]), rb = __byte_perm(rw[2], rw[3], selp[pr]);
+      rk[pr] = (ra & ~mhi[pr]) | (rb & mhi[pr]);
+    }
+    uint32_t packed;
+    const uint32_t nib = top2of4_packed(hk[0], hk[1], &packed);
+    const uint32_t p0 = nib & 3u, p1 = nib >> 2;
+    const int64_t t = t0 + r;
+    *reinterpret_cast<uint32_t*>(vals + t * (2 * G) + 2 * (g0 + g)) = packed;
+    if (relu_vals && apply)
+      *reinterpret_cast<uint32_t*>(relu_vals + t * (2 * G) + 2 * (g0 + g)) =
+          __byte_perm(rk[0], rk[1], 0x1010u + p0 * 0x22u + p1 * 0x2200u);
+    if (dense_out || relu_dense_out) {
+      const uint32_t kb = (1u << ((c4 >> (8 * p0)) & 0xFFu)) | (1u << ((c4 >> (8 * p1)) & 0xFFu));
+      uint32_t mk[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        mk[j] = (((kb >> (2 * j)) & 1u) * 0xFFFFu) | (((kb >> (2 * j + 1)) & 1u) * 0xFFFF0000u);
+      if (dense_out)
+        *reinterpret_cast<uint4*>(dense_out + t * F + c0 + g * M) =
+            make_uint4(hw[0] & mk[0], hw[1] & mk[1], hw[2] & mk[2], hw[3] & mk[3]);
+      if (relu_dense_out)
+        *reinterpret_cast<uint4*>(relu_dense_out + t * F + c0 + g * M) =
+            make_uint4(rw[0] & mk[0], rw[1] & mk[1], rw[2] & mk[2], rw[3] & mk[3]);
+    }
+    uint32_t word = nib;
+    word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 4;
+    word |= __shfl_down_sync(0xFFFFFFFFu, word, 2) << 8;
+    if (lead) {
+      const int64_t kw = (g0 + g) >> 2;
+      meta[t * (G >> 2) + kw] = (uint16_t)word;
+      if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(t, kw, 4 * G)) = (uint16_t)word;
+    }
+  }
+}
+
 }  // namespace
 
 int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
@@ -169,6 +324,22 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   dim3 grid((unsigned)((F + kCW - 1) / kCW), (unsigned)(T / V));
+  // fast path: groups of eight, strips whose group count divides the thread count, full warps per row step
+  const int tail = (int)(F % kCW);
+  const bool fast8 = (M == 8) && (tail == 0 || tail == 64 || tail == 128) && (V % 32 == 0);
+  if (fast8) {
+    static bool attr8[64] = {false};
+    if (dev < 0 || dev >= 64 || !attr8[dev]) {
+      SF_CUDA_TRY(cudaFuncSetAttribute(vnm8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       128 * (kCW + kPad) * 2 + kCW * 6));
+      if (dev >= 0 && dev < 64) attr8[dev] = true;
+    }
+    vnm8_kernel<<<grid, kThreads, smem, s>>>((const uint16_t*)P, T, F, ld, V, apply_sqrelu, (uint16_t*)vals,
+                                             (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
+                                             (uint16_t*)relu_vals, (uint16_t*)dense_out, (uint16_t*)relu_dense_out);
+    SF_LAUNCH_CHECK();
+    return SF_OK;
+  }
   vnm_kernel<<<grid, kThreads, smem, s>>>((const uint16_t*)P, T, F, ld, V, M, apply_sqrelu, (uint16_t*)vals,
                                           (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
                                           (uint16_t*)relu_vals, (uint16_t*)dense_out, (uint16_t*)relu_dense_out);

@@ -91,3 +91,20 @@ def test_empty_inputs_are_noops():
     w = torch.empty((0, 256), dtype=torch.bfloat16, device="cuda")
     vals, meta, _ = binding.sf_prune24_compress(w, 1, 0)
     assert vals.numel() == 0 and meta.numel() == 0
+
+
+def test_vnm_special_values_bit_exact():
+    """-0, subnormal squares, overflow to inf, exact ties at zero: packed arithmetic must match."""
+    rng = np.random.default_rng(3)
+    base = np.array([-0.0, 0.0, 1e-20, 3e-20, 1e-19, 1.5e19, 3e19, 1e-30, 0.5, -0.5, 2.0, 1e-10], dtype=np.float32)
+    x = base[rng.integers(0, base.size, size=(128, 512))]
+    p = synth.f32_to_bf16_bits(x)
+    for V in (64, 128):
+        ref = oracle.vnm_sparsify(p, V=V, M=8)
+        vals, meta, colidx, relu, dense = binding.sf_vnm_sparsify_act(to_dev(p), V, 8, want_dense=True)
+        torch.cuda.synchronize()
+        assert np.array_equal(colidx.cpu().numpy(), ref.colidx)
+        assert np.array_equal(bits(meta), ref.meta)
+        assert np.array_equal(bits(vals), ref.vals)
+        assert np.array_equal(bits(relu), ref.relu_vals)
+        assert np.array_equal(bits(dense), ref.dense)
