@@ -60,6 +60,127 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return float_to_bf16_bits(lo) | (float_to_bf16_bits(hi) << 16);
 }
 
+
+// ---- epilogue (shared by the one-CTA and the two-CTA kernels) ---------------------------------------
+// One epilogue warp owns TMEM lanes [32q, 32q+32) of a 128 x 256 accumulator tile whose first row is
+// m0 and first column n0; `taddr` is the TMEM address of (lane 32q, column 0) of that accumulator.
+constexpr int kAuxChunks = BN / 32;
+
+template <int kEpi>
+__device__ __forceinline__ void epi_prefetch(const GemmArgs& args, int64_t m0, int64_t n0, int q, int lane,
+                                             uint4 (&ax)[kEpi == EPI_DRELU_T ? kAuxChunks : 1][4]) {
+  if (kEpi == EPI_DRELU_T) {
+#pragma unroll
+    for (int ch = 0; ch < kAuxChunks; ++ch)
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        ax[kEpi == EPI_DRELU_T ? ch : 0][i] = __ldg(reinterpret_cast<const uint4*>(
+            reinterpret_cast<const uint16_t*>(args.aux) + (n0 + ch * 32 + i * 8 + (lane >> 2)) * args.ldaux + m0 +
+            q * 32 + (lane & 3) * 8));
+  }
+}
+
+template <int kEpi>
+__device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0, int q, int lane,
+                                         uint8_t* my_stage,
+                                         const uint4 (&ax)[kEpi == EPI_DRELU_T ? kAuxChunks : 1][4]) {
+  const int64_t row = m0 + q * 32 + lane;                                  // this thread's D row
+  auto chunk = [&](int ch, const uint4 (&a4)[4]) {
+    uint32_t v[32];
+    tmem_ld_32x32b_x32(taddr + ch * 32, v);
+    tmem_ld_wait();
+    const int64_t col0 = n0 + ch * 32;
+    if (kEpi == EPI_STORE || kEpi == EPI_SQRELU || kEpi == EPI_DRELU) {
+      uint16_t* crow = reinterpret_cast<uint16_t*>(args.C) + row * args.ldc + col0;
+      if (kEpi == EPI_STORE) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint4 o;
+          o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
+          o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
+          o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
+          o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+          reinterpret_cast<uint4*>(crow)[j] = o;
+        }
+      } else if (kEpi == EPI_SQRELU) {
+        uint16_t* hrow = reinterpret_cast<uint16_t*>(args.C2) + row * args.ldc2 + col0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint32_t y[4], h[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const uint32_t y0 = float_to_bf16_bits(__uint_as_float(v[8 * j + 2 * e]));
+            const uint32_t y1 = float_to_bf16_bits(__uint_as_float(v[8 * j + 2 * e + 1]));
+            const float f0 = fmaxf(bf16_bits_to_float(y0), 0.f), f1 = fmaxf(bf16_bits_to_float(y1), 0.f);
+            y[e] = y0 | (y1 << 16);
+            h[e] = pack_bf16x2(__fmul_rn(f0, f0), __fmul_rn(f1, f1));
+          }
+          reinterpret_cast<uint4*>(crow)[j] = make_uint4(y[0], y[1], y[2], y[3]);
+          reinterpret_cast<uint4*>(hrow)[j] = make_uint4(h[0], h[1], h[2], h[3]);
+        }
+      } else {  // EPI_DRELU: C = bf16(2 * acc * relu(aux))
+        const uint16_t* arow = reinterpret_cast<const uint16_t*>(args.aux) + row * args.ldaux + col0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint4 a = __ldg(reinterpret_cast<const uint4*>(arow) + j);
+          const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
+          uint32_t o[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float r0 = fmaxf(bf16_bits_to_float(aw[e] & 0xFFFFu), 0.f);
+            const float r1 = fmaxf(bf16_bits_to_float(aw[e] >> 16), 0.f);
+            const float d0 = __fmul_rn(__fmul_rn(2.f, __uint_as_float(v[8 * j + 2 * e])), r0);
+            const float d1 = __fmul_rn(__fmul_rn(2.f, __uint_as_float(v[8 * j + 2 * e + 1])), r1);
+            o[e] = pack_bf16x2(d0, d1);
+          }
+          reinterpret_cast<uint4*>(crow)[j] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+      }
+    } else {
+      // Transposed output: D row = feature (lane), D column = token. C is [N, M] row-major.
+      float r[32];
+      if (kEpi == EPI_DRELU_T) {
+        // aux[token, feature] chunk -> staging -> one column per lane
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          *reinterpret_cast<uint4*>(my_stage + (i * 8 + (lane >> 2)) * kEpiStageRow + (lane & 3) * 16) = a4[i];
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          r[j] = bf16_bits_to_float(*reinterpret_cast<const uint16_t*>(my_stage + j * kEpiStageRow + lane * 2));
+      }
+      __syncwarp();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        float x = __uint_as_float(v[j]);
+        uint32_t b;
+        if (kEpi == EPI_DRELU_T) {
+          // aux holds ReLU(y1) on the activation mask and +0 elsewhere: off-mask entries become +0
+          b = (r[j] == 0.f) ? 0u : float_to_bf16_bits(__fmul_rn(__fmul_rn(2.f, x), r[j]));
+        } else {
+          b = float_to_bf16_bits(x);
+        }
+        *reinterpret_cast<uint16_t*>(my_stage + j * kEpiStageRow + lane * 2) = (uint16_t)b;
+      }
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int t = i * 8 + (lane >> 2), seg = lane & 3;
+        const uint4 o = *reinterpret_cast<const uint4*>(my_stage + t * kEpiStageRow + seg * 16);
+        *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.C) + (col0 + t) * args.ldc + m0 + q * 32 + seg * 8) = o;
+      }
+    }
+        };
+  if (kEpi == EPI_DRELU_T) {
+#pragma unroll
+    for (int ch = 0; ch < BN / 32; ++ch) chunk(ch, ax[kEpi == EPI_DRELU_T ? ch : 0]);
+  } else {
+#pragma unroll 1
+    for (int ch = 0; ch < BN / 32; ++ch) chunk(ch, ax[0]);
+  }
+}
+
 template <int kMode, bool kAMN, bool kBMN, int kEpi>
 __global__ void __launch_bounds__(kMode == MODE_VENOM ? kThreadsVenom : kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
@@ -279,113 +400,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
       // The dy1 epilogue multiplies by a [token, feature] tile of the saved activations; its loads do
       // not depend on the accumulator, so they are issued before the wait and land during the main loop.
       uint4 ax[kEpi == EPI_DRELU_T ? BN / 32 : 1][4];
-      if (kEpi == EPI_DRELU_T) {
-#pragma unroll
-        for (int ch = 0; ch < BN / 32; ++ch)
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            ax[ch][i] = __ldg(reinterpret_cast<const uint4*>(
-                reinterpret_cast<const uint16_t*>(args.aux) + (n0 + ch * 32 + i * 8 + (lane >> 2)) * args.ldaux + m0 +
-                q * 32 + (lane & 3) * 8));
-      }
+      epi_prefetch<kEpi>(args, m0, n0, q, lane, ax);
       if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
-      const int64_t row = m0 + q * 32 + lane;                                  // this thread's D row
-      auto chunk = [&](int ch, const uint4 (&a4)[4]) {
-        uint32_t v[32];
-        tmem_ld_32x32b_x32(taddr + ch * 32, v);
-        tmem_ld_wait();
-        const int64_t col0 = n0 + ch * 32;
-        if (kEpi == EPI_STORE || kEpi == EPI_SQRELU || kEpi == EPI_DRELU) {
-          uint16_t* crow = reinterpret_cast<uint16_t*>(args.C) + row * args.ldc + col0;
-          if (kEpi == EPI_STORE) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint4 o;
-              o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
-              o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
-              o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
-              o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
-              reinterpret_cast<uint4*>(crow)[j] = o;
-            }
-          } else if (kEpi == EPI_SQRELU) {
-            uint16_t* hrow = reinterpret_cast<uint16_t*>(args.C2) + row * args.ldc2 + col0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint32_t y[4], h[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const uint32_t y0 = float_to_bf16_bits(__uint_as_float(v[8 * j + 2 * e]));
-                const uint32_t y1 = float_to_bf16_bits(__uint_as_float(v[8 * j + 2 * e + 1]));
-                const float f0 = fmaxf(bf16_bits_to_float(y0), 0.f), f1 = fmaxf(bf16_bits_to_float(y1), 0.f);
-                y[e] = y0 | (y1 << 16);
-                h[e] = pack_bf16x2(__fmul_rn(f0, f0), __fmul_rn(f1, f1));
-              }
-              reinterpret_cast<uint4*>(crow)[j] = make_uint4(y[0], y[1], y[2], y[3]);
-              reinterpret_cast<uint4*>(hrow)[j] = make_uint4(h[0], h[1], h[2], h[3]);
-            }
-          } else {  // EPI_DRELU: C = bf16(2 * acc * relu(aux))
-            const uint16_t* arow = reinterpret_cast<const uint16_t*>(args.aux) + row * args.ldaux + col0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const uint4 a = __ldg(reinterpret_cast<const uint4*>(arow) + j);
-              const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
-              uint32_t o[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float r0 = fmaxf(bf16_bits_to_float(aw[e] & 0xFFFFu), 0.f);
-                const float r1 = fmaxf(bf16_bits_to_float(aw[e] >> 16), 0.f);
-                const float d0 = __fmul_rn(__fmul_rn(2.f, __uint_as_float(v[8 * j + 2 * e])), r0);
-                const float d1 = __fmul_rn(__fmul_rn(2.f, __uint_as_float(v[8 * j + 2 * e + 1])), r1);
-                o[e] = pack_bf16x2(d0, d1);
-              }
-              reinterpret_cast<uint4*>(crow)[j] = make_uint4(o[0], o[1], o[2], o[3]);
-            }
-          }
-        } else {
-          // Transposed output: D row = feature (lane), D column = token. C is [N, M] row-major.
-          float r[32];
-          if (kEpi == EPI_DRELU_T) {
-            // aux[token, feature] chunk -> staging -> one column per lane
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              *reinterpret_cast<uint4*>(my_stage + (i * 8 + (lane >> 2)) * kEpiStageRow + (lane & 3) * 16) = a4[i];
-            __syncwarp();
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              r[j] = bf16_bits_to_float(*reinterpret_cast<const uint16_t*>(my_stage + j * kEpiStageRow + lane * 2));
-          }
-          __syncwarp();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            float x = __uint_as_float(v[j]);
-            uint32_t b;
-            if (kEpi == EPI_DRELU_T) {
-              // aux holds ReLU(y1) on the activation mask and +0 elsewhere: off-mask entries become +0
-              b = (r[j] == 0.f) ? 0u : float_to_bf16_bits(__fmul_rn(__fmul_rn(2.f, x), r[j]));
-            } else {
-              b = float_to_bf16_bits(x);
-            }
-            *reinterpret_cast<uint16_t*>(my_stage + j * kEpiStageRow + lane * 2) = (uint16_t)b;
-          }
-          __syncwarp();
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int t = i * 8 + (lane >> 2), seg = lane & 3;
-            const uint4 o = *reinterpret_cast<const uint4*>(my_stage + t * kEpiStageRow + seg * 16);
-            *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.C) + (col0 + t) * args.ldc + m0 + q * 32 + seg * 8) = o;
-          }
-        }
-            };
-      if (kEpi == EPI_DRELU_T) {
-#pragma unroll
-        for (int ch = 0; ch < BN / 32; ++ch) chunk(ch, ax[ch]);
-      } else {
-#pragma unroll 1
-        for (int ch = 0; ch < BN / 32; ++ch) chunk(ch, ax[0]);
-      }
+      epi_tile<kEpi>(args, taddr, m0, n0, q, lane, my_stage, ax);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&ctl->tmem_empty[acc]);
@@ -401,6 +420,203 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---- two-CTA kernel (cta_group::2) -----------------------------------------------------------------
+// A cluster of two CTAs computes one 256 x 256 tile: CTA r holds rows [128r, 128r+128) of A and of
+// the accumulator, and columns [128r, 128r+128) of B; the leader (rank 0) issues MMAs that read both
+// CTAs' shared memory. Each CTA therefore fetches half as much B per unit of tensor work as the
+// one-CTA kernel, which is what bounds the 2:4 and dense products. No TMA multicast is used: each
+// CTA loads its own halves, with completion bytes routed to the leader's barrier.
+constexpr int kThreads2 = 192;
+__host__ __device__ constexpr int stage_bytes2(bool sparse) { return sparse ? (8192 + 16384 + 2048) : (16384 + 16384); }
+__host__ __device__ constexpr int num_stages2(bool sparse) { return sparse ? 8 : 6; }
+__host__ __device__ constexpr int smem_bytes2(bool sparse) {
+  return 1024 + num_stages2(sparse) * stage_bytes2(sparse) + kEpiStageBytes + 512;
+}
+
+struct SmemCtl2 {
+  uint64_t full[8];
+  uint64_t empty[8];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int kMode, bool kAMN, bool kBMN, int kEpi>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+                const __grid_constant__ CUtensorMap tmapMeta, const GemmArgs args) {
+  extern __shared__ uint8_t smem_dyn[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  constexpr bool kSparse = kMode == MODE_SPARSE24;
+  constexpr int kStages = num_stages2(kSparse);
+  constexpr int kAStageBytes = kSparse ? 8192 : 16384;
+  constexpr int kBHalfBytes = 16384;
+  constexpr int kStageBytes = stage_bytes2(kSparse);
+  constexpr int kAccBufs = kSparse ? 1 : 2;
+  constexpr int kMmaPerStage = kSparse ? 2 : 4;
+  uint8_t* epi_stage = smem + kStages * kStageBytes;
+  SmemCtl2* ctl = reinterpret_cast<SmemCtl2*>(epi_stage + kEpiStageBytes);
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();               // 0 = leader
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const int num_m_tiles = args.num_m_tiles;              // 256-row tiles
+  const int num_tiles = num_m_tiles * args.num_n_tiles;
+  const int nkb = args.num_k_blocks;
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&tmapA);
+    prefetch_tmap(&tmapB);
+    if (kSparse) prefetch_tmap(&tmapMeta);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&ctl->full[s], 1);
+      mbar_init(&ctl->empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&ctl->tmem_full[b], 1);
+      mbar_init(&ctl->tmem_empty[b], 8);                 // 4 epilogue warps in each CTA of the pair
+    }
+    ctl->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_2cta(&ctl->tmem_base, kTmemCols);
+    tmem_relinquish_2cta();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                    // both CTAs' barriers and TMEM are ready
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+
+  if (warp == 0) {
+    // =========================== TMA producer (both CTAs) ===========================
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      const int m0 = mt * 256 + (int)rank * 128;         // this CTA's rows of A / D
+      const int nb0 = nt * BN + (int)rank * 128;         // this CTA's columns of B
+      for (int kb = 0; kb < nkb; ++kb) {
+        if (!mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+        if (lane == 0) {
+          uint8_t* sA = smem + stage * kStageBytes;
+          uint8_t* sB = sA + kAStageBytes;
+          uint8_t* sM = sB + kBHalfBytes;
+          uint64_t* bar = &ctl->full[stage];
+          const bool load_meta = kSparse && ((kb & 1) == 0);
+          if (rank == 0) {
+            // the leader's barrier collects the bytes of both CTAs
+            mbar_arrive_expect_tx(bar, 2u * ((uint32_t)kAStageBytes + (uint32_t)kBHalfBytes +
+                                             (load_meta ? (uint32_t)kMetaStageBytes : 0u)));
+          }
+          if (kMode == MODE_DENSE) {
+            if (!kAMN) {
+              tma_load_2d_2cta(sA, &tmapA, bar, kb * 64, m0);
+            } else {
+              tma_load_2d_2cta(sA, &tmapA, bar, m0, kb * 64);
+              tma_load_2d_2cta(sA + 8192, &tmapA, bar, m0 + 64, kb * 64);
+            }
+          } else {
+            tma_load_2d_2cta(sA, &tmapA, bar, kb * 32, m0);
+          }
+          if (load_meta) {
+            // metadata atoms are rows of 2 x 1 KB in a [2 * atoms, 256] uint32 view
+            const int atom = (m0 >> 7) * (nkb >> 1) + (kb >> 1);
+            tma_load_2d_2cta(sM, &tmapMeta, bar, 0, 2 * atom);
+          }
+          if (!kBMN) {
+            tma_load_2d_2cta(sB, &tmapB, bar, kb * 64, nb0);                   // box {64 k, 128 n}
+          } else {
+            tma_load_2d_2cta(sB, &tmapB, bar, nb0, kb * 64);                   // box {64 n, 64 k}
+            tma_load_2d_2cta(sB + 8192, &tmapB, bar, nb0 + 64, kb * 64);
+          }
+        }
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    // =========================== MMA issuer (leader CTA only) ===========================
+    if (rank == 0 && lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16(256, BN, kAMN, kBMN, kSparse);
+      uint32_t stage = 0, phase = 0;
+      uint32_t acc = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        if (!mbar_wait(&ctl->tmem_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + acc * BN;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!mbar_wait(&ctl->full[stage], phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sA = smem_u32(smem + stage * kStageBytes);
+          const uint32_t sB = sA + kAStageBytes;
+          const uint32_t sM = sB + kBHalfBytes;
+          if (kSparse && (kb & 1) == 0)
+            tmem_cp_128x128b_2cta(tmem_base + kMetaTmemCol, smem_desc(sM, 128, 128, kSwizzleNone));
+#pragma unroll
+          for (int k = 0; k < kMmaPerStage; ++k) {
+            uint64_t adesc, bdesc;
+            if (kMode == MODE_DENSE) {
+              adesc = kAMN ? smem_desc(sA + k * 2048, 8192, 1024, kSwizzle128B)
+                           : smem_desc(sA + k * 32, 16, 1024, kSwizzle128B);
+            } else {
+              adesc = smem_desc(sA + k * 32, 16, 512, 4 /* 64 B swizzle */);
+            }
+            if (kBMN) bdesc = smem_desc(sB + k * (kSparse ? 4096 : 2048), 8192, 1024, kSwizzle128B);
+            else      bdesc = smem_desc(sB + k * (kSparse ? 64 : 32), 16, 1024, kSwizzle128B);
+            const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
+            if (kSparse) {
+              const uint32_t col = (uint32_t)((kb & 1) * 2 + k);
+              mma_sp_f16_2cta(tmem_d, adesc, bdesc, tmem_base + kMetaTmemCol + (col & ~1u), idesc | (col & 1u), accum);
+            } else {
+              mma_f16_2cta(tmem_d, adesc, bdesc, idesc, accum);
+            }
+          }
+          mma_commit_2cta(&ctl->empty[stage]);             // frees the stage in both CTAs
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        mma_commit_2cta(&ctl->tmem_full[acc]);             // accumulator ready, both CTAs
+        if (++acc == (uint32_t)kAccBufs) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else {
+    // =========================== epilogue (warps 2..5, both CTAs) ===========================
+    const int q = warp & 3;
+    uint8_t* my_stage = epi_stage + q * 32 * kEpiStageRow;
+    uint32_t acc = 0, acc_phase = 0;
+    bool ok = true;
+    for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      const int64_t m0 = (int64_t)mt * 256 + (int64_t)rank * 128, n0 = (int64_t)nt * BN;
+      uint4 ax[kEpi == EPI_DRELU_T ? kAuxChunks : 1][4];
+      epi_prefetch<kEpi>(args, m0, n0, q, lane, ax);
+      if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
+      epi_tile<kEpi>(args, taddr, m0, n0, q, lane, my_stage, ax);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(&ctl->tmem_empty[acc]);
+      if (++acc == (uint32_t)kAccBufs) { acc = 0; acc_phase ^= 1; }
+    }
+  }
+
+  // =========================== teardown ===========================
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && ctl->abort_flag) atomicExch(args.status, 1);
+  cluster_sync_all();                                    // the peer is done with our shared memory and barriers
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_2cta(tmem_base, kTmemCols);
   }
 }
 
@@ -423,16 +639,18 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// 2D bf16 tensor map over a row-major [rows, cols] matrix; box = {box_cols, box_rows}.
+// 2D tensor map over a row-major [rows, cols] matrix of 2-byte (bf16) or 4-byte (uint32) elements;
+// box = {box_cols, box_rows}.
 int make_tmap(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
-              uint32_t box_rows, CUtensorMapSwizzle swz) {
+              uint32_t box_rows, CUtensorMapSwizzle swz, bool u32 = false) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return cuda_fail(cudaErrorUnknown);
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * (u32 ? 4 : 2)};
   cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  CUresult r = fn(m, u32 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                  const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -471,6 +689,36 @@ int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& a, 
   return SF_OK;
 }
 
+template <int kMode, bool kAMN, bool kBMN, int kEpi>
+int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tm, GemmArgs a, cudaStream_t s) {
+  auto kern = gemm_tc2_kernel<kMode, kAMN, kBMN, kEpi>;
+  constexpr int smem = smem_bytes2(kMode != MODE_DENSE);
+  static bool attr_done[64] = {false};
+  int dev = 0;
+  SF_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+    SF_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    if (dev >= 0 && dev < 64) attr_done[dev] = true;
+  }
+  a.num_m_tiles = (int)(a.M / 256);
+  const int tiles = a.num_m_tiles * a.num_n_tiles;
+  const int max_pairs = sm_count() / 2;
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  kern<<<2 * pairs, kThreads2, smem, s>>>(ta, tb, tm, a);
+  SF_LAUNCH_CHECK();
+  return SF_OK;
+}
+
+// The two-CTA kernels need M % 256 == 0; SF_ONE_CTA=1 in the environment forces the one-CTA kernels.
+bool use_two_cta(int64_t M) {
+  static int forced = -1;
+  if (forced < 0) {
+    const char* e = getenv("SF_ONE_CTA");
+    forced = (e && atoi(e) != 0) ? 1 : 0;
+  }
+  return forced == 0 && (M % 256 == 0);
+}
+
 }  // namespace
 
 int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64_t M, int64_t N, int64_t K, int epi,
@@ -478,12 +726,13 @@ int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64
                cudaStream_t s) {
   if (M % BM || N % BN || K % 64) return SF_ERR_SHAPE;
   if (M == 0 || N == 0) return SF_OK;
+  const bool two = use_two_cta(M);
   CUtensorMap ta, tb;
   int st;
   if (a_kmajor) st = make_tmap(&ta, A, M, K, K, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
   else          st = make_tmap(&ta, A, K, M, M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
   if (st != SF_OK) return st;
-  if (b_kmajor) st = make_tmap(&tb, B, N, K, K, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (b_kmajor) st = make_tmap(&tb, B, N, K, K, 64, two ? 128 : 256, CU_TENSOR_MAP_SWIZZLE_128B);
   else          st = make_tmap(&tb, B, K, N, N, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
   if (st != SF_OK) return st;
   GemmArgs a{};
@@ -491,7 +740,9 @@ int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64
   a.C = C; a.ldc = ldc; a.C2 = C2; a.ldc2 = ldc2; a.aux = aux; a.ldaux = ldaux;
   a.status = status;
   a.num_m_tiles = (int)(M / BM); a.num_n_tiles = (int)(N / BN); a.num_k_blocks = (int)(K / 64);
-#define SF_DENSE_CASE(AMN, BMN, EPI) return launch_one<MODE_DENSE, AMN, BMN, EPI>(ta, tb, a, s)
+#define SF_DENSE_CASE(AMN, BMN, EPI)                                              \
+  return two ? launch_two<MODE_DENSE, AMN, BMN, EPI>(ta, tb, ta, a, s)            \
+             : launch_one<MODE_DENSE, AMN, BMN, EPI>(ta, tb, a, s)
   const bool amn = !a_kmajor, bmn = !b_kmajor;
   if (epi == EPI_STORE) {
     if (!amn && !bmn) SF_DENSE_CASE(false, false, EPI_STORE);
@@ -511,17 +762,29 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, int
                   int epi, void* Ct, int64_t ldc, const void* aux, int64_t ldaux, int* status, cudaStream_t s) {
   if (M % BM || N % BN || K % 128) return SF_ERR_SHAPE;
   if (M == 0 || N == 0) return SF_OK;
-  CUtensorMap ta, tb;
+  const bool two = use_two_cta(M);
+  CUtensorMap ta, tb, tm;
   int st = make_tmap(&ta, a_vals, M, K / 2, K / 2, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B);
   if (st != SF_OK) return st;
-  st = make_tmap(&tb, B, N, K, K, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
+  st = make_tmap(&tb, B, N, K, K, 64, two ? 128 : 256, CU_TENSOR_MAP_SWIZZLE_128B);
   if (st != SF_OK) return st;
+  tm = ta;
+  if (two) {
+    // hardware-ordered metadata: 2 KB atoms viewed as two rows of 256 uint32
+    const int64_t atoms = (M / 128) * (K / 128);
+    st = make_tmap(&tm, meta_hw, 2 * atoms, 256, 256, 256, 2, CU_TENSOR_MAP_SWIZZLE_NONE, true);
+    if (st != SF_OK) return st;
+  }
   GemmArgs a{};
   a.M = M; a.N = N; a.K = K;
   a.C = Ct; a.ldc = ldc; a.aux = aux; a.ldaux = ldaux; a.meta_hw = meta_hw; a.status = status;
   a.num_m_tiles = (int)(M / BM); a.num_n_tiles = (int)(N / BN); a.num_k_blocks = (int)(K / 64);
-  if (epi == EPI_STORE_T) return launch_one<MODE_SPARSE24, false, false, EPI_STORE_T>(ta, tb, a, s);
-  if (epi == EPI_DRELU_T) return launch_one<MODE_SPARSE24, false, false, EPI_DRELU_T>(ta, tb, a, s);
+  if (epi == EPI_STORE_T)
+    return two ? launch_two<MODE_SPARSE24, false, false, EPI_STORE_T>(ta, tb, tm, a, s)
+               : launch_one<MODE_SPARSE24, false, false, EPI_STORE_T>(ta, tb, a, s);
+  if (epi == EPI_DRELU_T)
+    return two ? launch_two<MODE_SPARSE24, false, false, EPI_DRELU_T>(ta, tb, tm, a, s)
+               : launch_one<MODE_SPARSE24, false, false, EPI_DRELU_T>(ta, tb, a, s);
   return SF_ERR_UNSUPPORTED;
 }
 

@@ -18,7 +18,7 @@ def _f64(b):
 
 
 @pytest.mark.parametrize("a_k,b_k", [(True, True), (True, False), (False, True), (False, False)])
-@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (384, 512, 448)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (384, 512, 448), (256, 256, 128), (512, 768, 1024)])
 def test_dense_gemm_layouts(a_k, b_k, M, N, K):
     A = synth.normal_bf16((M, K) if a_k else (K, M), 0, 1, seed=1, stream=M + K)
     B = synth.normal_bf16((N, K) if b_k else (K, N), 0, 1, seed=2, stream=N + K)
@@ -39,7 +39,7 @@ def test_dense_gemm_exact_small_integers():
     assert np.array_equal(f32(C), (_f64(A) @ _f64(B).T).astype(np.float32))
 
 
-@pytest.mark.parametrize("Mr,Nc,K", [(128, 256, 128), (256, 512, 640), (384, 256, 1024)])
+@pytest.mark.parametrize("Mr,Nc,K", [(128, 256, 128), (256, 512, 640), (384, 256, 1024), (1024, 768, 2048)])
 def test_sparse24_gemm_against_oracle_packing(Mr, Nc, K):
     W = synth.prune_sweep_matrix(Mr, K, seed=Mr + K, tie_frac=0.1)
     W = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(W) * 50.0)       # O(1) magnitudes
