@@ -303,7 +303,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
           const uint32_t sM = sB + kBStageBytes;
           if (kSparse && (kb & 1) == 0) {
             // 128 rows x 16 B, no swizzle: 8-row core matrices 128 B apart
-            tmem_cp_128x128b(tmem_base + kMetaTmemCol, smem_desc(sM, 128, 128, kSwizzleNone));
+            tmem_cp_128x128b(tmem_base + kMetaTmemCol + 4u * ((uint32_t)(kb >> 1) & 1u),
+                             smem_desc(sM, 128, 128, kSwizzleNone));
           }
 #pragma unroll
           for (int k = 0; k < kMmaPerStage; ++k) {
@@ -323,7 +324,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             const uint32_t accum = (it > 0 || k > 0) ? 1u : 0u;
             if (kSparse) {
               const uint32_t col = (uint32_t)((kb & 1) * 2 + k);              // metadata column of this k step
-              mma_sp_f16(tmem_d, adesc, bdesc, tmem_base + kMetaTmemCol + (col & ~1u), idesc | (col & 1u), accum);
+              const uint32_t mbuf = kMetaTmemCol + 4u * ((uint32_t)(kb >> 1) & 1u);   // metadata double buffer
+              mma_sp_f16(tmem_d, adesc, bdesc, tmem_base + mbuf + (col & ~1u), idesc | (col & 1u), accum);
             } else {
               mma_f16(tmem_d, adesc, bdesc, idesc, accum);
             }
@@ -427,11 +429,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 // A cluster of two CTAs computes one 256 x 256 tile: CTA r holds rows [128r, 128r+128) of A and of
 // the accumulator, and columns [128r, 128r+128) of B; the leader (rank 0) issues MMAs that read both
 // CTAs' shared memory. Each CTA therefore fetches half as much B per unit of tensor work as the
-// one-CTA kernel, which is what bounds the 2:4 and dense products. No TMA multicast is used: each
-// CTA loads its own halves, with completion bytes routed to the leader's barrier.
+// one-CTA kernel. No TMA multicast is used: each CTA loads its own halves, with completion bytes
+// routed to the leader's barrier.
+// Stage = 64 K (dense, 4 MMAs of K=16) or 128 logical K (2:4, 4 MMAs of K=32 and one metadata atom):
+// four MMAs per barrier round trip keep the single issuing thread ahead of the tensor pipe.
 constexpr int kThreads2 = 192;
-__host__ __device__ constexpr int stage_bytes2(bool sparse) { return sparse ? (8192 + 16384 + 2048) : (16384 + 16384); }
-__host__ __device__ constexpr int num_stages2(bool sparse) { return sparse ? 8 : 6; }
+__host__ __device__ constexpr int stage_bytes2(bool sparse) { return sparse ? (16384 + 32768 + 2048) : (16384 + 16384); }
+__host__ __device__ constexpr int num_stages2(bool sparse) { return sparse ? 4 : 6; }
 __host__ __device__ constexpr int smem_bytes2(bool sparse) {
   return 1024 + num_stages2(sparse) * stage_bytes2(sparse) + kEpiStageBytes + 512;
 }
@@ -445,6 +449,10 @@ struct SmemCtl2 {
   int abort_flag;
 };
 
+__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
+  return (static_cast<uint64_t>(hi) << 32) | lo;
+}
+
 template <int kMode, bool kAMN, bool kBMN, int kEpi>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
@@ -453,11 +461,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   constexpr bool kSparse = kMode == MODE_SPARSE24;
   constexpr int kStages = num_stages2(kSparse);
-  constexpr int kAStageBytes = kSparse ? 8192 : 16384;
-  constexpr int kBHalfBytes = 16384;
+  constexpr int kBK = kSparse ? 128 : 64;                // logical K per stage
+  constexpr int kAStageBytes = 16384;
+  constexpr int kBHalfBytes = kSparse ? 32768 : 16384;
   constexpr int kStageBytes = stage_bytes2(kSparse);
   constexpr int kAccBufs = kSparse ? 1 : 2;
-  constexpr int kMmaPerStage = kSparse ? 2 : 4;
   uint8_t* epi_stage = smem + kStages * kStageBytes;
   SmemCtl2* ctl = reinterpret_cast<SmemCtl2*>(epi_stage + kEpiStageBytes);
   volatile int* abort_flag = &ctl->abort_flag;
@@ -467,7 +475,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const int num_m_tiles = args.num_m_tiles;              // 256-row tiles
   const int num_tiles = num_m_tiles * args.num_n_tiles;
-  const int nkb = args.num_k_blocks;
+  const int nkb = (int)(args.K / kBK);
 
   if (threadIdx.x == 0) {
     prefetch_tmap(&tmapA);
@@ -509,11 +517,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
           uint8_t* sB = sA + kAStageBytes;
           uint8_t* sM = sB + kBHalfBytes;
           uint64_t* bar = &ctl->full[stage];
-          const bool load_meta = kSparse && ((kb & 1) == 0);
           if (rank == 0) {
             // the leader's barrier collects the bytes of both CTAs
             mbar_arrive_expect_tx(bar, 2u * ((uint32_t)kAStageBytes + (uint32_t)kBHalfBytes +
-                                             (load_meta ? (uint32_t)kMetaStageBytes : 0u)));
+                                             (kSparse ? (uint32_t)kMetaStageBytes : 0u)));
           }
           if (kMode == MODE_DENSE) {
             if (!kAMN) {
@@ -522,19 +529,19 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
               tma_load_2d_2cta(sA, &tmapA, bar, m0, kb * 64);
               tma_load_2d_2cta(sA + 8192, &tmapA, bar, m0 + 64, kb * 64);
             }
+            if (!kBMN) {
+              tma_load_2d_2cta(sB, &tmapB, bar, kb * 64, nb0);                 // box {64 k, 128 n}
+            } else {
+              tma_load_2d_2cta(sB, &tmapB, bar, nb0, kb * 64);                 // box {64 n, 64 k}
+              tma_load_2d_2cta(sB + 8192, &tmapB, bar, nb0 + 64, kb * 64);
+            }
           } else {
-            tma_load_2d_2cta(sA, &tmapA, bar, kb * 32, m0);
-          }
-          if (load_meta) {
+            tma_load_2d_2cta(sA, &tmapA, bar, kb * 64, m0);                    // stored values: box {64, 128}
             // metadata atoms are rows of 2 x 1 KB in a [2 * atoms, 256] uint32 view
-            const int atom = (m0 >> 7) * (nkb >> 1) + (kb >> 1);
+            const int atom = (m0 >> 7) * nkb + kb;
             tma_load_2d_2cta(sM, &tmapMeta, bar, 0, 2 * atom);
-          }
-          if (!kBMN) {
-            tma_load_2d_2cta(sB, &tmapB, bar, kb * 64, nb0);                   // box {64 k, 128 n}
-          } else {
-            tma_load_2d_2cta(sB, &tmapB, bar, nb0, kb * 64);                   // box {64 n, 64 k}
-            tma_load_2d_2cta(sB + 8192, &tmapB, bar, nb0 + 64, kb * 64);
+            tma_load_2d_2cta(sB, &tmapB, bar, kb * 128, nb0);                  // two 64-wide K slabs
+            tma_load_2d_2cta(sB + 16384, &tmapB, bar, kb * 128 + 64, nb0);
           }
         }
         if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -544,6 +551,19 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     // =========================== MMA issuer (leader CTA only) ===========================
     if (rank == 0 && lane == 0) {
       constexpr uint32_t idesc = idesc_bf16(256, BN, kAMN, kBMN, kSparse);
+      // Descriptor halves that never change: high word = stride offset, version, swizzle; the low
+      // word is (address >> 4) | leading offset, advanced by plain 32-bit adds.
+      const uint32_t smem0 = smem_u32(smem);
+      const uint64_t a_proto = (kMode == MODE_DENSE && kAMN) ? smem_desc(0, 8192, 1024, kSwizzle128B)
+                                                             : smem_desc(0, 16, 1024, kSwizzle128B);
+      const uint64_t b_proto = kBMN ? smem_desc(0, 8192, 1024, kSwizzle128B) : smem_desc(0, 16, 1024, kSwizzle128B);
+      const uint64_t m_proto = smem_desc(0, 128, 128, kSwizzleNone);
+      const uint32_t a_hi = (uint32_t)(a_proto >> 32), b_hi = (uint32_t)(b_proto >> 32), m_hi = (uint32_t)(m_proto >> 32);
+      const uint32_t a_lo0 = (uint32_t)a_proto + (smem0 >> 4);
+      const uint32_t b_lo0 = (uint32_t)b_proto + ((smem0 + kAStageBytes) >> 4);
+      const uint32_t m_lo0 = (uint32_t)m_proto + ((smem0 + kAStageBytes + kBHalfBytes) >> 4);
+      // per-instruction advances of the low words (in 16-byte units)
+      constexpr uint32_t a_step = (kMode == MODE_DENSE && kAMN) ? (2048 >> 4) : (32 >> 4);
       uint32_t stage = 0, phase = 0;
       uint32_t acc = 0, acc_phase = 0;
       bool ok = true;
@@ -554,28 +574,21 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
         for (int kb = 0; kb < nkb; ++kb) {
           if (!mbar_wait(&ctl->full[stage], phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sA = smem_u32(smem + stage * kStageBytes);
-          const uint32_t sB = sA + kAStageBytes;
-          const uint32_t sM = sB + kBHalfBytes;
-          if (kSparse && (kb & 1) == 0)
-            tmem_cp_128x128b_2cta(tmem_base + kMetaTmemCol, smem_desc(sM, 128, 128, kSwizzleNone));
+          const uint32_t soff = stage * (uint32_t)(kStageBytes >> 4);
+          const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
+          const uint32_t mbuf = tmem_base + kMetaTmemCol + 4u * ((uint32_t)kb & 1u);   // metadata double buffer
+          if (kSparse) tmem_cp_128x128b_2cta(mbuf, desc64(m_lo0 + soff, m_hi));
 #pragma unroll
-          for (int k = 0; k < kMmaPerStage; ++k) {
-            uint64_t adesc, bdesc;
-            if (kMode == MODE_DENSE) {
-              adesc = kAMN ? smem_desc(sA + k * 2048, 8192, 1024, kSwizzle128B)
-                           : smem_desc(sA + k * 32, 16, 1024, kSwizzle128B);
-            } else {
-              adesc = smem_desc(sA + k * 32, 16, 512, 4 /* 64 B swizzle */);
-            }
-            if (kBMN) bdesc = smem_desc(sB + k * (kSparse ? 4096 : 2048), 8192, 1024, kSwizzle128B);
-            else      bdesc = smem_desc(sB + k * (kSparse ? 64 : 32), 16, 1024, kSwizzle128B);
+          for (int k = 0; k < 4; ++k) {
             const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
             if (kSparse) {
-              const uint32_t col = (uint32_t)((kb & 1) * 2 + k);
-              mma_sp_f16_2cta(tmem_d, adesc, bdesc, tmem_base + kMetaTmemCol + (col & ~1u), idesc | (col & 1u), accum);
+              // K = 32 per instruction: 32 B of stored A, 64 B of B inside a 64-wide K slab
+              const uint32_t bk = (uint32_t)((k >> 1) * (16384 >> 4) + (k & 1) * (64 >> 4));
+              mma_sp_f16_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi),
+                              mbuf + (uint32_t)(k & ~1), idesc | (uint32_t)(k & 1), accum);
             } else {
-              mma_f16_2cta(tmem_d, adesc, bdesc, idesc, accum);
+              const uint32_t bk = (uint32_t)k * (kBMN ? (2048 >> 4) : (32 >> 4));
+              mma_f16_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi), idesc, accum);
             }
           }
           mma_commit_2cta(&ctl->empty[stage]);             // frees the stage in both CTAs
@@ -764,7 +777,8 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, int
   if (M == 0 || N == 0) return SF_OK;
   const bool two = use_two_cta(M);
   CUtensorMap ta, tb, tm;
-  int st = make_tmap(&ta, a_vals, M, K / 2, K / 2, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B);
+  int st = two ? make_tmap(&ta, a_vals, M, K / 2, K / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)
+               : make_tmap(&ta, a_vals, M, K / 2, K / 2, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B);
   if (st != SF_OK) return st;
   st = make_tmap(&tb, B, N, K, K, 64, two ? 128 : 256, CU_TENSOR_MAP_SWIZZLE_128B);
   if (st != SF_OK) return st;
