@@ -121,6 +121,11 @@ SF_API int sf_vnm_sparsify_act(const void* preact, int64_t T, int64_t F, int64_t
  * sf_gemm_sparse24:  Ct[Nc,Mr] (transposed output!) with C[Mr,Nc] = A_s[Mr,K] B[Nc,K]^T where
  *     A_s is given packed: a_vals bf16 [Mr,K/2], a_meta canonical uint16 [Mr,K/16].
  *     This is y1 = X W1s^T with A_s = W1s, B = X, output y1 [T,F].  Mr % 128, Nc % 256, K % 128.
+ * sf_gemm_sparse24_rm:  C[Mr,Nc] (row-major) = A_s[Mr,K] op(B)^T with the same packed A_s;
+ *     b_kmajor = 1: B is [Nc,K] row-major; 0: B is stored [K,Nc] row-major. This is how V:N:M
+ *     activations with M <= 8 are multiplied: every such row is also a legal 2:4 row over all F
+ *     columns (y3 = y2 W2^T with B = W2 as stored; dX = dy1 W1 with B = W1 as stored).
+ *     Mr % 256, Nc % 256, K % 128.
  * sf_gemm_venom:  C[T,Nc] = A_vnm[T,F] Bt[F,Nc] with A_vnm in V:N:M packed form (vals, meta,
  *     colidx as produced by sf_vnm_sparsify_act) and Bt row-major [F,Nc] (rows are gathered by
  *     colidx).  T % 128, V in {64,128}, Nc % 256, (4F/M) % 128 == 0.
@@ -131,6 +136,8 @@ SF_API int sf_gemm_dense(const void* A, int a_kmajor, const void* B, int b_kmajo
                   int64_t Mr, int64_t Nc, int64_t K, void* workspace, void* stream);
 SF_API int sf_gemm_sparse24(const void* a_vals, const void* a_meta, const void* B, void* Ct,
                      int64_t Mr, int64_t Nc, int64_t K, void* workspace, void* stream);
+SF_API int sf_gemm_sparse24_rm(const void* a_vals, const void* a_meta, const void* B, int b_kmajor, void* C,
+                               int64_t Mr, int64_t Nc, int64_t K, void* workspace, void* stream);
 SF_API int sf_gemm_venom(const void* a_vals, const void* a_meta, const void* colidx, const void* Bt,
                   void* C, int64_t T, int64_t F, int64_t Nc, int V, int M,
                   void* workspace, void* stream);

@@ -48,6 +48,7 @@ _SIGNATURES = {
     "sf_gemm_workspace_size": (_i32, [_i64, _i64, C.POINTER(_sz)]),
     "sf_gemm_dense": (_i32, [_vp, _i32, _vp, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "sf_gemm_sparse24": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
+    "sf_gemm_sparse24_rm": (_i32, [_vp, _vp, _vp, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "sf_gemm_sparse24_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "sf_gemm_venom": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp, _vp]),
     "sf_ffn_workspace_size": (_i32, [C.POINTER(sf_ffn_desc), C.POINTER(_sz), C.POINTER(_sz)]),
@@ -200,6 +201,20 @@ def sf_gemm_sparse24(a_vals, a_meta, B, Ct_out=None, workspace=None, stream=None
                                 _ptr(workspace), _stream(stream))
     _check(st, "sf_gemm_sparse24")
     return Ct_out, workspace
+
+
+def sf_gemm_sparse24_rm(a_vals, a_meta, B, b_kmajor: bool, C_out=None, workspace=None, stream=None):
+    """C[Mr,Nc] = A_s[Mr,K] op(B)^T, row-major output; B is [Nc,K] (b_kmajor) or [K,Nc]."""
+    Mr, K = a_vals.shape[0], a_vals.shape[1] * 2
+    Nc = B.shape[0] if b_kmajor else B.shape[1]
+    if C_out is None:
+        C_out = torch.empty((Mr, Nc), dtype=B.dtype, device=B.device)
+    if workspace is None:
+        workspace = _workspace(sf_gemm_workspace_size(Mr, K), B.device)
+    st = lib().sf_gemm_sparse24_rm(_ptr(a_vals), _ptr(a_meta), _ptr(B), int(b_kmajor), _ptr(C_out), Mr, Nc, K,
+                                   _ptr(workspace), _stream(stream))
+    _check(st, "sf_gemm_sparse24_rm")
+    return C_out, workspace
 
 
 def sf_gemm_sparse24_noalloc(a_vals, a_meta, B, Ct_out, stream=None):

@@ -60,9 +60,12 @@ __global__ void pack_like_kernel(const uint16_t* __restrict__ dense, const uint1
 
 struct SparseLayout {
   // forward context
-  size_t y2_vals, relu_vals, meta, meta_hw, colidx, y2_dense, relu_dense, w2t, y1, ctx_total;
+  size_t y2_vals, relu_vals, meta, meta_hw, colidx, y2_dense, relu_dense, w2t, y1, vals24, meta24, meta24_hw,
+      ctx_total;
   // workspace (after the status block)
-  size_t w1_vals, w1_meta, w1_meta_hw, ws_y1, w2_vals, w2_meta, w2_meta_hw, dy1_dense, dy1_vals, ws_total;
+  size_t w1_vals, w1_meta, w1_meta_hw, ws_y1, w2_vals, w2_meta, w2_meta_hw, dy1_dense, dy1_vals, dy1_vals24,
+      ws_total;
+  bool plain24;   // activations are fed to the tensor cores as plain 2:4 over all F columns
 };
 
 SparseLayout sparse_layout(const sf_ffn_desc& d) {
@@ -79,6 +82,16 @@ SparseLayout sparse_layout(const sf_ffn_desc& d) {
   L.relu_dense = take(T * F * 2);
   L.w2t = take(F * D * 2);
   L.y1 = (d.flags & 1) ? take(T * F * 2) : (size_t)-1;
+  // M <= 8: every V:N:M row is also a legal 2:4 row over all F columns, and on this hardware the
+  // ungathered 2:4 product (twice the tensor work, no row gather) is the faster of the two.
+  L.plain24 = (d.M == 4) || (d.M == 8 && vnm_has_24_view(d.F, d.V, d.M));
+  if (d.M == 8 && L.plain24) {
+    L.vals24 = take(T * F);
+    L.meta24 = take(T * F / 8);
+    L.meta24_hw = take(T * F / 8);
+  } else {
+    L.vals24 = L.y2_vals; L.meta24 = L.meta; L.meta24_hw = L.meta_hw;   // M == 4: the packed form is already 2:4
+  }
   L.ctx_total = o;
   o = kStatusBytes;
   L.w1_vals = take(F * D);
@@ -90,6 +103,7 @@ SparseLayout sparse_layout(const sf_ffn_desc& d) {
   L.w2_meta_hw = take(F * D / 8);
   L.dy1_dense = take(T * F * 2);
   L.dy1_vals = take(T * 2 * G * 2);
+  L.dy1_vals24 = (d.M == 8 && L.plain24) ? take(T * F) : L.dy1_vals;
   L.ws_total = o;
   return L;
 }
@@ -185,7 +199,21 @@ int sf_gemm_sparse24(const void* a_vals, const void* a_meta, const void* B, void
   cudaStream_t s = (cudaStream_t)stream;
   uint8_t* hw = at(workspace, kStatusBytes);
   SF_TRY(launch_meta_reorder(a_meta, hw, Mr, K, s));
-  return gemm_sparse24(a_vals, hw, B, Mr, Nc, K, EPI_STORE_T, Ct, Mr, nullptr, 0, (int*)workspace, s);
+  return gemm_sparse24(a_vals, hw, B, true, Mr, Nc, K, EPI_STORE_T, Ct, Mr, nullptr, 0, (int*)workspace, s);
+}
+
+int sf_gemm_sparse24_rm(const void* a_vals, const void* a_meta, const void* B, int b_kmajor, void* C, int64_t Mr,
+                        int64_t Nc, int64_t K, void* workspace, void* stream) {
+  if (Mr < 0 || Nc < 0 || K <= 0 || Mr % 256 || Nc % 256 || K % 128) return SF_ERR_SHAPE;
+  if (Mr == 0 || Nc == 0) return SF_OK;
+  if (!a_vals || !a_meta || !B || !C || !workspace) return SF_ERR_NULL;
+  if (!aligned16(a_vals) || !aligned16(a_meta) || !aligned16(B) || !aligned16(C) || !aligned16(workspace))
+    return SF_ERR_ALIGN;
+  SF_TRY(check_arch());
+  cudaStream_t s = (cudaStream_t)stream;
+  uint8_t* hw = at(workspace, kStatusBytes);
+  SF_TRY(launch_meta_reorder(a_meta, hw, Mr, K, s));
+  return gemm_sparse24(a_vals, hw, B, b_kmajor != 0, Mr, Nc, K, EPI_STORE, C, Nc, nullptr, 0, (int*)workspace, s);
 }
 
 int sf_gemm_venom(const void* a_vals, const void* a_meta, const void* colidx, const void* Bt, void* C, int64_t T,
@@ -241,19 +269,29 @@ int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, co
   SF_TRY(launch_prune24(W1, d.F, d.D, d.D, 1, d.prune_mode, at(workspace, L.w1_vals), at(workspace, L.w1_meta),
                         at(workspace, L.w1_meta_hw), nullptr, s));
   trace_mark(s);
-  SF_TRY(gemm_sparse24(at(workspace, L.w1_vals), at(workspace, L.w1_meta_hw), X, d.F, d.T, d.D, EPI_STORE_T, y1,
+  SF_TRY(gemm_sparse24(at(workspace, L.w1_vals), at(workspace, L.w1_meta_hw), X, true, d.F, d.T, d.D, EPI_STORE_T, y1,
                        d.F, nullptr, 0, status, s));
   trace_mark(s);
   // lines 5-6: y2 = ReLU(y1)^2 in V:N:M form (+ what the backward pass needs)
+  const bool emit24 = L.plain24 && d.M == 8;
   SF_TRY(launch_vnm(y1, d.T, d.F, d.F, d.V, d.M, 1, at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta),
                     at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), at(fwd_ctx, L.relu_vals),
-                    at(fwd_ctx, L.y2_dense), at(fwd_ctx, L.relu_dense), s));
+                    at(fwd_ctx, L.y2_dense), at(fwd_ctx, L.relu_dense), emit24 ? at(fwd_ctx, L.vals24) : nullptr,
+                    emit24 ? at(fwd_ctx, L.meta24) : nullptr, emit24 ? at(fwd_ctx, L.meta24_hw) : nullptr, s));
   trace_mark(s);
-  // line 7: y3 = y2 W2^T with W2 dense; rows of W2^T are gathered by the kept columns
-  SF_TRY(launch_transpose(W2, at(fwd_ctx, L.w2t), d.D, d.F, s));
-  trace_mark(s);
-  SF_TRY(gemm_venom(at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), at(fwd_ctx, L.w2t), d.T,
-                    d.F, d.D, d.V, d.M, Y, d.D, status, s));
+  // line 7: y3 = y2 W2^T with W2 dense
+  if (L.plain24) {
+    // y2 as a 2:4 operand over all F columns against W2 [D, F] as it is stored (no transpose, no gather)
+    trace_mark(s);
+    SF_TRY(gemm_sparse24(at(fwd_ctx, L.vals24), at(fwd_ctx, L.meta24_hw), W2, true, d.T, d.D, d.F, EPI_STORE, Y, d.D,
+                         nullptr, 0, status, s));
+  } else {
+    // condensed V:N:M operand; rows of W2^T are gathered by the kept columns
+    SF_TRY(launch_transpose(W2, at(fwd_ctx, L.w2t), d.D, d.F, s));
+    trace_mark(s);
+    SF_TRY(gemm_venom(at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), at(fwd_ctx, L.w2t), d.T,
+                      d.F, d.D, d.V, d.M, Y, d.D, status, s));
+  }
   trace_mark(s);
   return SF_OK;
 }
@@ -271,18 +309,36 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
   // Algorithm 2 line 2: W2s = sparsify24(W2^T) along d_model (contiguous in the saved W2^T copy),
   // dy2 = dY W2s;  line 4: dy1 = 2 dy2 ReLU(y1) on y2's mask (fused into the product's epilogue)
   trace_mark(s);
-  SF_TRY(launch_prune24(at(fwd_ctx, L.w2t), d.F, d.D, d.D, 1, d.prune_mode, at(workspace, L.w2_vals),
-                        at(workspace, L.w2_meta), at(workspace, L.w2_meta_hw), nullptr, s));
+  if (L.plain24) {
+    // no W2^T copy exists on this path: prune the strided groups of W2 [D, F] directly
+    SF_TRY(launch_prune24(W2, d.D, d.F, d.F, 0, d.prune_mode, at(workspace, L.w2_vals), at(workspace, L.w2_meta),
+                          at(workspace, L.w2_meta_hw), nullptr, s));
+  } else {
+    SF_TRY(launch_prune24(at(fwd_ctx, L.w2t), d.F, d.D, d.D, 1, d.prune_mode, at(workspace, L.w2_vals),
+                          at(workspace, L.w2_meta), at(workspace, L.w2_meta_hw), nullptr, s));
+  }
   trace_mark(s);
-  SF_TRY(gemm_sparse24(at(workspace, L.w2_vals), at(workspace, L.w2_meta_hw), dY, d.F, d.T, d.D, EPI_DRELU_T,
+  SF_TRY(gemm_sparse24(at(workspace, L.w2_vals), at(workspace, L.w2_meta_hw), dY, true, d.F, d.T, d.D, EPI_DRELU_T,
                        at(workspace, L.dy1_dense), d.F, at(fwd_ctx, L.relu_dense), d.F, status, s));
   trace_mark(s);
-  SF_TRY(launch_pack_like(at(workspace, L.dy1_dense), at(fwd_ctx, L.meta), at(fwd_ctx, L.colidx),
-                          at(workspace, L.dy1_vals), d.T, d.F, d.V, d.M, s));
-  trace_mark(s);
-  // line 5: dX = dy1 W1 with W1 dense (rows gathered by the kept columns)
-  SF_TRY(gemm_venom(at(workspace, L.dy1_vals), at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), W1, d.T, d.F, d.D, d.V,
-                    d.M, dX, d.D, status, s));
+  // line 5: dX = dy1 W1 with W1 dense
+  if (L.plain24) {
+    // dy1 shares y2's positions: pack it with the same 2:4 metadata; W1 [F, D] is the MN-major operand
+    SF_TRY(launch_pack24(at(workspace, L.dy1_dense), at(fwd_ctx, L.meta24), at(workspace, L.dy1_vals24), d.T, d.F, s));
+    if ((d.flags & 1) && d.M == 8)    // debug: also the V:N:M-packed form
+      SF_TRY(launch_pack_like(at(workspace, L.dy1_dense), at(fwd_ctx, L.meta), at(fwd_ctx, L.colidx),
+                              at(workspace, L.dy1_vals), d.T, d.F, d.V, d.M, s));
+    trace_mark(s);
+    SF_TRY(gemm_sparse24(at(workspace, L.dy1_vals24), at(fwd_ctx, L.meta24_hw), W1, false, d.T, d.D, d.F, EPI_STORE,
+                         dX, d.D, nullptr, 0, status, s));
+  } else {
+    SF_TRY(launch_pack_like(at(workspace, L.dy1_dense), at(fwd_ctx, L.meta), at(fwd_ctx, L.colidx),
+                            at(workspace, L.dy1_vals), d.T, d.F, d.V, d.M, s));
+    trace_mark(s);
+    // rows of W1 gathered by the kept columns
+    SF_TRY(gemm_venom(at(workspace, L.dy1_vals), at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), W1, d.T, d.F, d.D,
+                      d.V, d.M, dX, d.D, status, s));
+  }
   trace_mark(s);
   // line 3: dW2 = dY^T y2 [D, F];  line 6: dW1 = dy1^T X [F, D]  (reduction over tokens)
   SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.y2_dense), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0,

@@ -540,8 +540,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
             // metadata atoms are rows of 2 x 1 KB in a [2 * atoms, 256] uint32 view
             const int atom = (m0 >> 7) * nkb + kb;
             tma_load_2d_2cta(sM, &tmapMeta, bar, 0, 2 * atom);
-            tma_load_2d_2cta(sB, &tmapB, bar, kb * 128, nb0);                  // two 64-wide K slabs
-            tma_load_2d_2cta(sB + 16384, &tmapB, bar, kb * 128 + 64, nb0);
+            if (!kBMN) {
+              tma_load_2d_2cta(sB, &tmapB, bar, kb * 128, nb0);                // two 64-wide K slabs
+              tma_load_2d_2cta(sB + 16384, &tmapB, bar, kb * 128 + 64, nb0);
+            } else {
+              tma_load_2d_2cta(sB, &tmapB, bar, nb0, kb * 128);                // two chunks {64 n, 128 k}
+              tma_load_2d_2cta(sB + 16384, &tmapB, bar, nb0 + 64, kb * 128);
+            }
           }
         }
         if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -556,7 +561,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
       const uint32_t smem0 = smem_u32(smem);
       const uint64_t a_proto = (kMode == MODE_DENSE && kAMN) ? smem_desc(0, 8192, 1024, kSwizzle128B)
                                                              : smem_desc(0, 16, 1024, kSwizzle128B);
-      const uint64_t b_proto = kBMN ? smem_desc(0, 8192, 1024, kSwizzle128B) : smem_desc(0, 16, 1024, kSwizzle128B);
+      const uint64_t b_proto = kBMN ? smem_desc(0, kSparse ? 16384 : 8192, 1024, kSwizzle128B)
+                                    : smem_desc(0, 16, 1024, kSwizzle128B);
       const uint64_t m_proto = smem_desc(0, 128, 128, kSwizzleNone);
       const uint32_t a_hi = (uint32_t)(a_proto >> 32), b_hi = (uint32_t)(b_proto >> 32), m_hi = (uint32_t)(m_proto >> 32);
       const uint32_t a_lo0 = (uint32_t)a_proto + (smem0 >> 4);
@@ -583,7 +589,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
             const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
             if (kSparse) {
               // K = 32 per instruction: 32 B of stored A, 64 B of B inside a 64-wide K slab
-              const uint32_t bk = (uint32_t)((k >> 1) * (16384 >> 4) + (k & 1) * (64 >> 4));
+              const uint32_t bk = kBMN ? (uint32_t)k * (4096 >> 4)      // 32 k rows of 128 B
+                                       : (uint32_t)((k >> 1) * (16384 >> 4) + (k & 1) * (64 >> 4));
               mma_sp_f16_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi),
                               mbuf + (uint32_t)(k & ~1), idesc | (uint32_t)(k & 1), accum);
             } else {
@@ -771,16 +778,20 @@ int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64
   return SF_ERR_UNSUPPORTED;
 }
 
-int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, int64_t M, int64_t N, int64_t K,
-                  int epi, void* Ct, int64_t ldc, const void* aux, int64_t ldaux, int* status, cudaStream_t s) {
+int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t M, int64_t N,
+                  int64_t K, int epi, void* C, int64_t ldc, const void* aux, int64_t ldaux, int* status,
+                  cudaStream_t s) {
   if (M % BM || N % BN || K % 128) return SF_ERR_SHAPE;
   if (M == 0 || N == 0) return SF_OK;
   const bool two = use_two_cta(M);
+  const bool plain = (epi == EPI_STORE);                 // row-major output, either B layout: two-CTA kernel only
+  if ((plain || !b_kmajor) && !two) return SF_ERR_UNSUPPORTED;
   CUtensorMap ta, tb, tm;
   int st = two ? make_tmap(&ta, a_vals, M, K / 2, K / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)
                : make_tmap(&ta, a_vals, M, K / 2, K / 2, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B);
   if (st != SF_OK) return st;
-  st = make_tmap(&tb, B, N, K, K, 64, two ? 128 : 256, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (b_kmajor) st = make_tmap(&tb, B, N, K, K, 64, two ? 128 : 256, CU_TENSOR_MAP_SWIZZLE_128B);
+  else          st = make_tmap(&tb, B, K, N, N, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
   if (st != SF_OK) return st;
   tm = ta;
   if (two) {
@@ -791,8 +802,12 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, int
   }
   GemmArgs a{};
   a.M = M; a.N = N; a.K = K;
-  a.C = Ct; a.ldc = ldc; a.aux = aux; a.ldaux = ldaux; a.meta_hw = meta_hw; a.status = status;
+  a.C = C; a.ldc = ldc; a.aux = aux; a.ldaux = ldaux; a.meta_hw = meta_hw; a.status = status;
   a.num_m_tiles = (int)(M / BM); a.num_n_tiles = (int)(N / BN); a.num_k_blocks = (int)(K / 64);
+  if (epi == EPI_STORE) {
+    if (b_kmajor) return launch_two<MODE_SPARSE24, false, false, EPI_STORE>(ta, tb, tm, a, s);
+    return launch_two<MODE_SPARSE24, false, true, EPI_STORE>(ta, tb, tm, a, s);
+  }
   if (epi == EPI_STORE_T)
     return two ? launch_two<MODE_SPARSE24, false, false, EPI_STORE_T>(ta, tb, tm, a, s)
                : launch_one<MODE_SPARSE24, false, false, EPI_STORE_T>(ta, tb, a, s);

@@ -37,9 +37,12 @@ struct GemmArgs {
 int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64_t M, int64_t N, int64_t K, int epi,
                void* C, int64_t ldc, void* C2, int64_t ldc2, const void* aux, int64_t ldaux, int* status,
                cudaStream_t s);
-// Ct[N,M] = (A_s[M,K] B[N,K]^T)^T with A_s 2:4-packed; epi in {EPI_STORE_T, EPI_DRELU_T}.
-int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, int64_t M, int64_t N, int64_t K,
-                  int epi, void* Ct, int64_t ldc, const void* aux, int64_t ldaux, int* status, cudaStream_t s);
+// A_s[M,K] 2:4-packed times B (b_kmajor: [N,K] row-major, else [K,N] row-major).
+// epi EPI_STORE_T / EPI_DRELU_T: transposed output Ct[N,M] (b_kmajor only); EPI_STORE: C[M,N]
+// (two-CTA kernel, M % 256 == 0).
+int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t M, int64_t N,
+                  int64_t K, int epi, void* C, int64_t ldc, const void* aux, int64_t ldaux, int* status,
+                  cudaStream_t s);
 // C[T,N] = A_vnm[T,F] Bt[F,N]; A_vnm packed (vals [T, 2F/Mv], hardware-ordered metadata, colidx).
 int gemm_venom(const void* a_vals, const uint8_t* meta_hw, const uint8_t* colidx, const void* Bt, int64_t T,
                int64_t F, int64_t N, int V, int Mv, void* C, int64_t ldc, int* status, cudaStream_t s);

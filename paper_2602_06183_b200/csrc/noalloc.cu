@@ -58,5 +58,5 @@ extern "C" int sf_gemm_sparse24_noalloc(const void* a_vals, const void* a_meta, 
   unsigned char* hw = scratch + kNoAllocStatusBytes;
   st = launch_meta_reorder(a_meta, hw, Mr, K, s);
   if (st != SF_OK) return st;
-  return gemm_sparse24(a_vals, hw, B, Mr, Nc, K, EPI_STORE_T, Ct, Mr, nullptr, 0, reinterpret_cast<int*>(scratch), s);
+  return gemm_sparse24(a_vals, hw, B, true, Mr, Nc, K, EPI_STORE_T, Ct, Mr, nullptr, 0, reinterpret_cast<int*>(scratch), s);
 }

@@ -175,7 +175,8 @@ __global__ void __launch_bounds__(kThreads)
 vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int V, int apply,
             uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
             uint8_t* __restrict__ colidx, uint16_t* __restrict__ relu_vals, uint16_t* __restrict__ dense_out,
-            uint16_t* __restrict__ relu_dense_out) {
+            uint16_t* __restrict__ relu_dense_out, uint16_t* __restrict__ vals24, uint16_t* __restrict__ meta24,
+            uint8_t* __restrict__ meta24_hw) {
   constexpr int M = 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   uint16_t* tile = reinterpret_cast<uint16_t*>(smem_raw);                        // [V][kCW + kPad]
@@ -305,14 +306,60 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
       meta[t * (G >> 2) + kw] = (uint16_t)word;
       if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(t, kw, 4 * G)) = (uint16_t)word;
     }
+    // The same row as a plain 2:4 operand over all F columns: two values per eight columns always
+    // satisfy "at most two per four", so each half-group stores its kept values (or zeros) and a
+    // legal position pair. A half-group with one kept value at position p pairs it with a zero
+    // at position 1 (p = 0) or 0 (p > 0).
+    if (vals24) {
+      const uint32_t ca = (c4 >> (8 * p0)) & 0xFFu, cb = (c4 >> (8 * p1)) & 0xFFu;     // kept columns, ca < cb
+      const uint32_t va = packed & 0xFFFFu, vb = packed >> 16;
+      uint32_t wlo, whi, nlo, nhi;
+      if (cb < 4u) {
+        wlo = packed; nlo = ca | (cb << 2); whi = 0u; nhi = 4u;
+      } else if (ca >= 4u) {
+        wlo = 0u; nlo = 4u; whi = packed; nhi = (ca - 4u) | ((cb - 4u) << 2);
+      } else {
+        const uint32_t pb = cb - 4u;
+        wlo = ca == 0u ? va : (va << 16); nlo = ca == 0u ? 4u : (ca << 2);
+        whi = pb == 0u ? vb : (vb << 16); nhi = pb == 0u ? 4u : (pb << 2);
+      }
+      *reinterpret_cast<uint2*>(vals24 + t * (F >> 1) + (g0 + g) * 4) = make_uint2(wlo, whi);
+      uint32_t mb = nlo | (nhi << 4);
+      mb |= __shfl_down_sync(0xFFFFFFFFu, mb, 1) << 8;
+      if ((g & 1) == 0) {
+        const int64_t kw24 = (g0 + g) >> 1;
+        meta24[t * (F >> 4) + kw24] = (uint16_t)mb;
+        *reinterpret_cast<uint16_t*>(meta24_hw + meta_hw_offset(t, kw24, F)) = (uint16_t)mb;
+      }
+    }
   }
 }
+
+// Gather a dense [R, K] matrix at the positions of canonical 2:4 metadata: vals[r, k/2] (bf16).
+__global__ void __launch_bounds__(256)
+pack24_kernel(const uint4* __restrict__ dense, const uint16_t* __restrict__ meta, uint4* __restrict__ vals,
+              int64_t R, int64_t K) {
+  const int64_t words = K >> 4;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= R * words) return;
+  const uint4 q0 = __ldg(dense + 2 * idx), q1 = __ldg(dense + 2 * idx + 1);
+  const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+  const uint32_t m = meta[idx];
+  uint32_t o[4];
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const uint32_t nib = (m >> (4 * g)) & 0xFu;
+    o[g] = __byte_perm(w[2 * g], w[2 * g + 1], 0x1010u + (nib & 3u) * 0x22u + (nib >> 2) * 0x2200u);
+  }
+  vals[idx] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 
 }  // namespace
 
 int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
                void* vals, void* meta, void* meta_hw, void* colidx, void* relu_vals, void* dense_out,
-               void* relu_dense_out, cudaStream_t s) {
+               void* relu_dense_out, void* vals24, void* meta24, void* meta24_hw, cudaStream_t s) {
   if (T == 0 || F == 0) return SF_OK;
   const size_t smem = (size_t)V * (kCW + kPad) * 2 + kCW * 4 + kCW + kCW;
   static bool attr_set[64] = {false};                         // per device
@@ -336,15 +383,31 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
     }
     vnm8_kernel<<<grid, kThreads, smem, s>>>((const uint16_t*)P, T, F, ld, V, apply_sqrelu, (uint16_t*)vals,
                                              (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
-                                             (uint16_t*)relu_vals, (uint16_t*)dense_out, (uint16_t*)relu_dense_out);
+                                             (uint16_t*)relu_vals, (uint16_t*)dense_out, (uint16_t*)relu_dense_out,
+                                             (uint16_t*)vals24, (uint16_t*)meta24, (uint8_t*)meta24_hw);
     SF_LAUNCH_CHECK();
     return SF_OK;
   }
+  if (vals24) return SF_ERR_UNSUPPORTED;                 // the plain-2:4 view is produced by the fast path only
   vnm_kernel<<<grid, kThreads, smem, s>>>((const uint16_t*)P, T, F, ld, V, M, apply_sqrelu, (uint16_t*)vals,
                                           (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
                                           (uint16_t*)relu_vals, (uint16_t*)dense_out, (uint16_t*)relu_dense_out);
   SF_LAUNCH_CHECK();
   return SF_OK;
+}
+
+int launch_pack24(const void* dense, const void* meta, void* vals, int64_t R, int64_t K, cudaStream_t s) {
+  const int64_t n = R * (K >> 4);
+  if (n == 0) return SF_OK;
+  pack24_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>((const uint4*)dense, (const uint16_t*)meta, (uint4*)vals, R, K);
+  SF_LAUNCH_CHECK();
+  return SF_OK;
+}
+
+// True when launch_vnm can also emit the plain-2:4 view (vals24 / meta24) for this shape.
+bool vnm_has_24_view(int64_t F, int V, int M) {
+  const int tail = (int)(F % kCW);
+  return (M == 8) && (tail == 0 || tail == 64 || tail == 128) && (V % 32 == 0);
 }
 
 }  // namespace sf

@@ -53,6 +53,20 @@ def test_sparse24_gemm_against_oracle_packing(Mr, Nc, K):
     assert rel_fro(f32(Ct), ref) < TOL
 
 
+@pytest.mark.parametrize("b_k", [True, False])
+@pytest.mark.parametrize("Mr,Nc,K", [(256, 256, 128), (512, 768, 1152)])
+def test_sparse24_gemm_row_major_output(b_k, Mr, Nc, K):
+    W = synth.prune_sweep_matrix(Mr, K, seed=Mr + K + 1, tie_frac=0.1)
+    W = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(W) * 50.0)
+    B = synth.normal_bf16((Nc, K) if b_k else (K, Nc), 0, 1, seed=4, stream=K)
+    p = oracle.prune24(W, group_dim=1, mode=0)
+    meta = torch.from_numpy(p.meta.view(np.int16)).cuda()
+    C, ws = binding.sf_gemm_sparse24_rm(to_dev(p.vals), meta, to_dev(B), b_k)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    Bf = _f64(B) if b_k else _f64(B).T
+    assert rel_fro(f32(C), _f64(p.dense) @ Bf.T) < TOL
+
+
 def test_sparse24_gemm_one_hot_metadata_probe():
     """Each kept value is a distinct power of two in an otherwise zero row and B is an identity
     slice, so the output says which K position every stored value was multiplied with."""
