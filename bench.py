@@ -52,7 +52,7 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                       "--format=csv,noheader,nounits", "-lms", "20"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
@@ -205,8 +205,10 @@ def run_ours(args, cfg):
         raise SystemExit("device status: a bounded wait expired")
 
     # ---- per-kernel times inside the step (events recorded by the library between its kernels)
-    names = ["prune24_W1", "gemm_sparse24_y1", "vnm_sparsify", "transpose_W2", "gemm_venom_y3",
-             None, "prune24_W2", "gemm_sparse24_dy1", "pack_dy1", "gemm_venom_dX", "gemm_dense_dW2", "gemm_dense_dW1"]
+    plain24 = (M <= 8)                       # activations multiplied as plain 2:4 operands (no row gather)
+    act_gemm = "gemm_sparse24" if plain24 else "gemm_venom"
+    names = ["prune24_W1", "gemm_sparse24_y1", "vnm_sparsify", "transpose_W2", f"{act_gemm}_y3",
+             None, "prune24_W2", "gemm_sparse24_dy1", "pack_dy1", f"{act_gemm}_dX", "gemm_dense_dW2", "gemm_dense_dW1"]
     with binding.StageTrace(13 * K) as tr:
         for _ in range(K):
             sparse_step()
@@ -218,34 +220,48 @@ def run_ours(args, cfg):
             if n:
                 per.setdefault(n, []).append(v)
     kern_ms = {n: float(np.mean(v)) for n, v in per.items()}
-    unit = 2.0 * T * D * F                                       # flop of one dense product
+    if plain24:
+        kern_ms.pop("transpose_W2", None)    # not launched on this path (zero-length interval)
+    unit = 2.0 * T * D * F                   # flop of one dense product
     peaks = _peaks()
-    # algorithmic work per launch: dense products 1 unit at the dense peak; 2:4 products 1 unit
-    # at twice the dense peak; Venom products 4/M of a unit at twice the dense peak.
-    alg = {"gemm_dense_dW2": (unit, 1.0), "gemm_dense_dW1": (unit, 1.0),
-           "gemm_sparse24_y1": (unit, 2.0), "gemm_sparse24_dy1": (unit, 2.0),
-           "gemm_venom_y3": (unit, 2.0 * M / 4.0), "gemm_venom_dX": (unit, 2.0 * M / 4.0)}
-    groups = {"gemm_dense(MN-major A,B)": ["gemm_dense_dW2", "gemm_dense_dW1"],
-              "gemm_sparse24": ["gemm_sparse24_y1", "gemm_sparse24_dy1"],
-              "gemm_venom": ["gemm_venom_y3", "gemm_venom_dX"]}
-    tot = {g: sum(kern_ms[k] for k in ks) for g, ks in groups.items()}
+    # Kernel groups by the device function that runs them. Algorithmic work per launch: one dense
+    # product (2*T*D*F flop) for every product; the peak it is held against is the measured dense
+    # bf16 GEMM peak for the dense kernel, twice that for the 2:4 kernel (nominal 2:4 ratio), and
+    # M/4 times more for the condensed Venom kernel.
+    groups = {
+        "gemm_tc2_kernel<dense, MN-major A and B> (dW2, dW1)": (["gemm_dense_dW2", "gemm_dense_dW1"], 1.0),
+        "gemm_tc2_kernel<2:4 sparse> (y1, dy1" + (", y3, dX)" if plain24 else ")"):
+            (["gemm_sparse24_y1", "gemm_sparse24_dy1"] + ([f"{act_gemm}_y3", f"{act_gemm}_dX"] if plain24 else []), 2.0),
+    }
+    if not plain24:
+        groups["gemm_tc_kernel<venom> (y3, dX)"] = ([f"{act_gemm}_y3", f"{act_gemm}_dX"], 2.0 * M / 4.0)
+    tot = {g: sum(kern_ms[k] for k in ks) for g, (ks, _) in groups.items()}
     dom = max(tot, key=tot.get)
-    ks = groups[dom]
+    ks, ratio = groups[dom]
     avg_ms = tot[dom] / len(ks)
-    achieved = alg[ks[0]][0] / (avg_ms / 1e3) / 1e12             # dense-equivalent TFLOP/s of the kernel
-    peak = peaks["bf16_tflops_sustained"] * alg[ks[0]][1]
+    achieved = unit / (avg_ms / 1e3) / 1e12                      # dense-equivalent TFLOP/s of the kernel
+    peak = peaks["bf16_tflops_sustained"] * ratio
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(tpath):
-        traffic = json.load(open(tpath)).get(dom)
+        traffic = json.load(open(tpath)).get(dom.split(" (")[0])
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": traffic, "peak_source": peaks["source"] + " (sustained bf16 GEMM"
-                + (", x nominal sparse ratio" if alg[ks[0]][1] != 1.0 else "") + ")",
-                "avg_launch_ms": avg_ms, "launches_per_step": len(ks)}
+                "frac": achieved / peak, "traffic": traffic,
+                "peak_source": peaks["source"] + " sustained bf16 GEMM" + (f" x {ratio:g} (nominal sparse ratio)" if ratio != 1.0 else ""),
+                "avg_launch_ms": avg_ms, "launches_per_step": len(ks),
+                "share_of_step": tot[dom] / sum(kern_ms.values()),
+                "other_groups": {g: {"avg_launch_ms": tot[g] / len(groups[g][0]),
+                                     "frac": unit / (tot[g] / len(groups[g][0]) / 1e3) / 1e12 / (peaks["bf16_tflops_sustained"] * groups[g][1])}
+                                 for g in groups if g != dom}}
     hbm = peaks["hbm_gbs"]
     prune_gbs = 3.125 * F * D / (kern_ms["prune24_W1"] / 1e3) / 1e9
-    vnm_bytes = T * F * (2 + 4.0 / M + 4.0 / M + 0.5 / M) + (T // V) * (F // M) * 4 + 2 * T * F * 2
+    # bytes the V:N:M kernel moves in the step: input, V:N:M-packed values + ReLU values + metadata
+    # (canonical and tensor-core order) + colidx, the two masked dense copies, and (M = 8) the 2:4 view
+    vnm_bytes = T * F * (2 + 4.0 / M + 4.0 / M + 1.0 / M) + (T // V) * (F // M) * 4 + 2 * T * F * 2
+    if plain24 and M == 8:
+        vnm_bytes += T * F * (1.0 + 0.25)
     vnm_gbs = vnm_bytes / (kern_ms["vnm_sparsify"] / 1e3) / 1e9
+    launches_per_step = 10 if plain24 else 11
 
     # ---- end to end through the host-buffer entry point (H2D of inputs and D2H of results timed)
     staging = torch.empty((binding.sf_ffn_host_staging_size(desc),), dtype=torch.uint8, device="cuda")
@@ -276,7 +292,7 @@ def run_ours(args, cfg):
         "roofline": roofline, "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e / K, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
-        "gpu_launches": 11 * K,
+        "gpu_launches": launches_per_step * K,
     }
 
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:
@@ -298,7 +314,7 @@ def run_ours(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4_d4096")

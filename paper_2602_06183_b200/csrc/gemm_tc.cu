@@ -20,8 +20,6 @@
 #include "tc_ptx.cuh"
 #include "gemm_tc.cuh"
 
-#include <cstdlib>
-
 namespace sf {
 
 namespace {
@@ -55,6 +53,19 @@ struct SmemCtl {
   uint32_t tmem_base;
   int abort_flag;
 };
+
+// Tile raster: bands of kRasterM tile rows, m fastest inside a band. The tiles that run at the same
+// time then form a near-square block (8 x ~9 for 74 CTA pairs), so a wave touches ~17 operand
+// panels instead of ~65 and operands larger than the L2 are not re-read once per tile column.
+constexpr int kRasterM = 8;
+__device__ __forceinline__ void tile_coords(int tile, int num_m, int num_n, int& mt, int& nt) {
+  const int per_band = kRasterM * num_n;
+  const int band = tile / per_band, rem = tile - band * per_band;
+  const int m_start = band * kRasterM;
+  const int gm = min(kRasterM, num_m - m_start);
+  nt = rem / gm;
+  mt = m_start + (rem - nt * gm);
+}
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return float_to_bf16_bits(lo) | (float_to_bf16_bits(hi) << 16);
@@ -199,8 +210,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
   constexpr int kAccBufs = kSparse ? 1 : 2;
   constexpr int kMmaPerStage = kSparse ? 2 : 4;      // dense: K=16 x4 = 64; sparse: logical K=32 x2 = 64
 
-  const int num_m_tiles = args.num_m_tiles, num_n_tiles = args.num_n_tiles;
-  const int num_tiles = num_m_tiles * num_n_tiles;
+  const int num_m_tiles = args.num_m_tiles, num_n_tiles_ = args.num_n_tiles;
+  const int num_tiles = num_m_tiles * num_n_tiles_;
   const int nkb = args.num_k_blocks;                 // 64-wide (logical) k blocks per sweep
   const int sweeps = (kMode == MODE_VENOM && args.V == 64) ? 2 : 1;
   const int iters = nkb * sweeps;
@@ -233,7 +244,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     uint32_t stage = 0, phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      int mt, nt;
+      tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
       const int m0 = mt * BM, n0 = nt * BN;
       for (int it = 0; it < iters; ++it) {
         const int sweep = it / nkb, kb = it - sweep * nkb;
@@ -351,7 +363,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     uint32_t stage = 0, phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      int mt, nt;
+      tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
       const int64_t n0 = (int64_t)nt * BN;
       for (int it = 0; it < iters; ++it) {
         const int sweep = it / nkb, kb = it - sweep * nkb;
@@ -397,7 +410,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      int mt, nt;
+      tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
       const int64_t m0 = (int64_t)mt * BM, n0 = (int64_t)nt * BN;
       // The dy1 epilogue multiplies by a [token, feature] tile of the saved activations; its loads do
       // not depend on the accumulator, so they are issued before the wait and land during the main loop.
@@ -473,8 +487,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();               // 0 = leader
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const int num_m_tiles = args.num_m_tiles;              // 256-row tiles
-  const int num_tiles = num_m_tiles * args.num_n_tiles;
+  const int num_m_tiles = args.num_m_tiles, num_n_tiles_ = args.num_n_tiles;   // 256-row tiles
+  const int num_tiles = num_m_tiles * num_n_tiles_;
   const int nkb = (int)(args.K / kBK);
 
   if (threadIdx.x == 0) {
@@ -507,7 +521,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     uint32_t stage = 0, phase = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      int mt, nt;
+      tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
       const int m0 = mt * 256 + (int)rank * 128;         // this CTA's rows of A / D
       const int nb0 = nt * BN + (int)rank * 128;         // this CTA's columns of B
       for (int kb = 0; kb < nkb; ++kb) {
@@ -613,7 +628,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-      const int mt = tile % num_m_tiles, nt = tile / num_m_tiles;
+      int mt, nt;
+      tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
       const int64_t m0 = (int64_t)mt * 256 + (int64_t)rank * 128, n0 = (int64_t)nt * BN;
       uint4 ax[kEpi == EPI_DRELU_T ? kAuxChunks : 1][4];
       epi_prefetch<kEpi>(args, m0, n0, q, lane, ax);
@@ -729,15 +745,8 @@ int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
   return SF_OK;
 }
 
-// The two-CTA kernels need M % 256 == 0; SF_ONE_CTA=1 in the environment forces the one-CTA kernels.
-bool use_two_cta(int64_t M) {
-  static int forced = -1;
-  if (forced < 0) {
-    const char* e = getenv("SF_ONE_CTA");
-    forced = (e && atoi(e) != 0) ? 1 : 0;
-  }
-  return forced == 0 && (M % 256 == 0);
-}
+// The two-CTA kernels need M % 256 == 0; other shapes run the one-CTA kernels.
+bool use_two_cta(int64_t M) { return M % 256 == 0; }
 
 }  // namespace
 
@@ -828,12 +837,7 @@ int gemm_venom(const void* a_vals, const uint8_t* meta_hw, const uint8_t* colidx
   st = make_tmap(&tb, Bt, F, N, N, 64, 1, CU_TENSOR_MAP_SWIZZLE_128B);        // row gather: one row per box
   if (st != SF_OK) return st;
   GemmArgs a{};
-  {
-    const char* e = getenv("SF_GATHER_TMA_GROUPS");
-    a.gather_tma_groups = e ? atoi(e) : 12;
-    if (a.gather_tma_groups < 0) a.gather_tma_groups = 0;
-    if (a.gather_tma_groups > 16) a.gather_tma_groups = 16;
-  }
+  a.gather_tma_groups = 12;      // measured optimum of the TMA : cp.async split (of 16 groups per stage)
   a.M = T; a.N = N; a.K = Kc;
   a.aux = Bt; a.ldaux = N;
   a.C = C; a.ldc = ldc; a.meta_hw = meta_hw; a.colidx = colidx; a.V = V; a.Mv = Mv; a.G = F / Mv;

@@ -136,13 +136,13 @@ prune24_cols_kernel(const uint16_t* __restrict__ W, int64_t Kd, int64_t Rc, int6
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
       const int kr = ch * 16 + g * 4;
-      uint32_t o0, o1;
-      const uint32_t nib = prune_group<kSoft>(tile[kr][c], tile[kr + 1][c], tile[kr + 2][c], tile[kr + 3][c], o0, o1);
-      packed[g] = o0 | (o1 << 16);
+      const uint32_t lo = (uint32_t)tile[kr][c] | ((uint32_t)tile[kr + 1][c] << 16);
+      const uint32_t hi = (uint32_t)tile[kr + 2][c] | ((uint32_t)tile[kr + 3][c] << 16);
+      const uint32_t nib = prune_group_packed<kSoft>(lo, hi, packed[g]);
       m |= nib << (4 * g);
       if (dense_out) {
         uint32_t d[4];
-        expand_group(nib, o0, o1, d);
+        expand_group(nib, packed[g] & 0xFFFFu, packed[g] >> 16, d);
         tile[kr][c] = (uint16_t)d[0];
         tile[kr + 1][c] = (uint16_t)d[1];
         tile[kr + 2][c] = (uint16_t)d[2];
