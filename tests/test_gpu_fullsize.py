@@ -1,0 +1,117 @@
+"""Parity at the benchmark's full sizes, on outputs the oracle can compute one sample at a time.
+
+FFN step (the launch configuration bench.py times): whole V-blocks of tokens are checked for
+y1 / masks / y2 / y3 / dy1 / dX, and whole M-groups of features (all tokens) for dW1 / dW2 — the
+V:N:M selection of a block only needs its own rows, and that of a group only its own columns, so
+both samples are exact restrictions of the full problem. Standalone prune / sparsify sweeps are
+checked bit for bit on sampled rows / blocks of the full-size matrices.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_06183_b200 import binding, synth
+from util import to_dev, bits, f32, rel_fro
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+@pytest.mark.parametrize("name", ["c4_d4096", "c5_d8192"])
+def test_ffn_step_full_size_sampled(name):
+    cfg = synth.FFN_CONFIGS[name]
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    G = F // M
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
+    desc = binding.make_desc(T, D, F, V, M, flags=1)
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    dX_, dW1_, dW2_, ddY = (to_dev(a) for a in (X, W1, W2, dY))
+    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+    gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
+    binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
+    binding.sf_sparse_ffn_bwd(desc, ddY, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+
+    y1_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y1).view(T, F)
+    vals_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y2_VALS).view(T, 2 * G)
+    relu_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_RELU_VALS).view(T, 2 * G)
+    meta_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_META).view(T, G // 4)
+    cidx_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_COLIDX).view(T // V, G, 4)
+    dy1v_dev = binding.sf_ctx_view(desc, ws, binding.SF_CTX_DY1_VALS).view(T, 2 * G)
+
+    # ---- sample 1: two whole V-blocks of tokens (first and last), all features
+    blocks = [0, T // V - 1]
+    rows = np.concatenate([np.arange(b * V, (b + 1) * V) for b in blocks])
+    rows_t = torch.from_numpy(rows).cuda()
+    y1_rows = bits(y1_dev[rows_t])
+    free = oracle.sparse_ffn_fwd(X[rows], W1, W2, V=V, M=M)
+    assert rel_fro(oracle.bf16_to_f32(y1_rows), oracle.bf16_to_f32(free.y1b)) < TOL
+    fwd = oracle.sparse_ffn_fwd(X[rows], W1, W2, V=V, M=M, forced_y1b=y1_rows)
+    assert np.array_equal(cidx_dev[torch.tensor(blocks).cuda()].cpu().numpy(), fwd.act.colidx)
+    assert np.array_equal(bits(meta_dev[rows_t]), fwd.act.meta)
+    assert np.array_equal(bits(vals_dev[rows_t]), fwd.act.vals)
+    assert np.array_equal(bits(relu_dev[rows_t]), fwd.act.relu_vals)
+    assert rel_fro(f32(Y[rows_t]), fwd.y3) < TOL
+    bwd = oracle.sparse_ffn_bwd(dY[rows], X[rows], W1, W2, fwd)
+    assert rel_fro(oracle.bf16_to_f32(bits(dy1v_dev[rows_t])), oracle.bf16_to_f32(bwd.dy1_vals)) < TOL
+    assert rel_fro(f32(gX[rows_t]), bwd.dX) < TOL
+
+    # ---- sample 2: four whole M-groups of features, all tokens -> columns of dW2, rows of dW1
+    groups = [0, G // 3, (2 * G) // 3, G - 1]
+    cols = np.concatenate([np.arange(g * M, (g + 1) * M) for g in groups])
+    cols_t = torch.from_numpy(cols).cuda()
+    y1_cols = bits(y1_dev[:, cols_t])
+    act = oracle.vnm_sparsify(y1_cols, V=V, M=M)
+    # the GPU's masks for these groups are the oracle's on the same pre-activations
+    assert np.array_equal(cidx_dev[:, torch.tensor(groups).cuda()].cpu().numpy(), act.colidx)
+    f64 = lambda b: oracle.bf16_to_f32(b).astype(np.float64)
+    dW2_ref = f64(dY).T @ f64(act.dense)                                  # [D, |cols|]
+    assert rel_fro(f32(gW2[:, cols_t]), dW2_ref) < TOL
+    w2s_cols = oracle.prune24(np.ascontiguousarray(W2[:, cols]), group_dim=0).dense   # groups along D
+    dy2 = (f64(dY) @ f64(w2s_cols)).astype(np.float32)
+    relu = np.maximum(oracle.bf16_to_f32(y1_cols), 0)
+    dy1 = oracle.f32_to_bf16((np.float32(2.0) * dy2 * relu).astype(np.float32)).reshape(dy2.shape)
+    dy1 = np.where(act.mask, dy1, np.uint16(0))
+    dW1_ref = f64(dy1).T @ f64(X)                                          # [|cols|, D]
+    assert rel_fro(f32(gW1[cols_t]), dW1_ref) < TOL
+
+
+@pytest.mark.parametrize("rows,cols", synth.PRUNE_SWEEP_SHAPES)
+def test_prune_sweep_full_size_sampled_rows(rows, cols):
+    w = synth.prune_sweep_matrix(rows, cols, seed=1000 + rows % 97 + cols % 89, tie_frac=0.05)
+    wd = to_dev(w)
+    rng = np.random.default_rng(rows)
+    for mode in (0, 1):
+        vals, meta, _ = binding.sf_prune24_compress(wd, 1, mode)
+        sample = np.sort(rng.choice(rows, size=192, replace=False))
+        ref = oracle.prune24(w[sample], group_dim=1, mode=mode)
+        st = torch.from_numpy(sample).cuda()
+        assert np.array_equal(bits(meta[st]), ref.meta)
+        assert np.array_equal(bits(vals[st]), ref.vals)
+    # strided groups: sampled output rows are sampled input columns
+    vals, meta, _ = binding.sf_prune24_compress(wd, 0, 0)
+    sample = np.sort(rng.choice(cols, size=64, replace=False))
+    ref = oracle.prune24(np.ascontiguousarray(w[:, sample]), group_dim=0, mode=0)
+    st = torch.from_numpy(sample).cuda()
+    assert np.array_equal(bits(meta[st]), ref.meta)
+    assert np.array_equal(bits(vals[st]), ref.vals)
+
+
+@pytest.mark.parametrize("V,M", [(64, 8), (128, 8), (64, 16), (128, 16)])
+def test_act_sweep_full_size_sampled_blocks(V, M):
+    T = F = 16384
+    p = synth.act_sweep_matrix(T, F, seed=2000)
+    vals, meta, colidx, relu, _ = binding.sf_vnm_sparsify_act(to_dev(p), V, M)
+    torch.cuda.synchronize()
+    blocks = [0, 7, T // V - 1]
+    for b in blocks:
+        ref = oracle.vnm_sparsify(p[b * V:(b + 1) * V], V=V, M=M)
+        sl = slice(b * V, (b + 1) * V)
+        assert np.array_equal(colidx[b].cpu().numpy(), ref.colidx[0])
+        assert np.array_equal(bits(meta[sl]), ref.meta)
+        assert np.array_equal(bits(vals[sl]), ref.vals)
+        assert np.array_equal(bits(relu[sl]), ref.relu_vals)
+    # the sparsity the paper quotes for trained models: about 90 % zeros before the format's own pruning
+    zero_frac = float((oracle.bf16_to_f32(p[:1024]) <= 0).mean())
+    assert 0.88 < zero_frac < 0.93
