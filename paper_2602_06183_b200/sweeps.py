@@ -1,0 +1,141 @@
+"""Stand-alone throughput sweeps of the bandwidth kernels and single products (one JSON line each).
+
+    python -m paper_2602_06183_b200.sweeps [--which prune,act,gemm,c5]
+
+prune: 2:4 prune + compress on the weight shapes of the sweep configuration (both group directions,
+       hard and soft), GB/s at 3.125 algorithmic bytes per element.
+act:   SquaredReLU + V:N:M sparsify on 16384 x 16384 pre-activations with ~90 % negatives,
+       V in {64, 128}, M in {8, 16}.
+gemm:  dense vs 2:4 vs Venom products at the paper's micro-benchmark shape (m, n, k) = (4096, 16384, 4096)
+       and at the FFN shapes.
+c5:    sparse and dense step of the d_model = 8192 layer.
+Inputs larger than the L2; times are CUDA-event averages over 20 launches after 3 warm-ups.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+import torch
+
+from . import binding, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    return json.load(open(p))["hbm_gbs"] if os.path.exists(p) else 6650.0
+
+
+def _time(fn, iters=20, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def _dev(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def prune_sweep():
+    peak = _hbm_peak()
+    for i, (rows, cols) in enumerate(synth.PRUNE_SWEEP_SHAPES):
+        w = _dev(synth.prune_sweep_matrix(rows, cols, seed=1000 + i))
+        for group_dim in (1, 0):
+            for mode in (0, 1):
+                out = binding.sf_prune24_compress(w, group_dim, mode)
+                ms = _time(lambda: binding.sf_prune24_compress(w, group_dim, mode, out=out))
+                gbs = 3.125 * rows * cols / (ms / 1e3) / 1e9
+                print(json.dumps({"kernel": "prune24_compress", "rows": rows, "cols": cols, "group_dim": group_dim,
+                                  "prune_mode": mode, "us": ms * 1e3, "GBps": gbs, "frac_of_measured_hbm": gbs / peak}))
+
+
+def act_sweep():
+    peak = _hbm_peak()
+    T = F = 16384
+    p = _dev(synth.act_sweep_matrix(T, F, seed=2000))
+    for V in (64, 128):
+        for M in (8, 16):
+            out = binding.sf_vnm_sparsify_act(p, V, M)
+            ms = _time(lambda: binding.sf_vnm_sparsify_act(p, V, M, out=out))
+            nbytes = T * F * (2 + 4.0 / M + 4.0 / M + 0.5 / M) + (T // V) * (F // M) * 4
+            gbs = nbytes / (ms / 1e3) / 1e9
+            print(json.dumps({"kernel": "vnm_sparsify_act", "T": T, "F": F, "V": V, "M": M, "us": ms * 1e3,
+                              "bytes_per_element": nbytes / (T * F), "GBps": gbs, "frac_of_measured_hbm": gbs / peak}))
+
+
+def gemm_sweep():
+    for (m, n, k) in [(4096, 16384, 4096), (16384, 8192, 4096), (8192, 4096, 16384)]:
+        A = torch.randn((m, k), device="cuda").to(torch.bfloat16)
+        B = torch.randn((n, k), device="cuda").to(torch.bfloat16)
+        C = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
+        ws = torch.zeros((binding.sf_gemm_workspace_size(m, k),), dtype=torch.uint8, device="cuda")
+        ms_d = _time(lambda: binding.sf_gemm_dense(A, True, B, True, C_out=C, workspace=ws))
+        vals, meta, _ = binding.sf_prune24_compress(A, 1, 0)
+        ms_p = _time(lambda: binding.sf_prune24_compress(A, 1, 0, out=(vals, meta, None)))
+        ms_s = _time(lambda: binding.sf_gemm_sparse24_rm(vals, meta, B, True, C_out=C, workspace=ws))
+        fl = 2.0 * m * n * k
+        print(json.dumps({"shape_mnk": [m, n, k], "dense_ms": ms_d, "dense_tflops": fl / ms_d / 1e9,
+                          "sparse24_ms": ms_s, "sparse24_dense_equiv_tflops": fl / ms_s / 1e9,
+                          "prune_ms": ms_p, "speedup_gemm_only": ms_d / ms_s,
+                          "speedup_with_prune": ms_d / (ms_s + ms_p)}))
+    # Venom (condensed, gathered) vs the same V:N:M operand as plain 2:4, M = 8 and 16
+    T, F, N = 8192, 16384, 4096
+    for M in (8, 16):
+        G = F // M
+        P = _dev(synth.normal_bf16((T, F), 0.0, 1.0, seed=7))
+        vals, meta, colidx, _, _ = binding.sf_vnm_sparsify_act(P, 128, M)
+        Bt = torch.randn((F, N), device="cuda").to(torch.bfloat16)
+        C = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+        ws = torch.zeros((binding.sf_gemm_workspace_size(T, F),), dtype=torch.uint8, device="cuda")
+        ms_v = _time(lambda: binding.sf_gemm_venom(vals, meta, colidx, Bt, 128, M, C_out=C, workspace=ws))
+        print(json.dumps({"kernel": "gemm_venom", "T": T, "F": F, "N": N, "V": 128, "M": M, "ms": ms_v,
+                          "dense_equiv_tflops": 2.0 * T * F * N / ms_v / 1e9}))
+
+
+def c5_step():
+    cfg = synth.FFN_CONFIGS["c5_d8192"]
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    X, W1, W2, dY = (_dev(a) for a in synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"]))
+    desc = binding.make_desc(T, D, F, V, M)
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+    gX, gW1, gW2 = torch.empty_like(X), torch.empty_like(W1), torch.empty_like(W2)
+
+    def sparse():
+        binding.sf_sparse_ffn_fwd(desc, X, W1, W2, Y, ctx, ws)
+        binding.sf_sparse_ffn_bwd(desc, dY, X, W1, W2, ctx, gX, gW1, gW2, ws)
+
+    def dense():
+        binding.sf_dense_ffn_fwd(desc, X, W1, W2, Y, ctx, ws)
+        binding.sf_dense_ffn_bwd(desc, dY, X, W1, W2, ctx, gX, gW1, gW2, ws)
+
+    ms_s, ms_d = _time(sparse, iters=10), _time(dense, iters=10)
+    fl = 12.0 * T * D * F
+    print(json.dumps({"workload": "c5_d8192", "sparse_step_ms": ms_s, "dense_step_ms": ms_d,
+                      "sparse_dense_equiv_tflops": fl / ms_s / 1e9, "dense_tflops": fl / ms_d / 1e9,
+                      "speedup": ms_d / ms_s, "status": binding.sf_check_status(ws)}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--which", default="prune,act,gemm,c5")
+    args = ap.parse_args()
+    from . import build
+    build.build()
+    for w in args.which.split(","):
+        {"prune": prune_sweep, "act": act_sweep, "gemm": gemm_sweep, "c5": c5_step}[w]()
+
+
+if __name__ == "__main__":
+    main()
