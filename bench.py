@@ -130,7 +130,7 @@ def run_reference(args, cfg):
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
-    from paper_2602_06183_b200 import binding, build, synth
+    from paper_2602_06183_b200 import binding, build, replicas, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -163,8 +163,7 @@ def run_ours(args, cfg):
         binding.sf_dense_ffn_bwd(desc, ddY, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     def timed(fn, steps):
@@ -175,12 +174,7 @@ def run_ours(args, cfg):
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return replicas.max_over_ranks(e0.elapsed_time(e1), device="cuda")
 
     for _ in range(W if args.quick else max(W, 3)):
         sparse_step()
@@ -191,7 +185,7 @@ def run_ours(args, cfg):
     ms = timed(sparse_step, K)
     clocks = sampler.stop() if sampler else None
     flop_step = 12.0 * T * D * F
-    value = world * flop_step * K / (ms / 1e3) / 1e12
+    value = replicas.aggregate_tflops(flop_step, K, ms)
 
     if args.quick:
         if rank == 0:
@@ -273,7 +267,7 @@ def run_ours(args, cfg):
 
     host_step()
     ms_e2e = timed(host_step, K)
-    e2e_val = world * flop_step * K / (ms_e2e / 1e3) / 1e12
+    e2e_val = replicas.aggregate_tflops(flop_step, K, ms_e2e)
     h2d = 2 * T * D * 2 + 2 * F * D * 2
     d2h = h2d
 
@@ -285,7 +279,7 @@ def run_ours(args, cfg):
                    "prune_mode": args.prune_mode, "parallelism": f"replicas x{world}",
                    "l2": "per-step inputs (402 MB of operands, >2 GB of intermediates) exceed the 126 MB L2"},
         "dense_step_ms": ms_dense / K, "speedup_vs_dense_step": ms_dense / ms,
-        "dense_step_tflops": world * flop_step * K / (ms_dense / 1e3) / 1e12,
+        "dense_step_tflops": replicas.aggregate_tflops(flop_step, K, ms_dense),
         "kernel_ms": kern_ms,
         "prune24_gbs": prune_gbs, "prune24_frac_of_hbm": prune_gbs / hbm,
         "vnm_sparsify_gbs": vnm_gbs, "vnm_frac_of_hbm": vnm_gbs / hbm,
