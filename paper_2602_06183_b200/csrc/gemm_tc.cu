@@ -96,10 +96,7 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
                                          uint8_t* my_stage,
                                          const uint4 (&ax)[kEpi == EPI_DRELU_T ? kAuxChunks : 1][4]) {
   const int64_t row = m0 + q * 32 + lane;                                  // this thread's D row
-  auto chunk = [&](int ch, const uint4 (&a4)[4]) {
-    uint32_t v[32];
-    tmem_ld_32x32b_x32(taddr + ch * 32, v);
-    tmem_ld_wait();
+  auto chunk = [&](int ch, const uint4 (&a4)[4], const uint32_t (&v)[32]) {
     const int64_t col0 = n0 + ch * 32;
     if (kEpi == EPI_STORE || kEpi == EPI_SQRELU || kEpi == EPI_DRELU) {
       uint16_t* crow = reinterpret_cast<uint16_t*>(args.C) + row * args.ldc + col0;
@@ -183,12 +180,29 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
       }
     }
         };
+  // Two register buffers: the TMEM load of the next 32 columns is in flight while this one is converted.
+  uint32_t va[32], vb[32];
+  tmem_ld_32x32b_x32(taddr, va);
   if (kEpi == EPI_DRELU_T) {
 #pragma unroll
-    for (int ch = 0; ch < BN / 32; ++ch) chunk(ch, ax[kEpi == EPI_DRELU_T ? ch : 0]);
+    for (int ch = 0; ch < BN / 32; ch += 2) {
+      tmem_ld_wait_on(va);
+      tmem_ld_32x32b_x32(taddr + (ch + 1) * 32, vb);
+      chunk(ch, ax[kEpi == EPI_DRELU_T ? ch : 0], va);
+      tmem_ld_wait_on(vb);
+      if (ch + 2 < BN / 32) tmem_ld_32x32b_x32(taddr + (ch + 2) * 32, va);
+      chunk(ch + 1, ax[kEpi == EPI_DRELU_T ? ch + 1 : 0], vb);
+    }
   } else {
 #pragma unroll 1
-    for (int ch = 0; ch < BN / 32; ++ch) chunk(ch, ax[0]);
+    for (int ch = 0; ch < BN / 32; ch += 2) {
+      tmem_ld_wait_on(va);
+      tmem_ld_32x32b_x32(taddr + (ch + 1) * 32, vb);
+      chunk(ch, ax[0], va);
+      tmem_ld_wait_on(vb);
+      if (ch + 2 < BN / 32) tmem_ld_32x32b_x32(taddr + (ch + 2) * 32, va);
+      chunk(ch + 1, ax[0], vb);
+    }
   }
 }
 
