@@ -92,6 +92,15 @@ def _oracle_step(X, W1, W2, dY, V, M):
 
 
 def _cpu_threads():
+    """Threads the oracle's float64 products run on (numpy's BLAS pool); its element-wise parts
+    (selection, rounding) are single-threaded numpy."""
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
     try:
         return len(os.sched_getaffinity(0))
     except Exception:

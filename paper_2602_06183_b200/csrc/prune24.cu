@@ -12,34 +12,8 @@ namespace sf {
 
 namespace {
 
-// Selection for one group given the four raw bf16 patterns; returns nibble, writes the two
-// packed output patterns (hard: kept bits; soft: shrunk by the third-ranked magnitude).
-template <bool kSoft>
-__device__ __forceinline__ uint32_t prune_group(uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                                uint32_t& o0, uint32_t& o1) {
-  const uint32_t a[4] = {a0, a1, a2, a3};
-  uint32_t third;
-  const uint32_t nib = top2of4(a0 & 0x7FFFu, a1 & 0x7FFFu, a2 & 0x7FFFu, a3 & 0x7FFFu, &third);
-  const uint32_t p0 = nib & 3u, p1 = nib >> 2;
-  // register-only selects (no dynamic indexing into local memory)
-  uint32_t v0 = p0 == 0 ? a[0] : p0 == 1 ? a[1] : a[2];
-  uint32_t v1 = p1 == 1 ? a[1] : p1 == 2 ? a[2] : a[3];
-  if (kSoft) {
-    const uint32_t tk = (third == 0 ? a[0] : third == 1 ? a[1] : third == 2 ? a[2] : a[3]) & 0x7FFFu;
-    const float t = bf16_bits_to_float(tk);
-    const float f0 = bf16_bits_to_float(v0), f1 = bf16_bits_to_float(v1);
-    const float s0 = f0 > 0.f ? __fsub_rn(f0, t) : (f0 < 0.f ? __fadd_rn(f0, t) : 0.f);
-    const float s1 = f1 > 0.f ? __fsub_rn(f1, t) : (f1 < 0.f ? __fadd_rn(f1, t) : 0.f);
-    v0 = float_to_bf16_bits(s0);
-    v1 = float_to_bf16_bits(s1);
-  }
-  o0 = v0;
-  o1 = v1;
-  return nib;
-}
-
-// Packed variant for the row kernel: lo/hi hold the group's four patterns; returns the nibble and
-// the two kept (hard) or shrunk (soft) values packed into one word.
+// Selection for one group: lo/hi hold the group's four bf16 patterns; returns the nibble and the two
+// kept (hard) or shrunk by the third-ranked magnitude (soft) values packed into one word.
 template <bool kSoft>
 __device__ __forceinline__ uint32_t prune_group_packed(uint32_t lo, uint32_t hi, uint32_t& packed) {
   uint32_t third;

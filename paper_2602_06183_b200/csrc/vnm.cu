@@ -14,9 +14,10 @@ namespace sf {
 
 namespace {
 
-constexpr int kCW = 256;          // columns per CTA strip
+constexpr int kCW = 256;          // columns per CTA strip (>= 4 groups of the widest M)
 constexpr int kPad = 8;           // 16 B row padding (bank spread)
 constexpr int kThreads = 256;
+static_assert(kThreads >= kCW && kThreads % (kCW / 8) == 0, "one thread per strip column in the ranking steps");
 
 __device__ __forceinline__ void sqrelu_bits(uint32_t x, bool apply, uint32_t& h, uint32_t& relu) {
   if (!apply) { h = x; relu = 0; return; }
@@ -76,7 +77,8 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
   __syncthreads();
 
   // ---- pass A: column scores (sequential float32 adds, rows in ascending order)
-  {
+  // (the strip is kCW columns wide; threads beyond it only help with loads, pass B and stores)
+  if (tid < kCW) {
     const int j = tid;
     float s = 0.f;
     if (j < cvalid) {
@@ -89,7 +91,7 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
     score[j] = __float_as_uint(s);
   }
   __syncthreads();
-  {
+  if (tid < kCW) {
     const int j = tid, jm = j % M, base = j - jm;
     const uint32_t s = score[j];
     int rank = 0;
@@ -100,7 +102,7 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
     keepf[j] = rank < 4;
   }
   __syncthreads();
-  {
+  if (tid < kCW) {
     const int j = tid, jm = j % M, base = j - jm;
     if (keepf[j] && j < cvalid) {
       int pos = 0;
@@ -217,7 +219,7 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
     score[2 * tid + 1] = __float_as_uint(s1);
   }
   __syncthreads();
-  {
+  if (tid < kCW) {
     const int j = tid, jm = j & 7, base = j - jm;
     const uint32_t s = score[j];
     int rank = 0;
@@ -229,7 +231,7 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
     keepf[j] = rank < 4;
   }
   __syncthreads();
-  {
+  if (tid < kCW) {
     const int j = tid, jm = j & 7, base = j - jm;
     if (keepf[j] && j < cvalid) {
       int pos = 0;
@@ -245,10 +247,11 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
   }
 
   // pass B: a thread serves one group g = tid % ng for rows tid / ng, tid / ng + kThreads / ng, ...
-  const int g = tid % ng, rstep = kThreads / ng;
+  // Everything that depends only on (thread, group) is computed once; the row loop advances
+  // pointers by constant strides.
+  const int g = tid % ng, rstep = kThreads / ng, r0 = tid / ng;
   const int64_t g0 = c0 / M;
   const uint32_t c4 = *reinterpret_cast<const uint32_t*>(cidx + g * 4);
-  // per-thread constants: permute selectors / half masks that pick the kept columns out of a group
   uint32_t selp[2], mhi[2];
 #pragma unroll
   for (int pr = 0; pr < 2; ++pr) {
@@ -257,9 +260,26 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
     selp[pr] = sa | ((sa + 1u) << 4) | (sb << 8) | ((sb + 1u) << 12);
     mhi[pr] = ((ca & 4u) ? 0x0000FFFFu : 0u) | ((cb & 4u) ? 0xFFFF0000u : 0u);   // take from columns 4..7
   }
-  const bool lead = (g & 3) == 0;
-  for (int r = tid / ng; r < V; r += rstep) {
-    const uint4 q = *reinterpret_cast<const uint4*>(tile + r * kRow + g * M);
+  const bool lead4 = (g & 3) == 0, lead2 = (g & 1) == 0;
+  const bool want_relu = relu_vals && apply, want24 = vals24 != nullptr;
+  const int64_t trow = t0 + r0;
+  const uint16_t* tp = tile + r0 * kRow + g * M;
+  uint16_t* p_vals = vals + trow * (2 * G) + 2 * (g0 + g);
+  uint16_t* p_relu = want_relu ? relu_vals + trow * (2 * G) + 2 * (g0 + g) : nullptr;
+  uint16_t* p_dense = dense_out ? dense_out + trow * F + c0 + g * M : nullptr;
+  uint16_t* p_rdense = relu_dense_out ? relu_dense_out + trow * F + c0 + g * M : nullptr;
+  uint16_t* p_v24 = want24 ? vals24 + trow * (F >> 1) + (g0 + g) * 4 : nullptr;
+  uint16_t* p_meta = meta + trow * (G >> 2) + ((g0 + g) >> 2);
+  uint16_t* p_m24 = want24 ? meta24 + trow * (F >> 4) + ((g0 + g) >> 1) : nullptr;
+  // tensor-core-ordered copies: rows of one strip share their 128-row block, so the atom is fixed
+  const int64_t kw = (g0 + g) >> 2, kw24 = (g0 + g) >> 1;
+  uint8_t* hw_atom = meta_hw ? meta_hw + meta_hw_offset(t0 & ~int64_t(127), kw, 4 * G) : nullptr;
+  uint8_t* hw24_atom = want24 ? meta24_hw + meta_hw_offset(t0 & ~int64_t(127), kw24, F) : nullptr;
+  const int s_vals = rstep * (int)(2 * G), s_dense = rstep * (int)F, s_v24 = rstep * (int)(F >> 1);
+  const int s_meta = rstep * (int)(G >> 2), s_m24 = rstep * (int)(F >> 4);
+  const bool any_dense = dense_out || relu_dense_out;
+  for (int r = r0; r < V; r += rstep) {
+    const uint4 q = *reinterpret_cast<const uint4*>(tp);
     uint32_t rw[4] = {q.x, q.y, q.z, q.w}, hw[4];
     if (apply) {
 #pragma unroll
@@ -269,69 +289,72 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
       for (int j = 0; j < 4; ++j) hw[j] = rw[j];
     }
     // kept columns c0 < c1 | c2 < c3 as two packed pairs
-    uint32_t hk[2], rk[2];
-#pragma unroll
-    for (int pr = 0; pr < 2; ++pr) {
-      const uint32_t a = __byte_perm(hw[0], hw[1], selp[pr]), b = __byte_perm(hw[2], hw[3], selp[pr]);
-      hk[pr] = (a & ~mhi[pr]) | (b & mhi[pr]);
-      const uint32_t ra = __byte_perm(rw[0], rw[1], selp[pr]), rb = __byte_perm(rw[2], rw[3], selp[pr]);
-      rk[pr] = (ra & ~mhi[pr]) | (rb & mhi[pr]);
-    }
+    const uint32_t a0 = __byte_perm(hw[0], hw[1], selp[0]), b0 = __byte_perm(hw[2], hw[3], selp[0]);
+    const uint32_t a1 = __byte_perm(hw[0], hw[1], selp[1]), b1 = __byte_perm(hw[2], hw[3], selp[1]);
+    const uint32_t hk0 = (a0 & ~mhi[0]) | (b0 & mhi[0]), hk1 = (a1 & ~mhi[1]) | (b1 & mhi[1]);
     uint32_t packed;
-    const uint32_t nib = top2of4_packed(hk[0], hk[1], &packed);
+    const uint32_t nib = top2of4_packed(hk0, hk1, &packed);
     const uint32_t p0 = nib & 3u, p1 = nib >> 2;
-    const int64_t t = t0 + r;
-    *reinterpret_cast<uint32_t*>(vals + t * (2 * G) + 2 * (g0 + g)) = packed;
-    if (relu_vals && apply)
-      *reinterpret_cast<uint32_t*>(relu_vals + t * (2 * G) + 2 * (g0 + g)) =
-          __byte_perm(rk[0], rk[1], 0x1010u + p0 * 0x22u + p1 * 0x2200u);
-    if (dense_out || relu_dense_out) {
-      const uint32_t kb = (1u << ((c4 >> (8 * p0)) & 0xFFu)) | (1u << ((c4 >> (8 * p1)) & 0xFFu));
+    *reinterpret_cast<uint32_t*>(p_vals) = packed;
+    const uint32_t ca = (c4 >> (8 * p0)) & 0xFFu, cb = (c4 >> (8 * p1)) & 0xFFu;         // kept columns, ca < cb
+    if (want_relu) {
+      // the two kept ReLU values straight from the group's words (columns ca, cb)
+      const uint32_t sel = 2u * (ca & 3u) | ((2u * (ca & 3u) + 1u) << 4) | ((2u * (cb & 3u)) << 8) | ((2u * (cb & 3u) + 1u) << 12);
+      const uint32_t ra = __byte_perm(rw[0], rw[1], sel), rb = __byte_perm(rw[2], rw[3], sel);
+      const uint32_t mh = ((ca & 4u) ? 0x0000FFFFu : 0u) | ((cb & 4u) ? 0xFFFF0000u : 0u);
+      *reinterpret_cast<uint32_t*>(p_relu) = (ra & ~mh) | (rb & mh);
+    }
+    if (any_dense) {
+      const uint32_t kb = (1u << ca) | (1u << cb);
       uint32_t mk[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j)
         mk[j] = (((kb >> (2 * j)) & 1u) * 0xFFFFu) | (((kb >> (2 * j + 1)) & 1u) * 0xFFFF0000u);
-      if (dense_out)
-        *reinterpret_cast<uint4*>(dense_out + t * F + c0 + g * M) =
-            make_uint4(hw[0] & mk[0], hw[1] & mk[1], hw[2] & mk[2], hw[3] & mk[3]);
-      if (relu_dense_out)
-        *reinterpret_cast<uint4*>(relu_dense_out + t * F + c0 + g * M) =
-            make_uint4(rw[0] & mk[0], rw[1] & mk[1], rw[2] & mk[2], rw[3] & mk[3]);
+      if (dense_out) *reinterpret_cast<uint4*>(p_dense) = make_uint4(hw[0] & mk[0], hw[1] & mk[1], hw[2] & mk[2], hw[3] & mk[3]);
+      if (relu_dense_out) *reinterpret_cast<uint4*>(p_rdense) = make_uint4(rw[0] & mk[0], rw[1] & mk[1], rw[2] & mk[2], rw[3] & mk[3]);
     }
     uint32_t word = nib;
     word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 4;
     word |= __shfl_down_sync(0xFFFFFFFFu, word, 2) << 8;
-    if (lead) {
-      const int64_t kw = (g0 + g) >> 2;
-      meta[t * (G >> 2) + kw] = (uint16_t)word;
-      if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(t, kw, 4 * G)) = (uint16_t)word;
+    // offset of row r's word inside a metadata atom (r < 128)
+    const uint32_t hw_row = (uint32_t)(((t0 + r) & 127) >> 4) * 256u + (uint32_t)((t0 + r) & 7) * 16u +
+                            (uint32_t)(((t0 + r) >> 3) & 1) * 2u;
+    if (lead4) {
+      *p_meta = (uint16_t)word;
+      if (hw_atom) *reinterpret_cast<uint16_t*>(hw_atom + hw_row) = (uint16_t)word;
     }
     // The same row as a plain 2:4 operand over all F columns: two values per eight columns always
     // satisfy "at most two per four", so each half-group stores its kept values (or zeros) and a
     // legal position pair. A half-group with one kept value at position p pairs it with a zero
     // at position 1 (p = 0) or 0 (p > 0).
-    if (vals24) {
-      const uint32_t ca = (c4 >> (8 * p0)) & 0xFFu, cb = (c4 >> (8 * p1)) & 0xFFu;     // kept columns, ca < cb
+    if (want24) {
       const uint32_t va = packed & 0xFFFFu, vb = packed >> 16;
-      uint32_t wlo, whi, nlo, nhi;
-      if (cb < 4u) {
-        wlo = packed; nlo = ca | (cb << 2); whi = 0u; nhi = 4u;
-      } else if (ca >= 4u) {
-        wlo = 0u; nlo = 4u; whi = packed; nhi = (ca - 4u) | ((cb - 4u) << 2);
-      } else {
-        const uint32_t pb = cb - 4u;
-        wlo = ca == 0u ? va : (va << 16); nlo = ca == 0u ? 4u : (ca << 2);
-        whi = pb == 0u ? vb : (vb << 16); nhi = pb == 0u ? 4u : (pb << 2);
-      }
-      *reinterpret_cast<uint2*>(vals24 + t * (F >> 1) + (g0 + g) * 4) = make_uint2(wlo, whi);
+      const bool both_lo = cb < 4u, both_hi = ca >= 4u;
+      const uint32_t pb = cb & 3u, pa = ca & 3u;
+      // split case values / nibbles
+      const uint32_t s_wlo = pa == 0u ? va : (va << 16), s_nlo = pa == 0u ? 4u : (pa << 2);
+      const uint32_t s_whi = pb == 0u ? vb : (vb << 16), s_nhi = pb == 0u ? 4u : (pb << 2);
+      const uint32_t pair_nib = pa | (pb << 2);
+      const uint32_t wlo = both_lo ? packed : (both_hi ? 0u : s_wlo);
+      const uint32_t whi = both_hi ? packed : (both_lo ? 0u : s_whi);
+      const uint32_t nlo = both_lo ? pair_nib : (both_hi ? 4u : s_nlo);
+      const uint32_t nhi = both_hi ? pair_nib : (both_lo ? 4u : s_nhi);
+      *reinterpret_cast<uint2*>(p_v24) = make_uint2(wlo, whi);
       uint32_t mb = nlo | (nhi << 4);
       mb |= __shfl_down_sync(0xFFFFFFFFu, mb, 1) << 8;
-      if ((g & 1) == 0) {
-        const int64_t kw24 = (g0 + g) >> 1;
-        meta24[t * (F >> 4) + kw24] = (uint16_t)mb;
-        *reinterpret_cast<uint16_t*>(meta24_hw + meta_hw_offset(t, kw24, F)) = (uint16_t)mb;
+      if (lead2) {
+        *p_m24 = (uint16_t)mb;
+        *reinterpret_cast<uint16_t*>(hw24_atom + hw_row) = (uint16_t)mb;
       }
+      p_v24 += s_v24;
+      p_m24 += s_m24;
     }
+    tp += rstep * kRow;
+    p_vals += s_vals;
+    if (want_relu) p_relu += s_vals;
+    if (dense_out) p_dense += s_dense;
+    if (relu_dense_out) p_rdense += s_dense;
+    p_meta += s_meta;
   }
 }
 
