@@ -89,9 +89,15 @@ def gemm_sweep():
                           "sparse24_ms": ms_s, "sparse24_dense_equiv_tflops": fl / ms_s / 1e9,
                           "prune_ms": ms_p, "speedup_gemm_only": ms_d / ms_s,
                           "speedup_with_prune": ms_d / (ms_s + ms_p)}))
-    # Venom (condensed, gathered) vs the same V:N:M operand as plain 2:4, M = 8 and 16
+    # Venom (condensed operand, gathered B rows) at the sparsities of Table 5 and below
     T, F, N = 8192, 16384, 4096
-    for M in (8, 16):
+    A = torch.randn((T, F), device="cuda").to(torch.bfloat16)
+    Bd = torch.randn((N, F), device="cuda").to(torch.bfloat16)
+    Cd = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    wsd = torch.zeros((binding.sf_gemm_workspace_size(T, F),), dtype=torch.uint8, device="cuda")
+    ms_dense = _time(lambda: binding.sf_gemm_dense(A, True, Bd, True, C_out=Cd, workspace=wsd))
+    del A, Bd, Cd
+    for M in (8, 16, 32, 64):
         G = F // M
         P = _dev(synth.normal_bf16((T, F), 0.0, 1.0, seed=7))
         vals, meta, colidx, _, _ = binding.sf_vnm_sparsify_act(P, 128, M)
@@ -99,8 +105,9 @@ def gemm_sweep():
         C = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
         ws = torch.zeros((binding.sf_gemm_workspace_size(T, F),), dtype=torch.uint8, device="cuda")
         ms_v = _time(lambda: binding.sf_gemm_venom(vals, meta, colidx, Bt, 128, M, C_out=C, workspace=ws))
-        print(json.dumps({"kernel": "gemm_venom", "T": T, "F": F, "N": N, "V": 128, "M": M, "ms": ms_v,
-                          "dense_equiv_tflops": 2.0 * T * F * N / ms_v / 1e9}))
+        print(json.dumps({"kernel": "gemm_venom", "T": T, "F": F, "N": N, "V": 128, "M": M,
+                          "sparsity_pct": 100.0 * (1 - 2.0 / M), "ms": ms_v, "dense_ms": ms_dense,
+                          "speedup_vs_dense": ms_dense / ms_v, "dense_equiv_tflops": 2.0 * T * F * N / ms_v / 1e9}))
 
 
 def c5_step():

@@ -79,6 +79,20 @@ def test_sparse_ffn_v128_m16():
         assert rel_fro(g[k], ref) < TOL, k
 
 
+@pytest.mark.parametrize("V,M", [(64, 4), (128, 32)])
+def test_sparse_ffn_other_group_widths(V, M):
+    """M = 4 is 2:4 activation sparsity (every column kept, the plain-2:4 path); M = 32 runs the
+    condensed, gathered Venom product."""
+    cfg = dict(T=512, D=256, F=2048, V=V, N=2, M=M, sigma_w=0.05, seed=23 + M)
+    (X, W1, W2, dY), g = _run_sparse(cfg)
+    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, forced_y1b=g["y1"])
+    assert np.array_equal(g["colidx"], fwd.act.colidx) and np.array_equal(g["meta"], fwd.act.meta)
+    assert np.array_equal(g["y2_vals"], fwd.act.vals)
+    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd)
+    for k, ref in (("Y", fwd.y3), ("dX", bwd.dX), ("dW1", bwd.dW1), ("dW2", bwd.dW2)):
+        assert rel_fro(g[k], ref) < TOL, k
+
+
 def test_dense_ffn_c1():
     cfg = synth.FFN_CONFIGS["c1_small"]
     T, D, F = cfg["T"], cfg["D"], cfg["F"]
