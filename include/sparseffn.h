@@ -170,7 +170,10 @@ SF_API int sf_gemm_sparse24_noalloc(const void* a_vals, const void* a_meta, cons
  *
  * sf_sparse_ffn_fwd:  W1s = prune24(W1 along D);  y1 = X W1s^T;  y2 = V:N:M(ReLU(y1)^2);
  *                     Y = y2 W2^T  (W2 dense).  Saves packed y2, packed ReLU(y1), metadata,
- *                     column indices (and y1 if flags bit0) in fwd_ctx.
+ *                     column indices (and y1 if flags bit0) in fwd_ctx. For M <= 8 the product
+ *                     consumes y2 as a plain 2:4 operand over all F columns (identical result,
+ *                     no row gather); for M >= 16 it consumes the condensed V:N:M operand and
+ *                     gathers the kept rows of W2^T.
  * sf_sparse_ffn_bwd:  W2s = prune24(W2 along D);  dy2 = dY W2s;  dy1 = 2 dy2 ReLU(y1) on y2's
  *                     mask;  dX = dy1 W1 (W1 dense);  dW1 = dy1^T X [F,D];  dW2 = dY^T y2 [D,F].
  * sf_dense_ffn_fwd/bwd: the same equations with no pruning; fwd_ctx holds y1 (bf16 [T,F]).
@@ -194,7 +197,9 @@ typedef enum sf_ctx_field {
   SF_CTX_META = 2,      /* uint16 [T, F/(4M)] canonical */
   SF_CTX_COLIDX = 3,    /* uint8 [T/V, F/M, 4] */
   SF_CTX_Y1 = 4,        /* bf16 [T, F] (only with flags bit0) */
-  SF_CTX_DY1_VALS = 5   /* bf16 [T, 2F/M], lives in the WORKSPACE after sf_sparse_ffn_bwd */
+  SF_CTX_DY1_VALS = 5   /* bf16 [T, 2F/M], lives in the WORKSPACE after sf_sparse_ffn_bwd; for M == 8 it
+                           is only written when flags bit0 is set (the products then consume dy1 in
+                           its 2:4 form over all F columns instead) */
 } sf_ctx_field;
 SF_API int sf_ctx_view(const sf_ffn_desc* desc, const void* fwd_ctx_or_workspace, int field,
                 const void** ptr, size_t* bytes);

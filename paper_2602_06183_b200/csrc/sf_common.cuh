@@ -88,7 +88,7 @@ __device__ __forceinline__ uint32_t top2of4_packed(uint32_t lo, uint32_t hi, uin
 
 // ---- internal launchers (defined in the .cu files) ---------------------------------------
 // meta_hw (optional) receives the same metadata words in the order the sparse tensor-core
-// instruction reads them (see gemm_sparse.cu); requires R % 128 == 0 and K % 128 == 0.
+// instruction reads them (see meta_hw_offset below); requires R % 128 == 0 and K % 128 == 0.
 int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int group_dim, int prune_mode,
                    void* vals, void* meta, void* meta_hw, void* dense_out, cudaStream_t s);
 int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
