@@ -135,6 +135,40 @@ def test_step_from_host_buffers_matches_device_path():
     assert np.array_equal(as_f32(hdW1), g["dW1"]) and np.array_equal(as_f32(hdW2), g["dW2"])
 
 
+def test_sparse_step_replays_from_a_cuda_graph():
+    """The step enqueues kernels only (no allocation, no synchronisation), so it can be captured
+    once and replayed; the replay must reproduce the eager results bit for bit."""
+    cfg = synth.FFN_CONFIGS["c1_small"]
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
+    desc = binding.make_desc(T, D, F, V, M)
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
+    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+    gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
+
+    def step():
+        binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
+        binding.sf_sparse_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+
+    step()                                          # eager run (also does the one-time kernel set-up)
+    torch.cuda.synchronize()
+    eager = [t.clone() for t in (Y, gX, gW1, gW2)]
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    for t in (Y, gX, gW1, gW2):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    for a, b in zip(eager, (Y, gX, gW1, gW2)):
+        assert torch.equal(a, b)
+
+
 def test_ffn_rejects_ragged_shapes():
     desc = binding.make_desc(1000, 256, 1024, 64, 8)
     with pytest.raises(binding.SparseFFNError) as e:
