@@ -33,6 +33,8 @@ FFN_CONFIGS = {
     # one eighth of c4's tokens with the full-size layer: weights (134 MB each) still exceed the
     # L2, device footprint ~1.5 GB; used for profiler captures that must stay small
     "c4_slice": dict(T=1024, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
+    # the same slice with groups of 16 (87.5 % sparse activations): exercises the condensed Venom products
+    "c4_slice_m16": dict(T=1024, D=4096, F=16384, V=128, N=2, M=16, sigma_w=0.02, seed=4),
     "c5_d8192": dict(T=16384, D=8192, F=28672, V=128, N=2, M=8, sigma_w=0.015, seed=5),
 }
 
