@@ -93,6 +93,21 @@ def test_sparse_ffn_other_group_widths(V, M):
         assert rel_fro(g[k], ref) < TOL, k
 
 
+@pytest.mark.parametrize("T,D,F,V,M", [(256, 256, 256, 128, 8), (256, 256, 256, 64, 8), (512, 512, 512, 128, 16),
+                                       (768, 256, 1280, 128, 8)])
+def test_sparse_ffn_smallest_and_odd_tile_counts(T, D, F, V, M):
+    """One tile per product, fewer k-blocks than pipeline stages, tile counts that are not a
+    multiple of the raster band."""
+    cfg = dict(T=T, D=D, F=F, V=V, N=2, M=M, sigma_w=0.05, seed=T + F + V)
+    (X, W1, W2, dY), g = _run_sparse(cfg)
+    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, forced_y1b=g["y1"])
+    assert np.array_equal(g["colidx"], fwd.act.colidx) and np.array_equal(g["meta"], fwd.act.meta)
+    assert np.array_equal(g["y2_vals"], fwd.act.vals)
+    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd)
+    for k, ref in (("Y", fwd.y3), ("dX", bwd.dX), ("dW1", bwd.dW1), ("dW2", bwd.dW2)):
+        assert rel_fro(g[k], ref) < TOL, k
+
+
 def test_dense_ffn_c1():
     cfg = synth.FFN_CONFIGS["c1_small"]
     T, D, F = cfg["T"], cfg["D"], cfg["F"]
