@@ -268,8 +268,10 @@ def run_ours(args, cfg):
 
     # ---- end to end through the host-buffer entry point (H2D of inputs and D2H of results timed)
     staging = torch.empty((binding.sf_ffn_host_staging_size(desc),), dtype=torch.uint8, device="cuda")
-    hY, hdX = torch.empty_like(hX), torch.empty_like(hX)
-    hgW1, hgW2 = torch.empty_like(hW1), torch.empty_like(hW2)
+    # (empty_like of a pinned tensor is pageable: ask for pinned results explicitly)
+    hY, hdX = torch.empty_like(hX, pin_memory=True), torch.empty_like(hX, pin_memory=True)
+    hgW1, hgW2 = torch.empty_like(hW1, pin_memory=True), torch.empty_like(hW2, pin_memory=True)
+    assert all(t.is_pinned() for t in (hX, hW1, hW2, hdY, hY, hdX, hgW1, hgW2))
 
     def host_step():
         binding.sf_ffn_step_host(desc, False, hX, hW1, hW2, hdY, hY, hdX, hgW1, hgW2, staging, ctx, ws)

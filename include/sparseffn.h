@@ -204,10 +204,17 @@ typedef enum sf_ctx_field {
 SF_API int sf_ctx_view(const sf_ffn_desc* desc, const void* fwd_ctx_or_workspace, int field,
                 const void** ptr, size_t* bytes);
 
-/* One whole training step from HOST buffers (pinned memory recommended): copies X, W1, W2, dY
- * to the device staging area inside `workspace`, runs sf_sparse_ffn_fwd + sf_sparse_ffn_bwd
- * (dense != 0: the dense pair), copies Y, dX, dW1, dW2 back, all on `stream`. Does not
- * synchronise. host_* pointers are HOST pointers; `device_staging` is a DEVICE buffer of
+/* One whole training step from HOST buffers (pinned memory is needed for the copies to overlap):
+ * uploads X, W1, W2, dY into `device_staging`, runs sf_sparse_ffn_fwd + sf_sparse_ffn_bwd
+ * (dense != 0: the dense pair) on `stream`, and downloads Y, dX, dW2, dW1. Uploads run on a
+ * library-owned copy stream in the order X, W1, W2, dY, and each kernel waits only for the
+ * operands it reads (the W1 prune and the y1 product start while W2 and dY are still in flight);
+ * downloads run on a second copy stream, each as soon as its product is complete. Work already
+ * on `stream` is ordered before the first upload, and `stream` is complete only after the last
+ * download, so a cudaStreamSynchronize(stream) covers the whole step. Does not synchronise the
+ * host. The two copy streams and nine events are created once per device on the first call (make
+ * that call before any stream capture); calls on one device must not overlap on the host.
+ * host_* pointers are HOST pointers; `device_staging` is a DEVICE buffer of
  * sf_ffn_host_staging_size() bytes. */
 SF_API int sf_ffn_host_staging_size(const sf_ffn_desc* desc, size_t* bytes);
 SF_API int sf_ffn_step_host(const sf_ffn_desc* desc, int dense, const void* host_X, const void* host_W1,

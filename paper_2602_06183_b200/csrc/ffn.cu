@@ -1,6 +1,7 @@
 // Step orchestration (Algorithms 1 and 2; Eqs. 1-8 for the dense phase) and the product entry
 // points of the C ABI. Everything is enqueued on the caller's stream; buffers are carved out of
-// the caller's context / workspace; nothing is allocated here.
+// the caller's context / workspace; no device memory is allocated here. (The host-buffer step
+// additionally owns two copy streams and a few events per device, created on first use.)
 #include "sf_common.cuh"
 #include "gemm_tc.cuh"
 
@@ -21,6 +22,51 @@ int g_trace_cap = 0, g_trace_n = 0;
 
 inline void trace_mark(cudaStream_t s) {
   if (g_trace_events && g_trace_n < g_trace_cap) cudaEventRecord(g_trace_events[g_trace_n++], s);
+}
+
+// Copy/compute overlap of the host-buffer step: while sf_ffn_step_host runs, the step functions wait
+// for an operand's upload right before its first use and signal a result as soon as its product is
+// enqueued. Null outside sf_ffn_step_host.
+struct StepHooks {
+  cudaEvent_t w2_ready;      // forward: waited before the first kernel that reads W2
+  cudaEvent_t dx_done;       // backward: recorded after the dX product
+  cudaEvent_t dw2_done;      // backward: recorded after the dW2 product
+};
+const StepHooks* g_hooks = nullptr;
+
+inline void hook_wait_w2(cudaStream_t s) {
+  if (g_hooks) cudaStreamWaitEvent(s, g_hooks->w2_ready, 0);
+}
+inline void hook_dx_done(cudaStream_t s) {
+  if (g_hooks) cudaEventRecord(g_hooks->dx_done, s);
+}
+inline void hook_dw2_done(cudaStream_t s) {
+  if (g_hooks) cudaEventRecord(g_hooks->dw2_done, s);
+}
+
+// Per-device copy streams and events of the host-buffer step, created on first use.
+struct HostStepResources {
+  bool ready = false;
+  cudaStream_t up = nullptr, down = nullptr;
+  cudaEvent_t begin, xw1, w2, dy, y, dx, dw2, dw1, done;
+};
+constexpr int kMaxDevices = 64;
+HostStepResources g_host_step[kMaxDevices];
+
+int host_step_resources(HostStepResources** out) {
+  int dev = 0;
+  SF_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return SF_ERR_UNSUPPORTED;
+  HostStepResources& r = g_host_step[dev];
+  if (!r.ready) {
+    SF_CUDA_TRY(cudaStreamCreateWithFlags(&r.up, cudaStreamNonBlocking));
+    SF_CUDA_TRY(cudaStreamCreateWithFlags(&r.down, cudaStreamNonBlocking));
+    for (cudaEvent_t* e : {&r.begin, &r.xw1, &r.w2, &r.dy, &r.y, &r.dx, &r.dw2, &r.dw1, &r.done})
+      SF_CUDA_TRY(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+    r.ready = true;
+  }
+  *out = &r;
+  return SF_OK;
 }
 
 // ---- small helper kernels -------------------------------------------------------------------
@@ -280,6 +326,7 @@ int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, co
                     emit24 ? at(fwd_ctx, L.meta24) : nullptr, emit24 ? at(fwd_ctx, L.meta24_hw) : nullptr, s));
   trace_mark(s);
   // line 7: y3 = y2 W2^T with W2 dense
+  hook_wait_w2(s);
   if (L.plain24) {
     // y2 as a 2:4 operand over all F columns against W2 [D, F] as it is stored (no transpose, no gather)
     trace_mark(s);
@@ -340,10 +387,12 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
                       d.V, d.M, dX, d.D, status, s));
   }
   trace_mark(s);
+  hook_dx_done(s);
   // line 3: dW2 = dY^T y2 [D, F];  line 6: dW1 = dy1^T X [F, D]  (reduction over tokens)
   SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.y2_dense), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0,
                     nullptr, 0, status, s));
   trace_mark(s);
+  hook_dw2_done(s);
   SF_TRY(gemm_dense(at(workspace, L.dy1_dense), false, X, false, d.F, d.D, d.T, EPI_STORE, dW1, d.D, nullptr, 0,
                     nullptr, 0, status, s));
   trace_mark(s);
@@ -364,6 +413,7 @@ int sf_dense_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, con
   SF_TRY(gemm_dense(X, true, W1, true, d.T, d.F, d.D, EPI_SQRELU, at(fwd_ctx, L.y1), d.F, at(fwd_ctx, L.h), d.F,
                     nullptr, 0, status, s));
   trace_mark(s);
+  hook_wait_w2(s);
   SF_TRY(gemm_dense(at(fwd_ctx, L.h), true, W2, true, d.T, d.D, d.F, EPI_STORE, Y, d.D, nullptr, 0, nullptr, 0,
                     status, s));
   trace_mark(s);
@@ -388,10 +438,12 @@ int sf_dense_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, con
   // Eq. 7: dX = dy1 W1
   SF_TRY(gemm_dense(dy1, true, W1, false, d.T, d.D, d.F, EPI_STORE, dX, d.D, nullptr, 0, nullptr, 0, status, s));
   trace_mark(s);
+  hook_dx_done(s);
   // Eq. 5: dW2 = dY^T h [D, F];  Eq. 8: dW1 = dy1^T X [F, D]
   SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.h), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0, nullptr, 0,
                     status, s));
   trace_mark(s);
+  hook_dw2_done(s);
   SF_TRY(gemm_dense(dy1, false, X, false, d.F, d.D, d.T, EPI_STORE, dW1, d.D, nullptr, 0, nullptr, 0, status, s));
   trace_mark(s);
   return SF_OK;
@@ -444,21 +496,53 @@ int sf_ffn_step_host(const sf_ffn_desc* desc, int dense, const void* host_X, con
   void *dW1in = base + 4 * act, *dW2in = base + 4 * act + wgt, *ddW1 = base + 4 * act + 2 * wgt,
        *ddW2 = base + 4 * act + 3 * wgt;
   cudaStream_t s = (cudaStream_t)stream;
-  SF_CUDA_TRY(cudaMemcpyAsync(dXin, host_X, T * D * 2, cudaMemcpyHostToDevice, s));
-  SF_CUDA_TRY(cudaMemcpyAsync(dW1in, host_W1, F * D * 2, cudaMemcpyHostToDevice, s));
-  SF_CUDA_TRY(cudaMemcpyAsync(dW2in, host_W2, F * D * 2, cudaMemcpyHostToDevice, s));
-  SF_CUDA_TRY(cudaMemcpyAsync(ddY, host_dY, T * D * 2, cudaMemcpyHostToDevice, s));
-  if (dense) {
-    SF_TRY(sf_dense_ffn_fwd(desc, dXin, dW1in, dW2in, dYout, fwd_ctx, workspace, stream));
-    SF_TRY(sf_dense_ffn_bwd(desc, ddY, dXin, dW1in, dW2in, fwd_ctx, ddX, ddW1, ddW2, workspace, stream));
-  } else {
-    SF_TRY(sf_sparse_ffn_fwd(desc, dXin, dW1in, dW2in, dYout, fwd_ctx, workspace, stream));
-    SF_TRY(sf_sparse_ffn_bwd(desc, ddY, dXin, dW1in, dW2in, fwd_ctx, ddX, ddW1, ddW2, workspace, stream));
+  HostStepResources* r = nullptr;
+  SF_TRY(host_step_resources(&r));
+  // uploads, in the order the step first needs them, on their own stream behind everything already on `stream`
+  SF_CUDA_TRY(cudaEventRecord(r->begin, s));
+  SF_CUDA_TRY(cudaStreamWaitEvent(r->up, r->begin, 0));
+  SF_CUDA_TRY(cudaMemcpyAsync(dXin, host_X, T * D * 2, cudaMemcpyHostToDevice, r->up));
+  SF_CUDA_TRY(cudaMemcpyAsync(dW1in, host_W1, F * D * 2, cudaMemcpyHostToDevice, r->up));
+  SF_CUDA_TRY(cudaEventRecord(r->xw1, r->up));
+  SF_CUDA_TRY(cudaMemcpyAsync(dW2in, host_W2, F * D * 2, cudaMemcpyHostToDevice, r->up));
+  SF_CUDA_TRY(cudaEventRecord(r->w2, r->up));
+  SF_CUDA_TRY(cudaMemcpyAsync(ddY, host_dY, T * D * 2, cudaMemcpyHostToDevice, r->up));
+  SF_CUDA_TRY(cudaEventRecord(r->dy, r->up));
+
+  const StepHooks hooks{r->w2, r->dx, r->dw2};
+  g_hooks = &hooks;
+  int rc = SF_OK;
+  do {
+    if (cudaStreamWaitEvent(s, r->xw1, 0) != cudaSuccess) { rc = SF_ERR_CUDA; break; }
+    rc = dense ? sf_dense_ffn_fwd(desc, dXin, dW1in, dW2in, dYout, fwd_ctx, workspace, stream)
+               : sf_sparse_ffn_fwd(desc, dXin, dW1in, dW2in, dYout, fwd_ctx, workspace, stream);
+    if (rc != SF_OK) break;
+    if (cudaEventRecord(r->y, s) != cudaSuccess || cudaStreamWaitEvent(s, r->dy, 0) != cudaSuccess) {
+      rc = SF_ERR_CUDA;
+      break;
+    }
+    rc = dense ? sf_dense_ffn_bwd(desc, ddY, dXin, dW1in, dW2in, fwd_ctx, ddX, ddW1, ddW2, workspace, stream)
+               : sf_sparse_ffn_bwd(desc, ddY, dXin, dW1in, dW2in, fwd_ctx, ddX, ddW1, ddW2, workspace, stream);
+  } while (false);
+  g_hooks = nullptr;
+  // a failure past this point still has to rejoin the upload stream, or a capture of `stream` would dangle
+  if (rc != SF_OK) {
+    cudaStreamWaitEvent(s, r->dy, 0);
+    return rc;
   }
-  SF_CUDA_TRY(cudaMemcpyAsync(host_Y, dYout, T * D * 2, cudaMemcpyDeviceToHost, s));
-  SF_CUDA_TRY(cudaMemcpyAsync(host_dX, ddX, T * D * 2, cudaMemcpyDeviceToHost, s));
-  SF_CUDA_TRY(cudaMemcpyAsync(host_dW1, ddW1, F * D * 2, cudaMemcpyDeviceToHost, s));
-  SF_CUDA_TRY(cudaMemcpyAsync(host_dW2, ddW2, F * D * 2, cudaMemcpyDeviceToHost, s));
+  SF_CUDA_TRY(cudaEventRecord(r->dw1, s));
+  // downloads, each as soon as its product has finished, on a second stream
+  SF_CUDA_TRY(cudaStreamWaitEvent(r->down, r->y, 0));
+  SF_CUDA_TRY(cudaMemcpyAsync(host_Y, dYout, T * D * 2, cudaMemcpyDeviceToHost, r->down));
+  SF_CUDA_TRY(cudaStreamWaitEvent(r->down, r->dx, 0));
+  SF_CUDA_TRY(cudaMemcpyAsync(host_dX, ddX, T * D * 2, cudaMemcpyDeviceToHost, r->down));
+  SF_CUDA_TRY(cudaStreamWaitEvent(r->down, r->dw2, 0));
+  SF_CUDA_TRY(cudaMemcpyAsync(host_dW2, ddW2, F * D * 2, cudaMemcpyDeviceToHost, r->down));
+  SF_CUDA_TRY(cudaStreamWaitEvent(r->down, r->dw1, 0));
+  SF_CUDA_TRY(cudaMemcpyAsync(host_dW1, ddW1, F * D * 2, cudaMemcpyDeviceToHost, r->down));
+  SF_CUDA_TRY(cudaEventRecord(r->done, r->down));
+  // `stream` is complete only when the last download is
+  SF_CUDA_TRY(cudaStreamWaitEvent(s, r->done, 0));
   return SF_OK;
 }
 

@@ -140,14 +140,46 @@ def test_step_from_host_buffers_matches_device_path():
     staging = torch.empty((binding.sf_ffn_host_staging_size(desc),), dtype=torch.uint8, device="cuda")
     pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
     hX, hW1, hW2, hdY = pin(X), pin(W1), pin(W2), pin(dY)
-    hY, hdX = torch.empty_like(hX), torch.empty_like(hX)
-    hdW1, hdW2 = torch.empty_like(hW1), torch.empty_like(hW2)
+    hY, hdX = torch.empty_like(hX, pin_memory=True), torch.empty_like(hX, pin_memory=True)
+    hdW1, hdW2 = torch.empty_like(hW1, pin_memory=True), torch.empty_like(hW2, pin_memory=True)
     binding.sf_ffn_step_host(desc, False, hX, hW1, hW2, hdY, hY, hdX, hdW1, hdW2, staging, ctx, ws)
     assert binding.sf_check_status(ws) == binding.SF_OK
     (_, _, _, _), g = _run_sparse(cfg)
     as_f32 = lambda t: t.view(torch.bfloat16).float().numpy()
     assert np.array_equal(as_f32(hY), g["Y"]) and np.array_equal(as_f32(hdX), g["dX"])
     assert np.array_equal(as_f32(hdW1), g["dW1"]) and np.array_equal(as_f32(hdW2), g["dW2"])
+
+
+@pytest.mark.parametrize("dense", [False, True])
+def test_back_to_back_host_steps_do_not_race(dense):
+    """Uploads and downloads run on the library's own copy streams. Two steps with different inputs
+    that share one staging area, context and workspace, enqueued without a synchronisation between
+    them, must each give the result of running alone: the second step's uploads may not overtake the
+    first step's kernels, and its kernels may not overtake the first step's downloads."""
+    cfg = synth.FFN_CONFIGS["c1_small"]
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    desc = binding.make_desc(T, D, F, V, M)
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    staging = torch.empty((binding.sf_ffn_host_staging_size(desc),), dtype=torch.uint8, device="cuda")
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
+    ins = [tuple(pin(a) for a in synth.ffn_inputs(T, D, F, cfg["sigma_w"], seed)) for seed in (11, 12)]
+    outs = lambda i: tuple(torch.empty_like(i[k], pin_memory=True) for k in (0, 0, 1, 2))   # Y, dX, dW1, dW2
+
+    def run(pairs):
+        for i, o in pairs:
+            binding.sf_ffn_step_host(desc, dense, i[0], i[1], i[2], i[3], o[0], o[1], o[2], o[3], staging, ctx, ws)
+        assert binding.sf_check_status(ws) == binding.SF_OK
+
+    alone = [outs(i) for i in ins]
+    for i, o in zip(ins, alone):
+        run([(i, o)])
+    assert not torch.equal(alone[0][0], alone[1][0])
+    for _ in range(3):
+        together = [outs(i) for i in ins]
+        run(list(zip(ins, together)))
+        for a, b in zip(alone, together):
+            for x, y in zip(a, b):
+                assert torch.equal(x, y)
 
 
 def test_sparse_step_replays_from_a_cuda_graph():
