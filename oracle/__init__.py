@@ -3,7 +3,8 @@
 A plain, slow, numpy implementation of what the hot path computes, written from the paper:
 2:4 magnitude pruning with optional soft-thresholding (Section 2.2), the V:N:M activation
 format (Section 2.3), SquaredReLU (Eq. 2) and the masked FFN forward/backward products
-(Eqs. 1-8 with the operand colouring of Algorithms 1 and 2).
+(Eqs. 1-8 with the operand colouring of Algorithms 1 and 2), and the sparse/dense step
+schedule with the paper's speed-up arithmetic (Sections 3.1, 5.1, 5.3.2; `oracle.schedule`).
 
 Nothing in here is shared with, imported by, or derived from the CUDA path. Only the tests,
 the smoke check and the benchmark's CPU-baseline leg may import this package; the product
