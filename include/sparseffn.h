@@ -222,6 +222,46 @@ SF_API int sf_ffn_step_host(const sf_ffn_desc* desc, int dense, const void* host
                      void* host_dW1, void* host_dW2, void* device_staging, void* fwd_ctx,
                      void* workspace, void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * Sparse/dense step schedule (Section 5.3.2) and speed-up arithmetic (Sections 3.1 and 5.1).
+ * Host-side logic; nothing here touches the GPU except the two dispatchers.
+ *
+ * A run of `total_steps` steps (0-based index) is: `warmup_steps` dense steps (the paper starts
+ * V:N:M sparsification only after a dense warm-up, 1000 steps there), then `sparse_steps` sparse
+ * steps, then dense steps to the end (sparse first, dense afterwards to recover accuracy).
+ * SF_ERR_SHAPE when a count is negative, total_steps <= 0, the two phases exceed the run, or
+ * `step` lies outside [0, total_steps).
+ *
+ * sf_schedule_speedup:    time of total_steps dense steps / time of the mixed schedule when a
+ *                         sparse step is `sparse_step_speedup` times faster than a dense one
+ *                         (Section 5.1's example: 2.2x on half of the steps -> 1.37x).
+ * sf_ffn_flop_fraction:   FFN share of the training FLOPs, 18DF / (6(3DF + 2D(Nq + Nkv)H))
+ *                         (Section 3.1).
+ * sf_end_to_end_speedup:  1 / ((1 - f) + f / s): the whole-model effect of an s-times faster
+ *                         FFN whose share of the time is f (Section 3.1 takes the FLOP share as
+ *                         the time share).
+ * sf_ffn_fwd_scheduled /  run the forward / backward step of the kind the schedule assigns to
+ * sf_ffn_bwd_scheduled:   `step`; arguments as sf_sparse_ffn_fwd/bwd. Context and workspace of
+ *                         sf_ffn_workspace_size() fit both kinds. Call both with the same step. */
+typedef struct sf_schedule {
+  int64_t warmup_steps;
+  int64_t sparse_steps;
+  int64_t total_steps;
+} sf_schedule;
+typedef enum sf_step_kind { SF_STEP_DENSE = 0, SF_STEP_SPARSE = 1 } sf_step_kind;
+SF_API int sf_schedule_step_kind(const sf_schedule* schedule, int64_t step, int* kind);
+SF_API int sf_schedule_speedup(const sf_schedule* schedule, double sparse_step_speedup, double* speedup);
+SF_API int sf_ffn_flop_fraction(int64_t D, int64_t F, int64_t n_q_heads, int64_t n_kv_heads, int64_t head_dim,
+                         double* fraction);
+SF_API int sf_end_to_end_speedup(double ffn_fraction, double ffn_speedup, double* speedup);
+SF_API int sf_ffn_fwd_scheduled(const sf_schedule* schedule, int64_t step, const sf_ffn_desc* desc,
+                         const void* X, const void* W1, const void* W2, void* Y, void* fwd_ctx,
+                         void* workspace, void* stream);
+SF_API int sf_ffn_bwd_scheduled(const sf_schedule* schedule, int64_t step, const sf_ffn_desc* desc,
+                         const void* dY, const void* X, const void* W1, const void* W2,
+                         const void* fwd_ctx, void* dX, void* dW1, void* dW2, void* workspace,
+                         void* stream);
+
 /* Stage tracing, a measurement aid (the paper has no counterpart). `events` is a caller-owned HOST
  * array of `capacity` cudaEvent_t handles (created with timing enabled) that must stay valid until
  * tracing is switched off with capacity 0. While set, every FFN step call records one event

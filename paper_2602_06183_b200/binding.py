@@ -29,6 +29,13 @@ class sf_ffn_desc(C.Structure):
                 ("prune_mode", C.c_int32), ("flags", C.c_int32)]
 
 
+class sf_schedule(C.Structure):
+    _fields_ = [("warmup_steps", C.c_int64), ("sparse_steps", C.c_int64), ("total_steps", C.c_int64)]
+
+
+SF_STEP_DENSE, SF_STEP_SPARSE = 0, 1
+
+
 class SparseFFNError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -59,6 +66,14 @@ _SIGNATURES = {
     "sf_ctx_view": (_i32, [C.POINTER(sf_ffn_desc), _vp, _i32, C.POINTER(_vp), C.POINTER(_sz)]),
     "sf_ffn_host_staging_size": (_i32, [C.POINTER(sf_ffn_desc), C.POINTER(_sz)]),
     "sf_ffn_step_host": (_i32, [C.POINTER(sf_ffn_desc), _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_schedule_step_kind": (_i32, [C.POINTER(sf_schedule), _i64, C.POINTER(_i32)]),
+    "sf_schedule_speedup": (_i32, [C.POINTER(sf_schedule), C.c_double, C.POINTER(C.c_double)]),
+    "sf_ffn_flop_fraction": (_i32, [_i64, _i64, _i64, _i64, _i64, C.POINTER(C.c_double)]),
+    "sf_end_to_end_speedup": (_i32, [C.c_double, C.c_double, C.POINTER(C.c_double)]),
+    "sf_ffn_fwd_scheduled": (_i32, [C.POINTER(sf_schedule), _i64, C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp,
+                                    _vp, _vp]),
+    "sf_ffn_bwd_scheduled": (_i32, [C.POINTER(sf_schedule), _i64, C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp,
+                                    _vp, _vp, _vp, _vp, _vp]),
     "sf_trace_set": (_i32, [C.POINTER(_vp), _i32]),
     "sf_trace_count": (_i32, []),
     "sf_check_status": (_i32, [_vp, _vp]),
@@ -302,6 +317,45 @@ def sf_ffn_step_host(desc, dense: bool, hX, hW1, hW2, hdY, hY, hdX, hdW1, hdW2, 
     _check(lib().sf_ffn_step_host(C.byref(desc), int(dense), _ptr(hX), _ptr(hW1), _ptr(hW2), _ptr(hdY), _ptr(hY),
                                   _ptr(hdX), _ptr(hdW1), _ptr(hdW2), _ptr(staging), _ptr(fwd_ctx), _ptr(workspace),
                                   _stream(stream)), "sf_ffn_step_host")
+
+
+def make_schedule(warmup_steps: int, sparse_steps: int, total_steps: int) -> sf_schedule:
+    return sf_schedule(warmup_steps, sparse_steps, total_steps)
+
+
+def sf_schedule_step_kind(schedule, step: int) -> int:
+    kind = _i32(0)
+    _check(lib().sf_schedule_step_kind(C.byref(schedule), step, C.byref(kind)), "sf_schedule_step_kind")
+    return kind.value
+
+
+def sf_schedule_speedup(schedule, sparse_step_speedup: float) -> float:
+    out = C.c_double(0)
+    _check(lib().sf_schedule_speedup(C.byref(schedule), sparse_step_speedup, C.byref(out)), "sf_schedule_speedup")
+    return out.value
+
+
+def sf_ffn_flop_fraction(D: int, F: int, n_q_heads: int, n_kv_heads: int, head_dim: int) -> float:
+    out = C.c_double(0)
+    _check(lib().sf_ffn_flop_fraction(D, F, n_q_heads, n_kv_heads, head_dim, C.byref(out)), "sf_ffn_flop_fraction")
+    return out.value
+
+
+def sf_end_to_end_speedup(ffn_fraction: float, ffn_speedup: float) -> float:
+    out = C.c_double(0)
+    _check(lib().sf_end_to_end_speedup(ffn_fraction, ffn_speedup, C.byref(out)), "sf_end_to_end_speedup")
+    return out.value
+
+
+def sf_ffn_fwd_scheduled(schedule, step: int, desc, X, W1, W2, Y, fwd_ctx, workspace, stream=None):
+    _check(lib().sf_ffn_fwd_scheduled(C.byref(schedule), step, C.byref(desc), _ptr(X), _ptr(W1), _ptr(W2), _ptr(Y),
+                                      _ptr(fwd_ctx), _ptr(workspace), _stream(stream)), "sf_ffn_fwd_scheduled")
+
+
+def sf_ffn_bwd_scheduled(schedule, step: int, desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stream=None):
+    _check(lib().sf_ffn_bwd_scheduled(C.byref(schedule), step, C.byref(desc), _ptr(dY), _ptr(X), _ptr(W1), _ptr(W2),
+                                      _ptr(fwd_ctx), _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace),
+                                      _stream(stream)), "sf_ffn_bwd_scheduled")
 
 
 def sf_check_status(workspace, stream=None) -> int:

@@ -55,3 +55,37 @@ def test_null_and_alignment_rejected_before_launch(lib):
     assert lib.sf_vnm_sparsify_act(None, 128, 256, 256, 64, 2, 8, 1, None, None, None, None, None, None) == binding.SF_ERR_NULL
     # empty inputs are a no-op
     assert lib.sf_prune24_compress(None, 0, 256, 256, 1, 0, None, None, None, None) == binding.SF_OK
+
+
+def test_schedule_logic_matches_the_oracle(lib):
+    """The schedule functions are host arithmetic, so they are compared with the oracle here."""
+    from oracle import schedule as S
+    for warm, sparse, total in [(0, 0, 1), (0, 5, 5), (3, 4, 12), (1000, 30000, 60000), (2, 0, 9)]:
+        sc = binding.make_schedule(warm, sparse, total)
+        probe = sorted({0, max(warm - 1, 0), warm, min(warm + sparse, total - 1), max(warm + sparse - 1, 0), total - 1})
+        for step in probe:
+            assert binding.sf_schedule_step_kind(sc, step) == S.step_kind(step, warm, sparse, total)
+        for s in (1.0, 1.22, 2.2, 7.0):
+            assert binding.sf_schedule_speedup(sc, s) == pytest.approx(S.schedule_speedup(sparse, total, s), rel=1e-14)
+    for args in [(2048, 8192, 32, 8, 64), (4096, 16384, 32, 8, 128), (16384, 53248, 128, 8, 128)]:
+        assert binding.sf_ffn_flop_fraction(*args) == pytest.approx(S.ffn_flop_fraction(*args), rel=1e-14)
+    for f, s in [(0.0, 3.0), (0.5, 2.0), (0.82, 1.22), (1.0, 7.0)]:
+        assert binding.sf_end_to_end_speedup(f, s) == pytest.approx(S.end_to_end_speedup(f, s), rel=1e-14)
+
+
+def test_schedule_rejects_bad_arguments(lib):
+    kind, out = C.c_int(), C.c_double()
+    sc = binding.make_schedule(3, 4, 12)
+    assert lib.sf_schedule_step_kind(None, 0, C.byref(kind)) == binding.SF_ERR_NULL
+    assert lib.sf_schedule_step_kind(C.byref(sc), 0, None) == binding.SF_ERR_NULL
+    assert lib.sf_schedule_step_kind(C.byref(sc), 12, C.byref(kind)) == binding.SF_ERR_SHAPE
+    assert lib.sf_schedule_step_kind(C.byref(sc), -1, C.byref(kind)) == binding.SF_ERR_SHAPE
+    for bad in [(-1, 4, 12), (3, -4, 12), (3, 4, 0), (9, 4, 12)]:
+        b = binding.make_schedule(*bad)
+        assert lib.sf_schedule_step_kind(C.byref(b), 0, C.byref(kind)) == binding.SF_ERR_SHAPE
+        assert lib.sf_schedule_speedup(C.byref(b), 2.0, C.byref(out)) == binding.SF_ERR_SHAPE
+    assert lib.sf_schedule_speedup(C.byref(sc), 0.0, C.byref(out)) == binding.SF_ERR_SHAPE
+    assert lib.sf_end_to_end_speedup(1.5, 2.0, C.byref(out)) == binding.SF_ERR_SHAPE
+    assert lib.sf_ffn_flop_fraction(0, 8, 1, 1, 1, C.byref(out)) == binding.SF_ERR_SHAPE
+    # a step outside the schedule is rejected before any pointer is looked at
+    assert lib.sf_ffn_fwd_scheduled(C.byref(sc), 99, None, None, None, None, None, None, None, None) == binding.SF_ERR_SHAPE

@@ -225,3 +225,36 @@ def test_ffn_rejects_ragged_shapes():
     with pytest.raises(binding.SparseFFNError) as e:
         binding.sf_ffn_workspace_size(desc)
     assert e.value.status == binding.SF_ERR_UNSUPPORTED
+
+
+def test_scheduled_steps_dispatch_to_the_right_kind():
+    """A short run (2 warm-up, 3 sparse, 2 dense): every scheduled step reproduces, bit for bit,
+    the direct call of the kind the schedule assigns to it."""
+    cfg = synth.FFN_CONFIGS["c1_small"]
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
+    desc = binding.make_desc(T, D, F, V, M)
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
+
+    def run(fwd, bwd):
+        Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+        gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
+        fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
+        bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+        assert binding.sf_check_status(ws) == binding.SF_OK
+        return Y, gX, gW1, gW2
+
+    direct = {binding.SF_STEP_SPARSE: run(binding.sf_sparse_ffn_fwd, binding.sf_sparse_ffn_bwd),
+              binding.SF_STEP_DENSE: run(binding.sf_dense_ffn_fwd, binding.sf_dense_ffn_bwd)}
+    assert not torch.equal(direct[0][0], direct[1][0])
+    sc = binding.make_schedule(2, 3, 7)
+    kinds = []
+    for step in range(7):
+        kind = binding.sf_schedule_step_kind(sc, step)
+        kinds.append(kind)
+        got = run(lambda *a: binding.sf_ffn_fwd_scheduled(sc, step, *a),
+                  lambda *a: binding.sf_ffn_bwd_scheduled(sc, step, *a))
+        for a, b in zip(got, direct[kind]):
+            assert torch.equal(a, b)
+    assert kinds == [0, 0, 1, 1, 1, 0, 0]
