@@ -262,6 +262,16 @@ SF_API int sf_ffn_bwd_scheduled(const sf_schedule* schedule, int64_t step, const
                          const void* fwd_ctx, void* dX, void* dW1, void* dW2, void* workspace,
                          void* stream);
 
+/* Tensor-pipe calibration, a measurement aid (the paper has no counterpart). One CTA per SM (or
+ * one CTA pair per two SMs when two_cta != 0) issues 4 * iters tcgen05.mma instructions back to
+ * back on operands that already sit in shared memory: 128 x 256 x 16 per CTA for sparse == 0,
+ * 128 x 256 x 32 logical K with 2:4 metadata for sparse != 0; no loads, no epilogue. `cycles`
+ * (DEVICE pointer, int64, 8-byte aligned) receives the SM clocks CTA 0 spent from its first issue
+ * to the completion of its last instruction; clocks per instruction = *cycles / (4 * iters).
+ * `workspace` is any device buffer whose first int is a zeroed status word (a bounded wait that
+ * expires sets it; read it with sf_check_status). 1 <= iters <= 2^20. Enqueues on `stream`. */
+SF_API int sf_probe_mma_rate(int sparse, int two_cta, int iters, void* cycles, void* workspace, void* stream);
+
 /* Stage tracing, a measurement aid (the paper has no counterpart). `events` is a caller-owned HOST
  * array of `capacity` cudaEvent_t handles (created with timing enabled) that must stay valid until
  * tracing is switched off with capacity 0. While set, every FFN step call records one event

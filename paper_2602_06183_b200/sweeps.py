@@ -1,6 +1,6 @@
 """Stand-alone throughput sweeps of the bandwidth kernels and single products (one JSON line each).
 
-    python -m paper_2602_06183_b200.sweeps [--which prune,act,gemm,c5]
+    python -m paper_2602_06183_b200.sweeps [--which prune,act,gemm,c5,mma,power]
 
 prune: 2:4 prune + compress on the weight shapes of the sweep configuration (both group directions,
        hard and soft), GB/s at 3.125 algorithmic bytes per element.
@@ -9,6 +9,10 @@ act:   SquaredReLU + V:N:M sparsify on 16384 x 16384 pre-activations with ~90 % 
 gemm:  dense vs 2:4 vs Venom products at the paper's micro-benchmark shape (m, n, k) = (4096, 16384, 4096)
        and at the FFN shapes.
 c5:    sparse and dense step of the d_model = 8192 layer.
+mma:   clocks per tcgen05.mma issued back to back from shared memory (dense / 2:4, one CTA / CTA pair):
+       what the tensor pipe can do for the product kernels' tile shapes.
+power: seconds-long loops of the dense and the 2:4 product on random and on all-zero operands with
+       SM clock and board power sampled by nvidia-smi: separates the power cap from the kernel.
 Inputs larger than the L2; times are CUDA-event averages over 20 launches after 3 warm-ups.
 """
 from __future__ import annotations
@@ -134,6 +138,69 @@ def c5_step():
                       "speedup": ms_d / ms_s, "status": binding.sf_check_status(ws)}))
 
 
+def mma_rate():
+    for sparse, two in [(False, False), (True, False), (False, True), (True, True)]:
+        clk = binding.sf_probe_mma_rate(sparse, two)
+        macs = 128 * 256 * (32 if sparse else 16)               # dense-equivalent MACs per instruction per SM
+        print(json.dumps({"probe": "mma_rate", "operand": "2:4" if sparse else "dense",
+                          "cta_group": 2 if two else 1, "tile_per_cta": [128, 256, 32 if sparse else 16],
+                          "clk_per_mma": round(clk, 1), "dense_equiv_flop_per_clk_per_sm": round(2 * macs / clk)}))
+
+
+def _sampled_loop(fn, seconds=2.5):
+    """Run fn back to back for `seconds`; median SM clock / power over the last two thirds of the samples."""
+    import statistics
+    import subprocess
+    import time
+    q = "clocks.sm,power.draw,clocks_event_reasons.sw_power_cap,clocks_event_reasons.hw_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown"
+    dev = str(torch.cuda.current_device())
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        dev = vis.split(",")[int(dev)]
+    p = subprocess.Popen(["nvidia-smi", "-i", dev, f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "50"],
+                         stdout=subprocess.PIPE, text=True)
+    for _ in range(10):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n, t0 = 0, time.time()
+    e0.record()
+    while time.time() - t0 < seconds:
+        for _ in range(50):
+            fn()
+        n += 50
+        torch.cuda.synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    p.terminate()
+    rows = [l.split(", ") for l in p.communicate()[0].strip().splitlines() if l.count(",") >= 4]
+    rows = rows[len(rows) // 3:] or [["0", "0", "", "", ""]]
+    return {"ms": e0.elapsed_time(e1) / n,
+            "sm_mhz_median": statistics.median(float(r[0]) for r in rows),
+            "power_w_median": statistics.median(float(r[1]) for r in rows),
+            "sw_power_cap_share": sum(r[2].strip() == "Active" for r in rows) / len(rows),
+            "hw_or_thermal_slowdown_samples": sum(r[3].strip() == "Active" or r[4].strip() == "Active" for r in rows)}
+
+
+def power_loops():
+    m, n, k = 16384, 8192, 4096
+    fl = 2.0 * m * n * k
+    for data in ("randn", "zeros"):
+        gen = (lambda s: torch.randn(s, device="cuda")) if data == "randn" else (lambda s: torch.zeros(s, device="cuda"))
+        A, B = gen((m, k)).to(torch.bfloat16), gen((n, k)).to(torch.bfloat16)
+        C = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
+        ws = torch.zeros((binding.sf_gemm_workspace_size(m, k),), dtype=torch.uint8, device="cuda")
+        vals, meta, _ = binding.sf_prune24_compress(A, 1, 0)
+        for kind, fn in [("dense", lambda: binding.sf_gemm_dense(A, True, B, True, C_out=C, workspace=ws)),
+                         ("sparse24", lambda: binding.sf_gemm_sparse24_rm(vals, meta, B, True, C_out=C, workspace=ws))]:
+            r = _sampled_loop(fn)
+            r.update({"probe": "sustained_loop", "data": data, "kernel": kind, "shape_mnk": [m, n, k],
+                      "dense_equiv_tflops": fl / r["ms"] / 1e9,
+                      "tflops_per_ghz": fl / r["ms"] / 1e9 / max(r["sm_mhz_median"] / 1e3, 1e-9)})
+            print(json.dumps(r))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--which", default="prune,act,gemm,c5")
@@ -141,7 +208,8 @@ def main():
     from . import build
     build.build()
     for w in args.which.split(","):
-        {"prune": prune_sweep, "act": act_sweep, "gemm": gemm_sweep, "c5": c5_step}[w]()
+        {"prune": prune_sweep, "act": act_sweep, "gemm": gemm_sweep, "c5": c5_step, "mma": mma_rate,
+         "power": power_loops}[w]()
 
 
 if __name__ == "__main__":

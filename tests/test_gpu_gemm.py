@@ -111,3 +111,15 @@ def test_gemm_shape_errors():
     with pytest.raises(binding.SparseFFNError) as e:
         binding.sf_gemm_dense(A, True, B, True)
     assert e.value.status == binding.SF_ERR_SHAPE
+
+
+def test_mma_rate_probe_reports_the_pipe_rates():
+    """Back-to-back issue from shared memory: a dense 128x256x16 instruction takes 128 clocks
+    (8192 flop/clk/SM, the nominal rate); the 2:4 instruction has twice the logical K and must not
+    take more than 1.3x as long on a CTA pair, nor be faster than the dense one."""
+    dense = binding.sf_probe_mma_rate(False, True, iters=4000)
+    sparse = binding.sf_probe_mma_rate(True, True, iters=4000)
+    one = binding.sf_probe_mma_rate(True, False, iters=4000)
+    assert 120 < dense < 140
+    assert dense * 0.95 < sparse < dense * 1.3
+    assert sparse <= one * 1.02
