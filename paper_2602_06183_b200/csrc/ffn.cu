@@ -32,7 +32,7 @@ struct StepHooks {
   cudaEvent_t dx_done;       // backward: recorded after the dX product
   cudaEvent_t dw2_done;      // backward: recorded after the dW2 product
 };
-const StepHooks* g_hooks = nullptr;
+thread_local const StepHooks* g_hooks = nullptr;   // per host thread: other threads' steps see no hooks
 
 inline void hook_wait_w2(cudaStream_t s) {
   if (g_hooks) cudaStreamWaitEvent(s, g_hooks->w2_ready, 0);
