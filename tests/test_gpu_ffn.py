@@ -258,3 +258,31 @@ def test_scheduled_steps_dispatch_to_the_right_kind():
         for a, b in zip(got, direct[kind]):
             assert torch.equal(a, b)
     assert kinds == [0, 0, 1, 1, 1, 0, 0]
+
+
+def _legal_random_configs(n, seed):
+    """Seeded draw of legal step shapes: T, D, F multiples of 256, V in {64, 128}, M in {4..32},
+    condensed reduction 4F/M a multiple of 128, both prune modes, symmetric or ~90 %-negative
+    pre-activations."""
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < n:
+        T, D, F = (int(rng.integers(1, 4)) * 256 for _ in range(3))
+        F *= int(rng.integers(1, 3))
+        V, M = int(rng.choice([64, 128])), int(rng.choice([4, 8, 16, 32]))
+        if (4 * F // M) % 128:
+            continue
+        out.append((T, D, F, V, M, int(rng.integers(0, 2)), float(rng.choice([0.0, -1.3])), int(rng.integers(1, 1 << 20))))
+    return out
+
+
+@pytest.mark.parametrize("T,D,F,V,M,prune_mode,act_shift,seed", _legal_random_configs(10, seed=20260206))
+def test_sparse_ffn_random_legal_shapes(T, D, F, V, M, prune_mode, act_shift, seed):
+    cfg = dict(T=T, D=D, F=F, V=V, N=2, M=M, sigma_w=0.05, seed=seed)
+    (X, W1, W2, dY), g = _run_sparse(cfg, prune_mode, act_shift)
+    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, prune_mode=prune_mode, forced_y1b=g["y1"])
+    assert np.array_equal(g["colidx"], fwd.act.colidx) and np.array_equal(g["meta"], fwd.act.meta)
+    assert np.array_equal(g["y2_vals"], fwd.act.vals) and np.array_equal(g["relu_vals"], fwd.act.relu_vals)
+    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd, prune_mode=prune_mode)
+    for k, ref in (("Y", fwd.y3), ("dX", bwd.dX), ("dW1", bwd.dW1), ("dW2", bwd.dW2)):
+        assert rel_fro(g[k], ref) < TOL, k
