@@ -47,28 +47,41 @@ __device__ __forceinline__ void write_group_dense(uint16_t* drow, int M, uint32_
   }
 }
 
+__device__ __forceinline__ uint32_t relu2(uint32_t w) {
+  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&w);
+  __nv_bfloat162 z = __hmax2(x, __float2bfloat162_rn(0.f));
+  return *reinterpret_cast<uint32_t*>(&z);
+}
+__device__ __forceinline__ uint32_t sq2(uint32_t r) {
+  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&r);
+  __nv_bfloat162 z = __hmul2(x, x);
+  return *reinterpret_cast<uint32_t*>(&z);
+}
+
+// kW: strip width in columns (128 for M <= 32: half the shared memory, twice the resident CTAs; 256 for M = 64).
+template <int kW>
 __global__ void __launch_bounds__(kThreads)
 vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply,
            uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
            uint8_t* __restrict__ colidx, uint16_t* __restrict__ relu_vals, uint16_t* __restrict__ dense_out,
            uint16_t* __restrict__ relu_dense_out) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  uint16_t* tile = reinterpret_cast<uint16_t*>(smem_raw);                        // [V][kCW + kPad]
-  uint32_t* score = reinterpret_cast<uint32_t*>(tile + (size_t)V * (kCW + kPad)); // [kCW] float bits
-  uint8_t* keepf = reinterpret_cast<uint8_t*>(score + kCW);                       // [kCW]
-  uint8_t* cidx = keepf + kCW;                                                    // [kCW / 4][4]
-  constexpr int kRow = kCW + kPad;
+  uint16_t* tile = reinterpret_cast<uint16_t*>(smem_raw);                        // [V][kW + kPad]
+  uint32_t* score = reinterpret_cast<uint32_t*>(tile + (size_t)V * (kW + kPad)); // [kW] float bits
+  uint8_t* keepf = reinterpret_cast<uint8_t*>(score + kW);                       // [kW]
+  uint8_t* cidx = keepf + kW;                                                    // [kW / 4][4]
+  constexpr int kRow = kW + kPad;
 
   const int tid = threadIdx.x;
-  const int64_t c0 = (int64_t)blockIdx.x * kCW;
+  const int64_t c0 = (int64_t)blockIdx.x * kW;
   const int64_t blk = blockIdx.y;
   const int64_t t0 = blk * V;
-  const int cvalid = (int)min((int64_t)kCW, F - c0);
+  const int cvalid = (int)min((int64_t)kW, F - c0);
   const int64_t G = F / M;
 
   // ---- stage the strip
-  for (int i = tid; i < V * (kCW / 8); i += kThreads) {
-    const int r = i / (kCW / 8), cc = (i % (kCW / 8)) * 8;
+  for (int i = tid; i < V * (kW / 8); i += kThreads) {
+    const int r = i / (kW / 8), cc = (i % (kW / 8)) * 8;
     if (cc < cvalid) {
       const uint4 q = __ldg(reinterpret_cast<const uint4*>(P + (t0 + r) * ld + c0 + cc));
       *reinterpret_cast<uint4*>(tile + r * kRow + cc) = q;
@@ -76,22 +89,41 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
   }
   __syncthreads();
 
-  // ---- pass A: column scores (sequential float32 adds, rows in ascending order)
-  // (the strip is kCW columns wide; threads beyond it only help with loads, pass B and stores)
-  if (tid < kCW) {
-    const int j = tid;
-    float s = 0.f;
-    if (j < cvalid) {
-      for (int r = 0; r < V; ++r) {
-        uint32_t h, relu;
-        sqrelu_bits(tile[r * kRow + j], apply, h, relu);
-        s = __fadd_rn(s, bf16_bits_to_float(h & 0x7FFFu));
+  // ---- pass A: column scores (sequential float32 adds, rows in ascending order), two columns per
+  // thread on packed bf16 pairs: max with zero, then one correctly rounded bf16 multiply (equal to
+  // rounding the exact float32 square)
+  if (tid < kW / 2) {
+    float s0 = 0.f, s1 = 0.f;
+    if (2 * tid < cvalid) {
+      const uint32_t* col = reinterpret_cast<const uint32_t*>(tile) + tid;
+      // eight rows per trip: the loads and the packed arithmetic of a trip are independent, only the
+      // two add chains are sequential; a tail loop takes V % 8 rows
+      int r = 0;
+      for (; r + 8 <= V; r += 8) {
+        uint32_t h[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const uint32_t w = col[(r + u) * (kRow / 2)];
+          h[u] = apply ? sq2(relu2(w)) : (w & 0x7FFF7FFFu);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          s0 = __fadd_rn(s0, __uint_as_float(h[u] << 16));
+          s1 = __fadd_rn(s1, __uint_as_float(h[u] & 0xFFFF0000u));
+        }
+      }
+      for (; r < V; ++r) {
+        const uint32_t w = col[r * (kRow / 2)];
+        const uint32_t h = apply ? sq2(relu2(w)) : (w & 0x7FFF7FFFu);
+        s0 = __fadd_rn(s0, __uint_as_float(h << 16));
+        s1 = __fadd_rn(s1, __uint_as_float(h & 0xFFFF0000u));
       }
     }
-    score[j] = __float_as_uint(s);
+    score[2 * tid] = __float_as_uint(s0);
+    score[2 * tid + 1] = __float_as_uint(s1);
   }
   __syncthreads();
-  if (tid < kCW) {
+  if (tid < kW) {
     const int j = tid, jm = j % M, base = j - jm;
     const uint32_t s = score[j];
     int rank = 0;
@@ -102,7 +134,7 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
     keepf[j] = rank < 4;
   }
   __syncthreads();
-  if (tid < kCW) {
+  if (tid < kW) {
     const int j = tid, jm = j % M, base = j - jm;
     if (keepf[j] && j < cvalid) {
       int pos = 0;
@@ -162,17 +194,7 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
 // rounding the exact float32 square), whole 16-byte groups from shared memory, byte permutes with
 // selectors that depend only on the block's kept columns (constant per thread: a thread always
 // serves the same group of the strip), and mask words for the dense copies.
-__device__ __forceinline__ uint32_t relu2(uint32_t w) {
-  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&w);
-  __nv_bfloat162 z = __hmax2(x, __float2bfloat162_rn(0.f));
-  return *reinterpret_cast<uint32_t*>(&z);
-}
-__device__ __forceinline__ uint32_t sq2(uint32_t r) {
-  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&r);
-  __nv_bfloat162 z = __hmul2(x, x);
-  return *reinterpret_cast<uint32_t*>(&z);
-}
-
+template <int kW>
 __global__ void __launch_bounds__(kThreads)
 vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int V, int apply,
             uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
@@ -181,21 +203,21 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
             uint8_t* __restrict__ meta24_hw) {
   constexpr int M = 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  uint16_t* tile = reinterpret_cast<uint16_t*>(smem_raw);                        // [V][kCW + kPad]
-  uint32_t* score = reinterpret_cast<uint32_t*>(tile + (size_t)V * (kCW + kPad));
-  uint8_t* keepf = reinterpret_cast<uint8_t*>(score + kCW);
-  uint8_t* cidx = keepf + kCW;
-  constexpr int kRow = kCW + kPad;
+  uint16_t* tile = reinterpret_cast<uint16_t*>(smem_raw);                        // [V][kW + kPad]
+  uint32_t* score = reinterpret_cast<uint32_t*>(tile + (size_t)V * (kW + kPad));
+  uint8_t* keepf = reinterpret_cast<uint8_t*>(score + kW);
+  uint8_t* cidx = keepf + kW;
+  constexpr int kRow = kW + kPad;
 
   const int tid = threadIdx.x;
-  const int64_t c0 = (int64_t)blockIdx.x * kCW;
+  const int64_t c0 = (int64_t)blockIdx.x * kW;
   const int64_t blk = blockIdx.y;
   const int64_t t0 = blk * V;
-  const int cvalid = (int)min((int64_t)kCW, F - c0);
+  const int cvalid = (int)min((int64_t)kW, F - c0);
   const int64_t G = F / M;
 
-  for (int i = tid; i < V * (kCW / 8); i += kThreads) {
-    const int r = i / (kCW / 8), cc = (i % (kCW / 8)) * 8;
+  for (int i = tid; i < V * (kW / 8); i += kThreads) {
+    const int r = i / (kW / 8), cc = (i % (kW / 8)) * 8;
     if (cc < cvalid) {
       const uint4 q = __ldg(reinterpret_cast<const uint4*>(P + (t0 + r) * ld + c0 + cc));
       *reinterpret_cast<uint4*>(tile + r * kRow + cc) = q;
@@ -204,22 +226,31 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
   __syncthreads();
 
   // pass A: two columns per thread, rows first to last, one float32 add per element
-  if (tid < kCW / 2) {
+  if (tid < kW / 2) {
     float s0 = 0.f, s1 = 0.f;
     if (2 * tid < cvalid) {
       const uint32_t* col = reinterpret_cast<const uint32_t*>(tile) + tid;
-      for (int r = 0; r < V; ++r) {
-        const uint32_t w = col[r * (kRow / 2)];
-        const uint32_t h = apply ? sq2(relu2(w)) : (w & 0x7FFF7FFFu);
-        s0 = __fadd_rn(s0, __uint_as_float(h << 16));
-        s1 = __fadd_rn(s1, __uint_as_float(h & 0xFFFF0000u));
+      // eight rows per trip (V is a multiple of 8): the loads and the packed arithmetic of a trip are
+      // independent, only the two add chains are sequential
+      for (int r = 0; r < V; r += 8) {
+        uint32_t h[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const uint32_t w = col[(r + u) * (kRow / 2)];
+          h[u] = apply ? sq2(relu2(w)) : (w & 0x7FFF7FFFu);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          s0 = __fadd_rn(s0, __uint_as_float(h[u] << 16));
+          s1 = __fadd_rn(s1, __uint_as_float(h[u] & 0xFFFF0000u));
+        }
       }
     }
     score[2 * tid] = __float_as_uint(s0);
     score[2 * tid + 1] = __float_as_uint(s1);
   }
   __syncthreads();
-  if (tid < kCW) {
+  if (tid < kW) {
     const int j = tid, jm = j & 7, base = j - jm;
     const uint32_t s = score[j];
     int rank = 0;
@@ -231,7 +262,7 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
     keepf[j] = rank < 4;
   }
   __syncthreads();
-  if (tid < kCW) {
+  if (tid < kW) {
     const int j = tid, jm = j & 7, base = j - jm;
     if (keepf[j] && j < cvalid) {
       int pos = 0;
@@ -389,8 +420,10 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
   int dev = 0;
   SF_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    SF_CUDA_TRY(cudaFuncSetAttribute(vnm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    SF_CUDA_TRY(cudaFuncSetAttribute(vnm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      128 * (kCW + kPad) * 2 + kCW * 6));
+    SF_CUDA_TRY(cudaFuncSetAttribute(vnm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     128 * (128 + kPad) * 2 + 128 * 6));
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   dim3 grid((unsigned)((F + kCW - 1) / kCW), (unsigned)(T / V));
@@ -398,23 +431,40 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
   const int tail = (int)(F % kCW);
   const bool fast8 = (M == 8) && (tail == 0 || tail == 64 || tail == 128) && (V % 32 == 0);
   if (fast8) {
+    // 256-column strips measured as fast as 128-column ones at V = 128 and 15 % faster at V = 64
+    // (the kernel is bound by instruction issue, not by resident CTAs)
+    constexpr int kW8 = 256;
     static bool attr8[64] = {false};
     if (dev < 0 || dev >= 64 || !attr8[dev]) {
-      SF_CUDA_TRY(cudaFuncSetAttribute(vnm8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       128 * (kCW + kPad) * 2 + kCW * 6));
+      SF_CUDA_TRY(cudaFuncSetAttribute(vnm8_kernel<kW8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       128 * (kW8 + kPad) * 2 + kW8 * 6));
       if (dev >= 0 && dev < 64) attr8[dev] = true;
     }
-    vnm8_kernel<<<grid, kThreads, smem, s>>>((const uint16_t*)P, T, F, ld, V, apply_sqrelu, (uint16_t*)vals,
-                                             (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
-                                             (uint16_t*)relu_vals, (uint16_t*)dense_out, (uint16_t*)relu_dense_out,
-                                             (uint16_t*)vals24, (uint16_t*)meta24, (uint8_t*)meta24_hw);
+    const size_t smem8 = (size_t)V * (kW8 + kPad) * 2 + kW8 * 6;
+    dim3 grid8((unsigned)((F + kW8 - 1) / kW8), (unsigned)(T / V));
+    vnm8_kernel<kW8><<<grid8, kThreads, smem8, s>>>((const uint16_t*)P, T, F, ld, V, apply_sqrelu, (uint16_t*)vals,
+                                                    (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
+                                                    (uint16_t*)relu_vals, (uint16_t*)dense_out,
+                                                    (uint16_t*)relu_dense_out, (uint16_t*)vals24, (uint16_t*)meta24,
+                                                    (uint8_t*)meta24_hw);
     SF_LAUNCH_CHECK();
     return SF_OK;
   }
   if (vals24) return SF_ERR_UNSUPPORTED;                 // the plain-2:4 view is produced by the fast path only
-  vnm_kernel<<<grid, kThreads, smem, s>>>((const uint16_t*)P, T, F, ld, V, M, apply_sqrelu, (uint16_t*)vals,
-                                          (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
-                                          (uint16_t*)relu_vals, (uint16_t*)dense_out, (uint16_t*)relu_dense_out);
+  if (M <= 32) {
+    // narrow strips: 128 / M >= 4 groups per strip
+    const size_t smem_n = (size_t)V * (128 + kPad) * 2 + 128 * 6;
+    dim3 grid_n((unsigned)((F + 127) / 128), (unsigned)(T / V));
+    vnm_kernel<128><<<grid_n, kThreads, smem_n, s>>>((const uint16_t*)P, T, F, ld, V, M, apply_sqrelu, (uint16_t*)vals,
+                                                      (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
+                                                      (uint16_t*)relu_vals, (uint16_t*)dense_out,
+                                                      (uint16_t*)relu_dense_out);
+  } else {
+    vnm_kernel<256><<<grid, kThreads, smem, s>>>((const uint16_t*)P, T, F, ld, V, M, apply_sqrelu, (uint16_t*)vals,
+                                                  (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
+                                                  (uint16_t*)relu_vals, (uint16_t*)dense_out,
+                                                  (uint16_t*)relu_dense_out);
+  }
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
