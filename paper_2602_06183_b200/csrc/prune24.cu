@@ -2,7 +2,8 @@
 //
 // Streaming, HBM-bound kernels: 2 B read + 1 B packed values + 1/8 B metadata per element.
 //   * contiguous groups: one thread owns 16 consecutive elements of a row (four groups, one
-//     metadata word): two 128-bit loads, one 128-bit store of packed values, one 16-bit store.
+//     metadata word): two 128-bit loads, one 128-bit store of packed values, one 16-bit store;
+//     a warp owns 32 consecutive chunks of a row, so no index is ever divided.
 //   * strided groups (groups along dim 0, output K-major): a CTA stages a [128 x 64] panel in
 //     shared memory, selects per column, and writes the transposed packed panel with 128-bit
 //     stores through a padded staging buffer.
@@ -36,15 +37,20 @@ __device__ __forceinline__ void expand_group(uint32_t nib, uint32_t v0, uint32_t
   for (int i = 0; i < 4; ++i) d[i] = (p0 == (uint32_t)i) ? v0 : (p1 == (uint32_t)i) ? v1 : 0u;
 }
 
+// A warp owns 32 consecutive 16-element chunks of one row (1 KB of input); the eight warps of a CTA take
+// eight consecutive rows. Grid = (chunks / 32, rows / 8 folded over y and z): no index division.
+constexpr int kRowsPerCta = 8;
+
 template <bool kSoft>
 __global__ void __launch_bounds__(256)
-prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int64_t cols, int64_t ld,
+prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t ld,
                     uint4* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
                     uint4* __restrict__ dense_out) {
-  const int64_t words_per_row = cols >> 4;                       // 16-element chunks per row
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= rows * words_per_row) return;
-  const int64_t r = idx / words_per_row, kw = idx - r * words_per_row;
+  const int words_per_row = cols >> 4;                           // 16-element chunks per row
+  const int kw = (int)blockIdx.x * 32 + (int)(threadIdx.x & 31);
+  const int64_t r = ((int64_t)blockIdx.z * gridDim.y + blockIdx.y) * kRowsPerCta + (threadIdx.x >> 5);
+  if (kw >= words_per_row || r >= rows) return;
+  const int64_t idx = r * words_per_row + kw;
 
   const uint4* src = W + ((r * ld) >> 3) + (kw << 1);
   const uint4 q0 = __ldg(src), q1 = __ldg(src + 1);
@@ -64,7 +70,13 @@ prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int64_t cols, int
   }
   vals[idx] = make_uint4(packed[0], packed[1], packed[2], packed[3]);       // [R, K/2] bf16: 8 per chunk
   meta[idx] = (uint16_t)m;
-  if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(r, kw, cols)) = (uint16_t)m;
+  if (meta_hw) {
+    // tensor-core order (see meta_hw_offset), with the row part shared by the warp
+    const uint32_t mi = (uint32_t)r & 127u, kwi = (uint32_t)kw & 7u;
+    const int64_t atom = (r >> 7) * (int64_t)(cols >> 7) + (kw >> 3);
+    const uint32_t in_atom = (mi >> 4) * 256u + (kwi & 1u) * 128u + (mi & 7u) * 16u + (kwi >> 1) * 4u + ((mi >> 3) & 1u) * 2u;
+    *reinterpret_cast<uint16_t*>(meta_hw + atom * 2048 + in_atom) = (uint16_t)m;
+  }
   if (dense_out) {
     uint4* dst = dense_out + ((r * cols) >> 3) + (kw << 1);
     dst[0] = make_uint4(dense[0], dense[1], dense[2], dense[3]);
@@ -73,78 +85,131 @@ prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int64_t cols, int
 }
 
 // Strided groups. W is [Kd, Rc] row-major (Kd = rows = reduction dim, Rc = cols); outputs are
-// vals [Rc, Kd/2], meta [Rc, Kd/16]. Panel: 128 reduction rows x 64 columns per CTA.
+// vals [Rc, Kd/2], meta [Rc, Kd/16]. Panel: 128 reduction rows x 64 columns.
+// Persistent CTAs walk the panels; the next panel streams into a second shared-memory tile with
+// cp.async while the current one is selected and stored, so loads, arithmetic and stores overlap.
 constexpr int kPanelK = 128, kPanelC = 64;
 constexpr int kStageRow = (kPanelK / 2) * 2 + 16;   // packed bytes per column + 16 B pad
+constexpr int kColsTileBytes = kPanelK * (kPanelC + 8) * 2, kColsStageBytes = kPanelC * kStageRow;
+constexpr int kColsSmemBytes = 2 * kColsTileBytes + kColsStageBytes + kPanelC * (kPanelK / 16) * 2;
+constexpr int kColsCtasPerSm = 4;
+static_assert(kPanelK / 16 == 8 && kPanelC == 64, "index shifts in prune24_cols_kernel assume a 128 x 64 panel");
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
 
 template <bool kSoft>
 __global__ void __launch_bounds__(256)
 prune24_cols_kernel(const uint16_t* __restrict__ W, int64_t Kd, int64_t Rc, int64_t ld,
                     uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
-                    uint16_t* __restrict__ dense_out) {
-  __shared__ __align__(16) uint16_t tile[kPanelK][kPanelC + 8];          // +8: 16 B pad per row
-  __shared__ __align__(16) uint8_t stage[kPanelC][kStageRow];
-  __shared__ uint16_t mstage[kPanelC][kPanelK / 16];
-
-  const int64_t c0 = (int64_t)blockIdx.x * kPanelC;
-  const int64_t k0 = (int64_t)blockIdx.y * kPanelK;
+                    uint16_t* __restrict__ dense_out, int panels_x, int num_panels) {
+  extern __shared__ __align__(16) uint8_t cols_smem[];
+  typedef uint16_t TileRow[kPanelC + 8];                                 // +8: 16 B pad per row
+  typedef uint8_t StageRow[kStageRow];
+  typedef uint16_t MetaRow[kPanelK / 16];
+  StageRow* stage = reinterpret_cast<StageRow*>(cols_smem + 2 * kColsTileBytes);                       // [kPanelC]
+  MetaRow* mstage = reinterpret_cast<MetaRow*>(cols_smem + 2 * kColsTileBytes + kColsStageBytes);      // [kPanelC]
   const int tid = threadIdx.x;
-  const int kvalid = (int)min((int64_t)kPanelK, Kd - k0);               // multiple of 16
-  const int cvalid = (int)min((int64_t)kPanelC, Rc - c0);               // multiple of 8
 
-  // load: 8 threads x 16 B per row of 64 columns
-  for (int i = tid; i < kPanelK * (kPanelC / 8); i += 256) {
-    const int kr = i >> 3, cc = (i & 7) << 3;
-    if (kr < kvalid && cc < cvalid) {
-      const uint4 q = __ldg(reinterpret_cast<const uint4*>(W + (k0 + kr) * ld + c0 + cc));
-      *reinterpret_cast<uint4*>(&tile[kr][cc]) = q;
-    }
-  }
-  __syncthreads();
-
-  // select: lanes along columns (conflict-free), one thread per (column, 16-row chunk)
-  for (int i = tid; i < kPanelC * (kPanelK / 16); i += 256) {
-    const int c = i & (kPanelC - 1), ch = i >> 6;                        // ch: chunk of 16 rows
-    if (c >= cvalid || ch * 16 >= kvalid) continue;
-    uint32_t packed[4], m = 0;
+  // 8 threads x 16 B per row of 64 columns
+  auto prefetch = [&](int panel, int buf) {
+    const int py = panel / panels_x, px = panel - py * panels_x;
+    const int64_t c0 = (int64_t)px * kPanelC, k0 = (int64_t)py * kPanelK;
+    const int kvalid = (int)min((int64_t)kPanelK, Kd - k0), cvalid = (int)min((int64_t)kPanelC, Rc - c0);
+    TileRow* tile = reinterpret_cast<TileRow*>(cols_smem + buf * kColsTileBytes);
 #pragma unroll
-    for (int g = 0; g < 4; ++g) {
-      const int kr = ch * 16 + g * 4;
-      const uint32_t lo = (uint32_t)tile[kr][c] | ((uint32_t)tile[kr + 1][c] << 16);
-      const uint32_t hi = (uint32_t)tile[kr + 2][c] | ((uint32_t)tile[kr + 3][c] << 16);
-      const uint32_t nib = prune_group_packed<kSoft>(lo, hi, packed[g]);
-      m |= nib << (4 * g);
-      if (dense_out) {
-        uint32_t d[4];
-        expand_group(nib, packed[g] & 0xFFFFu, packed[g] >> 16, d);
-        tile[kr][c] = (uint16_t)d[0];
-        tile[kr + 1][c] = (uint16_t)d[1];
-        tile[kr + 2][c] = (uint16_t)d[2];
-        tile[kr + 3][c] = (uint16_t)d[3];
+    for (int u = 0; u < kPanelK * (kPanelC / 8) / 256; ++u) {
+      const int i = tid + u * 256;
+      const int kr = i >> 3, cc = (i & 7) << 3;
+      if (kr < kvalid && cc < cvalid) cp_async16(&tile[kr][cc], W + (k0 + kr) * ld + c0 + cc);
+    }
+    cp_async_commit();
+  };
+
+  int buf = 0;
+  if ((int)blockIdx.x < num_panels) prefetch(blockIdx.x, 0);
+  for (int panel = blockIdx.x; panel < num_panels; panel += gridDim.x, buf ^= 1) {
+    const int next = panel + (int)gridDim.x;
+    if (next < num_panels) {
+      prefetch(next, buf ^ 1);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
+    __syncthreads();            // this panel's tile is complete; the previous panel's stage has been drained
+
+    const int py = panel / panels_x, px = panel - py * panels_x;
+    const int64_t c0 = (int64_t)px * kPanelC, k0 = (int64_t)py * kPanelK;
+    const int kvalid = (int)min((int64_t)kPanelK, Kd - k0);               // multiple of 16
+    const int cvalid = (int)min((int64_t)kPanelC, Rc - c0);               // multiple of 8
+    TileRow* tile = reinterpret_cast<TileRow*>(cols_smem + buf * kColsTileBytes);
+
+    // select: one thread per (column pair, 16-row chunk); lanes run along column pairs, so the 32-bit
+    // loads of a warp are conflict-free, and two byte permutes turn two rows into the two columns' pairs
+    for (int i = tid; i < (kPanelC / 2) * (kPanelK / 16); i += 256) {
+      const int cp = i & (kPanelC / 2 - 1), ch = i >> 5;                   // ch: chunk of 16 rows
+      const int c = 2 * cp;
+      if (c >= cvalid || ch * 16 >= kvalid) continue;                      // cvalid is even: the pair is whole
+      uint32_t packed[2][4], m[2] = {0, 0};
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const int kr = ch * 16 + g * 4;
+        uint32_t rw[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) rw[j] = *reinterpret_cast<const uint32_t*>(&tile[kr + j][c]);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const uint32_t sel = e ? 0x7632u : 0x5410u;
+          const uint32_t lo = __byte_perm(rw[0], rw[1], sel), hi = __byte_perm(rw[2], rw[3], sel);
+          const uint32_t nib = prune_group_packed<kSoft>(lo, hi, packed[e][g]);
+          m[e] |= nib << (4 * g);
+          if (dense_out) {
+            uint32_t d[4];
+            expand_group(nib, packed[e][g] & 0xFFFFu, packed[e][g] >> 16, d);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) tile[kr + j][c + e] = (uint16_t)d[j];
+          }
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        *reinterpret_cast<uint4*>(&stage[c + e][ch * 16]) = make_uint4(packed[e][0], packed[e][1], packed[e][2], packed[e][3]);
+        mstage[c + e][ch] = (uint16_t)m[e];
       }
     }
-    *reinterpret_cast<uint4*>(&stage[c][ch * 16]) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-    mstage[c][ch] = (uint16_t)m;
-  }
-  __syncthreads();
+    __syncthreads();
 
-  // store packed values: per column kvalid/2 elements = kvalid bytes, 16 B per thread
-  const int chunks = kvalid >> 4;
-  for (int i = tid; i < kPanelC * chunks; i += 256) {
-    const int c = i / chunks, ch = i - c * chunks;
-    if (c >= cvalid) continue;
-    const uint4 q = *reinterpret_cast<const uint4*>(&stage[c][ch * 16]);
-    *reinterpret_cast<uint4*>(vals + (c0 + c) * (Kd >> 1) + (k0 >> 1) + ch * 8) = q;
-    const uint16_t mw = mstage[c][ch];
-    const int64_t kw = (k0 >> 4) + ch;
-    meta[(c0 + c) * (Kd >> 4) + kw] = mw;
-    if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(c0 + c, kw, Kd)) = mw;
-  }
-  if (dense_out) {
-    for (int i = tid; i < kPanelK * (kPanelC / 8); i += 256) {
-      const int kr = i >> 3, cc = (i & 7) << 3;
-      if (kr < kvalid && cc < cvalid)
-        *reinterpret_cast<uint4*>(dense_out + (k0 + kr) * Rc + c0 + cc) = *reinterpret_cast<const uint4*>(&tile[kr][cc]);
+    // store packed values: per column kvalid/2 elements = kvalid bytes, 16 B per thread
+    const int chunks = kvalid >> 4;
+    const bool full = chunks == kPanelK / 16;
+    for (int i = tid; i < kPanelC * chunks; i += 256) {
+      const int c = full ? (i >> 3) : (i / chunks), ch = i - c * chunks;
+      if (c >= cvalid) continue;
+      const uint4 q = *reinterpret_cast<const uint4*>(&stage[c][ch * 16]);
+      const int64_t orow = c0 + c;
+      *reinterpret_cast<uint4*>(vals + orow * (Kd >> 1) + (k0 >> 1) + ch * 8) = q;
+      const uint16_t mw = mstage[c][ch];
+      const int64_t kw = (k0 >> 4) + ch;
+      meta[orow * (Kd >> 4) + kw] = mw;
+      if (meta_hw) {
+        const uint32_t mi = (uint32_t)orow & 127u, kwi = (uint32_t)kw & 7u;
+        const int64_t atom = (orow >> 7) * (Kd >> 7) + (kw >> 3);
+        const uint32_t in_atom = (mi >> 4) * 256u + (kwi & 1u) * 128u + (mi & 7u) * 16u + (kwi >> 1) * 4u + ((mi >> 3) & 1u) * 2u;
+        *reinterpret_cast<uint16_t*>(meta_hw + atom * 2048 + in_atom) = mw;
+      }
+    }
+    if (dense_out) {
+      for (int i = tid; i < kPanelK * (kPanelC / 8); i += 256) {
+        const int kr = i >> 3, cc = (i & 7) << 3;
+        if (kr < kvalid && cc < cvalid)
+          *reinterpret_cast<uint4*>(dense_out + (k0 + kr) * Rc + c0 + cc) = *reinterpret_cast<const uint4*>(&tile[kr][cc]);
+      }
+      __syncthreads();          // this tile is overwritten by the prefetch two panels ahead
     }
   }
 }
@@ -189,22 +254,43 @@ int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int gr
                    void* vals, void* meta, void* meta_hw, void* dense_out, cudaStream_t s) {
   if (rows == 0 || cols == 0) return SF_OK;
   if (group_dim == 1) {
-    const int64_t n = rows * (cols >> 4);
-    const unsigned grid = (unsigned)((n + 255) / 256);
+    if (cols > (int64_t)1 << 30) return SF_ERR_SHAPE;
+    const int64_t row_ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
+    const int64_t gy = row_ctas < 32768 ? row_ctas : 32768;
+    const int64_t gz = (row_ctas + gy - 1) / gy;
+    if (gz > 65535) return SF_ERR_SHAPE;
+    dim3 grid((unsigned)(((cols >> 4) + 31) / 32), (unsigned)gy, (unsigned)gz);
     if (prune_mode == 0)
-      prune24_rows_kernel<false><<<grid, 256, 0, s>>>((const uint4*)W, rows, cols, ld, (uint4*)vals,
+      prune24_rows_kernel<false><<<grid, 256, 0, s>>>((const uint4*)W, rows, (int)cols, ld, (uint4*)vals,
                                                       (uint16_t*)meta, (uint8_t*)meta_hw, (uint4*)dense_out);
     else
-      prune24_rows_kernel<true><<<grid, 256, 0, s>>>((const uint4*)W, rows, cols, ld, (uint4*)vals,
+      prune24_rows_kernel<true><<<grid, 256, 0, s>>>((const uint4*)W, rows, (int)cols, ld, (uint4*)vals,
                                                      (uint16_t*)meta, (uint8_t*)meta_hw, (uint4*)dense_out);
   } else {
-    dim3 grid((unsigned)((cols + kPanelC - 1) / kPanelC), (unsigned)((rows + kPanelK - 1) / kPanelK));
+    const int64_t px = (cols + kPanelC - 1) / kPanelC, py = (rows + kPanelK - 1) / kPanelK;
+    if (px * py > (int64_t)1 << 30) return SF_ERR_SHAPE;
+    const int num_panels = (int)(px * py);
+    static bool attr_done[64] = {false};
+    static int sms[64] = {0};
+    int dev = 0;
+    SF_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return SF_ERR_UNSUPPORTED;
+    if (!attr_done[dev]) {
+      SF_CUDA_TRY(cudaFuncSetAttribute(prune24_cols_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kColsSmemBytes));
+      SF_CUDA_TRY(cudaFuncSetAttribute(prune24_cols_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kColsSmemBytes));
+      SF_CUDA_TRY(cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev));
+      attr_done[dev] = true;
+    }
+    const int resident = sms[dev] * kColsCtasPerSm;
+    const unsigned grid = (unsigned)(num_panels < resident ? num_panels : resident);
     if (prune_mode == 0)
-      prune24_cols_kernel<false><<<grid, 256, 0, s>>>((const uint16_t*)W, rows, cols, ld, (uint16_t*)vals,
-                                                      (uint16_t*)meta, (uint8_t*)meta_hw, (uint16_t*)dense_out);
+      prune24_cols_kernel<false><<<grid, 256, kColsSmemBytes, s>>>((const uint16_t*)W, rows, cols, ld, (uint16_t*)vals,
+                                                                   (uint16_t*)meta, (uint8_t*)meta_hw,
+                                                                   (uint16_t*)dense_out, (int)px, num_panels);
     else
-      prune24_cols_kernel<true><<<grid, 256, 0, s>>>((const uint16_t*)W, rows, cols, ld, (uint16_t*)vals,
-                                                     (uint16_t*)meta, (uint8_t*)meta_hw, (uint16_t*)dense_out);
+      prune24_cols_kernel<true><<<grid, 256, kColsSmemBytes, s>>>((const uint16_t*)W, rows, cols, ld, (uint16_t*)vals,
+                                                                  (uint16_t*)meta, (uint8_t*)meta_hw,
+                                                                  (uint16_t*)dense_out, (int)px, num_panels);
   }
   SF_LAUNCH_CHECK();
   return SF_OK;
