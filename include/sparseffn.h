@@ -197,9 +197,15 @@ typedef enum sf_ctx_field {
   SF_CTX_META = 2,      /* uint16 [T, F/(4M)] canonical */
   SF_CTX_COLIDX = 3,    /* uint8 [T/V, F/M, 4] */
   SF_CTX_Y1 = 4,        /* bf16 [T, F] (only with flags bit0) */
-  SF_CTX_DY1_VALS = 5   /* bf16 [T, 2F/M], lives in the WORKSPACE after sf_sparse_ffn_bwd; for M == 8 it
+  SF_CTX_DY1_VALS = 5,  /* bf16 [T, 2F/M], lives in the WORKSPACE after sf_sparse_ffn_bwd; for M == 8 it
                            is only written when flags bit0 is set (the products then consume dy1 in
                            its 2:4 form over all F columns instead) */
+  SF_CTX_Y2_VALS24 = 6, /* bf16 [T, F/2]: y2 as a plain 2:4 operand over all F columns (M <= 8 only,
+                           else SF_ERR_UNSUPPORTED): two stored values per four columns, explicit
+                           zeros where a half-group keeps fewer than two */
+  SF_CTX_Y2_META24 = 7, /* uint16 [T, F/16] canonical metadata of that operand (M <= 8 only) */
+  SF_CTX_DY1_VALS24 = 8 /* bf16 [T, F/2]: dy1 at the positions of SF_CTX_Y2_META24; lives in the WORKSPACE
+                           after sf_sparse_ffn_bwd (M <= 8 only) */
 } sf_ctx_field;
 SF_API int sf_ctx_view(const sf_ffn_desc* desc, const void* fwd_ctx_or_workspace, int field,
                 const void** ptr, size_t* bytes);

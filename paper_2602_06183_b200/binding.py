@@ -21,6 +21,7 @@ SF_ERR_NULL, SF_ERR_SHAPE, SF_ERR_ALIGN, SF_ERR_WORKSPACE = -1, -2, -3, -4
 SF_ERR_ARCH, SF_ERR_CUDA, SF_ERR_TIMEOUT, SF_ERR_UNSUPPORTED = -5, -6, -7, -8
 
 SF_CTX_Y2_VALS, SF_CTX_RELU_VALS, SF_CTX_META, SF_CTX_COLIDX, SF_CTX_Y1, SF_CTX_DY1_VALS = range(6)
+SF_CTX_Y2_VALS24, SF_CTX_Y2_META24, SF_CTX_DY1_VALS24 = 6, 7, 8
 
 
 class sf_ffn_desc(C.Structure):
@@ -295,7 +296,8 @@ def sf_dense_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stre
 
 
 _CTX_DTYPES = {SF_CTX_Y2_VALS: torch.bfloat16, SF_CTX_RELU_VALS: torch.bfloat16, SF_CTX_META: torch.int16,
-               SF_CTX_COLIDX: torch.uint8, SF_CTX_Y1: torch.bfloat16, SF_CTX_DY1_VALS: torch.bfloat16}
+               SF_CTX_COLIDX: torch.uint8, SF_CTX_Y1: torch.bfloat16, SF_CTX_DY1_VALS: torch.bfloat16,
+               SF_CTX_Y2_VALS24: torch.bfloat16, SF_CTX_Y2_META24: torch.int16, SF_CTX_DY1_VALS24: torch.bfloat16}
 
 
 def sf_ctx_view(desc, buf: torch.Tensor, field: int) -> torch.Tensor:

@@ -465,6 +465,15 @@ int sf_ctx_view(const sf_ffn_desc* desc, const void* buf, int field, const void*
       if (!(d.flags & 1)) return SF_ERR_UNSUPPORTED;
       off = L.y1; n = T * F * 2; break;
     case SF_CTX_DY1_VALS: off = L.dy1_vals; n = T * 2 * G * 2; break;
+    case SF_CTX_Y2_VALS24:
+      if (!L.plain24) return SF_ERR_UNSUPPORTED;
+      off = L.vals24; n = T * F; break;
+    case SF_CTX_Y2_META24:
+      if (!L.plain24) return SF_ERR_UNSUPPORTED;
+      off = L.meta24; n = T * F / 8; break;
+    case SF_CTX_DY1_VALS24:
+      if (!L.plain24) return SF_ERR_UNSUPPORTED;
+      off = L.dy1_vals24; n = T * F; break;
     default: return SF_ERR_SHAPE;
   }
   *ptr = at(buf, off);

@@ -68,6 +68,39 @@ def test_sparse_ffn_c1_teacher_forced(prune_mode, act_shift):
     assert rel_fro(g["Y"], free.y3) < 5e-2
 
 
+@pytest.mark.parametrize("M,act_shift", [(8, 0.0), (8, -1.3), (4, 0.0)])
+def test_plain_24_view_of_y2_and_dy1_is_exact(M, act_shift):
+    """For M <= 8 the products consume y2 / dy1 as plain 2:4 operands over all F columns. That view,
+    decompressed with its own metadata, must be the oracle's masked dense y2 bit for bit, hold at
+    most two entries per four columns with ascending positions, and dy1's view must be the masked
+    dense dy1 at the same positions."""
+    cfg = dict(synth.FFN_CONFIGS["c1_small"], M=M)
+    T, D, F, V = cfg["T"], cfg["D"], cfg["F"], cfg["V"]
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"], act_shift=act_shift)
+    desc = binding.make_desc(T, D, F, V, M, flags=1)
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
+    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+    gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
+    binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
+    binding.sf_sparse_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    y1 = bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y1)).reshape(T, F)
+    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, forced_y1b=y1)
+    v24 = bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y2_VALS24)).reshape(T, F // 2)
+    m24 = bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y2_META24)).reshape(T, F // 16)
+    nib = np.stack([(m24 >> np.uint16(4 * i)) & np.uint16(0xF) for i in range(4)], axis=-1)
+    assert ((nib & 3) < (nib >> 2)).all()                        # legal position pairs everywhere
+    assert np.array_equal(oracle.decompress24(v24, m24), fwd.act.dense)
+    # dy1 in the same positions: compare with the masked dense dy1 the oracle derives from the GPU's masks
+    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd)
+    d24 = bits(binding.sf_ctx_view(desc, ws, binding.SF_CTX_DY1_VALS24)).reshape(T, F // 2)
+    dy1_gpu = oracle.decompress24(d24, m24)
+    dy1_ref = oracle.decompress_vnm(bwd.dy1_vals, fwd.act.meta, fwd.act.colidx, V=V, M=M)
+    assert not (dy1_gpu[~fwd.act.mask] != 0).any()               # nothing outside y2's mask
+    assert rel_fro(oracle.bf16_to_f32(dy1_gpu), oracle.bf16_to_f32(dy1_ref)) < TOL
+
+
 def test_sparse_ffn_v128_m16():
     cfg = dict(T=512, D=256, F=2048, V=128, N=2, M=16, sigma_w=0.05, seed=17)
     (X, W1, W2, dY), g = _run_sparse(cfg)
