@@ -207,6 +207,8 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
   uint32_t* score = reinterpret_cast<uint32_t*>(tile + (size_t)V * (kW + kPad));
   uint8_t* keepf = reinterpret_cast<uint8_t*>(score + kW);
   uint8_t* cidx = keepf + kW;
+  uint4* sel_tab = reinterpret_cast<uint4*>(cidx + kW);                          // [kW / 8][7] selector words
+  uint8_t* nib_tab = reinterpret_cast<uint8_t*>(sel_tab + (kW / 8) * 7);         // [kW / 8][7] 2:4-view nibble pairs
   constexpr int kRow = kW + kPad;
 
   const int tid = threadIdx.x;
@@ -277,6 +279,38 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
     *reinterpret_cast<uint32_t*>(colidx + (blk * G + c0 / M + tid) * 4) = c4;
   }
 
+  // Selector table: a group's row keeps one of six position pairs (i < j) of its four kept columns.
+  // Everything the row loop derives from that pair -- byte-permute selectors that scatter the two
+  // kept values into the four dense words, pick the two ReLU values out of the row's words, and lay
+  // the pair out as a plain 2:4 operand with its nibble pair -- depends on (group, pair) only, so
+  // it is tabulated once per strip: slot = nibble % 7 is distinct for the six legal nibbles.
+  if (tid < ng * 6) {
+    const int ge = tid / 6, pe = tid - ge * 6;
+    const int pi = pe < 3 ? 0 : (pe < 5 ? 1 : 2), pj = pe < 3 ? pe + 1 : (pe < 5 ? pe - 1 : 3);
+    const uint32_t ca = cidx[ge * 4 + pi], cb = cidx[ge * 4 + pj];                // kept columns, ca < cb
+    const uint32_t nibp = (uint32_t)pi | ((uint32_t)pj << 2);
+    uint32_t sd[4];
+#pragma unroll
+    for (uint32_t j = 0; j < 4; ++j) {
+      const uint32_t lo = ca == 2 * j ? 0x10u : (cb == 2 * j ? 0x32u : 0x44u);
+      const uint32_t hi = ca == 2 * j + 1 ? 0x10u : (cb == 2 * j + 1 ? 0x32u : 0x44u);
+      sd[j] = lo | (hi << 8);
+    }
+    const uint32_t pa = ca & 3u, pb = cb & 3u;
+    const uint32_t s1 = (2u * pa) | ((2u * pa + 1u) << 4) | ((2u * pb) << 8) | ((2u * pb + 1u) << 12);
+    const uint32_t s2 = (ca < 4u ? 0x10u : 0x54u) | ((cb < 4u ? 0x32u : 0x76u) << 8);
+    const bool both_lo = cb < 4u, both_hi = ca >= 4u;
+    const uint32_t s_wlo = both_lo ? 0x3210u : (both_hi ? 0x4444u : (pa == 0u ? 0x4410u : 0x1044u));
+    const uint32_t s_whi = both_hi ? 0x3210u : (both_lo ? 0x4444u : (pb == 0u ? 0x4432u : 0x3244u));
+    const uint32_t pair_nib = pa | (pb << 2);
+    const uint32_t nlo = both_lo ? pair_nib : (both_hi ? 4u : (pa == 0u ? 4u : (pa << 2)));
+    const uint32_t nhi = both_hi ? pair_nib : (both_lo ? 4u : (pb == 0u ? 4u : (pb << 2)));
+    const int slot = ge * 7 + (int)(nibp % 7u);
+    sel_tab[slot] = make_uint4(sd[0] | (sd[1] << 16), sd[2] | (sd[3] << 16), s1 | (s2 << 16), s_wlo | (s_whi << 16));
+    nib_tab[slot] = (uint8_t)(nlo | (nhi << 4));
+  }
+  __syncthreads();
+
   // pass B: a thread serves one group g = tid % ng for rows tid / ng, tid / ng + kThreads / ng, ...
   // Everything that depends only on (thread, group) is computed once; the row loop advances
   // pointers by constant strides.
@@ -293,8 +327,11 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
   }
   const bool lead4 = (g & 3) == 0, lead2 = (g & 1) == 0;
   const bool want_relu = relu_vals && apply, want24 = vals24 != nullptr;
+  const bool need_relu_pair = want_relu || (relu_dense_out != nullptr);
   const int64_t trow = t0 + r0;
   const uint16_t* tp = tile + r0 * kRow + g * M;
+  const uint4* my_sel = sel_tab + g * 7;
+  const uint8_t* my_nib = nib_tab + g * 7;
   uint16_t* p_vals = vals + trow * (2 * G) + 2 * (g0 + g);
   uint16_t* p_relu = want_relu ? relu_vals + trow * (2 * G) + 2 * (g0 + g) : nullptr;
   uint16_t* p_dense = dense_out ? dense_out + trow * F + c0 + g * M : nullptr;
@@ -308,7 +345,6 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
   uint8_t* hw24_atom = want24 ? meta24_hw + meta_hw_offset(t0 & ~int64_t(127), kw24, F) : nullptr;
   const int s_vals = rstep * (int)(2 * G), s_dense = rstep * (int)F, s_v24 = rstep * (int)(F >> 1);
   const int s_meta = rstep * (int)(G >> 2), s_m24 = rstep * (int)(F >> 4);
-  const bool any_dense = dense_out || relu_dense_out;
   for (int r = r0; r < V; r += rstep) {
     const uint4 q = *reinterpret_cast<const uint4*>(tp);
     uint32_t rw[4] = {q.x, q.y, q.z, q.w}, hw[4];
@@ -325,25 +361,22 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
     const uint32_t hk0 = (a0 & ~mhi[0]) | (b0 & mhi[0]), hk1 = (a1 & ~mhi[1]) | (b1 & mhi[1]);
     uint32_t packed;
     const uint32_t nib = top2of4_packed(hk0, hk1, &packed);
-    const uint32_t p0 = nib & 3u, p1 = nib >> 2;
     *reinterpret_cast<uint32_t*>(p_vals) = packed;
-    const uint32_t ca = (c4 >> (8 * p0)) & 0xFFu, cb = (c4 >> (8 * p1)) & 0xFFu;         // kept columns, ca < cb
-    if (want_relu) {
-      // the two kept ReLU values straight from the group's words (columns ca, cb)
-      const uint32_t sel = 2u * (ca & 3u) | ((2u * (ca & 3u) + 1u) << 4) | ((2u * (cb & 3u)) << 8) | ((2u * (cb & 3u) + 1u) << 12);
-      const uint32_t ra = __byte_perm(rw[0], rw[1], sel), rb = __byte_perm(rw[2], rw[3], sel);
-      const uint32_t mh = ((ca & 4u) ? 0x0000FFFFu : 0u) | ((cb & 4u) ? 0xFFFF0000u : 0u);
-      *reinterpret_cast<uint32_t*>(p_relu) = (ra & ~mh) | (rb & mh);
+    // this row's pair -> its tabulated selectors (nib % 7 without a division: nib < 16)
+    const uint32_t slot = nib - 7u * ((nib * 37u) >> 8);
+    const uint4 sel = my_sel[slot];
+    if (need_relu_pair) {
+      // the two kept ReLU values straight from the group's words
+      const uint32_t x = __byte_perm(rw[0], rw[1], sel.z), y = __byte_perm(rw[2], rw[3], sel.z);
+      const uint32_t rpair = __byte_perm(x, y, sel.z >> 16);
+      if (want_relu) *reinterpret_cast<uint32_t*>(p_relu) = rpair;
+      if (relu_dense_out)
+        *reinterpret_cast<uint4*>(p_rdense) = make_uint4(__byte_perm(rpair, 0u, sel.x), __byte_perm(rpair, 0u, sel.x >> 16),
+                                                         __byte_perm(rpair, 0u, sel.y), __byte_perm(rpair, 0u, sel.y >> 16));
     }
-    if (any_dense) {
-      const uint32_t kb = (1u << ca) | (1u << cb);
-      uint32_t mk[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        mk[j] = (((kb >> (2 * j)) & 1u) * 0xFFFFu) | (((kb >> (2 * j + 1)) & 1u) * 0xFFFF0000u);
-      if (dense_out) *reinterpret_cast<uint4*>(p_dense) = make_uint4(hw[0] & mk[0], hw[1] & mk[1], hw[2] & mk[2], hw[3] & mk[3]);
-      if (relu_dense_out) *reinterpret_cast<uint4*>(p_rdense) = make_uint4(rw[0] & mk[0], rw[1] & mk[1], rw[2] & mk[2], rw[3] & mk[3]);
-    }
+    if (dense_out)
+      *reinterpret_cast<uint4*>(p_dense) = make_uint4(__byte_perm(packed, 0u, sel.x), __byte_perm(packed, 0u, sel.x >> 16),
+                                                      __byte_perm(packed, 0u, sel.y), __byte_perm(packed, 0u, sel.y >> 16));
     uint32_t word = nib;
     word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 4;
     word |= __shfl_down_sync(0xFFFFFFFFu, word, 2) << 8;
@@ -359,19 +392,8 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
     // legal position pair. A half-group with one kept value at position p pairs it with a zero
     // at position 1 (p = 0) or 0 (p > 0).
     if (want24) {
-      const uint32_t va = packed & 0xFFFFu, vb = packed >> 16;
-      const bool both_lo = cb < 4u, both_hi = ca >= 4u;
-      const uint32_t pb = cb & 3u, pa = ca & 3u;
-      // split case values / nibbles
-      const uint32_t s_wlo = pa == 0u ? va : (va << 16), s_nlo = pa == 0u ? 4u : (pa << 2);
-      const uint32_t s_whi = pb == 0u ? vb : (vb << 16), s_nhi = pb == 0u ? 4u : (pb << 2);
-      const uint32_t pair_nib = pa | (pb << 2);
-      const uint32_t wlo = both_lo ? packed : (both_hi ? 0u : s_wlo);
-      const uint32_t whi = both_hi ? packed : (both_lo ? 0u : s_whi);
-      const uint32_t nlo = both_lo ? pair_nib : (both_hi ? 4u : s_nlo);
-      const uint32_t nhi = both_hi ? pair_nib : (both_lo ? 4u : s_nhi);
-      *reinterpret_cast<uint2*>(p_v24) = make_uint2(wlo, whi);
-      uint32_t mb = nlo | (nhi << 4);
+      *reinterpret_cast<uint2*>(p_v24) = make_uint2(__byte_perm(packed, 0u, sel.w), __byte_perm(packed, 0u, sel.w >> 16));
+      uint32_t mb = my_nib[slot];
       mb |= __shfl_down_sync(0xFFFFFFFFu, mb, 1) << 8;
       if (lead2) {
         *p_m24 = (uint16_t)mb;
@@ -437,10 +459,10 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
     static bool attr8[64] = {false};
     if (dev < 0 || dev >= 64 || !attr8[dev]) {
       SF_CUDA_TRY(cudaFuncSetAttribute(vnm8_kernel<kW8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       128 * (kW8 + kPad) * 2 + kW8 * 6));
+                                       128 * (kW8 + kPad) * 2 + kW8 * 6 + (kW8 / 8) * 7 * 17));
       if (dev >= 0 && dev < 64) attr8[dev] = true;
     }
-    const size_t smem8 = (size_t)V * (kW8 + kPad) * 2 + kW8 * 6;
+    const size_t smem8 = (size_t)V * (kW8 + kPad) * 2 + kW8 * 6 + (kW8 / 8) * 7 * 17;
     dim3 grid8((unsigned)((F + kW8 - 1) / kW8), (unsigned)(T / V));
     vnm8_kernel<kW8><<<grid8, kThreads, smem8, s>>>((const uint16_t*)P, T, F, ld, V, apply_sqrelu, (uint16_t*)vals,
                                                     (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
