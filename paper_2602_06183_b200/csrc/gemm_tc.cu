@@ -75,29 +75,32 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // ---- epilogue (shared by the one-CTA and the two-CTA kernels) ---------------------------------------
 // One epilogue warp owns TMEM lanes [32q, 32q+32) of a 128 x 256 accumulator tile whose first row is
 // m0 and first column n0; `taddr` is the TMEM address of (lane 32q, column 0) of that accumulator.
-constexpr int kAuxChunks = BN / 32;
-
-template <int kEpi>
+// kTileN: accumulator columns of the tile (a multiple of 32). Columns at or beyond args.N (a ragged last
+// tile, whole 32-column chunks only since N % 32 == 0) are neither prefetched nor stored.
+template <int kEpi, int kTileN = BN>
 __device__ __forceinline__ void epi_prefetch(const GemmArgs& args, int64_t m0, int64_t n0, int q, int lane,
-                                             uint4 (&ax)[kEpi == EPI_DRELU_T ? kAuxChunks : 1][4]) {
+                                             uint4 (&ax)[kEpi == EPI_DRELU_T ? kTileN / 32 : 1][4]) {
   if (kEpi == EPI_DRELU_T) {
 #pragma unroll
-    for (int ch = 0; ch < kAuxChunks; ++ch)
+    for (int ch = 0; ch < kTileN / 32; ++ch) {
+      if (n0 + ch * 32 >= args.N) break;
 #pragma unroll
       for (int i = 0; i < 4; ++i)
         ax[kEpi == EPI_DRELU_T ? ch : 0][i] = __ldg(reinterpret_cast<const uint4*>(
             reinterpret_cast<const uint16_t*>(args.aux) + (n0 + ch * 32 + i * 8 + (lane >> 2)) * args.ldaux + m0 +
             q * 32 + (lane & 3) * 8));
+    }
   }
 }
 
-template <int kEpi>
+template <int kEpi, int kTileN = BN>
 __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0, int q, int lane,
                                          uint8_t* my_stage,
-                                         const uint4 (&ax)[kEpi == EPI_DRELU_T ? kAuxChunks : 1][4]) {
+                                         const uint4 (&ax)[kEpi == EPI_DRELU_T ? kTileN / 32 : 1][4]) {
   const int64_t row = m0 + q * 32 + lane;                                  // this thread's D row
   auto chunk = [&](int ch, const uint4 (&a4)[4], const uint32_t (&v)[32]) {
     const int64_t col0 = n0 + ch * 32;
+    if (col0 >= args.N) return;                                            // ragged last tile (warp-uniform)
     if (kEpi == EPI_STORE || kEpi == EPI_SQRELU || kEpi == EPI_DRELU) {
       uint16_t* crow = reinterpret_cast<uint16_t*>(args.C) + row * args.ldc + col0;
       if (kEpi == EPI_STORE) {
@@ -183,25 +186,40 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
   // Two register buffers: the TMEM load of the next 32 columns is in flight while this one is converted.
   uint32_t va[32], vb[32];
   tmem_ld_32x32b_x32(taddr, va);
+  constexpr int kChunks = kTileN / 32;
   if (kEpi == EPI_DRELU_T) {
 #pragma unroll
-    for (int ch = 0; ch < BN / 32; ch += 2) {
+    for (int ch = 0; ch < kChunks; ch += 2) {
       tmem_ld_wait_on(va);
-      tmem_ld_32x32b_x32(taddr + (ch + 1) * 32, vb);
+      if (ch + 1 < kChunks) tmem_ld_32x32b_x32(taddr + (ch + 1) * 32, vb);
       chunk(ch, ax[kEpi == EPI_DRELU_T ? ch : 0], va);
-      tmem_ld_wait_on(vb);
-      if (ch + 2 < BN / 32) tmem_ld_32x32b_x32(taddr + (ch + 2) * 32, va);
-      chunk(ch + 1, ax[kEpi == EPI_DRELU_T ? ch + 1 : 0], vb);
+      if (ch + 1 < kChunks) {
+        tmem_ld_wait_on(vb);
+        if (ch + 2 < kChunks) tmem_ld_32x32b_x32(taddr + (ch + 2) * 32, va);
+        chunk(ch + 1, ax[kEpi == EPI_DRELU_T ? (ch + 1 < kChunks ? ch + 1 : ch) : 0], vb);
+      }
     }
-  } else {
+  } else if (kChunks % 2 == 0) {
 #pragma unroll 1
-    for (int ch = 0; ch < BN / 32; ch += 2) {
+    for (int ch = 0; ch < kChunks; ch += 2) {
       tmem_ld_wait_on(va);
       tmem_ld_32x32b_x32(taddr + (ch + 1) * 32, vb);
       chunk(ch, ax[0], va);
       tmem_ld_wait_on(vb);
-      if (ch + 2 < BN / 32) tmem_ld_32x32b_x32(taddr + (ch + 2) * 32, va);
+      if (ch + 2 < kChunks) tmem_ld_32x32b_x32(taddr + (ch + 2) * 32, va);
       chunk(ch + 1, ax[0], vb);
+    }
+  } else {
+#pragma unroll
+    for (int ch = 0; ch < kChunks; ch += 2) {
+      tmem_ld_wait_on(va);
+      if (ch + 1 < kChunks) tmem_ld_32x32b_x32(taddr + (ch + 1) * 32, vb);
+      chunk(ch, ax[0], va);
+      if (ch + 1 < kChunks) {
+        tmem_ld_wait_on(vb);
+        if (ch + 2 < kChunks) tmem_ld_32x32b_x32(taddr + (ch + 2) * 32, va);
+        chunk(ch + 1, ax[0], vb);
+      }
     }
   }
 }
@@ -462,10 +480,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 // Stage = 64 K (dense, 4 MMAs of K=16) or 128 logical K (2:4, 4 MMAs of K=32 and one metadata atom):
 // four MMAs per barrier round trip keep the single issuing thread ahead of the tensor pipe.
 constexpr int kThreads2 = 192;
-__host__ __device__ constexpr int stage_bytes2(bool sparse) { return sparse ? (16384 + 32768 + 2048) : (16384 + 16384); }
+__host__ __device__ constexpr int stage_bytes2(bool sparse, int bn = BN) {
+  return sparse ? (16384 + 2 * (bn / 2) * 128 + 2048) : (16384 + 16384);
+}
 __host__ __device__ constexpr int num_stages2(bool sparse) { return sparse ? 4 : 6; }
-__host__ __device__ constexpr int smem_bytes2(bool sparse) {
-  return 1024 + num_stages2(sparse) * stage_bytes2(sparse) + kEpiStageBytes + 512;
+__host__ __device__ constexpr int smem_bytes2(bool sparse, int bn = BN) {
+  return 1024 + num_stages2(sparse) * stage_bytes2(sparse, bn) + kEpiStageBytes + 512;
 }
 
 struct SmemCtl2 {
@@ -481,7 +501,7 @@ __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
   return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 
-template <int kMode, bool kAMN, bool kBMN, int kEpi>
+template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                 const __grid_constant__ CUtensorMap tmapMeta, const GemmArgs args) {
@@ -491,9 +511,17 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   constexpr int kStages = num_stages2(kSparse);
   constexpr int kBK = kSparse ? 128 : 64;                // logical K per stage
   constexpr int kAStageBytes = 16384;
-  constexpr int kBHalfBytes = kSparse ? 32768 : 16384;
-  constexpr int kStageBytes = stage_bytes2(kSparse);
-  constexpr int kAccBufs = kSparse ? 1 : 2;
+  constexpr int kBSlabBytes = (kBN / 2) * 128;            // this CTA's half of B for one 64-wide K slab
+  constexpr int kBHalfBytes = kSparse ? 2 * kBSlabBytes : kBSlabBytes;
+  constexpr int kStageBytes = stage_bytes2(kSparse, kBN);
+  // 2:4 mode: TMEM holds the metadata next to the accumulators, so 256-column tiles leave room for one
+  // accumulator only; 224-column tiles fit two (448 columns + 8 of metadata) and the epilogue of a tile
+  // then overlaps the main loop of the next.
+  constexpr int kAccBufs = (kSparse && kBN > 248) ? 1 : 2;
+  constexpr uint32_t kMetaCol = kSparse ? (uint32_t)(kAccBufs * kBN) : 0u;
+  static_assert(kBN % 32 == 0 && kBN <= 256, "tile width");
+  static_assert(!(kMode == MODE_DENSE) || kBN == BN, "dense mode uses 256-column tiles");
+  static_assert(!kBMN || kBN == BN, "MN-major B is loaded in 64-column chunks");
   uint8_t* epi_stage = smem + kStages * kStageBytes;
   SmemCtl2* ctl = reinterpret_cast<SmemCtl2*>(epi_stage + kEpiStageBytes);
   volatile int* abort_flag = &ctl->abort_flag;
@@ -538,7 +566,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
       int mt, nt;
       tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
       const int m0 = mt * 256 + (int)rank * 128;         // this CTA's rows of A / D
-      const int nb0 = nt * BN + (int)rank * 128;         // this CTA's columns of B
+      const int nb0 = nt * kBN + (int)rank * (kBN / 2);  // this CTA's columns of B
       for (int kb = 0; kb < nkb; ++kb) {
         if (!mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
         if (lane == 0) {
@@ -571,7 +599,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
             tma_load_2d_2cta(sM, &tmapMeta, bar, 0, 2 * atom);
             if (!kBMN) {
               tma_load_2d_2cta(sB, &tmapB, bar, kb * 128, nb0);                // two 64-wide K slabs
-              tma_load_2d_2cta(sB + 16384, &tmapB, bar, kb * 128 + 64, nb0);
+              tma_load_2d_2cta(sB + kBSlabBytes, &tmapB, bar, kb * 128 + 64, nb0);
             } else {
               tma_load_2d_2cta(sB, &tmapB, bar, nb0, kb * 128);                // two chunks {64 n, 128 k}
               tma_load_2d_2cta(sB + 16384, &tmapB, bar, nb0 + 64, kb * 128);
@@ -584,7 +612,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   } else if (warp == 1) {
     // =========================== MMA issuer (leader CTA only) ===========================
     if (rank == 0 && lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(256, BN, kAMN, kBMN, kSparse);
+      constexpr uint32_t idesc = idesc_bf16(256, kBN, kAMN, kBMN, kSparse);
       // Descriptor halves that never change: high word = stride offset, version, swizzle; the low
       // word is (address >> 4) | leading offset, advanced by plain 32-bit adds.
       const uint32_t smem0 = smem_u32(smem);
@@ -605,13 +633,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
       for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
         if (!mbar_wait(&ctl->tmem_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t tmem_d = tmem_base + acc * BN;
+        const uint32_t tmem_d = tmem_base + acc * kBN;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!mbar_wait(&ctl->full[stage], phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t soff = stage * (uint32_t)(kStageBytes >> 4);
           const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
-          const uint32_t mbuf = tmem_base + kMetaTmemCol + 4u * ((uint32_t)kb & 1u);   // metadata double buffer
+          const uint32_t mbuf = tmem_base + kMetaCol + 4u * ((uint32_t)kb & 1u);       // metadata double buffer
           if (kSparse) tmem_cp_128x128b_2cta(mbuf, desc64(m_lo0 + soff, m_hi));
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
@@ -619,7 +647,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
             if (kSparse) {
               // K = 32 per instruction: 32 B of stored A, 64 B of B inside a 64-wide K slab
               const uint32_t bk = kBMN ? (uint32_t)k * (4096 >> 4)      // 32 k rows of 128 B
-                                       : (uint32_t)((k >> 1) * (16384 >> 4) + (k & 1) * (64 >> 4));
+                                       : (uint32_t)((k >> 1) * (kBSlabBytes >> 4) + (k & 1) * (64 >> 4));
               mma_sp_f16_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi),
                               mbuf + (uint32_t)(k & ~1), idesc | (uint32_t)(k & 1), accum);
             } else {
@@ -644,13 +672,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
       int mt, nt;
       tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
-      const int64_t m0 = (int64_t)mt * 256 + (int64_t)rank * 128, n0 = (int64_t)nt * BN;
-      uint4 ax[kEpi == EPI_DRELU_T ? kAuxChunks : 1][4];
-      epi_prefetch<kEpi>(args, m0, n0, q, lane, ax);
+      const int64_t m0 = (int64_t)mt * 256 + (int64_t)rank * 128, n0 = (int64_t)nt * kBN;
+      uint4 ax[kEpi == EPI_DRELU_T ? kBN / 32 : 1][4];
+      epi_prefetch<kEpi, kBN>(args, m0, n0, q, lane, ax);
       if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
-      epi_tile<kEpi>(args, taddr, m0, n0, q, lane, my_stage, ax);
+      const uint32_t taddr = tmem_base + acc * kBN + ((uint32_t)(q * 32) << 16);
+      epi_tile<kEpi, kBN>(args, taddr, m0, n0, q, lane, my_stage, ax);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(&ctl->tmem_empty[acc]);
@@ -739,10 +767,10 @@ int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& a, 
   return SF_OK;
 }
 
-template <int kMode, bool kAMN, bool kBMN, int kEpi>
+template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN>
 int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tm, GemmArgs a, cudaStream_t s) {
-  auto kern = gemm_tc2_kernel<kMode, kAMN, kBMN, kEpi>;
-  constexpr int smem = smem_bytes2(kMode != MODE_DENSE);
+  auto kern = gemm_tc2_kernel<kMode, kAMN, kBMN, kEpi, kBN>;
+  constexpr int smem = smem_bytes2(kMode != MODE_DENSE, kBN);
   static bool attr_done[64] = {false};
   int dev = 0;
   SF_CUDA_TRY(cudaGetDevice(&dev));
@@ -751,6 +779,7 @@ int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
     if (dev >= 0 && dev < 64) attr_done[dev] = true;
   }
   a.num_m_tiles = (int)(a.M / 256);
+  a.num_n_tiles = (int)((a.N + kBN - 1) / kBN);
   const int tiles = a.num_m_tiles * a.num_n_tiles;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
@@ -758,6 +787,10 @@ int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
+
+// Tile width of the two-accumulator 2:4 variant (transposed-output products): 2 x 224 accumulator
+// columns + 8 metadata columns fit the 512 TMEM columns.
+constexpr int kNarrowBN = 224;
 
 // The two-CTA kernels need M % 256 == 0; other shapes run the one-CTA kernels.
 bool use_two_cta(int64_t M) { return M % 256 == 0; }
@@ -813,7 +846,9 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
   int st = two ? make_tmap(&ta, a_vals, M, K / 2, K / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)
                : make_tmap(&ta, a_vals, M, K / 2, K / 2, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B);
   if (st != SF_OK) return st;
-  if (b_kmajor) st = make_tmap(&tb, B, N, K, K, 64, two ? 128 : 256, CU_TENSOR_MAP_SWIZZLE_128B);
+  // transposed-output products on CTA pairs run 224-column tiles with two accumulators
+  const bool narrow = two && !plain;
+  if (b_kmajor) st = make_tmap(&tb, B, N, K, K, 64, two ? (narrow ? kNarrowBN / 2 : 128) : 256, CU_TENSOR_MAP_SWIZZLE_128B);
   else          st = make_tmap(&tb, B, K, N, N, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
   if (st != SF_OK) return st;
   tm = ta;
@@ -832,10 +867,10 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
     return launch_two<MODE_SPARSE24, false, true, EPI_STORE>(ta, tb, tm, a, s);
   }
   if (epi == EPI_STORE_T)
-    return two ? launch_two<MODE_SPARSE24, false, false, EPI_STORE_T>(ta, tb, tm, a, s)
+    return two ? launch_two<MODE_SPARSE24, false, false, EPI_STORE_T, kNarrowBN>(ta, tb, tm, a, s)
                : launch_one<MODE_SPARSE24, false, false, EPI_STORE_T>(ta, tb, a, s);
   if (epi == EPI_DRELU_T)
-    return two ? launch_two<MODE_SPARSE24, false, false, EPI_DRELU_T>(ta, tb, tm, a, s)
+    return two ? launch_two<MODE_SPARSE24, false, false, EPI_DRELU_T, kNarrowBN>(ta, tb, tm, a, s)
                : launch_one<MODE_SPARSE24, false, false, EPI_DRELU_T>(ta, tb, a, s);
   return SF_ERR_UNSUPPORTED;
 }
