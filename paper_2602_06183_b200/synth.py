@@ -35,6 +35,8 @@ FFN_CONFIGS = {
     "c4_slice": dict(T=1024, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
     # the same slice with groups of 16 (87.5 % sparse activations): exercises the condensed Venom products
     "c4_slice_m16": dict(T=1024, D=4096, F=16384, V=128, N=2, M=16, sigma_w=0.02, seed=4),
+    # c4 with groups of 16 (Table 5's 87.5 % row): the full-size case of the condensed Venom products
+    "c4_d4096_m16": dict(T=8192, D=4096, F=16384, V=128, N=2, M=16, sigma_w=0.02, seed=4),
     "c5_d8192": dict(T=16384, D=8192, F=28672, V=128, N=2, M=8, sigma_w=0.015, seed=5),
 }
 

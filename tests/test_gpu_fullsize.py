@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-2
 
 
-@pytest.mark.parametrize("name", ["c4_d4096", "c5_d8192"])
+@pytest.mark.parametrize("name", ["c4_d4096", "c4_d4096_m16", "c5_d8192"])
 def test_ffn_step_full_size_sampled(name):
     cfg = synth.FFN_CONFIGS[name]
     T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
