@@ -283,7 +283,8 @@ SF_API int sf_probe_mma_rate(int sparse, int two_cta, int iters, void* cycles, v
  * tracing is switched off with capacity 0. While set, every FFN step call records one event
  * before its first kernel and one after each kernel, in launch order, on the call's stream:
  *   sparse fwd: 6 events (prune W1 | y1 product | V:N:M | W2 transpose | y3 product)
- *   sparse bwd: 7 events (prune W2 | dy1 product | pack | dX product | dW2 product | dW1 product)
+ *   sparse bwd: 7 events (prune W2 | dy1 product | pack | dX product | dW2 product | dW1 product);
+ *               for M <= 8 the dy1 product packs its own output and the pack interval is empty
  *   dense fwd: 3 events, dense bwd: 5 events.
  * sf_trace_count returns how many events have been recorded since sf_trace_set. Not thread-safe. */
 SF_API int sf_trace_set(void** events, int capacity);

@@ -365,13 +365,14 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
                           at(workspace, L.w2_meta), at(workspace, L.w2_meta_hw), nullptr, s));
   }
   trace_mark(s);
+  // (M <= 8: the same epilogue also packs dy1 with y2's 2:4 metadata, the operand of the dX product)
   SF_TRY(gemm_sparse24(at(workspace, L.w2_vals), at(workspace, L.w2_meta_hw), dY, true, d.F, d.T, d.D, EPI_DRELU_T,
-                       at(workspace, L.dy1_dense), d.F, at(fwd_ctx, L.relu_dense), d.F, status, s));
+                       at(workspace, L.dy1_dense), d.F, at(fwd_ctx, L.relu_dense), d.F, status, s,
+                       L.plain24 ? at(fwd_ctx, L.meta24) : nullptr, L.plain24 ? at(workspace, L.dy1_vals24) : nullptr));
   trace_mark(s);
   // line 5: dX = dy1 W1 with W1 dense
   if (L.plain24) {
-    // dy1 shares y2's positions: pack it with the same 2:4 metadata; W1 [F, D] is the MN-major operand
-    SF_TRY(launch_pack24(at(workspace, L.dy1_dense), at(fwd_ctx, L.meta24), at(workspace, L.dy1_vals24), d.T, d.F, s));
+    // dy1 shares y2's positions and was packed by the product above; W1 [F, D] is the MN-major operand
     if ((d.flags & 1) && d.M == 8)    // debug: also the V:N:M-packed form
       SF_TRY(launch_pack_like(at(workspace, L.dy1_dense), at(fwd_ctx, L.meta), at(fwd_ctx, L.colidx),
                               at(workspace, L.dy1_vals), d.T, d.F, d.V, d.M, s));

@@ -150,6 +150,16 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
     } else {
       // Transposed output: D row = feature (lane), D column = token. C is [N, M] row-major.
       float r[32];
+      // optional packed copy: the metadata words of this chunk's 32 tokens (features m0 + 32q .. + 31)
+      const bool pack = kEpi == EPI_DRELU_T && args.pack_vals != nullptr;
+      uint32_t mw[4] = {0, 0, 0, 0};
+      if (pack) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          mw[i] = __ldg(reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(args.pack_meta) +
+                                                         (col0 + i * 8 + (lane >> 2)) * (args.M >> 3) +
+                                                         ((m0 + q * 32) >> 3)));
+      }
       if (kEpi == EPI_DRELU_T) {
         // aux[token, feature] chunk -> staging -> one column per lane
         __syncwarp();
@@ -180,6 +190,14 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
         const int t = i * 8 + (lane >> 2), seg = lane & 3;
         const uint4 o = *reinterpret_cast<const uint4*>(my_stage + t * kEpiStageRow + seg * 16);
         *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.C) + (col0 + t) * args.ldc + m0 + q * 32 + seg * 8) = o;
+        if (pack) {
+          // this lane's eight features are two groups of four: keep the two recorded positions of each
+          const uint32_t mb = (mw[i] >> (8 * seg)) & 0xFFu;
+          const uint32_t p0 = __byte_perm(o.x, o.y, 0x1010u + (mb & 3u) * 0x22u + ((mb >> 2) & 3u) * 0x2200u);
+          const uint32_t p1 = __byte_perm(o.z, o.w, 0x1010u + ((mb >> 4) & 3u) * 0x22u + (mb >> 6) * 0x2200u);
+          *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(args.pack_vals) + (col0 + t) * (args.M >> 1) +
+                                    ((m0 + q * 32 + seg * 8) >> 1)) = make_uint2(p0, p1);
+        }
       }
     }
         };
@@ -836,7 +854,8 @@ int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64
 
 int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t M, int64_t N,
                   int64_t K, int epi, void* C, int64_t ldc, const void* aux, int64_t ldaux, int* status,
-                  cudaStream_t s) {
+                  cudaStream_t s, const void* pack_meta, void* pack_vals) {
+  if ((pack_meta != nullptr) != (pack_vals != nullptr) || (pack_vals && epi != EPI_DRELU_T)) return SF_ERR_UNSUPPORTED;
   if (M % BM || N % BN || K % 128) return SF_ERR_SHAPE;
   if (M == 0 || N == 0) return SF_OK;
   const bool two = use_two_cta(M);
@@ -861,6 +880,7 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
   GemmArgs a{};
   a.M = M; a.N = N; a.K = K;
   a.C = C; a.ldc = ldc; a.aux = aux; a.ldaux = ldaux; a.meta_hw = meta_hw; a.status = status;
+  a.pack_meta = pack_meta; a.pack_vals = pack_vals;
   a.num_m_tiles = (int)(M / BM); a.num_n_tiles = (int)(N / BN); a.num_k_blocks = (int)(K / 64);
   if (epi == EPI_STORE) {
     if (b_kmajor) return launch_two<MODE_SPARSE24, false, false, EPI_STORE>(ta, tb, tm, a, s);

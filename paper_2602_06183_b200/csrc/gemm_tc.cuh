@@ -31,6 +31,9 @@ struct GemmArgs {
   int* status;              // device status word (set to 1 when a bounded wait expires)
   int num_m_tiles, num_n_tiles, num_k_blocks;
   int gather_tma_groups;    // Venom: groups (of 16 per stage) fetched by TMA row gather; the rest by cp.async
+  // EPI_DRELU_T only, optional: also emit the output packed as a 2:4 operand at given positions
+  const void* pack_meta;    // canonical 2:4 metadata [N, M/16] uint16 (rows = output rows of Ct)
+  void* pack_vals;          // bf16 [N, M/2]
 };
 
 // D[M,N] = op(A) op(B)^T, tiles 128 x 256, K % 64 == 0.
@@ -40,9 +43,11 @@ int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64
 // A_s[M,K] 2:4-packed times B (b_kmajor: [N,K] row-major, else [K,N] row-major).
 // epi EPI_STORE_T / EPI_DRELU_T: transposed output Ct[N,M] (b_kmajor only); EPI_STORE: C[M,N]
 // (two-CTA kernel, M % 256 == 0).
+// pack_meta / pack_vals (EPI_DRELU_T, optional): additionally write Ct gathered at the positions of the
+// canonical 2:4 metadata pack_meta [N, M/16] into pack_vals [N, M/2].
 int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t M, int64_t N,
                   int64_t K, int epi, void* C, int64_t ldc, const void* aux, int64_t ldaux, int* status,
-                  cudaStream_t s);
+                  cudaStream_t s, const void* pack_meta = nullptr, void* pack_vals = nullptr);
 // C[T,N] = A_vnm[T,F] Bt[F,N]; A_vnm packed (vals [T, 2F/Mv], hardware-ordered metadata, colidx).
 int gemm_venom(const void* a_vals, const uint8_t* meta_hw, const uint8_t* colidx, const void* Bt, int64_t T,
                int64_t F, int64_t N, int V, int Mv, void* C, int64_t ldc, int* status, cudaStream_t s);

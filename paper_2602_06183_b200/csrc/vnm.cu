@@ -411,26 +411,6 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
   }
 }
 
-// Gather a dense [R, K] matrix at the positions of canonical 2:4 metadata: vals[r, k/2] (bf16).
-__global__ void __launch_bounds__(256)
-pack24_kernel(const uint4* __restrict__ dense, const uint16_t* __restrict__ meta, uint4* __restrict__ vals,
-              int64_t R, int64_t K) {
-  const int64_t words = K >> 4;
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= R * words) return;
-  const uint4 q0 = __ldg(dense + 2 * idx), q1 = __ldg(dense + 2 * idx + 1);
-  const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
-  const uint32_t m = meta[idx];
-  uint32_t o[4];
-#pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    const uint32_t nib = (m >> (4 * g)) & 0xFu;
-    o[g] = __byte_perm(w[2 * g], w[2 * g + 1], 0x1010u + (nib & 3u) * 0x22u + (nib >> 2) * 0x2200u);
-  }
-  vals[idx] = make_uint4(o[0], o[1], o[2], o[3]);
-}
-
-
 }  // namespace
 
 int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
@@ -487,14 +467,6 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
                                                   (uint16_t*)relu_vals, (uint16_t*)dense_out,
                                                   (uint16_t*)relu_dense_out);
   }
-  SF_LAUNCH_CHECK();
-  return SF_OK;
-}
-
-int launch_pack24(const void* dense, const void* meta, void* vals, int64_t R, int64_t K, cudaStream_t s) {
-  const int64_t n = R * (K >> 4);
-  if (n == 0) return SF_OK;
-  pack24_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>((const uint4*)dense, (const uint16_t*)meta, (uint4*)vals, R, K);
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
