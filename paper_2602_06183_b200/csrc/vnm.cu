@@ -149,10 +149,83 @@ vnm_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, int
     *reinterpret_cast<uint32_t*>(colidx + (blk * G + c0 / M + tid) * 4) = c4;
   }
 
-  // ---- pass B: 2:4 inside the kept columns, one (row, group) item per thread
+  // ---- pass B: 2:4 inside the kept columns
+  const int64_t g0 = c0 / M;
+  const int rstep_fast = ng > 0 ? kThreads / ng : 0;
+  if (ng > 0 && kThreads % ng == 0 && (32 % ng == 0 || ng % 32 == 0) && V % rstep_fast == 0) {
+    // Fast form: a thread always serves group tid % ng, for rows tid / ng, tid / ng + kThreads / ng, ...;
+    // the four kept columns, hence the four shared-memory offsets, are fixed per thread. Packed bf16
+    // arithmetic on the four kept values only; the ReLU pair reuses the byte-permute selector of the
+    // value pair; the dense copies are built in registers and written with whole 16-byte stores.
+    const int g = tid % ng, rstep = rstep_fast, r0 = tid / ng;
+    const uint32_t c4 = *reinterpret_cast<const uint32_t*>(cidx + g * 4);
+    const uint16_t* tp = tile + r0 * kRow + g * M;
+    const int o0 = (int)(c4 & 0xFFu), o1 = (int)((c4 >> 8) & 0xFFu), o2 = (int)((c4 >> 16) & 0xFFu), o3 = (int)(c4 >> 24);
+    const bool lead4 = (g & 3) == 0;
+    const bool want_relu = relu_vals && apply;
+    const int64_t trow = t0 + r0;
+    uint16_t* p_vals = vals + trow * (2 * G) + 2 * (g0 + g);
+    uint16_t* p_relu = want_relu ? relu_vals + trow * (2 * G) + 2 * (g0 + g) : nullptr;
+    uint16_t* p_dense = dense_out ? dense_out + trow * F + c0 + g * M : nullptr;
+    uint16_t* p_rdense = relu_dense_out ? relu_dense_out + trow * F + c0 + g * M : nullptr;
+    uint16_t* p_meta = meta + trow * (G >> 2) + ((g0 + g) >> 2);
+    const int64_t kw = (g0 + g) >> 2;
+    const int64_t s_vals = (int64_t)rstep * (2 * G), s_dense = (int64_t)rstep * F, s_meta = (int64_t)rstep * (G >> 2);
+    for (int r = r0; r < V; r += rstep) {
+      const uint32_t lo = (uint32_t)tp[o0] | ((uint32_t)tp[o1] << 16), hi = (uint32_t)tp[o2] | ((uint32_t)tp[o3] << 16);
+      const uint32_t rl_lo = apply ? relu2(lo) : 0u, rl_hi = apply ? relu2(hi) : 0u;
+      const uint32_t h_lo = apply ? sq2(rl_lo) : lo, h_hi = apply ? sq2(rl_hi) : hi;
+      uint32_t packed;
+      const uint32_t nib = top2of4_packed(h_lo, h_hi, &packed);
+      const uint32_t p0 = nib & 3u, p1 = nib >> 2;
+      *reinterpret_cast<uint32_t*>(p_vals) = packed;
+      const uint32_t rpair = __byte_perm(rl_lo, rl_hi, 0x1010u + p0 * 0x22u + p1 * 0x2200u);
+      if (want_relu) *reinterpret_cast<uint32_t*>(p_relu) = rpair;
+      if (dense_out || relu_dense_out) {
+        // whole 16-byte stores only: word j of the group holds the value kept at column 2j or 2j + 1
+        const uint32_t ca = (c4 >> (8 * p0)) & 0xFFu, cb = (c4 >> (8 * p1)) & 0xFFu;       // kept columns, ca < cb
+        const uint32_t wa = ca >> 1, wb = cb >> 1, sa = 16u * (ca & 1u), sb = 16u * (cb & 1u);
+        const uint32_t ha = (packed & 0xFFFFu) << sa, hb = (packed >> 16) << sb;
+        const uint32_t ra = (rpair & 0xFFFFu) << sa, rb = (rpair >> 16) << sb;
+        if (M >= 8) {
+          for (int m8 = 0; m8 < M; m8 += 8) {
+            uint32_t dw[4], rw4[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t wj = (uint32_t)(m8 >> 1) + j;
+              const bool ia = wa == wj, ib = wb == wj;
+              dw[j] = (ia ? ha : 0u) | (ib ? hb : 0u);
+              rw4[j] = (ia ? ra : 0u) | (ib ? rb : 0u);
+            }
+            if (dense_out) *reinterpret_cast<uint4*>(p_dense + m8) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
+            if (relu_dense_out) *reinterpret_cast<uint4*>(p_rdense + m8) = make_uint4(rw4[0], rw4[1], rw4[2], rw4[3]);
+          }
+        } else {                                            // M == 4: one 8-byte group
+          const uint32_t d0 = (wa == 0u ? ha : 0u) | (wb == 0u ? hb : 0u), d1 = (wa == 1u ? ha : 0u) | (wb == 1u ? hb : 0u);
+          const uint32_t q0 = (wa == 0u ? ra : 0u) | (wb == 0u ? rb : 0u), q1 = (wa == 1u ? ra : 0u) | (wb == 1u ? rb : 0u);
+          if (dense_out) *reinterpret_cast<uint2*>(p_dense) = make_uint2(d0, d1);
+          if (relu_dense_out) *reinterpret_cast<uint2*>(p_rdense) = make_uint2(q0, q1);
+        }
+      }
+      uint32_t word = nib;
+      word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 4;
+      word |= __shfl_down_sync(0xFFFFFFFFu, word, 2) << 8;
+      if (lead4) {
+        *p_meta = (uint16_t)word;
+        if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(t0 + r, kw, 4 * G)) = (uint16_t)word;
+      }
+      tp += rstep * kRow;
+      p_vals += s_vals;
+      if (want_relu) p_relu += s_vals;
+      if (dense_out) p_dense += s_dense;
+      if (relu_dense_out) p_rdense += s_dense;
+      p_meta += s_meta;
+    }
+    return;
+  }
+  // General form (ragged strips, V not a multiple of the row step): one (row, group) item per thread
   const int items = V * ng;
   const int items_pad = (items + 31) & ~31;
-  const int64_t g0 = c0 / M;
   for (int i = tid; i < items_pad; i += kThreads) {
     const bool valid = i < items;
     const int r = valid ? i / ng : 0, g = valid ? i - r * ng : 0;
