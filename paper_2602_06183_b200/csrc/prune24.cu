@@ -248,6 +248,38 @@ transpose_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, in
   }
 }
 
+// Transpose for shapes that are multiples of 64: 16-byte global loads and stores on both sides.
+// Shared tile rows are 33 words apart, so the word stores of the load phase are conflict-free and the
+// strided 16-bit reads of the store phase collide two ways at most.
+__global__ void __launch_bounds__(256)
+transpose64_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, int64_t rows, int64_t cols) {
+  __shared__ uint32_t t[64 * 33];
+  const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
+  const int tid = threadIdx.x;
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int row = (tid >> 3) + 32 * j, c8 = (tid & 7) * 8;
+    const uint4 q = __ldg(reinterpret_cast<const uint4*>(in + (r0 + row) * cols + c0 + c8));
+    uint32_t* d = t + row * 33 + (c8 >> 1);
+    d[0] = q.x; d[1] = q.y; d[2] = q.z; d[3] = q.w;
+  }
+  __syncthreads();
+  const uint16_t* th = reinterpret_cast<const uint16_t*>(t);
+  const int lane = tid & 31, warp = tid >> 5;
+  const int r8 = lane & 7, cq = lane >> 3;
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int c = warp * 4 + cq + 32 * j;                    // output row inside the tile
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t a = th[(r8 * 8 + 2 * k) * 66 + c], b = th[(r8 * 8 + 2 * k + 1) * 66 + c];
+      w[k] = a | (b << 16);
+    }
+    *reinterpret_cast<uint4*>(out + (c0 + c) * rows + r0 + r8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
 }  // namespace
 
 int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int group_dim, int prune_mode,
@@ -299,7 +331,10 @@ int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int gr
 int launch_transpose(const void* in, void* out, int64_t rows, int64_t cols, cudaStream_t s) {
   if (rows == 0 || cols == 0) return SF_OK;
   dim3 grid((unsigned)((cols + 63) / 64), (unsigned)((rows + 63) / 64));
-  transpose_kernel<<<grid, 256, 0, s>>>((const uint16_t*)in, (uint16_t*)out, rows, cols);
+  if (rows % 64 == 0 && cols % 64 == 0)
+    transpose64_kernel<<<grid, 256, 0, s>>>((const uint16_t*)in, (uint16_t*)out, rows, cols);
+  else
+    transpose_kernel<<<grid, 256, 0, s>>>((const uint16_t*)in, (uint16_t*)out, rows, cols);
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
