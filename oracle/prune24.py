@@ -3,8 +3,8 @@
 Test infrastructure only (see the package docstring).
 
 What the paper fixes
-  * n:m format: in every group of four consecutive elements at most two are non-zero
-    (Section 1, definition of n:m sparsity).
+  * n:m format with n = 2, m = 4: a group of four neighbours holds no more than two non-zero
+    entries (Section 1's definition of n:m sparsity).
   * The mask is the magnitude-based one: the two largest magnitudes of the group stay
     (Section 2.2, first sentence); equal magnitudes are resolved towards the lower index.
   * Soft-thresholding (Section 2.2): with the group's magnitudes sorted

@@ -3,10 +3,10 @@
 Test infrastructure only (see the package docstring).
 
 What the paper fixes (Section 2.3, Table 5)
-  * The matrix is cut into sub-matrices of V rows by M columns; in each sub-matrix only four
-    columns are retained and the V x 4 matrix they form is 2:4-sparsified by greedy magnitude
-    pruning. The density is N/M with N = 2 (Table 5: M = 16, 32, 64 -> 87.5, 93.75, 96.875 %
-    sparsity).
+  * Blocks of V rows by M columns; a block keeps four of its M columns, and every row of the
+    block keeps the two larger magnitudes among those four (a 2:4 pattern chosen greedily by
+    magnitude). Density is therefore N/M with N = 2 (Table 5: M = 16, 32, 64 -> 87.5, 93.75,
+    96.875 % sparsity).
   * The activation is y2 = ReLU(y1)^2 (Eq. 2).
 
 Readings where the paper is silent or garbled

@@ -148,3 +148,53 @@ def test_tie_between_columns_goes_to_lower_index():
     assert tuple(res.colidx[0, 0]) == (0, 1, 2, 6)
     # within the row the single non-zero sits at position 3 and is kept with position 0
     assert (int(res.meta[0, 0]) & 0xF) == (0 | 3 << 2)
+
+
+def test_column_score_is_taken_on_the_squared_activation():
+    """With the activation on, the block's kept columns are ranked by the sum of h = ReLU(p)^2
+    (the stored activation y2 of Eq. 2, the tensor Section 2.3 sparsifies), not by the sum of the
+    un-squared ReLU(p). One column with a single 4 (sum 4, sum of squares 16) against columns of
+    three 2s (sum 6, sum of squares 12): the squares rank the single-4 column first, the plain
+    values would rank it last."""
+    V, M = 4, 8
+    p = np.full((V, 32), -1.0, dtype=np.float32)
+    p[0, 0] = 4.0                         # column 0: sum 4, sum of squares 16
+    for c in (1, 2, 3, 4):
+        p[0:3, c] = 2.0                   # columns 1-4: sum 6, sum of squares 12
+    res = vnm_sparsify(_bits(p), V=V, M=M, apply_sqrelu=True)
+    # squares: 16 > 12 = 12 = 12 = 12 -> columns 0, 1, 2, 3 (ties to the lower index)
+    assert tuple(res.colidx[0, 0]) == (0, 1, 2, 3)
+    # (un-squared sums would give 6, 6, 6, 6 > 4 -> columns 1, 2, 3, 4)
+    # row 0 keeps the 16 and the first 4 among the kept columns; the stored values are the squares
+    assert (int(res.meta[0, 0]) & 0xF) == (0 | 1 << 2)
+    assert bf16_to_f32(res.vals[0, :2]).tolist() == [16.0, 4.0]
+    assert bf16_to_f32(res.relu_vals[0, :2]).tolist() == [4.0, 2.0]
+
+
+def test_column_choice_brute_force_with_the_activation_on():
+    """Brute force over all C(M, 4) column subsets and all six row pairs on small signed integers
+    with SquaredReLU applied: the retained mass is the mass of max(p, 0)^2 (exact in float32)."""
+    rng = np.random.default_rng(11)
+    V, M = 8, 8
+    for trial in range(40):
+        p = rng.integers(-6, 7, size=(V, M * 4)).astype(np.float32)
+        res = vnm_sparsify(_bits(p), V=V, M=M, apply_sqrelu=True)
+        h = np.where(p > 0, p * p, 0.0).astype(np.float64)
+        for g in range(4):
+            blk = h[:, g * M:(g + 1) * M]
+            colmass = blk.sum(axis=0)
+            best, best_set = None, None
+            for s in itertools.combinations(range(M), 4):
+                m = colmass[list(s)].sum()
+                if best is None or m > best:
+                    best, best_set = m, s
+            assert tuple(res.colidx[0, g]) == best_set
+            for r in range(V):
+                four = blk[r, list(best_set)]
+                bp, bpair = None, None
+                for pair in itertools.combinations(range(4), 2):
+                    m = four[pair[0]] + four[pair[1]]
+                    if bp is None or m > bp:
+                        bp, bpair = m, pair
+                nib = (int(res.meta[r, 0]) >> (4 * g)) & 0xF
+                assert (nib & 3, nib >> 2) == bpair
