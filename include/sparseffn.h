@@ -14,8 +14,10 @@
  *     library never allocates or frees device memory and never synchronises, except where an
  *     entry point says so. Work is enqueued on the caller's stream (`stream` is a
  *     cudaStream_t passed as void*; NULL = the legacy default stream).
- *   - Return value: SF_OK (0) or a negative sf_status. No exceptions cross the boundary. On a
- *     non-zero return nothing has been launched.
+ *   - Return value: SF_OK (0) or a negative sf_status. No exceptions cross the boundary. Argument
+ *     errors (NULL, shape, alignment, workspace size, architecture) are found before anything is
+ *     enqueued; after an SF_ERR_CUDA some kernels of the call may already be enqueued and the
+ *     outputs are undefined.
  *   - Base pointers must be 16-byte aligned and leading dimensions multiples of 8 elements.
  *   - Canonical 2:4 metadata: one nibble per group of four, `pos0 | pos1 << 2` with
  *     pos0 < pos1 the kept positions; four consecutive groups of a row are packed
@@ -152,8 +154,10 @@ SF_API int sf_gemm_venom(const void* a_vals, const void* a_meta, const void* col
  *   - Limit: Mr * K / 8 <= 4 MiB (e.g. 4096 x 8192); larger shapes return SF_ERR_WORKSPACE.
  *   - The call itself allocates and frees nothing (no cudaMalloc / cudaFree, no allocating
  *     library routine). Inputs and output are the caller's, exactly as for sf_gemm_sparse24.
- *   - The first call on each device looks up the array's device address; make that first call
- *     outside any stream capture.
+ *   - The first call on each device looks up the array's device address, and that is also the
+ *     moment the CUDA runtime loads the module that contains the array (4 MiB + 256 B of device
+ *     memory, taken once per device by the runtime, not by this code). Make that first call at
+ *     start-up, outside any stream capture, from one host thread; later calls take no memory.
  *   - All calls share the one array: two calls that may overlap on the GPU (different streams,
  *     or different host threads) race on it. Serialise them on one stream.
  *   - A bounded-wait expiry is recorded in the built-in status word, which no call reads back;
@@ -268,15 +272,15 @@ SF_API int sf_ffn_bwd_scheduled(const sf_schedule* schedule, int64_t step, const
                          const void* fwd_ctx, void* dX, void* dW1, void* dW2, void* workspace,
                          void* stream);
 
-/* Tensor-pipe calibration, a measurement aid (the paper has no counterpart). One CTA per SM (or
- * one CTA pair per two SMs when two_cta != 0) issues 4 * iters tcgen05.mma instructions back to
- * back on operands that already sit in shared memory: 128 x 256 x 16 per CTA for sparse == 0,
- * 128 x 256 x 32 logical K with 2:4 metadata for sparse != 0; no loads, no epilogue. `cycles`
- * (DEVICE pointer, int64, 8-byte aligned) receives the SM clocks CTA 0 spent from its first issue
- * to the completion of its last instruction; clocks per instruction = *cycles / (4 * iters).
- * `workspace` is any device buffer whose first int is a zeroed status word (a bounded wait that
- * expires sets it; read it with sf_check_status). 1 <= iters <= 2^20. Enqueues on `stream`. */
-SF_API int sf_probe_mma_rate(int sparse, int two_cta, int iters, void* cycles, void* workspace, void* stream);
+/* Bounded-wait self-test (the paper has no counterpart). Every device-side wait of the tensor-core
+ * kernels gives up after a clock budget, raises the status word at the start of the workspace and
+ * lets its CTA leave; sf_check_status then reports SF_ERR_TIMEOUT. This call runs that mechanism
+ * in isolation: one CTA of one warp waits, with the same wait routine and a budget of
+ * `budget_clocks` SM clocks (1 <= budget_clocks <= 2^31), on an mbarrier that nothing completes.
+ * The wait runs out by construction, the kernel sets the status word and returns; nothing is
+ * left waiting and the context stays usable. `workspace`: device buffer whose first int is the
+ * (zeroed) status word. Enqueues on `stream`. */
+SF_API int sf_selftest_wait_expiry(void* workspace, int64_t budget_clocks, void* stream);
 
 /* Stage tracing, a measurement aid (the paper has no counterpart). `events` is a caller-owned HOST
  * array of `capacity` cudaEvent_t handles (created with timing enabled) that must stay valid until

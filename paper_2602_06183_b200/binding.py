@@ -75,7 +75,7 @@ _SIGNATURES = {
                                     _vp, _vp]),
     "sf_ffn_bwd_scheduled": (_i32, [C.POINTER(sf_schedule), _i64, C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp,
                                     _vp, _vp, _vp, _vp, _vp]),
-    "sf_probe_mma_rate": (_i32, [_i32, _i32, _i32, _vp, _vp, _vp]),
+    "sf_selftest_wait_expiry": (_i32, [_vp, _i64, _vp]),
     "sf_trace_set": (_i32, [C.POINTER(_vp), _i32]),
     "sf_trace_count": (_i32, []),
     "sf_check_status": (_i32, [_vp, _vp]),
@@ -361,16 +361,9 @@ def sf_ffn_bwd_scheduled(schedule, step: int, desc, dY, X, W1, W2, fwd_ctx, dX, 
                                       _stream(stream)), "sf_ffn_bwd_scheduled")
 
 
-def sf_probe_mma_rate(sparse: bool, two_cta: bool, iters: int = 20000) -> float:
-    """SM clocks per tcgen05.mma issued back to back from shared-memory operands (no loads)."""
-    cycles = torch.zeros((1,), dtype=torch.int64, device="cuda")
-    ws = torch.zeros((64,), dtype=torch.int32, device="cuda")
-    _check(lib().sf_probe_mma_rate(int(sparse), int(two_cta), iters, _ptr(cycles), _ptr(ws), _stream(None)),
-           "sf_probe_mma_rate")
-    st = sf_check_status(ws)
-    if st != SF_OK:
-        raise SparseFFNError(st, "sf_probe_mma_rate")
-    return float(cycles.item()) / (4.0 * iters)
+def sf_selftest_wait_expiry(workspace, budget_clocks: int = 1_000_000, stream=None) -> None:
+    """One bounded wait on a barrier nothing completes: sets the status word of ``workspace``."""
+    _check(lib().sf_selftest_wait_expiry(_ptr(workspace), budget_clocks, _stream(stream)), "sf_selftest_wait_expiry")
 
 
 def sf_check_status(workspace, stream=None) -> int:

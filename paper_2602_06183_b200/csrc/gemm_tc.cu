@@ -270,7 +270,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     prefetch_tmap(&tmapA);
     prefetch_tmap(&tmapB);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&ctl->full[s], kMode == MODE_VENOM ? 1 + 128 : 1);   // Venom: + every cp.async gather thread
+      mbar_init(&ctl->full[s], kMode == MODE_VENOM ? 1 + 128 : 1);   // Venom: + one arrival per cp.async gather thread
       mbar_init(&ctl->empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -411,6 +411,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     const int ntma = args.gather_tma_groups;
     const uint16_t* Bt = reinterpret_cast<const uint16_t*>(args.aux);
     uint32_t stage = 0, phase = 0;
+    int pending = -1;                      // cp.async warps: stage whose copies are issued but not yet signalled
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       int mt, nt;
@@ -444,15 +445,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
               asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
             }
           }
-          // The barrier's pending count is raised now and lowered when this thread's copies have
-          // landed; the plain arrive accounts for the thread itself. No blocking wait.
-          asm volatile("cp.async.mbarrier.arrive.shared::cta.b64 [%0];" ::"r"(smem_u32(&ctl->full[stage])) : "memory");
-          mbar_arrive(&ctl->full[stage]);
+          asm volatile("cp.async.commit_group;" ::: "memory");
+          // These copies are generic-proxy writes and the MMA reads the stage through the async proxy:
+          // a stage is signalled only after its copies have landed and a proxy fence has ordered them.
+          // The warps stay one stage ahead: signal the previous stage while this one is in flight.
+          if (pending >= 0) {
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+            fence_proxy_async_smem();
+            mbar_arrive(&ctl->full[pending]);
+          }
+          pending = (int)stage;
         }
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
     }
-    if (gw >= 8) asm volatile("cp.async.wait_all;" ::: "memory");
+    if (gw >= 8) {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      if (pending >= 0) {
+        fence_proxy_async_smem();
+        mbar_arrive(&ctl->full[pending]);
+      }
+    }
   } else {
     // =========================== epilogue (warps 2..5) ===========================
     const int q = warp & 3;                                                    // TMEM lane quadrant

@@ -57,15 +57,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Wait budget in SM clocks (~1.5 s at 1.4 GHz): far above any legitimate wait in these kernels.
 constexpr long long kWaitBudgetClocks = 2000000000LL;
 
-// Bounded wait. Returns false on expiry or when *abort_flag is set by another role.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait. Returns false on expiry (after `budget` SM clocks) or when *abort_flag is set by
+// another role.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          long long budget = kWaitBudgetClocks) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 0x3FFu) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitBudgetClocks) {
+      if (clock64() - t0 > budget) {
         *abort_flag = 1;
         return false;
       }

@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from paper_2602_06183_b200 import binding, synth
-from util import to_dev, bits, f32, rel_fro
+from util import to_dev, bits, f32, rel_fro, assert_close_elementwise, Guarded
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-2      # relative Frobenius error, bf16 outputs vs float64-accumulated reference
@@ -27,6 +27,7 @@ def test_dense_gemm_layouts(a_k, b_k, M, N, K):
     Af = _f64(A) if a_k else _f64(A).T
     Bf = _f64(B) if b_k else _f64(B).T
     assert rel_fro(f32(C), Af @ Bf.T) < TOL
+    assert_close_elementwise(f32(C), Af @ Bf.T, K, "dense product")
 
 
 def test_dense_gemm_exact_small_integers():
@@ -51,6 +52,7 @@ def test_sparse24_gemm_against_oracle_packing(Mr, Nc, K):
     ref = _f64(X) @ _f64(p.dense).T                                     # [Nc, Mr] = X W_s^T
     assert Ct.shape == (Nc, Mr)
     assert rel_fro(f32(Ct), ref) < TOL
+    assert_close_elementwise(f32(Ct), ref, K, "2:4 product")
 
 
 @pytest.mark.parametrize("b_k", [True, False])
@@ -65,6 +67,7 @@ def test_sparse24_gemm_row_major_output(b_k, Mr, Nc, K):
     assert binding.sf_check_status(ws) == binding.SF_OK
     Bf = _f64(B) if b_k else _f64(B).T
     assert rel_fro(f32(C), _f64(p.dense) @ Bf.T) < TOL
+    assert_close_elementwise(f32(C), _f64(p.dense) @ Bf.T, K, "2:4 product, row-major output")
 
 
 def test_sparse24_gemm_one_hot_metadata_probe():
@@ -92,17 +95,23 @@ def test_sparse24_gemm_one_hot_metadata_probe():
 
 
 @pytest.mark.parametrize("T,F,Nc,V,M", [(128, 256, 256, 128, 8), (256, 1024, 512, 128, 8), (256, 512, 256, 64, 8),
-                                        (128, 1024, 256, 128, 16), (128, 512, 256, 64, 4)])
+                                        (128, 1024, 256, 128, 16), (128, 512, 256, 64, 4),
+                                        # Table 5's group widths: 93.75 % and 96.875 % sparse
+                                        (256, 2048, 512, 128, 32), (256, 2048, 256, 64, 32),
+                                        (256, 4096, 512, 128, 64), (128, 4096, 256, 64, 64), (384, 2048, 768, 128, 64)])
 def test_venom_gemm_against_oracle_packing(T, F, Nc, V, M):
     P = synth.normal_bf16((T, F), 0.2, 1.0, seed=T + F + M)
     Bt = synth.normal_bf16((F, Nc), 0, 1, seed=7, stream=F)
     a = oracle.vnm_sparsify(P, V=V, M=M)
     meta = torch.from_numpy(a.meta.view(np.int16)).cuda()
     colidx = torch.from_numpy(a.colidx).cuda()
-    C, ws = binding.sf_gemm_venom(to_dev(a.vals), meta, colidx, to_dev(Bt), V, M)
+    out = Guarded((T, Nc), torch.bfloat16)
+    C, ws = binding.sf_gemm_venom(to_dev(a.vals), meta, colidx, to_dev(Bt), V, M, C_out=out.t)
     assert binding.sf_check_status(ws) == binding.SF_OK
+    out.check("Venom product output")
     ref = _f64(a.dense) @ _f64(Bt)
     assert rel_fro(f32(C), ref) < TOL
+    assert_close_elementwise(f32(C), ref, 4 * F // M, "Venom product")
 
 
 def test_gemm_shape_errors():
@@ -113,13 +122,17 @@ def test_gemm_shape_errors():
     assert e.value.status == binding.SF_ERR_SHAPE
 
 
-def test_mma_rate_probe_reports_the_pipe_rates():
-    """Back-to-back issue from shared memory: a dense 128x256x16 instruction takes 128 clocks
-    (8192 flop/clk/SM, the nominal rate); the 2:4 instruction has twice the logical K and must not
-    take more than 1.3x as long on a CTA pair, nor be faster than the dense one."""
-    dense = binding.sf_probe_mma_rate(False, True, iters=4000)
-    sparse = binding.sf_probe_mma_rate(True, True, iters=4000)
-    one = binding.sf_probe_mma_rate(True, False, iters=4000)
-    assert 120 < dense < 140
-    assert dense * 0.95 < sparse < dense * 1.3
-    assert sparse <= one * 1.02
+def test_bounded_wait_runs_out_and_is_reported():
+    """A wait on a barrier that nothing completes gives up after its clock budget, the kernel sets
+    the status word and returns; the host reads SF_ERR_TIMEOUT once, then SF_OK again, and the
+    context keeps working."""
+    ws = torch.zeros((256,), dtype=torch.uint8, device="cuda")
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    binding.sf_selftest_wait_expiry(ws, budget_clocks=1_000_000)
+    assert binding.sf_check_status(ws) == binding.SF_ERR_TIMEOUT
+    assert binding.sf_check_status(ws) == binding.SF_OK              # reported once, then cleared
+    A = synth.normal_bf16((128, 64), 0, 1, seed=1)
+    B = synth.normal_bf16((256, 64), 0, 1, seed=2)
+    Cm, ws2 = binding.sf_gemm_dense(to_dev(A), True, to_dev(B), True)
+    assert binding.sf_check_status(ws2) == binding.SF_OK
+    assert rel_fro(f32(Cm), _f64(A) @ _f64(B).T) < TOL
