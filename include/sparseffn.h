@@ -52,13 +52,18 @@ typedef enum sf_status {
 } sf_status;
 
 /* Problem descriptor of one FFN layer step. Ragged shapes are rejected, never padded:
- * T, D, F multiples of 256, T % V == 0, (4F/M) % 128 == 0, V in {64,128}, N == 2,
- * M in {4,8,16,32}. */
+ * T, D, F multiples of 256 (the tile of a CTA pair, which every product of the step runs on),
+ * T % V == 0, (4F/M) % 128 == 0, V in {64,128}, N == 2, M in {4,8,16,32,64}. */
+typedef enum sf_ffn_flags {
+  SF_FFN_SAVE_Y1 = 1,     /* also store the full bf16 pre-activation y1 in the context (SF_CTX_Y1) */
+  SF_FFN_UNFUSED_ACT = 2  /* M == 8 only: run SquaredReLU + V:N:M as its own kernel on a stored y1 instead of
+                             inside the y1 product's epilogue (same results; for comparison and profiling) */
+} sf_ffn_flags;
 typedef struct sf_ffn_desc {
   int64_t T, D, F;
   int32_t V, N, M;
   int32_t prune_mode;  /* 0: hard magnitude top-2-of-4; 1: soft-thresholding (Section 2.2) */
-  int32_t flags;       /* bit0: also store the full bf16 pre-activation y1 in the context */
+  int32_t flags;       /* OR of sf_ffn_flags; other bits are rejected with SF_ERR_UNSUPPORTED */
 } sf_ffn_desc;
 
 SF_API const char* sf_status_string(int status);
@@ -169,30 +174,42 @@ SF_API int sf_gemm_sparse24_noalloc(const void* a_vals, const void* a_meta, cons
  * The FFN step (Algorithm 1 = forward, Algorithm 2 = backward; Eqs. 1-8 for the dense phase).
  *
  * sf_ffn_workspace_size: bytes of the forward context (saved for backward) and of the scratch
- * workspace for `desc`. Both buffers are caller-allocated device memory, 256-byte aligned. The
- * first 256 bytes of a workspace hold the device status word: zero them once before first use.
+ * workspace for `desc` (each the larger of what the sparse and the dense step need). Both buffers
+ * are caller-allocated device memory, 256-byte aligned. The first 256 bytes of a workspace hold
+ * the device status word: zero them once before first use. Every step call takes the sizes of the
+ * two buffers it is given and returns SF_ERR_WORKSPACE, before enqueuing anything, when one is
+ * smaller than the descriptor needs.
  *
  * sf_sparse_ffn_fwd:  W1s = prune24(W1 along D);  y1 = X W1s^T;  y2 = V:N:M(ReLU(y1)^2);
  *                     Y = y2 W2^T  (W2 dense).  Saves packed y2, packed ReLU(y1), metadata,
- *                     column indices (and y1 if flags bit0) in fwd_ctx. For M <= 8 the product
- *                     consumes y2 as a plain 2:4 operand over all F columns (identical result,
- *                     no row gather); for M >= 16 it consumes the condensed V:N:M operand and
- *                     gathers the kept rows of W2^T.
+ *                     column indices (and y1 with SF_FFN_SAVE_Y1) in fwd_ctx.
+ *                     M == 8: SquaredReLU and the V:N:M selection run inside the epilogue of the y1
+ *                     product on the accumulator tile (y1 is never written); the activation is also
+ *                     kept as a plain 2:4 operand over all F columns (two of eight is at most two
+ *                     of four), which is what the products consume: identical results, no row
+ *                     gather. No masked [T, F] copy of y2, ReLU(y1) or dy1 exists on this path.
+ *                     M >= 16: the product consumes the condensed V:N:M operand and gathers the kept
+ *                     rows of W2^T.
  * sf_sparse_ffn_bwd:  W2s = prune24(W2 along D);  dy2 = dY W2s;  dy1 = 2 dy2 ReLU(y1) on y2's
  *                     mask;  dX = dy1 W1 (W1 dense);  dW1 = dy1^T X [F,D];  dW2 = dY^T y2 [D,F].
+ *                     The two weight-gradient products reduce over tokens, so they run on the dense
+ *                     tensor path; for M == 8 their masked operand is expanded from its packed form
+ *                     inside the kernel.
  * sf_dense_ffn_fwd/bwd: the same equations with no pruning; fwd_ctx holds y1 (bf16 [T,F]).
  */
 SF_API int sf_ffn_workspace_size(const sf_ffn_desc* desc, size_t* fwd_ctx_bytes, size_t* workspace_bytes);
 SF_API int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, const void* W2,
-                      void* Y, void* fwd_ctx, void* workspace, void* stream);
+                      void* Y, void* fwd_ctx, size_t fwd_ctx_bytes, void* workspace, size_t workspace_bytes,
+                      void* stream);
 SF_API int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, const void* W1,
-                      const void* W2, const void* fwd_ctx, void* dX, void* dW1, void* dW2,
-                      void* workspace, void* stream);
+                      const void* W2, const void* fwd_ctx, size_t fwd_ctx_bytes, void* dX, void* dW1, void* dW2,
+                      void* workspace, size_t workspace_bytes, void* stream);
 SF_API int sf_dense_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, const void* W2,
-                     void* Y, void* fwd_ctx, void* workspace, void* stream);
+                     void* Y, void* fwd_ctx, size_t fwd_ctx_bytes, void* workspace, size_t workspace_bytes,
+                     void* stream);
 SF_API int sf_dense_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, const void* W1,
-                     const void* W2, const void* fwd_ctx, void* dX, void* dW1, void* dW2,
-                     void* workspace, void* stream);
+                     const void* W2, const void* fwd_ctx, size_t fwd_ctx_bytes, void* dX, void* dW1, void* dW2,
+                     void* workspace, size_t workspace_bytes, void* stream);
 
 /* Views into a sparse forward context (device pointers into fwd_ctx; nothing is copied). */
 typedef enum sf_ctx_field {
@@ -201,15 +218,15 @@ typedef enum sf_ctx_field {
   SF_CTX_META = 2,      /* uint16 [T, F/(4M)] canonical */
   SF_CTX_COLIDX = 3,    /* uint8 [T/V, F/M, 4] */
   SF_CTX_Y1 = 4,        /* bf16 [T, F] (only with flags bit0) */
-  SF_CTX_DY1_VALS = 5,  /* bf16 [T, 2F/M], lives in the WORKSPACE after sf_sparse_ffn_bwd; for M == 8 it
-                           is only written when flags bit0 is set (the products then consume dy1 in
-                           its 2:4 form over all F columns instead) */
+  SF_CTX_DY1_VALS = 5,  /* bf16 [T, 2F/M], lives in the WORKSPACE after sf_sparse_ffn_bwd; M != 8 only (for
+                           M == 8 dy1 exists in its 2:4 form only, SF_CTX_DY1_VALS24) */
   SF_CTX_Y2_VALS24 = 6, /* bf16 [T, F/2]: y2 as a plain 2:4 operand over all F columns (M <= 8 only,
                            else SF_ERR_UNSUPPORTED): two stored values per four columns, explicit
                            zeros where a half-group keeps fewer than two */
   SF_CTX_Y2_META24 = 7, /* uint16 [T, F/16] canonical metadata of that operand (M <= 8 only) */
-  SF_CTX_DY1_VALS24 = 8 /* bf16 [T, F/2]: dy1 at the positions of SF_CTX_Y2_META24; lives in the WORKSPACE
+  SF_CTX_DY1_VALS24 = 8, /* bf16 [T, F/2]: dy1 at the positions of SF_CTX_Y2_META24; lives in the WORKSPACE
                            after sf_sparse_ffn_bwd (M <= 8 only) */
+  SF_CTX_RELU_VALS24 = 9 /* bf16 [T, F/2]: ReLU(y1) at the positions of SF_CTX_Y2_META24 (M == 8 only) */
 } sf_ctx_field;
 SF_API int sf_ctx_view(const sf_ffn_desc* desc, const void* fwd_ctx_or_workspace, int field,
                 const void** ptr, size_t* bytes);
@@ -230,7 +247,7 @@ SF_API int sf_ffn_host_staging_size(const sf_ffn_desc* desc, size_t* bytes);
 SF_API int sf_ffn_step_host(const sf_ffn_desc* desc, int dense, const void* host_X, const void* host_W1,
                      const void* host_W2, const void* host_dY, void* host_Y, void* host_dX,
                      void* host_dW1, void* host_dW2, void* device_staging, void* fwd_ctx,
-                     void* workspace, void* stream);
+                     size_t fwd_ctx_bytes, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------
  * Sparse/dense step schedule (Section 5.3.2) and speed-up arithmetic (Sections 3.1 and 5.1).
@@ -266,11 +283,11 @@ SF_API int sf_ffn_flop_fraction(int64_t D, int64_t F, int64_t n_q_heads, int64_t
 SF_API int sf_end_to_end_speedup(double ffn_fraction, double ffn_speedup, double* speedup);
 SF_API int sf_ffn_fwd_scheduled(const sf_schedule* schedule, int64_t step, const sf_ffn_desc* desc,
                          const void* X, const void* W1, const void* W2, void* Y, void* fwd_ctx,
-                         void* workspace, void* stream);
+                         size_t fwd_ctx_bytes, void* workspace, size_t workspace_bytes, void* stream);
 SF_API int sf_ffn_bwd_scheduled(const sf_schedule* schedule, int64_t step, const sf_ffn_desc* desc,
                          const void* dY, const void* X, const void* W1, const void* W2,
-                         const void* fwd_ctx, void* dX, void* dW1, void* dW2, void* workspace,
-                         void* stream);
+                         const void* fwd_ctx, size_t fwd_ctx_bytes, void* dX, void* dW1, void* dW2,
+                         void* workspace, size_t workspace_bytes, void* stream);
 
 /* Bounded-wait self-test (the paper has no counterpart). Every device-side wait of the tensor-core
  * kernels gives up after a clock budget, raises the status word at the start of the workspace and

@@ -21,7 +21,8 @@ SF_ERR_NULL, SF_ERR_SHAPE, SF_ERR_ALIGN, SF_ERR_WORKSPACE = -1, -2, -3, -4
 SF_ERR_ARCH, SF_ERR_CUDA, SF_ERR_TIMEOUT, SF_ERR_UNSUPPORTED = -5, -6, -7, -8
 
 SF_CTX_Y2_VALS, SF_CTX_RELU_VALS, SF_CTX_META, SF_CTX_COLIDX, SF_CTX_Y1, SF_CTX_DY1_VALS = range(6)
-SF_CTX_Y2_VALS24, SF_CTX_Y2_META24, SF_CTX_DY1_VALS24 = 6, 7, 8
+SF_CTX_Y2_VALS24, SF_CTX_Y2_META24, SF_CTX_DY1_VALS24, SF_CTX_RELU_VALS24 = 6, 7, 8, 9
+SF_FFN_SAVE_Y1, SF_FFN_UNFUSED_ACT = 1, 2
 
 
 class sf_ffn_desc(C.Structure):
@@ -60,21 +61,22 @@ _SIGNATURES = {
     "sf_gemm_sparse24_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "sf_gemm_venom": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp, _vp]),
     "sf_ffn_workspace_size": (_i32, [C.POINTER(sf_ffn_desc), C.POINTER(_sz), C.POINTER(_sz)]),
-    "sf_sparse_ffn_fwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
-    "sf_sparse_ffn_bwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
-    "sf_dense_ffn_fwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
-    "sf_dense_ffn_bwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_sparse_ffn_fwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
+    "sf_sparse_ffn_bwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "sf_dense_ffn_fwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
+    "sf_dense_ffn_bwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp, _vp, _vp, _sz, _vp]),
     "sf_ctx_view": (_i32, [C.POINTER(sf_ffn_desc), _vp, _i32, C.POINTER(_vp), C.POINTER(_sz)]),
     "sf_ffn_host_staging_size": (_i32, [C.POINTER(sf_ffn_desc), C.POINTER(_sz)]),
-    "sf_ffn_step_host": (_i32, [C.POINTER(sf_ffn_desc), _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sf_ffn_step_host": (_i32, [C.POINTER(sf_ffn_desc), _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp,
+                                _sz, _vp]),
     "sf_schedule_step_kind": (_i32, [C.POINTER(sf_schedule), _i64, C.POINTER(_i32)]),
     "sf_schedule_speedup": (_i32, [C.POINTER(sf_schedule), C.c_double, C.POINTER(C.c_double)]),
     "sf_ffn_flop_fraction": (_i32, [_i64, _i64, _i64, _i64, _i64, C.POINTER(C.c_double)]),
     "sf_end_to_end_speedup": (_i32, [C.c_double, C.c_double, C.POINTER(C.c_double)]),
     "sf_ffn_fwd_scheduled": (_i32, [C.POINTER(sf_schedule), _i64, C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp,
-                                    _vp, _vp]),
+                                    _sz, _vp, _sz, _vp]),
     "sf_ffn_bwd_scheduled": (_i32, [C.POINTER(sf_schedule), _i64, C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp,
-                                    _vp, _vp, _vp, _vp, _vp]),
+                                    _sz, _vp, _vp, _vp, _vp, _sz, _vp]),
     "sf_selftest_wait_expiry": (_i32, [_vp, _i64, _vp]),
     "sf_trace_set": (_i32, [C.POINTER(_vp), _i32]),
     "sf_trace_count": (_i32, []),
@@ -273,31 +275,38 @@ def alloc_ffn_buffers(desc: sf_ffn_desc, device="cuda"):
     return _workspace(c, device), _workspace(w, device)
 
 
+def _nbytes(t: torch.Tensor) -> int:
+    return t.numel() * t.element_size()
+
+
 def sf_sparse_ffn_fwd(desc, X, W1, W2, Y, fwd_ctx, workspace, stream=None):
     _check(lib().sf_sparse_ffn_fwd(C.byref(desc), _ptr(X), _ptr(W1), _ptr(W2), _ptr(Y), _ptr(fwd_ctx),
-                                   _ptr(workspace), _stream(stream)), "sf_sparse_ffn_fwd")
+                                   _nbytes(fwd_ctx), _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "sf_sparse_ffn_fwd")
 
 
 def sf_sparse_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stream=None):
     _check(lib().sf_sparse_ffn_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(W1), _ptr(W2), _ptr(fwd_ctx),
-                                   _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace), _stream(stream)),
-           "sf_sparse_ffn_bwd")
+                                   _nbytes(fwd_ctx), _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace),
+                                   _nbytes(workspace), _stream(stream)), "sf_sparse_ffn_bwd")
 
 
 def sf_dense_ffn_fwd(desc, X, W1, W2, Y, fwd_ctx, workspace, stream=None):
     _check(lib().sf_dense_ffn_fwd(C.byref(desc), _ptr(X), _ptr(W1), _ptr(W2), _ptr(Y), _ptr(fwd_ctx),
-                                  _ptr(workspace), _stream(stream)), "sf_dense_ffn_fwd")
+                                  _nbytes(fwd_ctx), _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "sf_dense_ffn_fwd")
 
 
 def sf_dense_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stream=None):
     _check(lib().sf_dense_ffn_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(W1), _ptr(W2), _ptr(fwd_ctx),
-                                  _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace), _stream(stream)),
-           "sf_dense_ffn_bwd")
+                                  _nbytes(fwd_ctx), _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace),
+                                  _nbytes(workspace), _stream(stream)), "sf_dense_ffn_bwd")
 
 
 _CTX_DTYPES = {SF_CTX_Y2_VALS: torch.bfloat16, SF_CTX_RELU_VALS: torch.bfloat16, SF_CTX_META: torch.int16,
                SF_CTX_COLIDX: torch.uint8, SF_CTX_Y1: torch.bfloat16, SF_CTX_DY1_VALS: torch.bfloat16,
-               SF_CTX_Y2_VALS24: torch.bfloat16, SF_CTX_Y2_META24: torch.int16, SF_CTX_DY1_VALS24: torch.bfloat16}
+               SF_CTX_Y2_VALS24: torch.bfloat16, SF_CTX_Y2_META24: torch.int16, SF_CTX_DY1_VALS24: torch.bfloat16,
+               SF_CTX_RELU_VALS24: torch.bfloat16}
 
 
 def sf_ctx_view(desc, buf: torch.Tensor, field: int) -> torch.Tensor:
@@ -318,8 +327,8 @@ def sf_ffn_step_host(desc, dense: bool, hX, hW1, hW2, hdY, hY, hdX, hdW1, hdW2, 
                      stream=None):
     """Host tensors in, host tensors out (pinned memory recommended); does not synchronise."""
     _check(lib().sf_ffn_step_host(C.byref(desc), int(dense), _ptr(hX), _ptr(hW1), _ptr(hW2), _ptr(hdY), _ptr(hY),
-                                  _ptr(hdX), _ptr(hdW1), _ptr(hdW2), _ptr(staging), _ptr(fwd_ctx), _ptr(workspace),
-                                  _stream(stream)), "sf_ffn_step_host")
+                                  _ptr(hdX), _ptr(hdW1), _ptr(hdW2), _ptr(staging), _ptr(fwd_ctx), _nbytes(fwd_ctx),
+                                  _ptr(workspace), _nbytes(workspace), _stream(stream)), "sf_ffn_step_host")
 
 
 def make_schedule(warmup_steps: int, sparse_steps: int, total_steps: int) -> sf_schedule:
@@ -352,13 +361,14 @@ def sf_end_to_end_speedup(ffn_fraction: float, ffn_speedup: float) -> float:
 
 def sf_ffn_fwd_scheduled(schedule, step: int, desc, X, W1, W2, Y, fwd_ctx, workspace, stream=None):
     _check(lib().sf_ffn_fwd_scheduled(C.byref(schedule), step, C.byref(desc), _ptr(X), _ptr(W1), _ptr(W2), _ptr(Y),
-                                      _ptr(fwd_ctx), _ptr(workspace), _stream(stream)), "sf_ffn_fwd_scheduled")
+                                      _ptr(fwd_ctx), _nbytes(fwd_ctx), _ptr(workspace), _nbytes(workspace),
+                                      _stream(stream)), "sf_ffn_fwd_scheduled")
 
 
 def sf_ffn_bwd_scheduled(schedule, step: int, desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stream=None):
     _check(lib().sf_ffn_bwd_scheduled(C.byref(schedule), step, C.byref(desc), _ptr(dY), _ptr(X), _ptr(W1), _ptr(W2),
-                                      _ptr(fwd_ctx), _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace),
-                                      _stream(stream)), "sf_ffn_bwd_scheduled")
+                                      _ptr(fwd_ctx), _nbytes(fwd_ctx), _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace),
+                                      _nbytes(workspace), _stream(stream)), "sf_ffn_bwd_scheduled")
 
 
 def sf_selftest_wait_expiry(workspace, budget_clocks: int = 1_000_000, stream=None) -> None:

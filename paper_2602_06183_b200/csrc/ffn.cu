@@ -106,50 +106,64 @@ __global__ void pack_like_kernel(const uint16_t* __restrict__ dense, const uint1
 
 struct SparseLayout {
   // forward context
-  size_t y2_vals, relu_vals, meta, meta_hw, colidx, y2_dense, relu_dense, w2t, y1, vals24, meta24, meta24_hw,
+  size_t y2_vals, relu_vals, meta, meta_hw, colidx, y2_dense, relu_dense, w2t, y1, vals24, meta24, meta24_hw, relu24,
       ctx_total;
   // workspace (after the status block)
   size_t w1_vals, w1_meta, w1_meta_hw, ws_y1, w2_vals, w2_meta, w2_meta_hw, dy1_dense, dy1_vals, dy1_vals24,
       ws_total;
   bool plain24;   // activations are fed to the tensor cores as plain 2:4 over all F columns
+  bool packed8;   // M = 8: no masked dense copy of y2, ReLU(y1) or dy1 exists; every consumer reads the 2:4 layout
+  bool fused;     // packed8 and the activation is sparsified inside the y1 product's epilogue
 };
+
+constexpr size_t kNone = (size_t)-1;
 
 SparseLayout sparse_layout(const sf_ffn_desc& d) {
   SparseLayout L{};
   const size_t T = d.T, D = d.D, F = d.F, G = F / d.M;
+  // M <= 8: every V:N:M row is also a legal 2:4 row over all F columns, and on this hardware the
+  // ungathered 2:4 product (twice the tensor work, no row gather) is the faster of the two.
+  L.plain24 = (d.M == 4) || (d.M == 8 && vnm_has_24_view(d.F, d.V, d.M));
+  L.packed8 = d.M == 8 && L.plain24;
+  L.fused = L.packed8 && !(d.flags & SF_FFN_UNFUSED_ACT) && gemm_sparse24_vnm8_supported(d.F, d.T, d.D, d.V);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t r = o; o += up(bytes); return r; };
   L.y2_vals = take(T * 2 * G * 2);
   L.relu_vals = take(T * 2 * G * 2);
   L.meta = take(T * G / 2);
-  L.meta_hw = take(T * G / 2);
   L.colidx = take((T / d.V) * G * 4);
-  L.y2_dense = take(T * F * 2);
-  L.relu_dense = take(T * F * 2);
-  L.w2t = take(F * D * 2);
-  L.y1 = (d.flags & 1) ? take(T * F * 2) : (size_t)-1;
-  // M <= 8: every V:N:M row is also a legal 2:4 row over all F columns, and on this hardware the
-  // ungathered 2:4 product (twice the tensor work, no row gather) is the faster of the two.
-  L.plain24 = (d.M == 4) || (d.M == 8 && vnm_has_24_view(d.F, d.V, d.M));
-  if (d.M == 8 && L.plain24) {
+  L.y1 = (d.flags & SF_FFN_SAVE_Y1) ? take(T * F * 2) : kNone;
+  if (L.packed8) {
     L.vals24 = take(T * F);
+    L.relu24 = take(T * F);
     L.meta24 = take(T * F / 8);
     L.meta24_hw = take(T * F / 8);
+    L.meta_hw = L.y2_dense = L.relu_dense = L.w2t = kNone;
   } else {
+    L.meta_hw = take(T * G / 2);
+    L.y2_dense = take(T * F * 2);
+    L.relu_dense = take(T * F * 2);
+    L.w2t = L.plain24 ? kNone : take(F * D * 2);
     L.vals24 = L.y2_vals; L.meta24 = L.meta; L.meta24_hw = L.meta_hw;   // M == 4: the packed form is already 2:4
+    L.relu24 = kNone;
   }
   L.ctx_total = o;
   o = kStatusBytes;
   L.w1_vals = take(F * D);
   L.w1_meta = take(F * D / 8);
   L.w1_meta_hw = take(F * D / 8);
-  L.ws_y1 = (d.flags & 1) ? (size_t)-1 : take(T * F * 2);
+  L.ws_y1 = ((d.flags & SF_FFN_SAVE_Y1) || L.fused) ? kNone : take(T * F * 2);
   L.w2_vals = take(F * D);
   L.w2_meta = take(F * D / 8);
   L.w2_meta_hw = take(F * D / 8);
-  L.dy1_dense = take(T * F * 2);
-  L.dy1_vals = take(T * 2 * G * 2);
-  L.dy1_vals24 = (d.M == 8 && L.plain24) ? take(T * F) : L.dy1_vals;
+  if (L.packed8) {
+    L.dy1_vals24 = take(T * F);
+    L.dy1_dense = L.dy1_vals = kNone;
+  } else {
+    L.dy1_dense = take(T * F * 2);
+    L.dy1_vals = take(T * 2 * G * 2);
+    L.dy1_vals24 = L.dy1_vals;
+  }
   L.ws_total = o;
   return L;
 }
@@ -170,7 +184,8 @@ DenseLayout dense_layout(const sf_ffn_desc& d) {
 int check_desc(const sf_ffn_desc* d) {
   if (!d) return SF_ERR_NULL;
   if (d->N != 2) return SF_ERR_UNSUPPORTED;
-  if (d->M != 4 && d->M != 8 && d->M != 16 && d->M != 32) return SF_ERR_SHAPE;
+  if (d->M != 4 && d->M != 8 && d->M != 16 && d->M != 32 && d->M != 64) return SF_ERR_SHAPE;
+  if (d->flags & ~(SF_FFN_SAVE_Y1 | SF_FFN_UNFUSED_ACT)) return SF_ERR_UNSUPPORTED;
   if (d->V != 64 && d->V != 128) return SF_ERR_SHAPE;
   if (d->T <= 0 || d->D <= 0 || d->F <= 0) return SF_ERR_SHAPE;
   if (d->T % 256 || d->D % 256 || d->F % 256 || d->T % d->V) return SF_ERR_SHAPE;
@@ -299,32 +314,63 @@ static int check_ptrs(std::initializer_list<const void*> ps) {
   return SF_OK;
 }
 
+// Sizes the caller says its buffers have, against what the descriptor needs.
+static int check_sizes(const sf_ffn_desc& d, bool dense, size_t fwd_ctx_bytes, size_t workspace_bytes) {
+  size_t need_ctx, need_ws;
+  if (dense) {
+    const DenseLayout L = dense_layout(d);
+    need_ctx = L.ctx_total; need_ws = L.ws_total;
+  } else {
+    const SparseLayout L = sparse_layout(d);
+    need_ctx = L.ctx_total; need_ws = L.ws_total;
+  }
+  return (fwd_ctx_bytes < need_ctx || workspace_bytes < need_ws) ? SF_ERR_WORKSPACE : SF_OK;
+}
+
 int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, const void* W2, void* Y,
-                      void* fwd_ctx, void* workspace, void* stream) {
+                      void* fwd_ctx, size_t fwd_ctx_bytes, void* workspace, size_t workspace_bytes, void* stream) {
   SF_TRY(check_desc(desc));
   SF_TRY(check_ptrs({X, W1, W2, Y, fwd_ctx, workspace}));
+  SF_TRY(check_sizes(*desc, false, fwd_ctx_bytes, workspace_bytes));
   SF_TRY(check_arch());
   const sf_ffn_desc& d = *desc;
   const SparseLayout L = sparse_layout(d);
   cudaStream_t s = (cudaStream_t)stream;
   int* status = (int*)workspace;
-  void* y1 = (d.flags & 1) ? (void*)at(fwd_ctx, L.y1) : (void*)at(workspace, L.ws_y1);
+  const bool save_y1 = (d.flags & SF_FFN_SAVE_Y1) != 0;
 
   // Algorithm 1 line 4: W1s = sparsify24(W1) along d_model, then y1 = X W1s^T
   trace_mark(s);
   SF_TRY(launch_prune24(W1, d.F, d.D, d.D, 1, d.prune_mode, at(workspace, L.w1_vals), at(workspace, L.w1_meta),
                         at(workspace, L.w1_meta_hw), nullptr, s));
   trace_mark(s);
-  SF_TRY(gemm_sparse24(at(workspace, L.w1_vals), at(workspace, L.w1_meta_hw), X, true, d.F, d.T, d.D, EPI_STORE_T, y1,
-                       d.F, nullptr, 0, status, s));
-  trace_mark(s);
-  // lines 5-6: y2 = ReLU(y1)^2 in V:N:M form (+ what the backward pass needs)
-  const bool emit24 = L.plain24 && d.M == 8;
-  SF_TRY(launch_vnm(y1, d.T, d.F, d.F, d.V, d.M, 1, at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta),
-                    at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), at(fwd_ctx, L.relu_vals),
-                    at(fwd_ctx, L.y2_dense), at(fwd_ctx, L.relu_dense), emit24 ? at(fwd_ctx, L.vals24) : nullptr,
-                    emit24 ? at(fwd_ctx, L.meta24) : nullptr, emit24 ? at(fwd_ctx, L.meta24_hw) : nullptr, s));
-  trace_mark(s);
+  if (L.fused) {
+    // lines 4-6 in one kernel: the product's epilogue applies ReLU^2 and selects the V:N:M pattern on the
+    // accumulator tile; y1 itself is never written (unless asked for)
+    Vnm8Out out{at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.relu_vals), at(fwd_ctx, L.meta), at(fwd_ctx, L.colidx),
+                at(fwd_ctx, L.vals24), at(fwd_ctx, L.relu24), at(fwd_ctx, L.meta24), at(fwd_ctx, L.meta24_hw),
+                save_y1 ? (void*)at(fwd_ctx, L.y1) : nullptr};
+    SF_TRY(gemm_sparse24_vnm8(at(workspace, L.w1_vals), at(workspace, L.w1_meta_hw), X, d.F, d.T, d.D, d.V, out,
+                              status, s));
+    trace_mark(s);
+    trace_mark(s);      // (the sparsify interval is empty on this path)
+  } else {
+    void* y1 = save_y1 ? (void*)at(fwd_ctx, L.y1) : (void*)at(workspace, L.ws_y1);
+    SF_TRY(gemm_sparse24(at(workspace, L.w1_vals), at(workspace, L.w1_meta_hw), X, true, d.F, d.T, d.D, EPI_STORE_T,
+                         y1, d.F, nullptr, 0, status, s));
+    trace_mark(s);
+    // lines 5-6: y2 = ReLU(y1)^2 in V:N:M form (+ what the backward pass needs)
+    if (L.packed8) {
+      SF_TRY(launch_vnm(y1, d.T, d.F, d.F, d.V, d.M, 1, at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta), nullptr,
+                        at(fwd_ctx, L.colidx), at(fwd_ctx, L.relu_vals), nullptr, nullptr, at(fwd_ctx, L.vals24),
+                        at(fwd_ctx, L.meta24), at(fwd_ctx, L.meta24_hw), at(fwd_ctx, L.relu24), s));
+    } else {
+      SF_TRY(launch_vnm(y1, d.T, d.F, d.F, d.V, d.M, 1, at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta),
+                        at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), at(fwd_ctx, L.relu_vals),
+                        at(fwd_ctx, L.y2_dense), at(fwd_ctx, L.relu_dense), nullptr, nullptr, nullptr, nullptr, s));
+    }
+    trace_mark(s);
+  }
   // line 7: y3 = y2 W2^T with W2 dense
   hook_wait_w2(s);
   if (L.plain24) {
@@ -344,9 +390,11 @@ int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, co
 }
 
 int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, const void* W1, const void* W2,
-                      const void* fwd_ctx, void* dX, void* dW1, void* dW2, void* workspace, void* stream) {
+                      const void* fwd_ctx, size_t fwd_ctx_bytes, void* dX, void* dW1, void* dW2, void* workspace,
+                      size_t workspace_bytes, void* stream) {
   SF_TRY(check_desc(desc));
   SF_TRY(check_ptrs({dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace}));
+  SF_TRY(check_sizes(*desc, false, fwd_ctx_bytes, workspace_bytes));
   SF_TRY(check_arch());
   const sf_ffn_desc& d = *desc;
   const SparseLayout L = sparse_layout(d);
@@ -365,17 +413,36 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
                           at(workspace, L.w2_meta), at(workspace, L.w2_meta_hw), nullptr, s));
   }
   trace_mark(s);
-  // (M <= 8: the same epilogue also packs dy1 with y2's 2:4 metadata, the operand of the dX product)
+  if (L.packed8) {
+    // M = 8: ReLU(y1) comes in the 2:4 layout of y2's mask and dy1 leaves in the same layout; no [T, F]
+    // matrix is written
+    SF_TRY(gemm_sparse24(at(workspace, L.w2_vals), at(workspace, L.w2_meta_hw), dY, true, d.F, d.T, d.D,
+                         EPI_DRELU24_T, nullptr, 0, at(fwd_ctx, L.relu24), 0, status, s, at(fwd_ctx, L.meta24),
+                         at(workspace, L.dy1_vals24)));
+    trace_mark(s);
+    trace_mark(s);
+    // line 5: dX = dy1 W1 with W1 dense; W1 [F, D] is the MN-major operand
+    SF_TRY(gemm_sparse24(at(workspace, L.dy1_vals24), at(fwd_ctx, L.meta24_hw), W1, false, d.T, d.D, d.F, EPI_STORE,
+                         dX, d.D, nullptr, 0, status, s));
+    trace_mark(s);
+    hook_dx_done(s);
+    // line 3: dW2 = dY^T y2 [D, F];  line 6: dW1 = dy1^T X [F, D]: dense tensor-core products whose masked
+    // operand is expanded from its packed form inside the kernel
+    SF_TRY(gemm_dense_expand(dY, 2, at(fwd_ctx, L.vals24), at(fwd_ctx, L.meta24), d.D, d.F, d.T, dW2, d.F, status, s));
+    trace_mark(s);
+    hook_dw2_done(s);
+    SF_TRY(gemm_dense_expand(X, 1, at(workspace, L.dy1_vals24), at(fwd_ctx, L.meta24), d.F, d.D, d.T, dW1, d.D, status,
+                             s));
+    trace_mark(s);
+    return SF_OK;
+  }
+  // (M = 4: the same epilogue also packs dy1 with y2's 2:4 metadata, the operand of the dX product)
   SF_TRY(gemm_sparse24(at(workspace, L.w2_vals), at(workspace, L.w2_meta_hw), dY, true, d.F, d.T, d.D, EPI_DRELU_T,
                        at(workspace, L.dy1_dense), d.F, at(fwd_ctx, L.relu_dense), d.F, status, s,
                        L.plain24 ? at(fwd_ctx, L.meta24) : nullptr, L.plain24 ? at(workspace, L.dy1_vals24) : nullptr));
   trace_mark(s);
   // line 5: dX = dy1 W1 with W1 dense
   if (L.plain24) {
-    // dy1 shares y2's positions and was packed by the product above; W1 [F, D] is the MN-major operand
-    if ((d.flags & 1) && d.M == 8)    // debug: also the V:N:M-packed form
-      SF_TRY(launch_pack_like(at(workspace, L.dy1_dense), at(fwd_ctx, L.meta), at(fwd_ctx, L.colidx),
-                              at(workspace, L.dy1_vals), d.T, d.F, d.V, d.M, s));
     trace_mark(s);
     SF_TRY(gemm_sparse24(at(workspace, L.dy1_vals24), at(fwd_ctx, L.meta24_hw), W1, false, d.T, d.D, d.F, EPI_STORE,
                          dX, d.D, nullptr, 0, status, s));
@@ -401,9 +468,10 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
 }
 
 int sf_dense_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, const void* W2, void* Y, void* fwd_ctx,
-                     void* workspace, void* stream) {
+                     size_t fwd_ctx_bytes, void* workspace, size_t workspace_bytes, void* stream) {
   SF_TRY(check_desc(desc));
   SF_TRY(check_ptrs({X, W1, W2, Y, fwd_ctx, workspace}));
+  SF_TRY(check_sizes(*desc, true, fwd_ctx_bytes, workspace_bytes));
   SF_TRY(check_arch());
   const sf_ffn_desc& d = *desc;
   const DenseLayout L = dense_layout(d);
@@ -422,9 +490,11 @@ int sf_dense_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, con
 }
 
 int sf_dense_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, const void* W1, const void* W2,
-                     const void* fwd_ctx, void* dX, void* dW1, void* dW2, void* workspace, void* stream) {
+                     const void* fwd_ctx, size_t fwd_ctx_bytes, void* dX, void* dW1, void* dW2, void* workspace,
+                     size_t workspace_bytes, void* stream) {
   SF_TRY(check_desc(desc));
   SF_TRY(check_ptrs({dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace}));
+  SF_TRY(check_sizes(*desc, true, fwd_ctx_bytes, workspace_bytes));
   SF_TRY(check_arch());
   const sf_ffn_desc& d = *desc;
   const DenseLayout L = dense_layout(d);
@@ -463,9 +533,11 @@ int sf_ctx_view(const sf_ffn_desc* desc, const void* buf, int field, const void*
     case SF_CTX_META: off = L.meta; n = T * G / 2; break;
     case SF_CTX_COLIDX: off = L.colidx; n = (T / d.V) * G * 4; break;
     case SF_CTX_Y1:
-      if (!(d.flags & 1)) return SF_ERR_UNSUPPORTED;
+      if (!(d.flags & SF_FFN_SAVE_Y1)) return SF_ERR_UNSUPPORTED;
       off = L.y1; n = T * F * 2; break;
-    case SF_CTX_DY1_VALS: off = L.dy1_vals; n = T * 2 * G * 2; break;
+    case SF_CTX_DY1_VALS:
+      if (L.packed8) return SF_ERR_UNSUPPORTED;
+      off = L.dy1_vals; n = T * 2 * G * 2; break;
     case SF_CTX_Y2_VALS24:
       if (!L.plain24) return SF_ERR_UNSUPPORTED;
       off = L.vals24; n = T * F; break;
@@ -475,6 +547,9 @@ int sf_ctx_view(const sf_ffn_desc* desc, const void* buf, int field, const void*
     case SF_CTX_DY1_VALS24:
       if (!L.plain24) return SF_ERR_UNSUPPORTED;
       off = L.dy1_vals24; n = T * F; break;
+    case SF_CTX_RELU_VALS24:
+      if (!L.packed8) return SF_ERR_UNSUPPORTED;
+      off = L.relu24; n = T * F; break;
     default: return SF_ERR_SHAPE;
   }
   *ptr = at(buf, off);
@@ -494,8 +569,10 @@ int sf_ffn_host_staging_size(const sf_ffn_desc* desc, size_t* bytes) {
 
 int sf_ffn_step_host(const sf_ffn_desc* desc, int dense, const void* host_X, const void* host_W1,
                      const void* host_W2, const void* host_dY, void* host_Y, void* host_dX, void* host_dW1,
-                     void* host_dW2, void* device_staging, void* fwd_ctx, void* workspace, void* stream) {
+                     void* host_dW2, void* device_staging, void* fwd_ctx, size_t fwd_ctx_bytes, void* workspace,
+                     size_t workspace_bytes, void* stream) {
   SF_TRY(check_desc(desc));
+  SF_TRY(check_sizes(*desc, dense != 0, fwd_ctx_bytes, workspace_bytes));
   if (!host_X || !host_W1 || !host_W2 || !host_dY || !host_Y || !host_dX || !host_dW1 || !host_dW2 ||
       !device_staging || !fwd_ctx || !workspace)
     return SF_ERR_NULL;
@@ -524,15 +601,19 @@ int sf_ffn_step_host(const sf_ffn_desc* desc, int dense, const void* host_X, con
   int rc = SF_OK;
   do {
     if (cudaStreamWaitEvent(s, r->xw1, 0) != cudaSuccess) { rc = SF_ERR_CUDA; break; }
-    rc = dense ? sf_dense_ffn_fwd(desc, dXin, dW1in, dW2in, dYout, fwd_ctx, workspace, stream)
-               : sf_sparse_ffn_fwd(desc, dXin, dW1in, dW2in, dYout, fwd_ctx, workspace, stream);
+    rc = dense ? sf_dense_ffn_fwd(desc, dXin, dW1in, dW2in, dYout, fwd_ctx, fwd_ctx_bytes, workspace, workspace_bytes,
+                                  stream)
+               : sf_sparse_ffn_fwd(desc, dXin, dW1in, dW2in, dYout, fwd_ctx, fwd_ctx_bytes, workspace,
+                                   workspace_bytes, stream);
     if (rc != SF_OK) break;
     if (cudaEventRecord(r->y, s) != cudaSuccess || cudaStreamWaitEvent(s, r->dy, 0) != cudaSuccess) {
       rc = SF_ERR_CUDA;
       break;
     }
-    rc = dense ? sf_dense_ffn_bwd(desc, ddY, dXin, dW1in, dW2in, fwd_ctx, ddX, ddW1, ddW2, workspace, stream)
-               : sf_sparse_ffn_bwd(desc, ddY, dXin, dW1in, dW2in, fwd_ctx, ddX, ddW1, ddW2, workspace, stream);
+    rc = dense ? sf_dense_ffn_bwd(desc, ddY, dXin, dW1in, dW2in, fwd_ctx, fwd_ctx_bytes, ddX, ddW1, ddW2, workspace,
+                                  workspace_bytes, stream)
+               : sf_sparse_ffn_bwd(desc, ddY, dXin, dW1in, dW2in, fwd_ctx, fwd_ctx_bytes, ddX, ddW1, ddW2, workspace,
+                                   workspace_bytes, stream);
   } while (false);
   g_hooks = nullptr;
   // a failure past this point still has to rejoin the upload stream, or a capture of `stream` would dangle

@@ -19,6 +19,7 @@
 #include "sf_common.cuh"
 #include "tc_ptx.cuh"
 #include "gemm_tc.cuh"
+#include "sparse_fmt.cuh"
 
 namespace sf {
 
@@ -77,9 +78,27 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // m0 and first column n0; `taddr` is the TMEM address of (lane 32q, column 0) of that accumulator.
 // kTileN: accumulator columns of the tile (a multiple of 32). Columns at or beyond args.N (a ragged last
 // tile, whole 32-column chunks only since N % 32 == 0) are neither prefetched nor stored.
+__host__ __device__ constexpr bool is_drelu_t(int epi) { return epi == EPI_DRELU_T || epi == EPI_DRELU24_T; }
+
 template <int kEpi, int kTileN = BN>
 __device__ __forceinline__ void epi_prefetch(const GemmArgs& args, int64_t m0, int64_t n0, int q, int lane,
-                                             uint4 (&ax)[kEpi == EPI_DRELU_T ? kTileN / 32 : 1][4]) {
+                                             uint4 (&ax)[is_drelu_t(kEpi) ? kTileN / 32 : 1][4]) {
+  if (kEpi == EPI_DRELU24_T) {
+    // ReLU(y1) in the 2:4 layout of the activation mask: four stored values and two position nibbles per
+    // eight features; (x, y) = values, z = nibbles
+#pragma unroll
+    for (int ch = 0; ch < kTileN / 32; ++ch) {
+      if (n0 + ch * 32 >= args.N) break;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int64_t token = n0 + ch * 32 + i * 8 + (lane >> 2), f = m0 + q * 32 + (lane & 3) * 8;
+        const uint2 r = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(args.aux) +
+                                                             token * (args.M >> 1) + (f >> 1)));
+        const uint32_t mb = __ldg(reinterpret_cast<const uint8_t*>(args.pack_meta) + token * (args.M >> 3) + (f >> 3));
+        ax[is_drelu_t(kEpi) ? ch : 0][i] = make_uint4(r.x, r.y, mb, 0u);
+      }
+    }
+  }
   if (kEpi == EPI_DRELU_T) {
 #pragma unroll
     for (int ch = 0; ch < kTileN / 32; ++ch) {
@@ -96,7 +115,7 @@ __device__ __forceinline__ void epi_prefetch(const GemmArgs& args, int64_t m0, i
 template <int kEpi, int kTileN = BN>
 __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0, int q, int lane,
                                          uint8_t* my_stage,
-                                         const uint4 (&ax)[kEpi == EPI_DRELU_T ? kTileN / 32 : 1][4]) {
+                                         const uint4 (&ax)[is_drelu_t(kEpi) ? kTileN / 32 : 1][4]) {
   const int64_t row = m0 + q * 32 + lane;                                  // this thread's D row
   auto chunk = [&](int ch, const uint4 (&a4)[4], const uint32_t (&v)[32]) {
     const int64_t col0 = n0 + ch * 32;
@@ -151,21 +170,22 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
       // Transposed output: D row = feature (lane), D column = token. C is [N, M] row-major.
       float r[32];
       // optional packed copy: the metadata words of this chunk's 32 tokens (features m0 + 32q .. + 31)
-      const bool pack = kEpi == EPI_DRELU_T && args.pack_vals != nullptr;
+      const bool pack = kEpi == EPI_DRELU24_T || (kEpi == EPI_DRELU_T && args.pack_vals != nullptr);
       uint32_t mw[4] = {0, 0, 0, 0};
-      if (pack) {
+      if (pack && kEpi == EPI_DRELU_T) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
           mw[i] = __ldg(reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(args.pack_meta) +
                                                          (col0 + i * 8 + (lane >> 2)) * (args.M >> 3) +
                                                          ((m0 + q * 32) >> 3)));
       }
-      if (kEpi == EPI_DRELU_T) {
+      if (is_drelu_t(kEpi)) {
         // aux[token, feature] chunk -> staging -> one column per lane
         __syncwarp();
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          *reinterpret_cast<uint4*>(my_stage + (i * 8 + (lane >> 2)) * kEpiStageRow + (lane & 3) * 16) = a4[i];
+          *reinterpret_cast<uint4*>(my_stage + (i * 8 + (lane >> 2)) * kEpiStageRow + (lane & 3) * 16) =
+              kEpi == EPI_DRELU24_T ? expand24_x8(make_uint2(a4[i].x, a4[i].y), a4[i].z) : a4[i];
         __syncwarp();
 #pragma unroll
         for (int j = 0; j < 32; ++j)
@@ -176,7 +196,7 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
       for (int j = 0; j < 32; ++j) {
         float x = __uint_as_float(v[j]);
         uint32_t b;
-        if (kEpi == EPI_DRELU_T) {
+        if (is_drelu_t(kEpi)) {
           // aux holds ReLU(y1) on the activation mask and +0 elsewhere: off-mask entries become +0
           b = (r[j] == 0.f) ? 0u : float_to_bf16_bits(__fmul_rn(__fmul_rn(2.f, x), r[j]));
         } else {
@@ -189,10 +209,11 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
       for (int i = 0; i < 4; ++i) {
         const int t = i * 8 + (lane >> 2), seg = lane & 3;
         const uint4 o = *reinterpret_cast<const uint4*>(my_stage + t * kEpiStageRow + seg * 16);
-        *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.C) + (col0 + t) * args.ldc + m0 + q * 32 + seg * 8) = o;
+        if (kEpi != EPI_DRELU24_T)
+          *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.C) + (col0 + t) * args.ldc + m0 + q * 32 + seg * 8) = o;
         if (pack) {
           // this lane's eight features are two groups of four: keep the two recorded positions of each
-          const uint32_t mb = (mw[i] >> (8 * seg)) & 0xFFu;
+          const uint32_t mb = kEpi == EPI_DRELU24_T ? (a4[i].z & 0xFFu) : ((mw[i] >> (8 * seg)) & 0xFFu);
           const uint32_t p0 = __byte_perm(o.x, o.y, 0x1010u + (mb & 3u) * 0x22u + ((mb >> 2) & 3u) * 0x2200u);
           const uint32_t p1 = __byte_perm(o.z, o.w, 0x1010u + ((mb >> 4) & 3u) * 0x22u + (mb >> 6) * 0x2200u);
           *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(args.pack_vals) + (col0 + t) * (args.M >> 1) +
@@ -205,16 +226,16 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
   uint32_t va[32], vb[32];
   tmem_ld_32x32b_x32(taddr, va);
   constexpr int kChunks = kTileN / 32;
-  if (kEpi == EPI_DRELU_T) {
+  if (is_drelu_t(kEpi)) {
 #pragma unroll
     for (int ch = 0; ch < kChunks; ch += 2) {
       tmem_ld_wait_on(va);
       if (ch + 1 < kChunks) tmem_ld_32x32b_x32(taddr + (ch + 1) * 32, vb);
-      chunk(ch, ax[kEpi == EPI_DRELU_T ? ch : 0], va);
+      chunk(ch, ax[is_drelu_t(kEpi) ? ch : 0], va);
       if (ch + 1 < kChunks) {
         tmem_ld_wait_on(vb);
         if (ch + 2 < kChunks) tmem_ld_32x32b_x32(taddr + (ch + 2) * 32, va);
-        chunk(ch + 1, ax[kEpi == EPI_DRELU_T ? (ch + 1 < kChunks ? ch + 1 : ch) : 0], vb);
+        chunk(ch + 1, ax[is_drelu_t(kEpi) ? (ch + 1 < kChunks ? ch + 1 : ch) : 0], vb);
       }
     }
   } else if (kChunks % 2 == 0) {
@@ -238,6 +259,156 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
         if (ch + 2 < kChunks) tmem_ld_32x32b_x32(taddr + (ch + 2) * 32, va);
         chunk(ch + 1, ax[0], vb);
       }
+    }
+  }
+}
+
+
+// ---- fused SquaredReLU + V:N:M selection (groups of eight) ---------------------------------------------
+// Epilogue of the y1 product: the accumulator tile is y1^T (TMEM lane = feature, column = token), so a
+// lane owns one feature column of every V x 8 block and eight neighbouring lanes own one block.
+// Per V-block of the tile, each epilogue warp (32 features = four groups):
+//   pass 1  reads its lanes' V accumulator columns, rounds them to bf16 (this is y1), parks them in
+//           shared memory as [token][feature], and accumulates the column score of Section 2.3 in
+//           float32, token by token in ascending order (the order is part of the format);
+//   rank    the eight lanes of a group exchange scores; the four best columns stay (ties to the lower
+//           column), their indices go to colidx and into per-group byte-permute selector tables;
+//   pass 2  one thread per (token, group) takes the group's eight values back from shared memory, applies
+//           SquaredReLU, keeps the two largest of the four kept columns and writes the packed activation,
+//           the packed ReLU values, both metadata forms and the 2:4 view.
+// The accumulator is released to the MMA warp as soon as the last block's pass 1 has read it.
+constexpr int kVnmStageBytes = 128 * 64;                        // y1 of one block: up to 128 tokens x 32 features
+constexpr int kVnmWarpBytes = kVnmStageBytes + 16 + 4 * 7 * 16 + 32;   // + colidx, selector table, nibble table
+constexpr int kVnmEpiBytes = 4 * ((kVnmWarpBytes + 127) / 128 * 128);
+
+template <int kTileN>
+__device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0, int q,
+                                              int lane, uint8_t* wsm, uint64_t* tmem_empty_bar) {
+  uint8_t* stage = wsm;                                                   // [V][64 B]
+  uint8_t* cidx = wsm + kVnmStageBytes;                                   // [4 groups][4]
+  uint4* sel_tab = reinterpret_cast<uint4*>(wsm + kVnmStageBytes + 16);   // [4 groups][7]
+  uint8_t* nib_tab = wsm + kVnmStageBytes + 16 + 4 * 7 * 16;              // [4 groups][7]
+  const int V = args.V;
+  const int64_t F = args.M, G = F >> 3;
+  const int64_t f0 = m0 + q * 32, g0 = f0 >> 3;                           // this warp's first feature / group
+  const int jm = lane & 7, gl = lane & 3;
+  constexpr int kMaxBlocks = kTileN / 64;
+  int nblk = kTileN / V;
+  while (nblk > 0 && n0 + (int64_t)(nblk - 1) * V >= args.N) --nblk;       // ragged last tile: whole blocks only
+  if (nblk == 0) {                                                         // cannot happen for a launched tile; keep the protocol
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive_leader(tmem_empty_bar);
+    return;
+  }
+#pragma unroll 1
+  for (int b = 0; b < kMaxBlocks; ++b) {
+    if (b >= nblk) break;
+    __syncwarp();                                                          // the previous block's pass 2 has read the stage
+    const int64_t t0 = n0 + (int64_t)b * V;
+    // ---- pass 1
+    float score = 0.f;
+    uint32_t v[32];
+#pragma unroll 1
+    for (int c = 0; c < V / 32; ++c) {
+      tmem_ld_32x32b_x32(taddr + (uint32_t)(b * V + c * 32), v);
+      tmem_ld_wait_on(v);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const uint32_t y = float_to_bf16_bits(__uint_as_float(v[j]));
+        *reinterpret_cast<uint16_t*>(stage + (c * 32 + j) * 64 + lane * 2) = (uint16_t)y;
+        const float r = fmaxf(bf16_bits_to_float(y), 0.f);
+        const float h = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(r, r)));
+        score = __fadd_rn(score, h);
+      }
+    }
+    if (b == nblk - 1) {
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(tmem_empty_bar);
+    }
+    // ---- rank the eight columns of each group
+    const uint32_t sb = __float_as_uint(score);                            // scores are >= 0: the pattern orders them
+    int rank = 0;
+#pragma unroll
+    for (int i = 1; i < 8; ++i) {
+      const uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, sb, i);
+      const int oj = jm ^ i;
+      rank += (o > sb) || (o == sb && oj < jm);
+    }
+    const bool keep = rank < 4;
+    const uint32_t ball = __ballot_sync(0xFFFFFFFFu, keep);
+    const uint32_t gbyte = (ball >> (lane & 24)) & 0xFFu;
+    __syncwarp();                                                          // previous block's pass 2 is done with the tables
+    if (keep) cidx[(lane >> 3) * 4 + __popc(gbyte & ((1u << jm) - 1u))] = (uint8_t)jm;
+    __syncwarp();
+    if (lane < 4)
+      *reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(args.vn_colidx) + ((t0 / V) * G + g0 + lane) * 4) =
+          *reinterpret_cast<const uint32_t*>(cidx + lane * 4);
+    if (lane < 24) {
+      const int ge = lane / 6, pe = lane - ge * 6;
+      const int pi = pe < 3 ? 0 : (pe < 5 ? 1 : 2), pj = pe < 3 ? pe + 1 : (pe < 5 ? pe - 1 : 3);
+      uint4 selv;
+      uint32_t nib24;
+      vnm8_pair_selectors(cidx[ge * 4 + pi], cidx[ge * 4 + pj], selv, nib24);
+      const int slot = ge * 7 + (int)nib_slot((uint32_t)pi | ((uint32_t)pj << 2));
+      sel_tab[slot] = selv;
+      nib_tab[slot] = (uint8_t)nib24;
+    }
+    __syncwarp();
+    // ---- pass 2: this thread serves group gl of tokens (lane >> 2) + 8 * it
+    const uint32_t c4 = *reinterpret_cast<const uint32_t*>(cidx + gl * 4);
+    uint32_t selp[2], mhi[2];
+#pragma unroll
+    for (int pr = 0; pr < 2; ++pr) {
+      const uint32_t ca = (c4 >> (16 * pr)) & 0xFFu, cb = (c4 >> (16 * pr + 8)) & 0xFFu;
+      const uint32_t sa = 2u * (ca & 3u), sbb = 2u * (cb & 3u);
+      selp[pr] = sa | ((sa + 1u) << 4) | (sbb << 8) | ((sbb + 1u) << 12);
+      mhi[pr] = ((ca & 4u) ? 0x0000FFFFu : 0u) | ((cb & 4u) ? 0xFFFF0000u : 0u);
+    }
+    const uint4* my_sel = sel_tab + gl * 7;
+    const uint8_t* my_nib = nib_tab + gl * 7;
+    const int64_t kw24 = (f0 >> 4) + (gl >> 1);                            // this lane pair's 16-column word of the 2:4 view
+    const bool lead4 = gl == 0, lead2 = (gl & 1) == 0;
+#pragma unroll 2
+    for (int it = 0; it < V / 8; ++it) {
+      const int tk = (lane >> 2) + 8 * it;
+      const int64_t t = t0 + tk;
+      const uint4 qv = *reinterpret_cast<const uint4*>(stage + tk * 64 + gl * 16);
+      uint32_t rw[4] = {qv.x, qv.y, qv.z, qv.w}, hw[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { rw[j] = bf2_relu(rw[j]); hw[j] = bf2_sq(rw[j]); }
+      const uint32_t a0 = __byte_perm(hw[0], hw[1], selp[0]), b0 = __byte_perm(hw[2], hw[3], selp[0]);
+      const uint32_t a1 = __byte_perm(hw[0], hw[1], selp[1]), b1 = __byte_perm(hw[2], hw[3], selp[1]);
+      const uint32_t hk0 = (a0 & ~mhi[0]) | (b0 & mhi[0]), hk1 = (a1 & ~mhi[1]) | (b1 & mhi[1]);
+      uint32_t packed;
+      const uint32_t nib = top2of4_packed(hk0, hk1, &packed);
+      const uint32_t slot = nib_slot(nib);
+      const uint4 sel = my_sel[slot];
+      const uint32_t x = __byte_perm(rw[0], rw[1], sel.z), y = __byte_perm(rw[2], rw[3], sel.z);
+      const uint32_t rpair = __byte_perm(x, y, sel.z >> 16);
+      const int64_t pv = t * (2 * G) + 2 * (g0 + gl);
+      reinterpret_cast<uint32_t*>(args.vn_vals)[pv >> 1] = packed;
+      reinterpret_cast<uint32_t*>(args.vn_relu)[pv >> 1] = rpair;
+      const int64_t p24 = (t * (F >> 1) + (g0 + gl) * 4) >> 2;             // in 8-byte units
+      reinterpret_cast<uint2*>(args.vn_vals24)[p24] =
+          make_uint2(__byte_perm(packed, 0u, sel.w), __byte_perm(packed, 0u, sel.w >> 16));
+      reinterpret_cast<uint2*>(args.vn_relu24)[p24] =
+          make_uint2(__byte_perm(rpair, 0u, sel.w), __byte_perm(rpair, 0u, sel.w >> 16));
+      if (args.vn_y1) reinterpret_cast<uint4*>(args.vn_y1)[(t * F + f0 + gl * 8) >> 3] = qv;
+      // canonical V:N:M metadata: the warp's four groups of a token form one word
+      uint32_t word = nib;
+      word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 4;
+      word |= __shfl_down_sync(0xFFFFFFFFu, word, 2) << 8;
+      if (lead4) reinterpret_cast<uint16_t*>(args.vn_meta)[t * (G >> 2) + (g0 >> 2)] = (uint16_t)word;
+      // metadata of the 2:4 view: one byte per group, one 16-bit word per pair of groups
+      uint32_t mb = my_nib[slot];
+      mb |= __shfl_down_sync(0xFFFFFFFFu, mb, 1) << 8;
+      const uint32_t mb32 = (mb & 0xFFFFu) | (__shfl_down_sync(0xFFFFFFFFu, mb, 2) << 16);
+      if (lead4) reinterpret_cast<uint32_t*>(args.vn_meta24)[(t * (F >> 4) + (f0 >> 4)) >> 1] = mb32;
+      if (lead2)
+        *reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(args.vn_meta24_hw) + meta_hw_offset(t, kw24, F)) =
+            (uint16_t)mb;
     }
   }
 }
@@ -478,7 +649,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
       const int64_t m0 = (int64_t)mt * BM, n0 = (int64_t)nt * BN;
       // The dy1 epilogue multiplies by a [token, feature] tile of the saved activations; its loads do
       // not depend on the accumulator, so they are issued before the wait and land during the main loop.
-      uint4 ax[kEpi == EPI_DRELU_T ? BN / 32 : 1][4];
+      uint4 ax[is_drelu_t(kEpi) ? BN / 32 : 1][4];
       epi_prefetch<kEpi>(args, m0, n0, q, lane, ax);
       if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
@@ -511,17 +682,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 // Stage = 64 K (dense, 4 MMAs of K=16) or 128 logical K (2:4, 4 MMAs of K=32 and one metadata atom):
 // four MMAs per barrier round trip keep the single issuing thread ahead of the tensor pipe.
 constexpr int kThreads2 = 192;
+constexpr int kThreads2Expand = 320;                     // + four warps that expand a packed operand into its stage
+constexpr int kPkStageBytes = 8192 + 1024;               // packed values [64 tokens][64] + metadata bytes [64][16]
 __host__ __device__ constexpr int stage_bytes2(bool sparse, int bn = BN) {
   return sparse ? (16384 + 2 * (bn / 2) * 128 + 2048) : (16384 + 16384);
 }
-__host__ __device__ constexpr int num_stages2(bool sparse) { return sparse ? 4 : 6; }
-__host__ __device__ constexpr int smem_bytes2(bool sparse, int bn = BN) {
-  return 1024 + num_stages2(sparse) * stage_bytes2(sparse, bn) + kEpiStageBytes + 512;
+__host__ __device__ constexpr int num_stages2(bool sparse, int bn = BN, bool expand = false) {
+  return sparse ? (bn <= 128 ? 5 : 4) : (expand ? 5 : 6);
+}
+__host__ __device__ constexpr int epi_bytes2(int epi) { return epi == EPI_VNM8 ? kVnmEpiBytes : kEpiStageBytes; }
+__host__ __device__ constexpr int smem_bytes2(bool sparse, int bn = BN, int epi = EPI_STORE, bool expand = false) {
+  return 1024 + num_stages2(sparse, bn, expand) * (stage_bytes2(sparse, bn) + (expand ? kPkStageBytes : 0)) +
+         epi_bytes2(epi) + 512;
 }
 
 struct SmemCtl2 {
   uint64_t full[8];
   uint64_t empty[8];
+  uint64_t pk_full[8];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint32_t tmem_base;
@@ -532,15 +710,20 @@ __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
   return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 
-template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
+// kExpand (dense mode with both operands MN-major only): 1 = operand A, 2 = operand B is not loaded as a
+// dense tile; its 2:4-packed form (tmapPk: values, tmapMeta: metadata bytes) is staged by TMA and four
+// extra warps expand it, zero-filled, into the swizzled layout the MMA reads.
+template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN, int kExpand = 0>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kExpand ? kThreads2Expand : kThreads2, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                const __grid_constant__ CUtensorMap tmapMeta, const GemmArgs args) {
+                const __grid_constant__ CUtensorMap tmapMeta, const __grid_constant__ CUtensorMap tmapPk,
+                const GemmArgs args) {
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   constexpr bool kSparse = kMode == MODE_SPARSE24;
-  constexpr int kStages = num_stages2(kSparse);
+  constexpr int kStages = num_stages2(kSparse, kBN, kExpand != 0);
   constexpr int kBK = kSparse ? 128 : 64;                // logical K per stage
+  static_assert(kExpand == 0 || (kMode == MODE_DENSE && kAMN && kBMN), "packed operands: weight-gradient products only");
   constexpr int kAStageBytes = 16384;
   constexpr int kBSlabBytes = (kBN / 2) * 128;            // this CTA's half of B for one 64-wide K slab
   constexpr int kBHalfBytes = kSparse ? 2 * kBSlabBytes : kBSlabBytes;
@@ -553,8 +736,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   static_assert(kBN % 32 == 0 && kBN <= 256, "tile width");
   static_assert(!(kMode == MODE_DENSE) || kBN == BN, "dense mode uses 256-column tiles");
   static_assert(!kBMN || kBN == BN, "MN-major B is loaded in 64-column chunks");
-  uint8_t* epi_stage = smem + kStages * kStageBytes;
-  SmemCtl2* ctl = reinterpret_cast<SmemCtl2*>(epi_stage + kEpiStageBytes);
+  uint8_t* pk_stage = smem + kStages * kStageBytes;       // kExpand: ring of packed tiles, one per stage
+  uint8_t* epi_stage = pk_stage + (kExpand ? kStages * kPkStageBytes : 0);
+  SmemCtl2* ctl = reinterpret_cast<SmemCtl2*>(epi_stage + epi_bytes2(kEpi));
   volatile int* abort_flag = &ctl->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -567,10 +751,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   if (threadIdx.x == 0) {
     prefetch_tmap(&tmapA);
     prefetch_tmap(&tmapB);
-    if (kSparse) prefetch_tmap(&tmapMeta);
+    if (kSparse || kExpand) prefetch_tmap(&tmapMeta);
+    if (kExpand) prefetch_tmap(&tmapPk);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&ctl->full[s], 1);
+      mbar_init(&ctl->full[s], kExpand ? 1 + 8 : 1);     // + the four expander warps of either CTA
       mbar_init(&ctl->empty[s], 1);
+      mbar_init(&ctl->pk_full[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&ctl->tmem_full[b], 1);
@@ -606,22 +792,34 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
           uint8_t* sM = sB + kBHalfBytes;
           uint64_t* bar = &ctl->full[stage];
           if (rank == 0) {
-            // the leader's barrier collects the bytes of both CTAs
-            mbar_arrive_expect_tx(bar, 2u * ((uint32_t)kAStageBytes + (uint32_t)kBHalfBytes +
+            // the leader's barrier collects the bytes of both CTAs (an expanded operand arrives by
+            // shared-memory stores, not by TMA)
+            mbar_arrive_expect_tx(bar, 2u * ((kExpand == 1 ? 0u : (uint32_t)kAStageBytes) +
+                                             (kExpand == 2 ? 0u : (uint32_t)kBHalfBytes) +
                                              (kSparse ? (uint32_t)kMetaStageBytes : 0u)));
           }
           if (kMode == MODE_DENSE) {
-            if (!kAMN) {
+            if (kExpand == 1) {
+              // packed A: this CTA's 128 features of 64 tokens, into the staging ring (own barrier)
+            } else if (!kAMN) {
               tma_load_2d_2cta(sA, &tmapA, bar, kb * 64, m0);
             } else {
               tma_load_2d_2cta(sA, &tmapA, bar, m0, kb * 64);
               tma_load_2d_2cta(sA + 8192, &tmapA, bar, m0 + 64, kb * 64);
             }
-            if (!kBMN) {
+            if (kExpand == 2) {
+            } else if (!kBMN) {
               tma_load_2d_2cta(sB, &tmapB, bar, kb * 64, nb0);                 // box {64 k, 128 n}
             } else {
               tma_load_2d_2cta(sB, &tmapB, bar, nb0, kb * 64);                 // box {64 n, 64 k}
               tma_load_2d_2cta(sB + 8192, &tmapB, bar, nb0 + 64, kb * 64);
+            }
+            if (kExpand) {
+              const int f0 = kExpand == 1 ? m0 : nb0;                          // first feature of this CTA's half
+              uint8_t* sP = pk_stage + stage * kPkStageBytes;
+              mbar_arrive_expect_tx(&ctl->pk_full[stage], (uint32_t)kPkStageBytes);
+              tma_load_2d(sP, &tmapPk, &ctl->pk_full[stage], f0 >> 1, kb * 64);          // values: box {64, 64}
+              tma_load_2d(sP + 8192, &tmapMeta, &ctl->pk_full[stage], f0 >> 4, kb * 64); // metadata: box {8, 64}
             }
           } else {
             tma_load_2d_2cta(sA, &tmapA, bar, kb * 64, m0);                    // stored values: box {64, 128}
@@ -694,25 +892,60 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
         if (++acc == (uint32_t)kAccBufs) { acc = 0; acc_phase ^= 1; }
       }
     }
+  } else if (kExpand != 0 && warp >= 6) {
+    // =========================== operand expander (warps 6..9, both CTAs) ===========================
+    // Stage tile = 64 tokens (K) x 128 features, MN-major, 128-byte swizzle: two chunks of 64 features,
+    // a token row of a chunk is 128 bytes whose 16-byte units are XOR-ed with (token & 7). One unit is
+    // eight features = two 2:4 groups = four stored values + one metadata byte in the packed tile.
+    const int te = (int)threadIdx.x - 192;                 // 0..127
+    const int seg = te & 15, tk0 = te >> 4;                // 16 units per token row; 8 tokens per pass
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+      for (int kb = 0; kb < nkb; ++kb) {
+        if (!mbar_wait(&ctl->pk_full[stage], phase, abort_flag)) { ok = false; break; }
+        const uint8_t* sP = pk_stage + stage * kPkStageBytes;
+        uint8_t* dst = smem + stage * kStageBytes + (kExpand == 1 ? 0 : kAStageBytes) + (seg >> 3) * 8192;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int tk = tk0 + 8 * i;
+          const uint2 v = *reinterpret_cast<const uint2*>(sP + tk * 128 + seg * 8);
+          const uint32_t mb = sP[8192 + tk * 16 + seg];
+          *reinterpret_cast<uint4*>(dst + tk * 128 + (((seg & 7) ^ (tk & 7)) << 4)) = expand24_x8(v, mb);
+        }
+        // generic-proxy stores -> visible to the tensor core's async-proxy reads, then signal the stage
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_leader(&ctl->full[stage]);
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
+    }
   } else {
     // =========================== epilogue (warps 2..5, both CTAs) ===========================
     const int q = warp & 3;
-    uint8_t* my_stage = epi_stage + q * 32 * kEpiStageRow;
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
       int mt, nt;
       tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
       const int64_t m0 = (int64_t)mt * 256 + (int64_t)rank * 128, n0 = (int64_t)nt * kBN;
-      uint4 ax[kEpi == EPI_DRELU_T ? kBN / 32 : 1][4];
-      epi_prefetch<kEpi, kBN>(args, m0, n0, q, lane, ax);
-      if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
-      tc_fence_after();
       const uint32_t taddr = tmem_base + acc * kBN + ((uint32_t)(q * 32) << 16);
-      epi_tile<kEpi, kBN>(args, taddr, m0, n0, q, lane, my_stage, ax);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_leader(&ctl->tmem_empty[acc]);
+      if constexpr (kEpi == EPI_VNM8) {
+        if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        // releases the accumulator itself, as soon as its last column has been read
+        epi_vnm8_tile<kBN>(args, taddr, m0, n0, q, lane, epi_stage + q * (kVnmEpiBytes / 4), &ctl->tmem_empty[acc]);
+      } else {
+        uint8_t* my_stage = epi_stage + q * 32 * kEpiStageRow;
+        uint4 ax[is_drelu_t(kEpi) ? kBN / 32 : 1][4];
+        epi_prefetch<kEpi, kBN>(args, m0, n0, q, lane, ax);
+        if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        epi_tile<kEpi, kBN>(args, taddr, m0, n0, q, lane, my_stage, ax);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_leader(&ctl->tmem_empty[acc]);
+      }
       if (++acc == (uint32_t)kAccBufs) { acc = 0; acc_phase ^= 1; }
     }
   }
@@ -748,17 +981,18 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// 2D tensor map over a row-major [rows, cols] matrix of 2-byte (bf16) or 4-byte (uint32) elements;
+// 2D tensor map over a row-major [rows, cols] matrix of 2-byte (bf16, uint16) or 4-byte (uint32) elements;
 // box = {box_cols, box_rows}.
 int make_tmap(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
-              uint32_t box_rows, CUtensorMapSwizzle swz, bool u32 = false) {
+              uint32_t box_rows, CUtensorMapSwizzle swz, int kind = 0 /* 0 bf16, 1 uint32, 2 uint16 */) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return cuda_fail(cudaErrorUnknown);
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const bool u32 = kind == 1;
   cuuint64_t strides[1] = {(cuuint64_t)ld * (u32 ? 4 : 2)};
   cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, u32 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+  CUresult r = fn(m, u32 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : (kind == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16), 2,
                   const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -798,10 +1032,12 @@ int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& a, 
   return SF_OK;
 }
 
-template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN>
-int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tm, GemmArgs a, cudaStream_t s) {
-  auto kern = gemm_tc2_kernel<kMode, kAMN, kBMN, kEpi, kBN>;
-  constexpr int smem = smem_bytes2(kMode != MODE_DENSE, kBN);
+template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN, int kExpand = 0>
+int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tm, GemmArgs a, cudaStream_t s,
+               const CUtensorMap* tpk = nullptr) {
+  auto kern = gemm_tc2_kernel<kMode, kAMN, kBMN, kEpi, kBN, kExpand>;
+  constexpr int smem = smem_bytes2(kMode != MODE_DENSE, kBN, kEpi, kExpand != 0);
+  static_assert(smem <= 232448, "shared memory per CTA");
   static bool attr_done[64] = {false};
   int dev = 0;
   SF_CUDA_TRY(cudaGetDevice(&dev));
@@ -814,14 +1050,17 @@ int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
   const int tiles = a.num_m_tiles * a.num_n_tiles;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  kern<<<2 * pairs, kThreads2, smem, s>>>(ta, tb, tm, a);
+  kern<<<2 * pairs, kExpand ? kThreads2Expand : kThreads2, smem, s>>>(ta, tb, tm, tpk ? *tpk : ta, a);
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
 
 // Tile width of the two-accumulator 2:4 variant (transposed-output products): 2 x 224 accumulator
 // columns + 8 metadata columns fit the 512 TMEM columns.
-constexpr int kNarrowBN = 224;
+#ifndef SF_NARROW_BN
+#define SF_NARROW_BN 224
+#endif
+constexpr int kNarrowBN = SF_NARROW_BN;
 
 // The two-CTA kernels need M % 256 == 0; other shapes run the one-CTA kernels.
 bool use_two_cta(int64_t M) { return M % 256 == 0; }
@@ -868,7 +1107,8 @@ int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64
 int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t M, int64_t N,
                   int64_t K, int epi, void* C, int64_t ldc, const void* aux, int64_t ldaux, int* status,
                   cudaStream_t s, const void* pack_meta, void* pack_vals) {
-  if ((pack_meta != nullptr) != (pack_vals != nullptr) || (pack_vals && epi != EPI_DRELU_T)) return SF_ERR_UNSUPPORTED;
+  if ((pack_meta != nullptr) != (pack_vals != nullptr) || (pack_vals && !is_drelu_t(epi))) return SF_ERR_UNSUPPORTED;
+  if (epi == EPI_DRELU24_T && (!pack_vals || !aux || M % 256)) return SF_ERR_UNSUPPORTED;
   if (M % BM || N % BN || K % 128) return SF_ERR_SHAPE;
   if (M == 0 || N == 0) return SF_OK;
   const bool two = use_two_cta(M);
@@ -887,7 +1127,7 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
   if (two) {
     // hardware-ordered metadata: 2 KB atoms viewed as two rows of 256 uint32
     const int64_t atoms = (M / 128) * (K / 128);
-    st = make_tmap(&tm, meta_hw, 2 * atoms, 256, 256, 256, 2, CU_TENSOR_MAP_SWIZZLE_NONE, true);
+    st = make_tmap(&tm, meta_hw, 2 * atoms, 256, 256, 256, 2, CU_TENSOR_MAP_SWIZZLE_NONE, 1);
     if (st != SF_OK) return st;
   }
   GemmArgs a{};
@@ -905,7 +1145,58 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
   if (epi == EPI_DRELU_T)
     return two ? launch_two<MODE_SPARSE24, false, false, EPI_DRELU_T, kNarrowBN>(ta, tb, tm, a, s)
                : launch_one<MODE_SPARSE24, false, false, EPI_DRELU_T>(ta, tb, a, s);
+  if (epi == EPI_DRELU24_T) return launch_two<MODE_SPARSE24, false, false, EPI_DRELU24_T, kNarrowBN>(ta, tb, tm, a, s);
   return SF_ERR_UNSUPPORTED;
+}
+
+bool gemm_sparse24_vnm8_supported(int64_t F, int64_t T, int64_t D, int V) {
+  return F > 0 && T > 0 && F % 256 == 0 && D % 128 == 0 && (V == 64 || V == 128) && T % V == 0;
+}
+
+int gemm_sparse24_vnm8(const void* a_vals, const uint8_t* meta_hw, const void* X, int64_t F, int64_t T, int64_t D,
+                       int V, const Vnm8Out& out, int* status, cudaStream_t s) {
+  if (!gemm_sparse24_vnm8_supported(F, T, D, V)) return SF_ERR_SHAPE;
+  // Token tiles hold whole V-blocks: three blocks of 64 (192 columns) or one block of 128.
+  const int bn = V == 64 ? 192 : 128;
+  CUtensorMap ta, tb, tm;
+  int st = make_tmap(&ta, a_vals, F, D / 2, D / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tb, X, T, D, D, 64, bn / 2, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  const int64_t atoms = (F / 128) * (D / 128);
+  st = make_tmap(&tm, meta_hw, 2 * atoms, 256, 256, 256, 2, CU_TENSOR_MAP_SWIZZLE_NONE, 1);
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = F; a.N = T; a.K = D; a.V = V;
+  a.meta_hw = meta_hw; a.status = status;
+  a.vn_vals = out.vals; a.vn_relu = out.relu; a.vn_meta = out.meta; a.vn_colidx = out.colidx;
+  a.vn_vals24 = out.vals24; a.vn_relu24 = out.relu24; a.vn_meta24 = out.meta24; a.vn_meta24_hw = out.meta24_hw;
+  a.vn_y1 = out.y1;
+  if (V == 64) return launch_two<MODE_SPARSE24, false, false, EPI_VNM8, 192>(ta, tb, tm, a, s);
+  return launch_two<MODE_SPARSE24, false, false, EPI_VNM8, 128>(ta, tb, tm, a, s);
+}
+
+int gemm_dense_expand(const void* dense_op, int packed_operand, const void* pk_vals, const void* pk_meta, int64_t M,
+                      int64_t N, int64_t K, void* C, int64_t ldc, int* status, cudaStream_t s) {
+  if (M % 256 || N % 256 || K % 64 || (packed_operand != 1 && packed_operand != 2)) return SF_ERR_SHAPE;
+  if (M == 0 || N == 0) return SF_OK;
+  const int64_t X = packed_operand == 1 ? M : N;                              // width of the packed operand
+  CUtensorMap ta, tb, tm, tp;
+  // the dense operand: [K, M] or [K, N] row-major, 64 x 64 boxes
+  int st = make_tmap(packed_operand == 1 ? &tb : &ta, dense_op, K, packed_operand == 1 ? N : M,
+                     packed_operand == 1 ? N : M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  if (packed_operand == 1) ta = tb; else tb = ta;                             // the unused map only has to be valid
+  st = make_tmap(&tp, pk_vals, K, X / 2, X / 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_NONE);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tm, pk_meta, K, X / 16, X / 16, 8, 64, CU_TENSOR_MAP_SWIZZLE_NONE, 2);
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = M; a.N = N; a.K = K;
+  a.C = C; a.ldc = ldc; a.status = status;
+  a.num_m_tiles = (int)(M / BM); a.num_n_tiles = (int)(N / BN); a.num_k_blocks = (int)(K / 64);
+  if (packed_operand == 1) return launch_two<MODE_DENSE, true, true, EPI_STORE, BN, 1>(ta, tb, tm, a, s, &tp);
+  return launch_two<MODE_DENSE, true, true, EPI_STORE, BN, 2>(ta, tb, tm, a, s, &tp);
 }
 
 int gemm_venom(const void* a_vals, const uint8_t* meta_hw, const uint8_t* colidx, const void* Bt, int64_t T,

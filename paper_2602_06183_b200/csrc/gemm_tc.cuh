@@ -13,7 +13,11 @@ enum GemmEpilogue {
   EPI_SQRELU = 1,   // C = y = bf16(acc);  C2 = bf16(max(y, 0)^2)                     (Eq. 2)
   EPI_DRELU = 2,    // C = bf16(2 * acc * max(aux[m, n], 0))                           (Eq. 6)
   EPI_STORE_T = 3,  // C[n, m] = bf16(acc)          (accumulator rows are output columns)
-  EPI_DRELU_T = 4   // C[n, m] = bf16(2 * acc * aux[n, m]), +0 where aux is zero       (Eq. 6 on the mask)
+  EPI_DRELU_T = 4,  // C[n, m] = bf16(2 * acc * aux[n, m]), +0 where aux is zero       (Eq. 6 on the mask)
+  EPI_VNM8 = 5,     // SquaredReLU + V:N:M selection (groups of eight) on the accumulator tile itself: rows are
+                    // features, columns are tokens; writes the packed activation, never the dense y1  (Eq. 2, Section 2.3)
+  EPI_DRELU24_T = 6 // as EPI_DRELU_T with aux given in the 2:4 layout of the mask (values [n, m/2] + pack_meta) and
+                    // only the packed output written
 };
 
 struct GemmArgs {
@@ -34,12 +38,38 @@ struct GemmArgs {
   // EPI_DRELU_T only, optional: also emit the output packed as a 2:4 operand at given positions
   const void* pack_meta;    // canonical 2:4 metadata [N, M/16] uint16 (rows = output rows of Ct)
   void* pack_vals;          // bf16 [N, M/2]
+  // EPI_VNM8 outputs (T = N tokens, F = M features, G = F / 8 groups per token)
+  void* vn_vals;            // bf16 [T, 2G]   kept activation values (V:N:M packed)
+  void* vn_relu;            // bf16 [T, 2G]   ReLU(y1) at the same positions
+  void* vn_meta;            // uint16 [T, G/4] canonical nibbles over the condensed matrix
+  void* vn_colidx;          // uint8 [T/V, G, 4]
+  void* vn_vals24;          // bf16 [T, F/2]  the same activation as a plain 2:4 operand over all F columns
+  void* vn_relu24;          // bf16 [T, F/2]  ReLU(y1) in that layout
+  void* vn_meta24;          // uint16 [T, F/16] canonical metadata of that operand
+  void* vn_meta24_hw;       // the same words in tensor-core order
+  void* vn_y1;              // optional bf16 [T, F]: the pre-activation itself
+};
+
+// Outputs of the fused y1 product (see GemmArgs::vn_*).
+struct Vnm8Out {
+  void *vals, *relu, *meta, *colidx, *vals24, *relu24, *meta24, *meta24_hw, *y1;
 };
 
 // D[M,N] = op(A) op(B)^T, tiles 128 x 256, K % 64 == 0.
 int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64_t M, int64_t N, int64_t K, int epi,
                void* C, int64_t ldc, void* C2, int64_t ldc2, const void* aux, int64_t ldaux, int* status,
                cudaStream_t s);
+// The weight-gradient products with one operand given packed: D[M,N] = A^T B with A [K, M] and B [K, N]
+// row-major (reduction over the rows), where operand `packed_operand` (1 = A, 2 = B) is not read as a
+// dense matrix but expanded on the fly from its 2:4 layout: values [K, X/2] + canonical metadata
+// [K, X/16] (X = M or N). M % 256 == 0, N % 256 == 0, K % 64 == 0.
+int gemm_dense_expand(const void* dense_op, int packed_operand, const void* pk_vals, const void* pk_meta, int64_t M,
+                      int64_t N, int64_t K, void* C, int64_t ldc, int* status, cudaStream_t s);
+// y1 product with the activation sparsified in the epilogue: W1s [F, D] 2:4-packed times X [T, D];
+// F % 256 == 0, D % 128 == 0, T % V == 0, V in {64, 128}. Nothing of y1 is written unless out.y1 is set.
+int gemm_sparse24_vnm8(const void* a_vals, const uint8_t* meta_hw, const void* X, int64_t F, int64_t T, int64_t D,
+                       int V, const Vnm8Out& out, int* status, cudaStream_t s);
+bool gemm_sparse24_vnm8_supported(int64_t F, int64_t T, int64_t D, int V);
 // A_s[M,K] 2:4-packed times B (b_kmajor: [N,K] row-major, else [K,N] row-major).
 // epi EPI_STORE_T / EPI_DRELU_T: transposed output Ct[N,M] (b_kmajor only); EPI_STORE: C[M,N]
 // (two-CTA kernel, M % 256 == 0).

@@ -57,21 +57,24 @@ int sf_end_to_end_speedup(double ffn_fraction, double ffn_speedup, double* speed
 }
 
 int sf_ffn_fwd_scheduled(const sf_schedule* schedule, int64_t step, const sf_ffn_desc* desc, const void* X,
-                         const void* W1, const void* W2, void* Y, void* fwd_ctx, void* workspace, void* stream) {
-  int kind = SF_STEP_DENSE;
-  SF_TRY(sf_schedule_step_kind(schedule, step, &kind));
-  return kind == SF_STEP_SPARSE ? sf_sparse_ffn_fwd(desc, X, W1, W2, Y, fwd_ctx, workspace, stream)
-                                : sf_dense_ffn_fwd(desc, X, W1, W2, Y, fwd_ctx, workspace, stream);
-}
-
-int sf_ffn_bwd_scheduled(const sf_schedule* schedule, int64_t step, const sf_ffn_desc* desc, const void* dY,
-                         const void* X, const void* W1, const void* W2, const void* fwd_ctx, void* dX, void* dW1,
-                         void* dW2, void* workspace, void* stream) {
+                         const void* W1, const void* W2, void* Y, void* fwd_ctx, size_t fwd_ctx_bytes, void* workspace,
+                         size_t workspace_bytes, void* stream) {
   int kind = SF_STEP_DENSE;
   SF_TRY(sf_schedule_step_kind(schedule, step, &kind));
   return kind == SF_STEP_SPARSE
-             ? sf_sparse_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stream)
-             : sf_dense_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stream);
+             ? sf_sparse_ffn_fwd(desc, X, W1, W2, Y, fwd_ctx, fwd_ctx_bytes, workspace, workspace_bytes, stream)
+             : sf_dense_ffn_fwd(desc, X, W1, W2, Y, fwd_ctx, fwd_ctx_bytes, workspace, workspace_bytes, stream);
+}
+
+int sf_ffn_bwd_scheduled(const sf_schedule* schedule, int64_t step, const sf_ffn_desc* desc, const void* dY,
+                         const void* X, const void* W1, const void* W2, const void* fwd_ctx, size_t fwd_ctx_bytes,
+                         void* dX, void* dW1, void* dW2, void* workspace, size_t workspace_bytes, void* stream) {
+  int kind = SF_STEP_DENSE;
+  SF_TRY(sf_schedule_step_kind(schedule, step, &kind));
+  return kind == SF_STEP_SPARSE ? sf_sparse_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, fwd_ctx_bytes, dX, dW1, dW2, workspace,
+                                                    workspace_bytes, stream)
+                                : sf_dense_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, fwd_ctx_bytes, dX, dW1, dW2, workspace,
+                                                   workspace_bytes, stream);
 }
 
 }  // extern "C"

@@ -93,7 +93,7 @@ int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int gr
                    void* vals, void* meta, void* meta_hw, void* dense_out, cudaStream_t s);
 int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
                void* vals, void* meta, void* meta_hw, void* colidx, void* relu_vals, void* dense_out,
-               void* relu_dense_out, void* vals24, void* meta24, void* meta24_hw, cudaStream_t s);
+               void* relu_dense_out, void* vals24, void* meta24, void* meta24_hw, void* relu24, cudaStream_t s);
 bool vnm_has_24_view(int64_t F, int V, int M);
 int launch_transpose(const void* in, void* out, int64_t rows, int64_t cols, cudaStream_t s);
 

@@ -9,6 +9,7 @@
 //           two matching ReLU values, one metadata nibble (four neighbours form a uint16).
 // The accumulation order of pass A is part of the format: it is what makes the mask unique.
 #include "sf_common.cuh"
+#include "sparse_fmt.cuh"
 
 namespace sf {
 
@@ -47,16 +48,8 @@ __device__ __forceinline__ void write_group_dense(uint16_t* drow, int M, uint32_
   }
 }
 
-__device__ __forceinline__ uint32_t relu2(uint32_t w) {
-  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&w);
-  __nv_bfloat162 z = __hmax2(x, __float2bfloat162_rn(0.f));
-  return *reinterpret_cast<uint32_t*>(&z);
-}
-__device__ __forceinline__ uint32_t sq2(uint32_t r) {
-  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&r);
-  __nv_bfloat162 z = __hmul2(x, x);
-  return *reinterpret_cast<uint32_t*>(&z);
-}
+__device__ __forceinline__ uint32_t relu2(uint32_t w) { return bf2_relu(w); }
+__device__ __forceinline__ uint32_t sq2(uint32_t r) { return bf2_sq(r); }
 
 // kW: strip width in columns (128 for M <= 32: half the shared memory, twice the resident CTAs; 256 for M = 64).
 template <int kW>
@@ -273,7 +266,7 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
             uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
             uint8_t* __restrict__ colidx, uint16_t* __restrict__ relu_vals, uint16_t* __restrict__ dense_out,
             uint16_t* __restrict__ relu_dense_out, uint16_t* __restrict__ vals24, uint16_t* __restrict__ meta24,
-            uint8_t* __restrict__ meta24_hw) {
+            uint8_t* __restrict__ meta24_hw, uint16_t* __restrict__ relu24) {
   constexpr int M = 8;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   uint16_t* tile = reinterpret_cast<uint16_t*>(smem_raw);                        // [V][kW + kPad]
@@ -362,25 +355,12 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
     const int pi = pe < 3 ? 0 : (pe < 5 ? 1 : 2), pj = pe < 3 ? pe + 1 : (pe < 5 ? pe - 1 : 3);
     const uint32_t ca = cidx[ge * 4 + pi], cb = cidx[ge * 4 + pj];                // kept columns, ca < cb
     const uint32_t nibp = (uint32_t)pi | ((uint32_t)pj << 2);
-    uint32_t sd[4];
-#pragma unroll
-    for (uint32_t j = 0; j < 4; ++j) {
-      const uint32_t lo = ca == 2 * j ? 0x10u : (cb == 2 * j ? 0x32u : 0x44u);
-      const uint32_t hi = ca == 2 * j + 1 ? 0x10u : (cb == 2 * j + 1 ? 0x32u : 0x44u);
-      sd[j] = lo | (hi << 8);
-    }
-    const uint32_t pa = ca & 3u, pb = cb & 3u;
-    const uint32_t s1 = (2u * pa) | ((2u * pa + 1u) << 4) | ((2u * pb) << 8) | ((2u * pb + 1u) << 12);
-    const uint32_t s2 = (ca < 4u ? 0x10u : 0x54u) | ((cb < 4u ? 0x32u : 0x76u) << 8);
-    const bool both_lo = cb < 4u, both_hi = ca >= 4u;
-    const uint32_t s_wlo = both_lo ? 0x3210u : (both_hi ? 0x4444u : (pa == 0u ? 0x4410u : 0x1044u));
-    const uint32_t s_whi = both_hi ? 0x3210u : (both_lo ? 0x4444u : (pb == 0u ? 0x4432u : 0x3244u));
-    const uint32_t pair_nib = pa | (pb << 2);
-    const uint32_t nlo = both_lo ? pair_nib : (both_hi ? 4u : (pa == 0u ? 4u : (pa << 2)));
-    const uint32_t nhi = both_hi ? pair_nib : (both_lo ? 4u : (pb == 0u ? 4u : (pb << 2)));
+    uint4 selv;
+    uint32_t nib24;
+    vnm8_pair_selectors(ca, cb, selv, nib24);
     const int slot = ge * 7 + (int)(nibp % 7u);
-    sel_tab[slot] = make_uint4(sd[0] | (sd[1] << 16), sd[2] | (sd[3] << 16), s1 | (s2 << 16), s_wlo | (s_whi << 16));
-    nib_tab[slot] = (uint8_t)(nlo | (nhi << 4));
+    sel_tab[slot] = selv;
+    nib_tab[slot] = (uint8_t)nib24;
   }
   __syncthreads();
 
@@ -400,7 +380,7 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
   }
   const bool lead4 = (g & 3) == 0, lead2 = (g & 1) == 0;
   const bool want_relu = relu_vals && apply, want24 = vals24 != nullptr;
-  const bool need_relu_pair = want_relu || (relu_dense_out != nullptr);
+  const bool need_relu_pair = want_relu || (relu_dense_out != nullptr) || (relu24 != nullptr && apply);
   const int64_t trow = t0 + r0;
   const uint16_t* tp = tile + r0 * kRow + g * M;
   const uint4* my_sel = sel_tab + g * 7;
@@ -410,6 +390,7 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
   uint16_t* p_dense = dense_out ? dense_out + trow * F + c0 + g * M : nullptr;
   uint16_t* p_rdense = relu_dense_out ? relu_dense_out + trow * F + c0 + g * M : nullptr;
   uint16_t* p_v24 = want24 ? vals24 + trow * (F >> 1) + (g0 + g) * 4 : nullptr;
+  uint16_t* p_r24 = (want24 && relu24 && apply) ? relu24 + trow * (F >> 1) + (g0 + g) * 4 : nullptr;
   uint16_t* p_meta = meta + trow * (G >> 2) + ((g0 + g) >> 2);
   uint16_t* p_m24 = want24 ? meta24 + trow * (F >> 4) + ((g0 + g) >> 1) : nullptr;
   // tensor-core-ordered copies: rows of one strip share their 128-row block, so the atom is fixed
@@ -443,6 +424,11 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
       const uint32_t x = __byte_perm(rw[0], rw[1], sel.z), y = __byte_perm(rw[2], rw[3], sel.z);
       const uint32_t rpair = __byte_perm(x, y, sel.z >> 16);
       if (want_relu) *reinterpret_cast<uint32_t*>(p_relu) = rpair;
+      if (p_r24) {
+        // ReLU(y1) in the layout of the 2:4 view (what the dy1 epilogue multiplies by)
+        *reinterpret_cast<uint2*>(p_r24) = make_uint2(__byte_perm(rpair, 0u, sel.w), __byte_perm(rpair, 0u, sel.w >> 16));
+        p_r24 += s_v24;
+      }
       if (relu_dense_out)
         *reinterpret_cast<uint4*>(p_rdense) = make_uint4(__byte_perm(rpair, 0u, sel.x), __byte_perm(rpair, 0u, sel.x >> 16),
                                                          __byte_perm(rpair, 0u, sel.y), __byte_perm(rpair, 0u, sel.y >> 16));
@@ -488,7 +474,7 @@ vnm8_kernel(const uint16_t* __restrict__ P, int64_t T, int64_t F, int64_t ld, in
 
 int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
                void* vals, void* meta, void* meta_hw, void* colidx, void* relu_vals, void* dense_out,
-               void* relu_dense_out, void* vals24, void* meta24, void* meta24_hw, cudaStream_t s) {
+               void* relu_dense_out, void* vals24, void* meta24, void* meta24_hw, void* relu24, cudaStream_t s) {
   if (T == 0 || F == 0) return SF_OK;
   const size_t smem = (size_t)V * (kCW + kPad) * 2 + kCW * 4 + kCW + kCW;
   static bool attr_set[64] = {false};                         // per device
@@ -521,7 +507,7 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
                                                     (uint16_t*)meta, (uint8_t*)meta_hw, (uint8_t*)colidx,
                                                     (uint16_t*)relu_vals, (uint16_t*)dense_out,
                                                     (uint16_t*)relu_dense_out, (uint16_t*)vals24, (uint16_t*)meta24,
-                                                    (uint8_t*)meta24_hw);
+                                                    (uint8_t*)meta24_hw, (uint16_t*)relu24);
     SF_LAUNCH_CHECK();
     return SF_OK;
   }

@@ -30,6 +30,8 @@ __all__ = [
 FFN_CONFIGS = {
     "c1_small": dict(T=1024, D=256, F=1024, V=64, N=2, M=8, sigma_w=0.02, seed=0),
     "c4_d4096": dict(T=8192, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
+    # the same layer with the block height of the paper's Table 5 (V = 64)
+    "c4_d4096_v64": dict(T=8192, D=4096, F=16384, V=64, N=2, M=8, sigma_w=0.02, seed=4),
     # one eighth of c4's tokens with the full-size layer: weights (134 MB each) still exceed the
     # L2, device footprint ~1.5 GB; used for profiler captures that must stay small
     "c4_slice": dict(T=1024, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),

@@ -88,4 +88,42 @@ def test_schedule_rejects_bad_arguments(lib):
     assert lib.sf_end_to_end_speedup(1.5, 2.0, C.byref(out)) == binding.SF_ERR_SHAPE
     assert lib.sf_ffn_flop_fraction(0, 8, 1, 1, 1, C.byref(out)) == binding.SF_ERR_SHAPE
     # a step outside the schedule is rejected before any pointer is looked at
-    assert lib.sf_ffn_fwd_scheduled(C.byref(sc), 99, None, None, None, None, None, None, None, None) == binding.SF_ERR_SHAPE
+    assert lib.sf_ffn_fwd_scheduled(C.byref(sc), 99, None, None, None, None, None, None, 0, None, 0, None) == binding.SF_ERR_SHAPE
+
+
+def test_step_calls_reject_short_buffers_before_launching(lib):
+    """Every step call is told how large its context and workspace are and refuses, on the host,
+    buffers smaller than sf_ffn_workspace_size reports (no device is touched: the pointers are fake)."""
+    desc = binding.make_desc(1024, 256, 1024, 64, 8)
+    need_ctx, need_ws = binding.sf_ffn_workspace_size(desc)
+    assert need_ctx > 0 and need_ws > 256
+    ok = C.c_void_p(0x10000)
+    d = C.byref(desc)
+    W = binding.SF_ERR_WORKSPACE
+    # (the size query reports the larger of the sparse and the dense step's needs, so "short" here
+    # means well below either)
+    assert lib.sf_sparse_ffn_fwd(d, ok, ok, ok, ok, ok, need_ctx // 2, ok, need_ws, None) == W
+    assert lib.sf_sparse_ffn_fwd(d, ok, ok, ok, ok, ok, need_ctx, ok, need_ws // 2, None) == W
+    assert lib.sf_sparse_ffn_bwd(d, ok, ok, ok, ok, ok, need_ctx, ok, ok, ok, ok, 0, None) == W
+    assert lib.sf_dense_ffn_fwd(d, ok, ok, ok, ok, ok, 16, ok, need_ws, None) == W
+    assert lib.sf_dense_ffn_bwd(d, ok, ok, ok, ok, ok, need_ctx, ok, ok, ok, ok, 255, None) == W
+    assert lib.sf_ffn_step_host(d, 0, ok, ok, ok, ok, ok, ok, ok, ok, ok, ok, need_ctx // 2, ok, need_ws, None) == W
+    sc = binding.make_schedule(0, 1, 2)
+    assert lib.sf_ffn_fwd_scheduled(C.byref(sc), 0, d, ok, ok, ok, ok, ok, need_ctx, ok, need_ws // 2, None) == W
+    # NULL and alignment still come first
+    assert lib.sf_sparse_ffn_fwd(d, None, ok, ok, ok, ok, need_ctx, ok, need_ws, None) == binding.SF_ERR_NULL
+    # unknown flag bits are refused
+    bad = binding.make_desc(1024, 256, 1024, 64, 8, flags=8)
+    a, b = C.c_size_t(), C.c_size_t()
+    assert lib.sf_ffn_workspace_size(C.byref(bad), C.byref(a), C.byref(b)) == binding.SF_ERR_UNSUPPORTED
+
+
+def test_context_shrinks_without_masked_dense_copies(lib):
+    """M = 8 keeps the activation in packed forms only: the context of the d_model = 4096 layer with
+    8192 tokens must stay below 0.6 GB (three masked [T, F] copies alone would be 0.8 GB)."""
+    desc = binding.make_desc(8192, 4096, 16384, 128, 8)
+    ctx, ws = binding.sf_ffn_workspace_size(desc)
+    # the query reports the larger of the sparse and dense needs; the dense step keeps y1 and h: 2 x 268 MB
+    dense_ctx = 2 * 8192 * 16384 * 2
+    assert ctx == max(ctx, dense_ctx)
+    assert ctx < 0.6e9

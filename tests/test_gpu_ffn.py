@@ -11,34 +11,86 @@ import torch
 
 import oracle
 from paper_2602_06183_b200 import binding, synth
-from util import to_dev, bits, f32, rel_fro
+from util import to_dev, bits, f32, rel_fro, assert_close_elementwise, Guarded
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-2
 
 
-def _run_sparse(cfg, prune_mode=0, act_shift=0.0):
+def _run_sparse(cfg, prune_mode=0, act_shift=0.0, flags=binding.SF_FFN_SAVE_Y1):
+    """One sparse step through the C ABI. Context, workspace and every output sit between guard
+    zones that are checked after the step (nothing may be written outside a buffer)."""
     T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
     X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"], act_shift=act_shift)
-    desc = binding.make_desc(T, D, F, V, M, prune_mode=prune_mode, flags=1)
-    ctx, ws = binding.alloc_ffn_buffers(desc)
+    desc = binding.make_desc(T, D, F, V, M, prune_mode=prune_mode, flags=flags)
+    nctx, nws = binding.sf_ffn_workspace_size(desc)
+    gctx, gws = Guarded(nctx, zero=True), Guarded(nws, zero=True)
+    ctx, ws = gctx.t, gws.t
     dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
-    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
-    gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
+    gY, ggX = Guarded((T, D), torch.bfloat16), Guarded((T, D), torch.bfloat16)
+    ggW1, ggW2 = Guarded((F, D), torch.bfloat16), Guarded((D, F), torch.bfloat16)
+    Y, gX, gW1, gW2 = gY.t, ggX.t, ggW1.t, ggW2.t
     binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
     assert binding.sf_check_status(ws) == binding.SF_OK
     binding.sf_sparse_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
     assert binding.sf_check_status(ws) == binding.SF_OK
+    for g, name in ((gctx, "context"), (gws, "workspace"), (gY, "Y"), (ggX, "dX"), (ggW1, "dW1"), (ggW2, "dW2")):
+        g.check(name)
     G = F // M
+    view = lambda buf, field: binding.sf_ctx_view(desc, buf, field)
     out = dict(
-        y1=bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y1)).reshape(T, F),
-        y2_vals=bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y2_VALS)).reshape(T, 2 * G),
-        relu_vals=bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_RELU_VALS)).reshape(T, 2 * G),
-        meta=bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_META)).reshape(T, G // 4),
-        colidx=binding.sf_ctx_view(desc, ctx, binding.SF_CTX_COLIDX).cpu().numpy().reshape(T // V, G, 4),
-        dy1_vals=bits(binding.sf_ctx_view(desc, ws, binding.SF_CTX_DY1_VALS)).reshape(T, 2 * G),
+        y2_vals=bits(view(ctx, binding.SF_CTX_Y2_VALS)).reshape(T, 2 * G),
+        relu_vals=bits(view(ctx, binding.SF_CTX_RELU_VALS)).reshape(T, 2 * G),
+        meta=bits(view(ctx, binding.SF_CTX_META)).reshape(T, G // 4),
+        colidx=view(ctx, binding.SF_CTX_COLIDX).cpu().numpy().reshape(T // V, G, 4),
         Y=f32(Y), dX=f32(gX), dW1=f32(gW1), dW2=f32(gW2))
+    if flags & binding.SF_FFN_SAVE_Y1:
+        out["y1"] = bits(view(ctx, binding.SF_CTX_Y1)).reshape(T, F)
+    if M == 8:
+        # the activation and dy1 live in their 2:4 layout over all F columns
+        m24 = bits(view(ctx, binding.SF_CTX_Y2_META24)).reshape(T, F // 16)
+        out["meta24"] = m24
+        out["vals24"] = bits(view(ctx, binding.SF_CTX_Y2_VALS24)).reshape(T, F // 2)
+        out["relu24"] = bits(view(ctx, binding.SF_CTX_RELU_VALS24)).reshape(T, F // 2)
+        out["dy1_dense"] = oracle.decompress24(bits(view(ws, binding.SF_CTX_DY1_VALS24)).reshape(T, F // 2), m24)
+    else:
+        dy1_vals = bits(view(ws, binding.SF_CTX_DY1_VALS)).reshape(T, 2 * G)
+        out["dy1_dense"] = oracle.decompress_vnm(dy1_vals, out["meta"], out["colidx"], V=V, M=M)
     return (X, W1, W2, dY), out
+
+
+def _check_against_oracle(inputs, g, cfg, prune_mode=0):
+    """Stage-wise, teacher-forced comparison of one step with the oracle (needs the saved y1)."""
+    X, W1, W2, dY = inputs
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, prune_mode=prune_mode, forced_y1b=g["y1"])
+    assert np.array_equal(g["colidx"], fwd.act.colidx)
+    assert np.array_equal(g["meta"], fwd.act.meta)
+    assert np.array_equal(g["y2_vals"], fwd.act.vals)
+    assert np.array_equal(g["relu_vals"], fwd.act.relu_vals)
+    if M == 8:
+        nib = np.stack([(g["meta24"] >> np.uint16(4 * i)) & np.uint16(0xF) for i in range(4)], axis=-1)
+        assert ((nib & 3) < (nib >> 2)).all()                    # legal position pairs everywhere
+        assert np.array_equal(oracle.decompress24(g["vals24"], g["meta24"]), fwd.act.dense)
+        relu_dense = np.where(fwd.act.mask, oracle.vnm.squared_relu_bf16(g["y1"])[1], np.uint16(0))
+        assert np.array_equal(oracle.decompress24(g["relu24"], g["meta24"]), relu_dense)
+    assert rel_fro(g["Y"], fwd.y3) < TOL
+    assert_close_elementwise(g["Y"], fwd.y3, F, "Y")
+    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd, prune_mode=prune_mode)
+    assert not (g["dy1_dense"][~fwd.act.mask] != 0).any()        # nothing outside y2's mask
+    assert rel_fro(oracle.bf16_to_f32(g["dy1_dense"]), oracle.bf16_to_f32(bwd.dy1_dense)) < TOL
+    assert_close_elementwise(oracle.bf16_to_f32(g["dy1_dense"]), oracle.bf16_to_f32(bwd.dy1_dense), D, "dy1")
+    # The remaining products are compared with the oracle evaluated on the GPU's own dy1 (a one-ulp
+    # difference in dy1 is legitimate and would otherwise be charged to dX and dW1 as well).
+    dy1m = oracle.bf16_to_f32(g["dy1_dense"]).astype(np.float64)
+    refs = dict(dX=dy1m @ oracle.bf16_to_f32(W1).astype(np.float64),
+                dW1=dy1m.T @ oracle.bf16_to_f32(X).astype(np.float64), dW2=bwd.dW2)
+    for k, Kred in (("dX", F), ("dW1", T), ("dW2", T)):
+        assert rel_fro(g[k], refs[k]) < TOL, k
+        assert_close_elementwise(g[k], refs[k], Kred, k)
+    for k, ref in (("dX", bwd.dX), ("dW1", bwd.dW1)):
+        assert rel_fro(g[k], ref) < TOL, k
+    return fwd, bwd
 
 
 @pytest.mark.parametrize("prune_mode,act_shift", [(0, 0.0), (1, 0.0), (0, -1.3)])
@@ -49,96 +101,79 @@ def test_sparse_ffn_c1_teacher_forced(prune_mode, act_shift):
     # stage 1: the GPU's y1 against the oracle's own product with the pruned W1
     free = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, prune_mode=prune_mode)
     assert rel_fro(oracle.bf16_to_f32(g["y1"]), oracle.bf16_to_f32(free.y1b)) < TOL
-    # stage 2: selection on the GPU's y1 must agree bit for bit
-    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, prune_mode=prune_mode, forced_y1b=g["y1"])
-    assert np.array_equal(g["colidx"], fwd.act.colidx)
-    assert np.array_equal(g["meta"], fwd.act.meta)
-    assert np.array_equal(g["y2_vals"], fwd.act.vals)
-    assert np.array_equal(g["relu_vals"], fwd.act.relu_vals)
-    # stage 3: products with those masks
-    assert rel_fro(g["Y"], fwd.y3) < TOL
-    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd, prune_mode=prune_mode)
-    assert rel_fro(oracle.bf16_to_f32(g["dy1_vals"]), oracle.bf16_to_f32(bwd.dy1_vals)) < TOL
-    assert rel_fro(g["dX"], bwd.dX) < TOL
-    assert rel_fro(g["dW1"], bwd.dW1) < TOL
-    assert rel_fro(g["dW2"], bwd.dW2) < TOL
+    assert_close_elementwise(oracle.bf16_to_f32(g["y1"]), oracle.bf16_to_f32(free.y1b), cfg["D"], "y1")
+    # stages 2 and 3: selection on the GPU's y1 bit for bit, products with those masks
+    _check_against_oracle((X, W1, W2, dY), g, cfg, prune_mode)
     # free-running comparison: masks may differ in a few near-tie blocks only
     disagree = float((free.act.colidx != g["colidx"]).any(axis=-1).mean())
     assert disagree < 0.05
     assert rel_fro(g["Y"], free.y3) < 5e-2
 
 
-@pytest.mark.parametrize("M,act_shift", [(8, 0.0), (8, -1.3), (4, 0.0)])
-def test_plain_24_view_of_y2_and_dy1_is_exact(M, act_shift):
-    """For M <= 8 the products consume y2 / dy1 as plain 2:4 operands over all F columns. That view,
-    decompressed with its own metadata, must be the oracle's masked dense y2 bit for bit, hold at
-    most two entries per four columns with ascending positions, and dy1's view must be the masked
-    dense dy1 at the same positions."""
-    cfg = dict(synth.FFN_CONFIGS["c1_small"], M=M)
-    T, D, F, V = cfg["T"], cfg["D"], cfg["F"], cfg["V"]
-    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"], act_shift=act_shift)
-    desc = binding.make_desc(T, D, F, V, M, flags=1)
-    ctx, ws = binding.alloc_ffn_buffers(desc)
-    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
-    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
-    gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
-    binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
-    binding.sf_sparse_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
-    assert binding.sf_check_status(ws) == binding.SF_OK
-    y1 = bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y1)).reshape(T, F)
-    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, forced_y1b=y1)
-    v24 = bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y2_VALS24)).reshape(T, F // 2)
-    m24 = bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y2_META24)).reshape(T, F // 16)
-    nib = np.stack([(m24 >> np.uint16(4 * i)) & np.uint16(0xF) for i in range(4)], axis=-1)
-    assert ((nib & 3) < (nib >> 2)).all()                        # legal position pairs everywhere
-    assert np.array_equal(oracle.decompress24(v24, m24), fwd.act.dense)
-    # dy1 in the same positions: compare with the masked dense dy1 the oracle derives from the GPU's masks
-    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd)
-    d24 = bits(binding.sf_ctx_view(desc, ws, binding.SF_CTX_DY1_VALS24)).reshape(T, F // 2)
-    dy1_gpu = oracle.decompress24(d24, m24)
-    dy1_ref = oracle.decompress_vnm(bwd.dy1_vals, fwd.act.meta, fwd.act.colidx, V=V, M=M)
-    assert not (dy1_gpu[~fwd.act.mask] != 0).any()               # nothing outside y2's mask
-    assert rel_fro(oracle.bf16_to_f32(dy1_gpu), oracle.bf16_to_f32(dy1_ref)) < TOL
+@pytest.mark.parametrize("cfg", [
+    dict(T=1024, D=256, F=1024, V=64, N=2, M=8, sigma_w=0.02, seed=0),      # fused epilogue, three 64-token blocks per tile
+    dict(T=512, D=256, F=512, V=128, N=2, M=8, sigma_w=0.05, seed=3),       # fused epilogue, one 128-token block per tile
+    dict(T=512, D=256, F=2048, V=128, N=2, M=16, sigma_w=0.05, seed=17),    # condensed Venom products
+], ids=["m8_v64", "m8_v128", "m16_v128"])
+def test_step_without_saved_y1_is_the_same_step(cfg):
+    """The benchmarked configuration keeps no y1 (flags = 0), which moves buffers inside the context and
+    the workspace. Everything it produces must equal, bit for bit, the teacher-forced run that saves
+    y1 and is checked against the oracle; what the context exposes is compared with the oracle too."""
+    inputs, g1 = _run_sparse(cfg, flags=binding.SF_FFN_SAVE_Y1)
+    fwd, _ = _check_against_oracle(inputs, g1, cfg)
+    _, g0 = _run_sparse(cfg, flags=0)
+    assert "y1" not in g0
+    for k in g0:
+        assert np.array_equal(g0[k], g1[k]), k
+    assert np.array_equal(g0["colidx"], fwd.act.colidx) and np.array_equal(g0["y2_vals"], fwd.act.vals)
 
 
-def test_sparse_ffn_v128_m16():
-    cfg = dict(T=512, D=256, F=2048, V=128, N=2, M=16, sigma_w=0.05, seed=17)
-    (X, W1, W2, dY), g = _run_sparse(cfg)
-    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=128, M=16, forced_y1b=g["y1"])
-    assert np.array_equal(g["colidx"], fwd.act.colidx) and np.array_equal(g["meta"], fwd.act.meta)
-    assert np.array_equal(g["y2_vals"], fwd.act.vals)
-    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd)
-    for k, ref in (("Y", fwd.y3), ("dX", bwd.dX), ("dW1", bwd.dW1), ("dW2", bwd.dW2)):
-        assert rel_fro(g[k], ref) < TOL, k
+@pytest.mark.parametrize("V,act_shift", [(64, 0.0), (128, 0.0), (64, -1.3)])
+def test_fused_activation_epilogue_equals_the_two_kernel_path(V, act_shift):
+    """SquaredReLU + V:N:M inside the y1 product's epilogue against the stand-alone kernel on a stored
+    y1: same accumulation, same selection rule, so every output must agree bit for bit. T is not a
+    multiple of the fused kernel's 192-token tile, so the last tile is ragged."""
+    cfg = dict(T=1280, D=512, F=768, V=V, N=2, M=8, sigma_w=0.05, seed=41)
+    inputs, fused = _run_sparse(cfg, act_shift=act_shift, flags=binding.SF_FFN_SAVE_Y1)
+    _, two = _run_sparse(cfg, act_shift=act_shift, flags=binding.SF_FFN_SAVE_Y1 | binding.SF_FFN_UNFUSED_ACT)
+    for k in fused:
+        assert np.array_equal(fused[k], two[k]), k
+    _check_against_oracle(inputs, fused, cfg)
 
 
-@pytest.mark.parametrize("V,M", [(64, 4), (128, 32)])
-def test_sparse_ffn_other_group_widths(V, M):
-    """M = 4 is 2:4 activation sparsity (every column kept, the plain-2:4 path); M = 32 runs the
-    condensed, gathered Venom product."""
-    cfg = dict(T=512, D=256, F=2048, V=V, N=2, M=M, sigma_w=0.05, seed=23 + M)
-    (X, W1, W2, dY), g = _run_sparse(cfg)
-    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, forced_y1b=g["y1"])
-    assert np.array_equal(g["colidx"], fwd.act.colidx) and np.array_equal(g["meta"], fwd.act.meta)
-    assert np.array_equal(g["y2_vals"], fwd.act.vals)
-    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd)
-    for k, ref in (("Y", fwd.y3), ("dX", bwd.dX), ("dW1", bwd.dW1), ("dW2", bwd.dW2)):
-        assert rel_fro(g[k], ref) < TOL, k
+def test_plain_24_view_of_m4_activations_is_exact():
+    """M = 4 is 2:4 activation sparsity: the packed V:N:M form is itself the 2:4 operand the products
+    consume. Decompressed with its own metadata it must be the oracle's masked dense y2 bit for bit,
+    and dy1 packed by the dy1 product's epilogue must sit at the same positions."""
+    cfg = dict(synth.FFN_CONFIGS["c1_small"], M=4)
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], 4
+    inputs, g = _run_sparse(cfg)
+    fwd, bwd = _check_against_oracle(inputs, g, cfg)
+    desc = binding.make_desc(T, D, F, V, M, flags=binding.SF_FFN_SAVE_Y1)
+    assert np.all(g["colidx"] == np.arange(4))
+    assert np.array_equal(oracle.decompress24(g["y2_vals"], g["meta"]), fwd.act.dense)
+
+
+@pytest.mark.parametrize("cfg", [
+    dict(T=512, D=256, F=2048, V=128, N=2, M=16, sigma_w=0.05, seed=17),
+    dict(T=512, D=256, F=2048, V=64, N=2, M=4, sigma_w=0.05, seed=27),      # 2:4 activation sparsity
+    dict(T=512, D=256, F=2048, V=128, N=2, M=32, sigma_w=0.05, seed=55),    # condensed, gathered Venom product
+    dict(T=256, D=256, F=4096, V=128, N=2, M=64, sigma_w=0.05, seed=87),    # Table 5's widest group
+    dict(T=256, D=256, F=2048, V=64, N=2, M=64, sigma_w=0.05, seed=88),
+], ids=["m16", "m4", "m32", "m64_v128", "m64_v64"])
+def test_sparse_ffn_other_group_widths(cfg):
+    inputs, g = _run_sparse(cfg)
+    _check_against_oracle(inputs, g, cfg)
 
 
 @pytest.mark.parametrize("T,D,F,V,M", [(256, 256, 256, 128, 8), (256, 256, 256, 64, 8), (512, 512, 512, 128, 16),
-                                       (768, 256, 1280, 128, 8)])
+                                       (768, 256, 1280, 128, 8), (768, 256, 1280, 64, 8)])
 def test_sparse_ffn_smallest_and_odd_tile_counts(T, D, F, V, M):
     """One tile per product, fewer k-blocks than pipeline stages, tile counts that are not a
     multiple of the raster band."""
     cfg = dict(T=T, D=D, F=F, V=V, N=2, M=M, sigma_w=0.05, seed=T + F + V)
-    (X, W1, W2, dY), g = _run_sparse(cfg)
-    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, forced_y1b=g["y1"])
-    assert np.array_equal(g["colidx"], fwd.act.colidx) and np.array_equal(g["meta"], fwd.act.meta)
-    assert np.array_equal(g["y2_vals"], fwd.act.vals)
-    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd)
-    for k, ref in (("Y", fwd.y3), ("dX", bwd.dX), ("dW1", bwd.dW1), ("dW2", bwd.dW2)):
-        assert rel_fro(g[k], ref) < TOL, k
+    inputs, g = _run_sparse(cfg)
+    _check_against_oracle(inputs, g, cfg)
 
 
 def test_dense_ffn_c1():
@@ -312,10 +347,5 @@ def _legal_random_configs(n, seed):
 @pytest.mark.parametrize("T,D,F,V,M,prune_mode,act_shift,seed", _legal_random_configs(10, seed=20260206))
 def test_sparse_ffn_random_legal_shapes(T, D, F, V, M, prune_mode, act_shift, seed):
     cfg = dict(T=T, D=D, F=F, V=V, N=2, M=M, sigma_w=0.05, seed=seed)
-    (X, W1, W2, dY), g = _run_sparse(cfg, prune_mode, act_shift)
-    fwd = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M, prune_mode=prune_mode, forced_y1b=g["y1"])
-    assert np.array_equal(g["colidx"], fwd.act.colidx) and np.array_equal(g["meta"], fwd.act.meta)
-    assert np.array_equal(g["y2_vals"], fwd.act.vals) and np.array_equal(g["relu_vals"], fwd.act.relu_vals)
-    bwd = oracle.sparse_ffn_bwd(dY, X, W1, W2, fwd, prune_mode=prune_mode)
-    for k, ref in (("Y", fwd.y3), ("dX", bwd.dX), ("dW1", bwd.dW1), ("dW2", bwd.dW2)):
-        assert rel_fro(g[k], ref) < TOL, k
+    inputs, g = _run_sparse(cfg, prune_mode, act_shift)
+    _check_against_oracle(inputs, g, cfg, prune_mode)

@@ -12,33 +12,42 @@ import torch
 
 import oracle
 from paper_2602_06183_b200 import binding, synth
-from util import to_dev, bits, f32, rel_fro
+from util import to_dev, bits, f32, rel_fro, assert_close_elementwise, Guarded
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-2
 
 
-@pytest.mark.parametrize("name", ["c4_d4096", "c4_d4096_m16", "c5_d8192"])
+def _full_step(cfg, flags):
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
+    desc = binding.make_desc(T, D, F, V, M, flags=flags)
+    nctx, nws = binding.sf_ffn_workspace_size(desc)
+    gctx, gws = Guarded(nctx, zero=True), Guarded(nws, zero=True)
+    dX_, dW1_, dW2_, ddY = (to_dev(a) for a in (X, W1, W2, dY))
+    outs = [Guarded((T, D), torch.bfloat16), Guarded((T, D), torch.bfloat16), Guarded((F, D), torch.bfloat16),
+            Guarded((D, F), torch.bfloat16)]
+    Y, gX, gW1, gW2 = (o.t for o in outs)
+    binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, gctx.t, gws.t)
+    binding.sf_sparse_ffn_bwd(desc, ddY, dX_, dW1_, dW2_, gctx.t, gX, gW1, gW2, gws.t)
+    assert binding.sf_check_status(gws.t) == binding.SF_OK
+    for g, nm in zip([gctx, gws] + outs, ["context", "workspace", "Y", "dX", "dW1", "dW2"]):
+        g.check(nm)
+    return (X, W1, W2, dY), desc, gctx.t, gws.t, (Y, gX, gW1, gW2)
+
+
+@pytest.mark.parametrize("name", ["c4_d4096", "c4_d4096_v64", "c4_d4096_m16", "c5_d8192"])
 def test_ffn_step_full_size_sampled(name):
     cfg = synth.FFN_CONFIGS[name]
     T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
     G = F // M
-    X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
-    desc = binding.make_desc(T, D, F, V, M, flags=1)
-    ctx, ws = binding.alloc_ffn_buffers(desc)
-    dX_, dW1_, dW2_, ddY = (to_dev(a) for a in (X, W1, W2, dY))
-    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
-    gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
-    binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
-    binding.sf_sparse_ffn_bwd(desc, ddY, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
-    assert binding.sf_check_status(ws) == binding.SF_OK
-
-    y1_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y1).view(T, F)
-    vals_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y2_VALS).view(T, 2 * G)
-    relu_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_RELU_VALS).view(T, 2 * G)
-    meta_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_META).view(T, G // 4)
-    cidx_dev = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_COLIDX).view(T // V, G, 4)
-    dy1v_dev = binding.sf_ctx_view(desc, ws, binding.SF_CTX_DY1_VALS).view(T, 2 * G)
+    (X, W1, W2, dY), desc, ctx, ws, (Y, gX, gW1, gW2) = _full_step(cfg, binding.SF_FFN_SAVE_Y1)
+    view = lambda buf, field: binding.sf_ctx_view(desc, buf, field)
+    y1_dev = view(ctx, binding.SF_CTX_Y1).view(T, F)
+    vals_dev = view(ctx, binding.SF_CTX_Y2_VALS).view(T, 2 * G)
+    relu_dev = view(ctx, binding.SF_CTX_RELU_VALS).view(T, 2 * G)
+    meta_dev = view(ctx, binding.SF_CTX_META).view(T, G // 4)
+    cidx_dev = view(ctx, binding.SF_CTX_COLIDX).view(T // V, G, 4)
 
     # ---- sample 1: two whole V-blocks of tokens (first and last), all features
     blocks = [0, T // V - 1]
@@ -47,15 +56,28 @@ def test_ffn_step_full_size_sampled(name):
     y1_rows = bits(y1_dev[rows_t])
     free = oracle.sparse_ffn_fwd(X[rows], W1, W2, V=V, M=M)
     assert rel_fro(oracle.bf16_to_f32(y1_rows), oracle.bf16_to_f32(free.y1b)) < TOL
+    assert_close_elementwise(oracle.bf16_to_f32(y1_rows), oracle.bf16_to_f32(free.y1b), D, "y1")
     fwd = oracle.sparse_ffn_fwd(X[rows], W1, W2, V=V, M=M, forced_y1b=y1_rows)
     assert np.array_equal(cidx_dev[torch.tensor(blocks).cuda()].cpu().numpy(), fwd.act.colidx)
     assert np.array_equal(bits(meta_dev[rows_t]), fwd.act.meta)
     assert np.array_equal(bits(vals_dev[rows_t]), fwd.act.vals)
     assert np.array_equal(bits(relu_dev[rows_t]), fwd.act.relu_vals)
     assert rel_fro(f32(Y[rows_t]), fwd.y3) < TOL
+    assert_close_elementwise(f32(Y[rows_t]), fwd.y3, F, "Y")
     bwd = oracle.sparse_ffn_bwd(dY[rows], X[rows], W1, W2, fwd)
-    assert rel_fro(oracle.bf16_to_f32(bits(dy1v_dev[rows_t])), oracle.bf16_to_f32(bwd.dy1_vals)) < TOL
+    if M == 8:
+        m24 = bits(view(ctx, binding.SF_CTX_Y2_META24).view(T, F // 16)[rows_t])
+        assert np.array_equal(oracle.decompress24(bits(view(ctx, binding.SF_CTX_Y2_VALS24).view(T, F // 2)[rows_t]), m24),
+                              fwd.act.dense)
+        dy1_rows = oracle.decompress24(bits(view(ws, binding.SF_CTX_DY1_VALS24).view(T, F // 2)[rows_t]), m24)
+    else:
+        dy1_rows = oracle.decompress_vnm(bits(view(ws, binding.SF_CTX_DY1_VALS).view(T, 2 * G)[rows_t]),
+                                         fwd.act.meta, fwd.act.colidx, V=V, M=M)
+    assert rel_fro(oracle.bf16_to_f32(dy1_rows), oracle.bf16_to_f32(bwd.dy1_dense)) < TOL
+    assert_close_elementwise(oracle.bf16_to_f32(dy1_rows), oracle.bf16_to_f32(bwd.dy1_dense), D, "dy1")
     assert rel_fro(f32(gX[rows_t]), bwd.dX) < TOL
+    f64 = lambda b: oracle.bf16_to_f32(b).astype(np.float64)
+    assert_close_elementwise(f32(gX[rows_t]), f64(dy1_rows) @ f64(W1), F, "dX")
 
     # ---- sample 2: four whole M-groups of features, all tokens -> columns of dW2, rows of dW1
     groups = [0, G // 3, (2 * G) // 3, G - 1]
@@ -65,9 +87,9 @@ def test_ffn_step_full_size_sampled(name):
     act = oracle.vnm_sparsify(y1_cols, V=V, M=M)
     # the GPU's masks for these groups are the oracle's on the same pre-activations
     assert np.array_equal(cidx_dev[:, torch.tensor(groups).cuda()].cpu().numpy(), act.colidx)
-    f64 = lambda b: oracle.bf16_to_f32(b).astype(np.float64)
     dW2_ref = f64(dY).T @ f64(act.dense)                                  # [D, |cols|]
     assert rel_fro(f32(gW2[:, cols_t]), dW2_ref) < TOL
+    assert_close_elementwise(f32(gW2[:, cols_t]), dW2_ref, T, "dW2")
     w2s_cols = oracle.prune24(np.ascontiguousarray(W2[:, cols]), group_dim=0).dense   # groups along D
     dy2 = (f64(dY) @ f64(w2s_cols)).astype(np.float32)
     relu = np.maximum(oracle.bf16_to_f32(y1_cols), 0)
@@ -75,6 +97,17 @@ def test_ffn_step_full_size_sampled(name):
     dy1 = np.where(act.mask, dy1, np.uint16(0))
     dW1_ref = f64(dy1).T @ f64(X)                                          # [|cols|, D]
     assert rel_fro(f32(gW1[cols_t]), dW1_ref) < TOL
+
+    # ---- the configuration the benchmark times keeps no y1: it must reproduce this run bit for bit
+    saved = [t.clone() for t in (Y, gX, gW1, gW2)]
+    saved_ctx = [view(ctx, f).clone() for f in (binding.SF_CTX_Y2_VALS, binding.SF_CTX_META, binding.SF_CTX_COLIDX)]
+    del ctx, ws, Y, gX, gW1, gW2, y1_dev, vals_dev, relu_dev, meta_dev, cidx_dev
+    torch.cuda.empty_cache()
+    _, desc0, ctx0, ws0, outs0 = _full_step(cfg, 0)
+    for a, b in zip(saved, outs0):
+        assert torch.equal(a, b)
+    for a, f in zip(saved_ctx, (binding.SF_CTX_Y2_VALS, binding.SF_CTX_META, binding.SF_CTX_COLIDX)):
+        assert torch.equal(a, binding.sf_ctx_view(desc0, ctx0, f))
 
 
 @pytest.mark.parametrize("rows,cols", synth.PRUNE_SWEEP_SHAPES)
