@@ -56,8 +56,16 @@ typedef enum sf_status {
  * T % V == 0, (4F/M) % 128 == 0, V in {64,128}, N == 2, M in {4,8,16,32,64}. */
 typedef enum sf_ffn_flags {
   SF_FFN_SAVE_Y1 = 1,     /* also store the full bf16 pre-activation y1 in the context (SF_CTX_Y1) */
-  SF_FFN_UNFUSED_ACT = 2  /* M == 8 only: run SquaredReLU + V:N:M as its own kernel on a stored y1 instead of
-                             inside the y1 product's epilogue (same results; for comparison and profiling) */
+  SF_FFN_UNFUSED_ACT = 2, /* M == 8: run SquaredReLU + V:N:M as its own kernel on a stored y1, never inside the
+                             y1 product's epilogue */
+  SF_FFN_FUSED_ACT = 4,   /* M == 8: run them inside the y1 product's epilogue whenever the shape allows. With
+                             neither bit the library fuses for V == 64 (token tiles of three blocks) and not for
+                             V == 128 (a one-block tile re-reads the weight operand too often). Same results
+                             either way, bit for bit. */
+  SF_FFN_PACKED_GRAD_OPERANDS = 8 /* M == 8: keep no masked [T, F] copy of y2 and dy1; the two weight-gradient
+                             products expand their operand from its packed form inside the kernel. Saves
+                             4*T*F bytes of context + workspace, costs about a third more time in those two
+                             products. Same results, bit for bit. */
 } sf_ffn_flags;
 typedef struct sf_ffn_desc {
   int64_t T, D, F;
@@ -187,14 +195,14 @@ SF_API int sf_gemm_sparse24_noalloc(const void* a_vals, const void* a_meta, cons
  *                     product on the accumulator tile (y1 is never written); the activation is also
  *                     kept as a plain 2:4 operand over all F columns (two of eight is at most two
  *                     of four), which is what the products consume: identical results, no row
- *                     gather. No masked [T, F] copy of y2, ReLU(y1) or dy1 exists on this path.
+ *                     gather. ReLU(y1) exists in that layout only.
  *                     M >= 16: the product consumes the condensed V:N:M operand and gathers the kept
  *                     rows of W2^T.
  * sf_sparse_ffn_bwd:  W2s = prune24(W2 along D);  dy2 = dY W2s;  dy1 = 2 dy2 ReLU(y1) on y2's
  *                     mask;  dX = dy1 W1 (W1 dense);  dW1 = dy1^T X [F,D];  dW2 = dY^T y2 [D,F].
  *                     The two weight-gradient products reduce over tokens, so they run on the dense
- *                     tensor path; for M == 8 their masked operand is expanded from its packed form
- *                     inside the kernel.
+ *                     tensor path on a masked [T, F] copy of y2 / dy1 written by the epilogue that
+ *                     produces it (or, with SF_FFN_PACKED_GRAD_OPERANDS, on the packed form).
  * sf_dense_ffn_fwd/bwd: the same equations with no pruning; fwd_ctx holds y1 (bf16 [T,F]).
  */
 SF_API int sf_ffn_workspace_size(const sf_ffn_desc* desc, size_t* fwd_ctx_bytes, size_t* workspace_bytes);

@@ -112,8 +112,10 @@ struct SparseLayout {
   size_t w1_vals, w1_meta, w1_meta_hw, ws_y1, w2_vals, w2_meta, w2_meta_hw, dy1_dense, dy1_vals, dy1_vals24,
       ws_total;
   bool plain24;   // activations are fed to the tensor cores as plain 2:4 over all F columns
-  bool packed8;   // M = 8: no masked dense copy of y2, ReLU(y1) or dy1 exists; every consumer reads the 2:4 layout
+  bool packed8;   // M = 8: ReLU(y1) and the operands of the sparse products exist in the 2:4 layout only
   bool fused;     // packed8 and the activation is sparsified inside the y1 product's epilogue
+  bool expand;    // packed8 and the weight-gradient products expand their masked operand from its packed form
+                  // (no masked [T, F] copy of y2 or dy1 exists at all)
 };
 
 constexpr size_t kNone = (size_t)-1;
@@ -125,7 +127,12 @@ SparseLayout sparse_layout(const sf_ffn_desc& d) {
   // ungathered 2:4 product (twice the tensor work, no row gather) is the faster of the two.
   L.plain24 = (d.M == 4) || (d.M == 8 && vnm_has_24_view(d.F, d.V, d.M));
   L.packed8 = d.M == 8 && L.plain24;
-  L.fused = L.packed8 && !(d.flags & SF_FFN_UNFUSED_ACT) && gemm_sparse24_vnm8_supported(d.F, d.T, d.D, d.V);
+  // The fused epilogue needs whole V-blocks inside a token tile: three blocks of 64 in a 192-column tile cost
+  // 9 % more operand traffic than the plain product's 224 columns, one block of 128 in a 128-column tile 28 %
+  // more, which outweighs the saved kernel: V = 128 fuses only on request.
+  const bool can_fuse = L.packed8 && gemm_sparse24_vnm8_supported(d.F, d.T, d.D, d.V);
+  L.fused = can_fuse && !(d.flags & SF_FFN_UNFUSED_ACT) && (d.V == 64 || (d.flags & SF_FFN_FUSED_ACT));
+  L.expand = L.packed8 && (d.flags & SF_FFN_PACKED_GRAD_OPERANDS);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t r = o; o += up(bytes); return r; };
   L.y2_vals = take(T * 2 * G * 2);
@@ -138,7 +145,8 @@ SparseLayout sparse_layout(const sf_ffn_desc& d) {
     L.relu24 = take(T * F);
     L.meta24 = take(T * F / 8);
     L.meta24_hw = take(T * F / 8);
-    L.meta_hw = L.y2_dense = L.relu_dense = L.w2t = kNone;
+    L.y2_dense = L.expand ? kNone : take(T * F * 2);
+    L.meta_hw = L.relu_dense = L.w2t = kNone;
   } else {
     L.meta_hw = take(T * G / 2);
     L.y2_dense = take(T * F * 2);
@@ -158,7 +166,8 @@ SparseLayout sparse_layout(const sf_ffn_desc& d) {
   L.w2_meta_hw = take(F * D / 8);
   if (L.packed8) {
     L.dy1_vals24 = take(T * F);
-    L.dy1_dense = L.dy1_vals = kNone;
+    L.dy1_dense = L.expand ? kNone : take(T * F * 2);
+    L.dy1_vals = kNone;
   } else {
     L.dy1_dense = take(T * F * 2);
     L.dy1_vals = take(T * 2 * G * 2);
@@ -185,7 +194,9 @@ int check_desc(const sf_ffn_desc* d) {
   if (!d) return SF_ERR_NULL;
   if (d->N != 2) return SF_ERR_UNSUPPORTED;
   if (d->M != 4 && d->M != 8 && d->M != 16 && d->M != 32 && d->M != 64) return SF_ERR_SHAPE;
-  if (d->flags & ~(SF_FFN_SAVE_Y1 | SF_FFN_UNFUSED_ACT)) return SF_ERR_UNSUPPORTED;
+  if (d->flags & ~(SF_FFN_SAVE_Y1 | SF_FFN_UNFUSED_ACT | SF_FFN_FUSED_ACT | SF_FFN_PACKED_GRAD_OPERANDS))
+    return SF_ERR_UNSUPPORTED;
+  if ((d->flags & SF_FFN_UNFUSED_ACT) && (d->flags & SF_FFN_FUSED_ACT)) return SF_ERR_UNSUPPORTED;
   if (d->V != 64 && d->V != 128) return SF_ERR_SHAPE;
   if (d->T <= 0 || d->D <= 0 || d->F <= 0) return SF_ERR_SHAPE;
   if (d->T % 256 || d->D % 256 || d->F % 256 || d->T % d->V) return SF_ERR_SHAPE;
@@ -349,7 +360,7 @@ int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, co
     // accumulator tile; y1 itself is never written (unless asked for)
     Vnm8Out out{at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.relu_vals), at(fwd_ctx, L.meta), at(fwd_ctx, L.colidx),
                 at(fwd_ctx, L.vals24), at(fwd_ctx, L.relu24), at(fwd_ctx, L.meta24), at(fwd_ctx, L.meta24_hw),
-                save_y1 ? (void*)at(fwd_ctx, L.y1) : nullptr};
+                save_y1 ? (void*)at(fwd_ctx, L.y1) : nullptr, L.expand ? nullptr : (void*)at(fwd_ctx, L.y2_dense)};
     SF_TRY(gemm_sparse24_vnm8(at(workspace, L.w1_vals), at(workspace, L.w1_meta_hw), X, d.F, d.T, d.D, d.V, out,
                               status, s));
     trace_mark(s);
@@ -362,7 +373,8 @@ int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, co
     // lines 5-6: y2 = ReLU(y1)^2 in V:N:M form (+ what the backward pass needs)
     if (L.packed8) {
       SF_TRY(launch_vnm(y1, d.T, d.F, d.F, d.V, d.M, 1, at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta), nullptr,
-                        at(fwd_ctx, L.colidx), at(fwd_ctx, L.relu_vals), nullptr, nullptr, at(fwd_ctx, L.vals24),
+                        at(fwd_ctx, L.colidx), at(fwd_ctx, L.relu_vals),
+                        L.expand ? nullptr : (void*)at(fwd_ctx, L.y2_dense), nullptr, at(fwd_ctx, L.vals24),
                         at(fwd_ctx, L.meta24), at(fwd_ctx, L.meta24_hw), at(fwd_ctx, L.relu24), s));
     } else {
       SF_TRY(launch_vnm(y1, d.T, d.F, d.F, d.V, d.M, 1, at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta),
@@ -414,11 +426,11 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
   }
   trace_mark(s);
   if (L.packed8) {
-    // M = 8: ReLU(y1) comes in the 2:4 layout of y2's mask and dy1 leaves in the same layout; no [T, F]
-    // matrix is written
+    // M = 8: ReLU(y1) comes in the 2:4 layout of y2's mask and dy1 leaves in the same layout (plus, unless
+    // the weight-gradient products expand their operands themselves, as a masked [T, F] matrix)
     SF_TRY(gemm_sparse24(at(workspace, L.w2_vals), at(workspace, L.w2_meta_hw), dY, true, d.F, d.T, d.D,
-                         EPI_DRELU24_T, nullptr, 0, at(fwd_ctx, L.relu24), 0, status, s, at(fwd_ctx, L.meta24),
-                         at(workspace, L.dy1_vals24)));
+                         EPI_DRELU24_T, L.expand ? nullptr : (void*)at(workspace, L.dy1_dense), d.F,
+                         at(fwd_ctx, L.relu24), 0, status, s, at(fwd_ctx, L.meta24), at(workspace, L.dy1_vals24)));
     trace_mark(s);
     trace_mark(s);
     // line 5: dX = dy1 W1 with W1 dense; W1 [F, D] is the MN-major operand
@@ -426,13 +438,24 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
                          dX, d.D, nullptr, 0, status, s));
     trace_mark(s);
     hook_dx_done(s);
-    // line 3: dW2 = dY^T y2 [D, F];  line 6: dW1 = dy1^T X [F, D]: dense tensor-core products whose masked
-    // operand is expanded from its packed form inside the kernel
-    SF_TRY(gemm_dense_expand(dY, 2, at(fwd_ctx, L.vals24), at(fwd_ctx, L.meta24), d.D, d.F, d.T, dW2, d.F, status, s));
+    // line 3: dW2 = dY^T y2 [D, F];  line 6: dW1 = dy1^T X [F, D]: dense tensor-core products (the reduction
+    // runs over tokens); their masked operand is a stored [T, F] matrix or is expanded from its packed form
+    // inside the kernel
+    if (L.expand) {
+      SF_TRY(gemm_dense_expand(dY, 2, at(fwd_ctx, L.vals24), at(fwd_ctx, L.meta24), d.D, d.F, d.T, dW2, d.F, status, s));
+    } else {
+      SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.y2_dense), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0,
+                        nullptr, 0, status, s));
+    }
     trace_mark(s);
     hook_dw2_done(s);
-    SF_TRY(gemm_dense_expand(X, 1, at(workspace, L.dy1_vals24), at(fwd_ctx, L.meta24), d.F, d.D, d.T, dW1, d.D, status,
-                             s));
+    if (L.expand) {
+      SF_TRY(gemm_dense_expand(X, 1, at(workspace, L.dy1_vals24), at(fwd_ctx, L.meta24), d.F, d.D, d.T, dW1, d.D,
+                               status, s));
+    } else {
+      SF_TRY(gemm_dense(at(workspace, L.dy1_dense), false, X, false, d.F, d.D, d.T, EPI_STORE, dW1, d.D, nullptr, 0,
+                        nullptr, 0, status, s));
+    }
     trace_mark(s);
     return SF_OK;
   }

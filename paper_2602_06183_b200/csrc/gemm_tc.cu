@@ -209,7 +209,7 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
       for (int i = 0; i < 4; ++i) {
         const int t = i * 8 + (lane >> 2), seg = lane & 3;
         const uint4 o = *reinterpret_cast<const uint4*>(my_stage + t * kEpiStageRow + seg * 16);
-        if (kEpi != EPI_DRELU24_T)
+        if (kEpi != EPI_DRELU24_T || args.C != nullptr)
           *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.C) + (col0 + t) * args.ldc + m0 + q * 32 + seg * 8) = o;
         if (pack) {
           // this lane's eight features are two groups of four: keep the two recorded positions of each
@@ -277,49 +277,54 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
 //           SquaredReLU, keeps the two largest of the four kept columns and writes the packed activation,
 //           the packed ReLU values, both metadata forms and the 2:4 view.
 // The accumulator is released to the MMA warp as soon as the last block's pass 1 has read it.
-constexpr int kVnmStageBytes = 128 * 64;                        // y1 of one block: up to 128 tokens x 32 features
-constexpr int kVnmWarpBytes = kVnmStageBytes + 16 + 4 * 7 * 16 + 32;   // + colidx, selector table, nibble table
-constexpr int kVnmEpiBytes = 4 * ((kVnmWarpBytes + 127) / 128 * 128);
+// Shared memory of one epilogue warp: y1 of one block as [token pair][feature] words (low half = even
+// token), then colidx, the selector table and the nibble table of the block.
+__host__ __device__ constexpr int vnm_stage_bytes(int V) { return V * 64; }
+__host__ __device__ constexpr int vnm_warp_bytes(int V) { return vnm_stage_bytes(V) + 16 + 4 * 7 * 16 + 48; }
+constexpr int kVnmEpiWarps = 8;                                  // two sets of four: one set per accumulator buffer
+__host__ __device__ constexpr int vnm_epi_bytes(int V) { return kVnmEpiWarps * vnm_warp_bytes(V); }
 
-template <int kTileN>
+template <int kTileN, int kV>
 __device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0, int q,
                                               int lane, uint8_t* wsm, uint64_t* tmem_empty_bar) {
-  uint8_t* stage = wsm;                                                   // [V][64 B]
-  uint8_t* cidx = wsm + kVnmStageBytes;                                   // [4 groups][4]
-  uint4* sel_tab = reinterpret_cast<uint4*>(wsm + kVnmStageBytes + 16);   // [4 groups][7]
-  uint8_t* nib_tab = wsm + kVnmStageBytes + 16 + 4 * 7 * 16;              // [4 groups][7]
-  const int V = args.V;
+  uint32_t* stage = reinterpret_cast<uint32_t*>(wsm);                     // [kV / 2][32 features]
+  uint8_t* cidx = wsm + vnm_stage_bytes(kV);                              // [4 groups][4]
+  uint4* sel_tab = reinterpret_cast<uint4*>(wsm + vnm_stage_bytes(kV) + 16);   // [4 groups][7]
+  uint8_t* nib_tab = wsm + vnm_stage_bytes(kV) + 16 + 4 * 7 * 16;         // [4 groups][7]
   const int64_t F = args.M, G = F >> 3;
   const int64_t f0 = m0 + q * 32, g0 = f0 >> 3;                           // this warp's first feature / group
   const int jm = lane & 7, gl = lane & 3;
-  constexpr int kMaxBlocks = kTileN / 64;
-  int nblk = kTileN / V;
-  while (nblk > 0 && n0 + (int64_t)(nblk - 1) * V >= args.N) --nblk;       // ragged last tile: whole blocks only
-  if (nblk == 0) {                                                         // cannot happen for a launched tile; keep the protocol
+  constexpr int kBlocks = kTileN / kV;
+  int nblk = kBlocks;
+  while (nblk > 0 && n0 + (int64_t)(nblk - 1) * kV >= args.N) --nblk;      // ragged last tile: whole blocks only
+  if (nblk == 0) {
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive_leader(tmem_empty_bar);
     return;
   }
+  // strides per token of the outputs this thread writes (in the units of its pointers)
+  const int sv = (int)G, s24 = (int)(F >> 3), sm = (int)(G >> 2), sm24 = (int)(F >> 5);
+  const bool lead4 = gl == 0, lead2 = (gl & 1) == 0;
 #pragma unroll 1
-  for (int b = 0; b < kMaxBlocks; ++b) {
+  for (int b = 0; b < kBlocks; ++b) {
     if (b >= nblk) break;
     __syncwarp();                                                          // the previous block's pass 2 has read the stage
-    const int64_t t0 = n0 + (int64_t)b * V;
-    // ---- pass 1
+    const int64_t t0 = n0 + (int64_t)b * kV;
+    // ---- pass 1: two tokens per step on packed bf16 pairs
     float score = 0.f;
     uint32_t v[32];
 #pragma unroll 1
-    for (int c = 0; c < V / 32; ++c) {
-      tmem_ld_32x32b_x32(taddr + (uint32_t)(b * V + c * 32), v);
+    for (int c = 0; c < kV / 32; ++c) {
+      tmem_ld_32x32b_x32(taddr + (uint32_t)(b * kV + c * 32), v);
       tmem_ld_wait_on(v);
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const uint32_t y = float_to_bf16_bits(__uint_as_float(v[j]));
-        *reinterpret_cast<uint16_t*>(stage + (c * 32 + j) * 64 + lane * 2) = (uint16_t)y;
-        const float r = fmaxf(bf16_bits_to_float(y), 0.f);
-        const float h = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(r, r)));
-        score = __fadd_rn(score, h);
+      for (int j = 0; j < 16; ++j) {
+        const uint32_t yp = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+        stage[(c * 16 + j) * 32 + lane] = yp;
+        const uint32_t hp = bf2_sq(bf2_relu(yp));
+        score = __fadd_rn(score, __uint_as_float(hp << 16));
+        score = __fadd_rn(score, __uint_as_float(hp & 0xFFFF0000u));
       }
     }
     if (b == nblk - 1) {
@@ -339,11 +344,10 @@ __device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t tad
     const bool keep = rank < 4;
     const uint32_t ball = __ballot_sync(0xFFFFFFFFu, keep);
     const uint32_t gbyte = (ball >> (lane & 24)) & 0xFFu;
-    __syncwarp();                                                          // previous block's pass 2 is done with the tables
     if (keep) cidx[(lane >> 3) * 4 + __popc(gbyte & ((1u << jm) - 1u))] = (uint8_t)jm;
     __syncwarp();
     if (lane < 4)
-      *reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(args.vn_colidx) + ((t0 / V) * G + g0 + lane) * 4) =
+      *reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(args.vn_colidx) + ((t0 / kV) * G + g0 + lane) * 4) =
           *reinterpret_cast<const uint32_t*>(cidx + lane * 4);
     if (lane < 24) {
       const int ge = lane / 6, pe = lane - ge * 6;
@@ -356,7 +360,7 @@ __device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t tad
       nib_tab[slot] = (uint8_t)nib24;
     }
     __syncwarp();
-    // ---- pass 2: this thread serves group gl of tokens (lane >> 2) + 8 * it
+    // ---- pass 2: this thread serves group gl of the token pairs (lane >> 2) + 8 * it
     const uint32_t c4 = *reinterpret_cast<const uint32_t*>(cidx + gl * 4);
     uint32_t selp[2], mhi[2];
 #pragma unroll
@@ -368,16 +372,25 @@ __device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t tad
     }
     const uint4* my_sel = sel_tab + gl * 7;
     const uint8_t* my_nib = nib_tab + gl * 7;
-    const int64_t kw24 = (f0 >> 4) + (gl >> 1);                            // this lane pair's 16-column word of the 2:4 view
-    const bool lead4 = gl == 0, lead2 = (gl & 1) == 0;
-#pragma unroll 2
-    for (int it = 0; it < V / 8; ++it) {
-      const int tk = (lane >> 2) + 8 * it;
-      const int64_t t = t0 + tk;
-      const uint4 qv = *reinterpret_cast<const uint4*>(stage + tk * 64 + gl * 16);
-      uint32_t rw[4] = {qv.x, qv.y, qv.z, qv.w}, hw[4];
+    // output pointers of this thread's first token; every pointer advances by a constant per token
+    const int64_t tf = t0 + 2 * (lane >> 2);
+    uint32_t* p_vals = reinterpret_cast<uint32_t*>(args.vn_vals) + tf * G + g0 + gl;
+    uint32_t* p_relu = reinterpret_cast<uint32_t*>(args.vn_relu) + tf * G + g0 + gl;
+    uint2* p_v24 = reinterpret_cast<uint2*>(args.vn_vals24) + tf * (F >> 3) + g0 + gl;
+    uint2* p_r24 = reinterpret_cast<uint2*>(args.vn_relu24) + tf * (F >> 3) + g0 + gl;
+    uint4* p_y1 = args.vn_y1 ? reinterpret_cast<uint4*>(args.vn_y1) + tf * (F >> 3) + g0 + gl : nullptr;
+    uint4* p_dense = args.vn_dense ? reinterpret_cast<uint4*>(args.vn_dense) + tf * (F >> 3) + g0 + gl : nullptr;
+    uint16_t* p_meta = reinterpret_cast<uint16_t*>(args.vn_meta) + tf * (G >> 2) + (g0 >> 2);
+    uint32_t* p_m24 = reinterpret_cast<uint32_t*>(args.vn_meta24) + tf * (F >> 5) + (f0 >> 5);
+    // tensor-core-ordered copy: the block lies inside one 128-row band, so the atom is fixed
+    const int64_t kw24 = (f0 >> 4) + (gl >> 1);
+    uint8_t* hw_atom = reinterpret_cast<uint8_t*>(args.vn_meta24_hw) + meta_hw_offset(t0 & ~int64_t(127), kw24, F);
+    const uint32_t* sp = stage + (lane >> 2) * 32 + gl * 8;
+
+    auto emit = [&](const uint32_t (&yw)[4], int dt, uint32_t trow) {
+      uint32_t rw[4], hw[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) { rw[j] = bf2_relu(rw[j]); hw[j] = bf2_sq(rw[j]); }
+      for (int j = 0; j < 4; ++j) { rw[j] = bf2_relu(yw[j]); hw[j] = bf2_sq(rw[j]); }
       const uint32_t a0 = __byte_perm(hw[0], hw[1], selp[0]), b0 = __byte_perm(hw[2], hw[3], selp[0]);
       const uint32_t a1 = __byte_perm(hw[0], hw[1], selp[1]), b1 = __byte_perm(hw[2], hw[3], selp[1]);
       const uint32_t hk0 = (a0 & ~mhi[0]) | (b0 & mhi[0]), hk1 = (a1 & ~mhi[1]) | (b1 & mhi[1]);
@@ -387,28 +400,45 @@ __device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t tad
       const uint4 sel = my_sel[slot];
       const uint32_t x = __byte_perm(rw[0], rw[1], sel.z), y = __byte_perm(rw[2], rw[3], sel.z);
       const uint32_t rpair = __byte_perm(x, y, sel.z >> 16);
-      const int64_t pv = t * (2 * G) + 2 * (g0 + gl);
-      reinterpret_cast<uint32_t*>(args.vn_vals)[pv >> 1] = packed;
-      reinterpret_cast<uint32_t*>(args.vn_relu)[pv >> 1] = rpair;
-      const int64_t p24 = (t * (F >> 1) + (g0 + gl) * 4) >> 2;             // in 8-byte units
-      reinterpret_cast<uint2*>(args.vn_vals24)[p24] =
-          make_uint2(__byte_perm(packed, 0u, sel.w), __byte_perm(packed, 0u, sel.w >> 16));
-      reinterpret_cast<uint2*>(args.vn_relu24)[p24] =
-          make_uint2(__byte_perm(rpair, 0u, sel.w), __byte_perm(rpair, 0u, sel.w >> 16));
-      if (args.vn_y1) reinterpret_cast<uint4*>(args.vn_y1)[(t * F + f0 + gl * 8) >> 3] = qv;
+      p_vals[dt * sv] = packed;
+      p_relu[dt * sv] = rpair;
+      p_v24[dt * s24] = make_uint2(__byte_perm(packed, 0u, sel.w), __byte_perm(packed, 0u, sel.w >> 16));
+      p_r24[dt * s24] = make_uint2(__byte_perm(rpair, 0u, sel.w), __byte_perm(rpair, 0u, sel.w >> 16));
+      if (p_y1) p_y1[dt * s24] = make_uint4(yw[0], yw[1], yw[2], yw[3]);
+      if (p_dense)
+        p_dense[dt * s24] = make_uint4(__byte_perm(packed, 0u, sel.x), __byte_perm(packed, 0u, sel.x >> 16),
+                                       __byte_perm(packed, 0u, sel.y), __byte_perm(packed, 0u, sel.y >> 16));
       // canonical V:N:M metadata: the warp's four groups of a token form one word
       uint32_t word = nib;
       word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 4;
       word |= __shfl_down_sync(0xFFFFFFFFu, word, 2) << 8;
-      if (lead4) reinterpret_cast<uint16_t*>(args.vn_meta)[t * (G >> 2) + (g0 >> 2)] = (uint16_t)word;
+      if (lead4) p_meta[dt * sm] = (uint16_t)word;
       // metadata of the 2:4 view: one byte per group, one 16-bit word per pair of groups
       uint32_t mb = my_nib[slot];
       mb |= __shfl_down_sync(0xFFFFFFFFu, mb, 1) << 8;
       const uint32_t mb32 = (mb & 0xFFFFu) | (__shfl_down_sync(0xFFFFFFFFu, mb, 2) << 16);
-      if (lead4) reinterpret_cast<uint32_t*>(args.vn_meta24)[(t * (F >> 4) + (f0 >> 4)) >> 1] = mb32;
-      if (lead2)
-        *reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(args.vn_meta24_hw) + meta_hw_offset(t, kw24, F)) =
-            (uint16_t)mb;
+      if (lead4) p_m24[dt * sm24] = mb32;
+      if (lead2) {
+        const uint32_t mi = trow & 127u;
+        *reinterpret_cast<uint16_t*>(hw_atom + (mi >> 4) * 256u + (mi & 7u) * 16u + ((mi >> 3) & 1u) * 2u) = (uint16_t)mb;
+      }
+    };
+#pragma unroll 1
+    for (int it = 0; it < kV / 16; ++it) {
+      const uint4 qa = *reinterpret_cast<const uint4*>(sp), qb = *reinterpret_cast<const uint4*>(sp + 4);
+      // de-interleave the token pair: low halves = even token, high halves = odd token
+      const uint32_t r0[4] = {__byte_perm(qa.x, qa.y, 0x5410), __byte_perm(qa.z, qa.w, 0x5410),
+                              __byte_perm(qb.x, qb.y, 0x5410), __byte_perm(qb.z, qb.w, 0x5410)};
+      const uint32_t r1[4] = {__byte_perm(qa.x, qa.y, 0x7632), __byte_perm(qa.z, qa.w, 0x7632),
+                              __byte_perm(qb.x, qb.y, 0x7632), __byte_perm(qb.z, qb.w, 0x7632)};
+      const uint32_t trow = (uint32_t)(tf & 127) + 16u * (uint32_t)it;
+      emit(r0, 0, trow);
+      emit(r1, 1, trow + 1u);
+      sp += 8 * 32;
+      p_vals += 16 * sv; p_relu += 16 * sv; p_v24 += 16 * s24; p_r24 += 16 * s24;
+      if (p_y1) p_y1 += 16 * s24;
+      if (p_dense) p_dense += 16 * s24;
+      p_meta += 16 * sm; p_m24 += 16 * sm24;
     }
   }
 }
@@ -682,18 +712,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 // Stage = 64 K (dense, 4 MMAs of K=16) or 128 logical K (2:4, 4 MMAs of K=32 and one metadata atom):
 // four MMAs per barrier round trip keep the single issuing thread ahead of the tensor pipe.
 constexpr int kThreads2 = 192;
-constexpr int kThreads2Expand = 320;                     // + four warps that expand a packed operand into its stage
+constexpr int kThreads2Expand = 448;                     // + eight warps that expand a packed operand into its stage
+constexpr int kThreads2Vnm = 320;                        // + a second set of four epilogue warps (one set per accumulator)
+__host__ __device__ constexpr int threads2(int epi, int expand) {
+  return expand ? kThreads2Expand : (epi == EPI_VNM8 ? kThreads2Vnm : kThreads2);
+}
 constexpr int kPkStageBytes = 8192 + 1024;               // packed values [64 tokens][64] + metadata bytes [64][16]
 __host__ __device__ constexpr int stage_bytes2(bool sparse, int bn = BN) {
   return sparse ? (16384 + 2 * (bn / 2) * 128 + 2048) : (16384 + 16384);
 }
 __host__ __device__ constexpr int num_stages2(bool sparse, int bn = BN, bool expand = false) {
-  return sparse ? (bn <= 128 ? 5 : 4) : (expand ? 5 : 6);
+  return sparse ? 4 : (expand ? 5 : 6);
 }
-__host__ __device__ constexpr int epi_bytes2(int epi) { return epi == EPI_VNM8 ? kVnmEpiBytes : kEpiStageBytes; }
+// the fused activation epilogue holds whole V-blocks per tile: 192 columns = three blocks of 64, 128 = one of 128
+__host__ __device__ constexpr int vnm_block(int bn) { return bn == 192 ? 64 : 128; }
+__host__ __device__ constexpr int epi_bytes2(int epi, int bn = BN) {
+  return epi == EPI_VNM8 ? vnm_epi_bytes(vnm_block(bn)) : kEpiStageBytes;
+}
 __host__ __device__ constexpr int smem_bytes2(bool sparse, int bn = BN, int epi = EPI_STORE, bool expand = false) {
   return 1024 + num_stages2(sparse, bn, expand) * (stage_bytes2(sparse, bn) + (expand ? kPkStageBytes : 0)) +
-         epi_bytes2(epi) + 512;
+         epi_bytes2(epi, bn) + 1024;
 }
 
 struct SmemCtl2 {
@@ -702,6 +740,7 @@ struct SmemCtl2 {
   uint64_t pk_full[8];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
+  uint2 expand_lut[16];      // byte-permute selectors of a 2:4 nibble (see the operand expander)
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -714,7 +753,7 @@ __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
 // dense tile; its 2:4-packed form (tmapPk: values, tmapMeta: metadata bytes) is staged by TMA and four
 // extra warps expand it, zero-filled, into the swizzled layout the MMA reads.
 template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN, int kExpand = 0>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kExpand ? kThreads2Expand : kThreads2, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(threads2(kEpi, kExpand), 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                 const __grid_constant__ CUtensorMap tmapMeta, const __grid_constant__ CUtensorMap tmapPk,
                 const GemmArgs args) {
@@ -738,7 +777,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   static_assert(!kBMN || kBN == BN, "MN-major B is loaded in 64-column chunks");
   uint8_t* pk_stage = smem + kStages * kStageBytes;       // kExpand: ring of packed tiles, one per stage
   uint8_t* epi_stage = pk_stage + (kExpand ? kStages * kPkStageBytes : 0);
-  SmemCtl2* ctl = reinterpret_cast<SmemCtl2*>(epi_stage + epi_bytes2(kEpi));
+  SmemCtl2* ctl = reinterpret_cast<SmemCtl2*>(epi_stage + epi_bytes2(kEpi, kBN));
   volatile int* abort_flag = &ctl->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -754,7 +793,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     if (kSparse || kExpand) prefetch_tmap(&tmapMeta);
     if (kExpand) prefetch_tmap(&tmapPk);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&ctl->full[s], kExpand ? 1 + 8 : 1);     // + the four expander warps of either CTA
+      mbar_init(&ctl->full[s], kExpand ? 1 + 16 : 1);    // + the eight expander warps of either CTA
       mbar_init(&ctl->empty[s], 1);
       mbar_init(&ctl->pk_full[s], 1);
     }
@@ -764,6 +803,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     }
     ctl->abort_flag = 0;
     fence_mbar_init();
+  }
+  if (kExpand && threadIdx.x >= 64 && threadIdx.x < 80) {
+    // nibble n = p0 | p1 << 2: output byte pair of column c takes stored value 0 (bytes 1,0) if c == p0,
+    // value 1 (bytes 3,2) if c == p1, else the zero operand (byte 4)
+    const uint32_t n = threadIdx.x - 64;
+    const uint32_t sel = 0x44444444u ^ (0x54u << (8u * (n & 3u))) ^ (0x76u << (8u * (n >> 2)));
+    ctl->expand_lut[n] = make_uint2(sel & 0xFFFFu, sel >> 16);
   }
   if (warp == 1) {
     tmem_alloc_2cta(&ctl->tmem_base, kTmemCols);
@@ -893,12 +939,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
       }
     }
   } else if (kExpand != 0 && warp >= 6) {
-    // =========================== operand expander (warps 6..9, both CTAs) ===========================
+    // =========================== operand expander (warps 6..13, both CTAs) ===========================
     // Stage tile = 64 tokens (K) x 128 features, MN-major, 128-byte swizzle: two chunks of 64 features,
     // a token row of a chunk is 128 bytes whose 16-byte units are XOR-ed with (token & 7). One unit is
     // eight features = two 2:4 groups = four stored values + one metadata byte in the packed tile.
-    const int te = (int)threadIdx.x - 192;                 // 0..127
-    const int seg = te & 15, tk0 = te >> 4;                // 16 units per token row; 8 tokens per pass
+    const int te = (int)threadIdx.x - 192;                 // 0..255
+    const int seg = te & 15, tk0 = te >> 4;                // 16 units per token row; 16 tokens per pass
+    const uint2* lut = ctl->expand_lut;
     uint32_t stage = 0, phase = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
@@ -906,12 +953,21 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
         if (!mbar_wait(&ctl->pk_full[stage], phase, abort_flag)) { ok = false; break; }
         const uint8_t* sP = pk_stage + stage * kPkStageBytes;
         uint8_t* dst = smem + stage * kStageBytes + (kExpand == 1 ? 0 : kAStageBytes) + (seg >> 3) * 8192;
+        uint2 v[4];
+        uint32_t mb[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int tk = tk0 + 8 * i;
-          const uint2 v = *reinterpret_cast<const uint2*>(sP + tk * 128 + seg * 8);
-          const uint32_t mb = sP[8192 + tk * 16 + seg];
-          *reinterpret_cast<uint4*>(dst + tk * 128 + (((seg & 7) ^ (tk & 7)) << 4)) = expand24_x8(v, mb);
+        for (int i = 0; i < 4; ++i) {
+          const int tk = tk0 + 16 * i;
+          v[i] = *reinterpret_cast<const uint2*>(sP + tk * 128 + seg * 8);
+          mb[i] = sP[8192 + tk * 16 + seg];
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int tk = tk0 + 16 * i;
+          const uint2 s0 = lut[mb[i] & 15u], s1 = lut[mb[i] >> 4];
+          *reinterpret_cast<uint4*>(dst + tk * 128 + (((seg & 7) ^ (tk & 7)) << 4)) =
+              make_uint4(__byte_perm(v[i].x, 0u, s0.x), __byte_perm(v[i].x, 0u, s0.y),
+                         __byte_perm(v[i].y, 0u, s1.x), __byte_perm(v[i].y, 0u, s1.y));
         }
         // generic-proxy stores -> visible to the tensor core's async-proxy reads, then signal the stage
         fence_proxy_async_smem();
@@ -920,9 +976,29 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
     }
+  } else if constexpr (kEpi == EPI_VNM8) {
+    // =========================== fused activation epilogue (warps 2..9, both CTAs) ===========================
+    // Two sets of four warps, one per accumulator buffer: set 0 takes this pair's even tiles, set 1 the odd
+    // ones, so each set has two main loops' time for one tile.
+    const int q = warp & 3, set = (warp - 2) >> 2;
+    constexpr int kV = vnm_block(kBN);
+    uint8_t* wsm = epi_stage + (set * 4 + q) * vnm_warp_bytes(kV);
+    uint32_t acc_phase = 0;
+    for (int tile = pair + set * num_pairs; tile < num_tiles; tile += 2 * num_pairs) {
+      int mt, nt;
+      tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
+      const int64_t m0 = (int64_t)mt * 256 + (int64_t)rank * 128, n0 = (int64_t)nt * kBN;
+      const uint32_t taddr = tmem_base + set * kBN + ((uint32_t)(q * 32) << 16);
+      if (!mbar_wait(&ctl->tmem_full[set], acc_phase, abort_flag)) break;
+      tc_fence_after();
+      // releases the accumulator itself, as soon as its last column has been read
+      epi_vnm8_tile<kBN, kV>(args, taddr, m0, n0, q, lane, wsm, &ctl->tmem_empty[set]);
+      acc_phase ^= 1;
+    }
   } else {
     // =========================== epilogue (warps 2..5, both CTAs) ===========================
     const int q = warp & 3;
+    uint8_t* my_stage = epi_stage + q * 32 * kEpiStageRow;
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
@@ -930,22 +1006,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
       tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
       const int64_t m0 = (int64_t)mt * 256 + (int64_t)rank * 128, n0 = (int64_t)nt * kBN;
       const uint32_t taddr = tmem_base + acc * kBN + ((uint32_t)(q * 32) << 16);
-      if constexpr (kEpi == EPI_VNM8) {
-        if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        // releases the accumulator itself, as soon as its last column has been read
-        epi_vnm8_tile<kBN>(args, taddr, m0, n0, q, lane, epi_stage + q * (kVnmEpiBytes / 4), &ctl->tmem_empty[acc]);
-      } else {
-        uint8_t* my_stage = epi_stage + q * 32 * kEpiStageRow;
-        uint4 ax[is_drelu_t(kEpi) ? kBN / 32 : 1][4];
-        epi_prefetch<kEpi, kBN>(args, m0, n0, q, lane, ax);
-        if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        epi_tile<kEpi, kBN>(args, taddr, m0, n0, q, lane, my_stage, ax);
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_leader(&ctl->tmem_empty[acc]);
-      }
+      uint4 ax[is_drelu_t(kEpi) ? kBN / 32 : 1][4];
+      epi_prefetch<kEpi, kBN>(args, m0, n0, q, lane, ax);
+      if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      epi_tile<kEpi, kBN>(args, taddr, m0, n0, q, lane, my_stage, ax);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(&ctl->tmem_empty[acc]);
       if (++acc == (uint32_t)kAccBufs) { acc = 0; acc_phase ^= 1; }
     }
   }
@@ -1050,7 +1118,7 @@ int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
   const int tiles = a.num_m_tiles * a.num_n_tiles;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  kern<<<2 * pairs, kExpand ? kThreads2Expand : kThreads2, smem, s>>>(ta, tb, tm, tpk ? *tpk : ta, a);
+  kern<<<2 * pairs, threads2(kEpi, kExpand), smem, s>>>(ta, tb, tm, tpk ? *tpk : ta, a);
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
@@ -1108,7 +1176,7 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
                   int64_t K, int epi, void* C, int64_t ldc, const void* aux, int64_t ldaux, int* status,
                   cudaStream_t s, const void* pack_meta, void* pack_vals) {
   if ((pack_meta != nullptr) != (pack_vals != nullptr) || (pack_vals && !is_drelu_t(epi))) return SF_ERR_UNSUPPORTED;
-  if (epi == EPI_DRELU24_T && (!pack_vals || !aux || M % 256)) return SF_ERR_UNSUPPORTED;
+  if (epi == EPI_DRELU24_T && (!pack_vals || !aux || M % 256)) return SF_ERR_UNSUPPORTED;   // C (dense copy) optional
   if (M % BM || N % BN || K % 128) return SF_ERR_SHAPE;
   if (M == 0 || N == 0) return SF_OK;
   const bool two = use_two_cta(M);
@@ -1171,7 +1239,7 @@ int gemm_sparse24_vnm8(const void* a_vals, const uint8_t* meta_hw, const void* X
   a.meta_hw = meta_hw; a.status = status;
   a.vn_vals = out.vals; a.vn_relu = out.relu; a.vn_meta = out.meta; a.vn_colidx = out.colidx;
   a.vn_vals24 = out.vals24; a.vn_relu24 = out.relu24; a.vn_meta24 = out.meta24; a.vn_meta24_hw = out.meta24_hw;
-  a.vn_y1 = out.y1;
+  a.vn_y1 = out.y1; a.vn_dense = out.dense;
   if (V == 64) return launch_two<MODE_SPARSE24, false, false, EPI_VNM8, 192>(ta, tb, tm, a, s);
   return launch_two<MODE_SPARSE24, false, false, EPI_VNM8, 128>(ta, tb, tm, a, s);
 }

@@ -48,11 +48,12 @@ struct GemmArgs {
   void* vn_meta24;          // uint16 [T, F/16] canonical metadata of that operand
   void* vn_meta24_hw;       // the same words in tensor-core order
   void* vn_y1;              // optional bf16 [T, F]: the pre-activation itself
+  void* vn_dense;           // optional bf16 [T, F]: the activation on its mask, +0 elsewhere
 };
 
 // Outputs of the fused y1 product (see GemmArgs::vn_*).
 struct Vnm8Out {
-  void *vals, *relu, *meta, *colidx, *vals24, *relu24, *meta24, *meta24_hw, *y1;
+  void *vals, *relu, *meta, *colidx, *vals24, *relu24, *meta24, *meta24_hw, *y1, *dense;
 };
 
 // D[M,N] = op(A) op(B)^T, tiles 128 x 256, K % 64 == 0.

@@ -35,6 +35,7 @@ FFN_CONFIGS = {
     # one eighth of c4's tokens with the full-size layer: weights (134 MB each) still exceed the
     # L2, device footprint ~1.5 GB; used for profiler captures that must stay small
     "c4_slice": dict(T=1024, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
+    "c4_slice_v64": dict(T=1024, D=4096, F=16384, V=64, N=2, M=8, sigma_w=0.02, seed=4),
     # the same slice with groups of 16 (87.5 % sparse activations): exercises the condensed Venom products
     "c4_slice_m16": dict(T=1024, D=4096, F=16384, V=128, N=2, M=16, sigma_w=0.02, seed=4),
     # c4 with groups of 16 (Table 5's 87.5 % row): the full-size case of the condensed Venom products

@@ -112,7 +112,7 @@ def test_sparse_ffn_c1_teacher_forced(prune_mode, act_shift):
 
 @pytest.mark.parametrize("cfg", [
     dict(T=1024, D=256, F=1024, V=64, N=2, M=8, sigma_w=0.02, seed=0),      # fused epilogue, three 64-token blocks per tile
-    dict(T=512, D=256, F=512, V=128, N=2, M=8, sigma_w=0.05, seed=3),       # fused epilogue, one 128-token block per tile
+    dict(T=512, D=256, F=512, V=128, N=2, M=8, sigma_w=0.05, seed=3),       # two-kernel path (the default for V = 128)
     dict(T=512, D=256, F=2048, V=128, N=2, M=16, sigma_w=0.05, seed=17),    # condensed Venom products
 ], ids=["m8_v64", "m8_v128", "m16_v128"])
 def test_step_without_saved_y1_is_the_same_step(cfg):
@@ -134,11 +134,16 @@ def test_fused_activation_epilogue_equals_the_two_kernel_path(V, act_shift):
     y1: same accumulation, same selection rule, so every output must agree bit for bit. T is not a
     multiple of the fused kernel's 192-token tile, so the last tile is ragged."""
     cfg = dict(T=1280, D=512, F=768, V=V, N=2, M=8, sigma_w=0.05, seed=41)
-    inputs, fused = _run_sparse(cfg, act_shift=act_shift, flags=binding.SF_FFN_SAVE_Y1)
-    _, two = _run_sparse(cfg, act_shift=act_shift, flags=binding.SF_FFN_SAVE_Y1 | binding.SF_FFN_UNFUSED_ACT)
+    Y1 = binding.SF_FFN_SAVE_Y1
+    inputs, fused = _run_sparse(cfg, act_shift=act_shift, flags=Y1 | binding.SF_FFN_FUSED_ACT)
+    _, two = _run_sparse(cfg, act_shift=act_shift, flags=Y1 | binding.SF_FFN_UNFUSED_ACT)
     for k in fused:
         assert np.array_equal(fused[k], two[k]), k
     _check_against_oracle(inputs, fused, cfg)
+    # and with the weight-gradient products reading the packed operands instead of masked [T, F] copies
+    _, packed = _run_sparse(cfg, act_shift=act_shift, flags=Y1 | binding.SF_FFN_FUSED_ACT | binding.SF_FFN_PACKED_GRAD_OPERANDS)
+    for k in fused:
+        assert np.array_equal(fused[k], packed[k]), k
 
 
 def test_plain_24_view_of_m4_activations_is_exact():
