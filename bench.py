@@ -3,14 +3,22 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-Prints ONE JSON line (rank 0). A "step" is one pass of the whole hot path: 2:4 prune of W1,
-sparse y1 product, SquaredReLU + V:N:M sparsify, Venom y3 product, 2:4 prune of W2, sparse dy1
-product, dy1 pack, Venom dX product and the two weight-gradient products, on synthetic inputs of
-the named workload (default: the d_model = 4096 FFN layer, 8192 tokens).
+Prints ONE JSON line (rank 0). For the FFN workloads a "step" is one pass of the whole hot path:
+2:4 prune of W1, the 2:4 y1 product with SquaredReLU + V:N:M selection (in its epilogue or as a
+second kernel, see config.path), the y3 product, 2:4 prune of W2, the 2:4 dy1 product with the
+dy1 epilogue, the dX product and the two weight-gradient products, on synthetic inputs of the named
+workload (default: the d_model = 4096 FFN layer, 8192 tokens).
 
 metric  = dense-equivalent TFLOP/s of the sparse step: 6 products x 2*T*D*F flop / step time.
-N > 1   = N independent replicas of the layer (the path has no exchange step), launched by
-          torchrun; the value is the aggregate over all ranks, timed as the max over ranks.
+value   = that metric over exactly K timed steps after W (>= 3) warm-up steps; per-kernel times come
+          from events the library records between its kernels inside the same K steps.
+sustained = the same step in K-step blocks alternating with dense-step blocks for at least
+          --sustain-seconds per arm (medians): what the part delivers once it sits on its power cap.
+N > 1   = N independent replicas of the layer (the path has no exchange step); `--gpus N` starts the
+          N ranks itself when it is not already running under torchrun; the value is the aggregate
+          over all ranks, timed as the max over ranks.
+Other workloads: c2_prune (2:4 prune + compress sweep), c3_act (SquaredReLU + V:N:M sweep), gemm_micro
+          (2:4 and Venom products against the dense product, the paper's micro-benchmark shapes).
 --impl reference times the CPU oracle (a deliberately plain numpy program) on a bounded sample.
 """
 from __future__ import annotations
@@ -18,6 +26,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import tempfile
@@ -30,6 +39,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "sparse_ffn_fwd_bwd_dense_equiv_tflops"
 UNIT = "TFLOP/s"
+SWEEP_WORKLOADS = ("c2_prune", "c3_act", "gemm_micro")
 
 
 def _peaks():
@@ -41,8 +51,14 @@ def _peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
+def _traffic():
+    """Per-launch DRAM traffic of the step's kernels from the committed single-pass ncu capture."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    return json.load(open(path)) if os.path.exists(path) else {}
+
+
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -50,8 +66,10 @@ class ClockSampler:
     def __init__(self, gpu_index: int):
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.p = None
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+        dev = vis.split(",")[gpu_index] if vis else str(gpu_index)
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.Q}",
+            self.p = subprocess.Popen(["nvidia-smi", f"--id={dev}", f"--query-gpu={self.Q}",
                                        "--format=csv,noheader,nounits", "-lms", "20"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
@@ -136,6 +154,18 @@ def run_reference(args, cfg):
     }))
 
 
+# ---- stage names in the order the library records its trace events (see sf_trace_set) ----------------
+TRACE_NAMES = ["prune24_W1", "gemm_y1", "vnm_sparsify", "transpose_W2", "gemm_y3",
+               None, "prune24_W2", "gemm_dy1", "pack_dy1", "gemm_dX", "gemm_dW2", "gemm_dW1"]
+
+
+def _step_path(V, M):
+    """Which kernels the library runs for this configuration (mirrors the rule in the step's layout)."""
+    if M == 8:
+        return "fused" if V == 64 else "two_kernel"
+    return "plain24" if M == 4 else "venom"
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -153,12 +183,12 @@ def run_ours(args, cfg):
     binding.lib()
 
     T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
-    K, W = args.steps, args.warmup
+    K, W = args.steps, max(args.warmup, 3) if not args.quick else args.warmup
     X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"] + rank)
     pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
     hX, hW1, hW2, hdY = pin(X), pin(W1), pin(W2), pin(dY)
     dX_, dW1_, dW2_, ddY = (h.cuda().view(torch.bfloat16) for h in (hX, hW1, hW2, hdY))
-    desc = binding.make_desc(T, D, F, V, M, prune_mode=args.prune_mode)
+    desc = binding.make_desc(T, D, F, V, M, prune_mode=args.prune_mode, flags=args.flags)
     ctx, ws = binding.alloc_ffn_buffers(desc)
     Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
     gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
@@ -185,91 +215,125 @@ def run_ours(args, cfg):
         barrier()
         return replicas.max_over_ranks(e0.elapsed_time(e1), device="cuda")
 
-    for _ in range(W if args.quick else max(W, 3)):
+    for _ in range(W):
         sparse_step()
     if binding.sf_check_status(ws) != binding.SF_OK:
         raise SystemExit("device status: a bounded wait expired during warm-up")
 
-    sampler = ClockSampler(local) if rank == 0 else None
-    ms = timed(sparse_step, K)
-    clocks = sampler.stop() if sampler else None
     flop_step = 12.0 * T * D * F
-    value = replicas.aggregate_tflops(flop_step, K, ms)
-
     if args.quick:
+        ms = timed(sparse_step, K)
         if rank == 0:
-            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
-                              "ms_per_step": ms / K, "config": {"workload": args.workload}, "quick": True}))
+            print(json.dumps({"metric": METRIC, "value": replicas.aggregate_tflops(flop_step, K, ms), "unit": UNIT,
+                              "n_gpus": world, "steps": K, "ms_per_step": ms / K,
+                              "config": {"workload": args.workload}, "quick": True}))
         return
+
+    # ---- the timed region: exactly K sparse steps; the library records an event between its kernels
+    sampler = ClockSampler(local) if rank == 0 else None
+    with binding.StageTrace(13 * K) as tr:
+        ms = timed(sparse_step, K)
+    clocks = sampler.stop() if sampler else None
+    value = replicas.aggregate_tflops(flop_step, K, ms)
+    d = tr.durations_ms()
+    per = {}
+    for s in range(K):
+        for n, v in zip(TRACE_NAMES, d[13 * s: 13 * s + 12]):
+            if n:
+                per.setdefault(n, []).append(v)
+    path = _step_path(V, M) if not (args.flags & (binding.SF_FFN_UNFUSED_ACT | binding.SF_FFN_FUSED_ACT)) else \
+        ("fused" if args.flags & binding.SF_FFN_FUSED_ACT else "two_kernel")
+    not_launched = {"fused": {"vnm_sparsify", "transpose_W2", "pack_dy1"}, "two_kernel": {"transpose_W2", "pack_dy1"},
+                    "plain24": {"transpose_W2", "pack_dy1"}, "venom": set()}[path]   # empty trace intervals
+    kern_ms = {n: float(np.mean(v)) for n, v in per.items() if n not in not_launched}
+    kern_sum = float(sum(kern_ms.values()))
+
     for _ in range(2):
         dense_step()
     ms_dense = timed(dense_step, K)
     if binding.sf_check_status(ws) != binding.SF_OK:
         raise SystemExit("device status: a bounded wait expired")
 
-    # ---- per-kernel times inside the step (events recorded by the library between its kernels)
-    plain24 = (M <= 8)                       # activations multiplied as plain 2:4 operands (no row gather)
-    act_gemm = "gemm_sparse24" if plain24 else "gemm_venom"
-    names = ["prune24_W1", "gemm_sparse24_y1", "vnm_sparsify", "transpose_W2", f"{act_gemm}_y3",
-             None, "prune24_W2", "gemm_sparse24_dy1", "pack_dy1", f"{act_gemm}_dX", "gemm_dense_dW2", "gemm_dense_dW1"]
-    with binding.StageTrace(13 * K) as tr:
-        for _ in range(K):
-            sparse_step()
-    d = tr.durations_ms()
-    per = {}
-    for s in range(K):
-        seg = d[13 * s: 13 * s + 12]
-        for n, v in zip(names, seg):
-            if n:
-                per.setdefault(n, []).append(v)
-    kern_ms = {n: float(np.mean(v)) for n, v in per.items()}
-    if plain24:
-        kern_ms.pop("transpose_W2", None)    # not launched on this path (zero-length interval)
-        kern_ms.pop("pack_dy1", None)        # dy1 is packed by the dy1 product's epilogue on this path
-    unit = 2.0 * T * D * F                   # flop of one dense product
+    # ---- sustained: alternate K-step blocks of the two arms until each has run for the target time
+    sustained = None
+    if args.sustain_seconds > 0:
+        target_ms = args.sustain_seconds * 1e3
+        blocks_s, blocks_d = [], []
+        sampler2 = ClockSampler(local) if rank == 0 else None
+        while sum(blocks_s) < target_ms or sum(blocks_d) < target_ms:
+            blocks_s.append(timed(sparse_step, K))
+            blocks_d.append(timed(dense_step, K))
+            if len(blocks_s) > 2000:
+                break
+        clocks2 = sampler2.stop() if sampler2 else None
+        ms_s, ms_d = float(np.median(blocks_s)) / K, float(np.median(blocks_d)) / K
+        sustained = {"ms_per_step": ms_s, "value": flop_step * world / (ms_s / 1e3) / 1e12, "dense_step_ms": ms_d,
+                     "speedup_vs_dense_step": ms_d / ms_s, "blocks_per_arm": len(blocks_s), "steps_per_block": K,
+                     "seconds_per_arm": sum(blocks_s) / 1e3, "clocks": clocks2}
+
+    # ---- roofline fractions on ALGORITHMIC work, against the measured peaks
     peaks = _peaks()
-    # Kernel groups by the device function that runs them. Algorithmic work per launch: one dense
-    # product (2*T*D*F flop) for every product; the peak it is held against is the measured dense
-    # bf16 GEMM peak for the dense kernel, twice that for the 2:4 kernel (nominal 2:4 ratio), and
-    # M/4 times more for the condensed Venom kernel.
-    groups = {
-        "gemm_tc2_kernel<dense, MN-major A and B> (dW2, dW1)": (["gemm_dense_dW2", "gemm_dense_dW1"], 1.0),
-        "gemm_tc2_kernel<2:4 sparse> (y1, dy1" + (", y3, dX)" if plain24 else ")"):
-            (["gemm_sparse24_y1", "gemm_sparse24_dy1"] + ([f"{act_gemm}_y3", f"{act_gemm}_dX"] if plain24 else []), 2.0),
-    }
-    if not plain24:
-        groups["gemm_tc_kernel<venom> (y3, dX)"] = ([f"{act_gemm}_y3", f"{act_gemm}_dX"], 2.0 * M / 4.0)
-    tot = {g: sum(kern_ms[k] for k in ks) for g, (ks, _) in groups.items()}
-    dom = max(tot, key=tot.get)
-    ks, ratio = groups[dom]
-    avg_ms = tot[dom] / len(ks)
-    achieved = unit / (avg_ms / 1e3) / 1e12                      # dense-equivalent TFLOP/s of the kernel
-    peak = peaks["bf16_tflops_sustained"] * ratio
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        traffic = json.load(open(tpath)).get(dom.split(" (")[0])
-    roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": traffic,
-                "peak_source": peaks["source"] + " sustained bf16 GEMM" + (f" x {ratio:g} (nominal sparse ratio)" if ratio != 1.0 else ""),
-                "avg_launch_ms": avg_ms, "launches_per_step": len(ks),
-                "share_of_step": tot[dom] / sum(kern_ms.values()),
-                "other_groups": {g: {"avg_launch_ms": tot[g] / len(groups[g][0]),
-                                     "frac": unit / (tot[g] / len(groups[g][0]) / 1e3) / 1e12 / (peaks["bf16_tflops_sustained"] * groups[g][1])}
-                                 for g in groups if g != dom}}
+    unit = 2.0 * T * D * F                   # flop of one dense product
+    # Tensor work in units of one dense product: the 2:4 products do 2*T*D*F dense-equivalent flop at the 2:4 peak
+    # (2 x dense), the V:N:M products (4/M) of that whichever kernel runs them, the weight-gradient products
+    # 2*T*D*F at the dense peak. The step loop runs for a long time at the power cap, so the peak is the SUSTAINED
+    # measured bf16 GEMM figure (the burst figure is printed beside it).
+    P = peaks["bf16_tflops_sustained"]
+    prod = {"gemm_y1": (1.0, 2.0), "gemm_dy1": (1.0, 2.0), "gemm_y3": (4.0 / M, 2.0), "gemm_dX": (4.0 / M, 2.0),
+            "gemm_dW2": (1.0, 1.0), "gemm_dW1": (1.0, 1.0)}
+    products = {}
+    for n, (alg, ratio) in prod.items():
+        t = kern_ms[n] / 1e3
+        products[n] = {"ms": kern_ms[n], "algorithmic_dense_equiv_tflops": alg * unit / t / 1e12,
+                       "peak_tflops": P * ratio, "frac": alg * unit / t / 1e12 / (P * ratio),
+                       "frac_of_burst_peak": alg * unit / t / 1e12 / (peaks["bf16_tflops"] * ratio)}
+    if path == "fused":
+        products["gemm_y1"]["includes"] = "SquaredReLU + V:N:M selection in the epilogue"
+    groups = {"2:4 tensor kernels (y1, dy1, y3, dX)": (["gemm_y1", "gemm_dy1", "gemm_y3", "gemm_dX"], 2.0),
+              "dense tensor kernel (dW2, dW1)": (["gemm_dW2", "gemm_dW1"], 1.0)}
+    gstat = {}
+    for g, (ks, ratio) in groups.items():
+        t = sum(kern_ms[k] for k in ks) / 1e3
+        alg = sum(prod[k][0] for k in ks) * unit
+        gstat[g] = {"ms": t * 1e3, "launches_per_step": len(ks), "achieved": alg / t / 1e12, "peak": P * ratio,
+                    "frac": alg / t / 1e12 / (P * ratio), "share_of_step": t * 1e3 / kern_sum}
+    dom = max(gstat, key=lambda g: gstat[g]["ms"])
+    traffic = _traffic()
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": gstat[dom]["achieved"], "peak": gstat[dom]["peak"],
+                "unit": "TFLOP/s", "frac": gstat[dom]["frac"],
+                "traffic": traffic.get("kernels", {}).get(dom), "traffic_captured_on": traffic.get("captured_on"),
+                "peak_source": peaks["source"] + " sustained bf16 GEMM x 2 (nominal 2:4 ratio)" if "2:4" in dom
+                else peaks["source"] + " sustained bf16 GEMM",
+                "work": "algorithmic dense-equivalent flop: 2TDF per 2:4 product, (4/M) 2TDF per V:N:M product",
+                "avg_launch_ms": gstat[dom]["ms"] / gstat[dom]["launches_per_step"],
+                "launches_per_step": gstat[dom]["launches_per_step"], "share_of_step": gstat[dom]["share_of_step"],
+                "other_groups": {g: v for g, v in gstat.items() if g != dom}}
+    floor_units = 0.5 + 0.5 + 2 * (4.0 / M) * 0.5 + 2.0
+    floor_ms = floor_units * unit / (P * 1e12) * 1e3
+    step_floor = {"dense_product_units": floor_units, "floor_ms": floor_ms, "frac": floor_ms / (ms / K),
+                  "frac_sustained": floor_ms / sustained["ms_per_step"] if sustained else None,
+                  "speedup_ceiling_vs_dense": 6.0 / floor_units}
+
+    # ---- bandwidth kernels on algorithmic bytes (3.125 B/element; 2 + 4/M + 0.5/M (+ 4/M ReLU values) + colidx)
     hbm = peaks["hbm_gbs"]
-    prune_gbs = 3.125 * F * D / (kern_ms["prune24_W1"] / 1e3) / 1e9
-    # bytes the V:N:M kernel moves in the step: input, V:N:M-packed values + ReLU values + metadata
-    # (canonical and tensor-core order) + colidx, the two masked dense copies, and (M = 8) the 2:4 view
-    vnm_bytes = T * F * (2 + 4.0 / M + 4.0 / M + 1.0 / M) + (T // V) * (F // M) * 4 + 2 * T * F * 2
-    if plain24 and M == 8:
-        vnm_bytes += T * F * (1.0 + 0.25)
-    vnm_gbs = vnm_bytes / (kern_ms["vnm_sparsify"] / 1e3) / 1e9
-    launches_per_step = 9 if plain24 else 11
+    bw = {}
+    for n in ("prune24_W1", "prune24_W2"):
+        gbs = 3.125 * F * D / (kern_ms[n] / 1e3) / 1e9
+        bw[n] = {"ms": kern_ms[n], "algorithmic_bytes": 3.125 * F * D, "gbs": gbs, "frac_of_hbm": gbs / hbm,
+                 "traffic_over_algorithmic": (traffic.get("kernels", {}).get(n) or 0) / (3.125 * F * D) or None}
+    vnm_alg = T * F * (2 + 4.0 / M + 0.5 / M + 4.0 / M) + (T // V) * (F // M) * 4
+    if "vnm_sparsify" in kern_ms:
+        gbs = vnm_alg / (kern_ms["vnm_sparsify"] / 1e3) / 1e9
+        bw["vnm_sparsify"] = {"ms": kern_ms["vnm_sparsify"], "algorithmic_bytes": vnm_alg, "gbs": gbs,
+                              "frac_of_hbm": gbs / hbm,
+                              "traffic_over_algorithmic": (traffic.get("kernels", {}).get("vnm_sparsify") or 0) / vnm_alg or None}
+    else:
+        bw["vnm_sparsify"] = {"fused_into": "gemm_y1", "algorithmic_bytes": vnm_alg - 2.0 * T * F,
+                              "note": "no separate kernel: y1 never leaves the chip"}
+    launches_per_step = len(kern_ms)
 
     # ---- end to end through the host-buffer entry point (H2D of inputs and D2H of results timed)
     staging = torch.empty((binding.sf_ffn_host_staging_size(desc),), dtype=torch.uint8, device="cuda")
-    # (empty_like of a pinned tensor is pageable: ask for pinned results explicitly)
     hY, hdX = torch.empty_like(hX, pin_memory=True), torch.empty_like(hX, pin_memory=True)
     hgW1, hgW2 = torch.empty_like(hW1, pin_memory=True), torch.empty_like(hW2, pin_memory=True)
     assert all(t.is_pinned() for t in (hX, hW1, hW2, hdY, hY, hdX, hgW1, hgW2))
@@ -284,22 +348,25 @@ def run_ours(args, cfg):
     d2h = h2d
 
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "T": T, "D": D, "F": F, "V": V, "N": 2, "M": M,
-                   "prune_mode": args.prune_mode, "parallelism": f"replicas x{world}",
-                   "l2": "per-step inputs (402 MB of operands, >2 GB of intermediates) exceed the 126 MB L2"},
+                   "prune_mode": args.prune_mode, "flags": args.flags, "path": path,
+                   "parallelism": f"replicas x{world}",
+                   "l2": f"per-step operands ({(2 * T * D + 2 * F * D) * 2 / 1e6:.0f} MB) and intermediates exceed the 126 MB L2"},
         "dense_step_ms": ms_dense / K, "speedup_vs_dense_step": ms_dense / ms,
         "dense_step_tflops": replicas.aggregate_tflops(flop_step, K, ms_dense),
-        "kernel_ms": kern_ms,
-        "prune24_gbs": prune_gbs, "prune24_frac_of_hbm": prune_gbs / hbm,
-        "vnm_sparsify_gbs": vnm_gbs, "vnm_frac_of_hbm": vnm_gbs / hbm,
+        "sustained": sustained,
+        "kernel_ms": kern_ms, "kernel_ms_sum": kern_sum, "kernel_ms_sum_over_step": kern_sum / (ms / K),
+        "products": products, "step_floor": step_floor, "bandwidth_kernels": bw,
         "roofline": roofline, "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e / K, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * K,
     }
+    if abs(kern_sum / (ms / K) - 1.0) > 0.05:
+        out["kernel_ms_note"] = "per-kernel times do not add up to the step time within 5 %: breakdown rejected"
 
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:
         Ts = V
@@ -317,6 +384,111 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+# ---- stand-alone sweeps (BASELINE configs 2 and 3, and the paper's product micro-benchmarks) ------------
+
+def _time_cuda(fn, iters=20, warm=3):
+    import torch
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def run_sweep(args):
+    """One JSON line: `results` holds one entry per swept shape; value = the worst fraction of the
+    measured HBM bandwidth (bandwidth sweeps) or the 2:4 speed-up at the paper's shape (gemm_micro)."""
+    import torch
+    from paper_2602_06183_b200 import binding, build, synth
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    build.build()
+    peaks = _peaks()
+    hbm = peaks["hbm_gbs"]
+    dev = lambda b: torch.from_numpy(np.ascontiguousarray(b).view(np.int16)).cuda().view(torch.bfloat16)
+    iters = max(args.steps, 5)
+    results = []
+    if args.workload == "c2_prune":
+        for i, (rows, cols) in enumerate(synth.PRUNE_SWEEP_SHAPES):
+            w = dev(synth.prune_sweep_matrix(rows, cols, seed=1000 + i))
+            for group_dim in (1, 0):
+                for mode in (0, 1):
+                    outb = binding.sf_prune24_compress(w, group_dim, mode)
+                    ms = _time_cuda(lambda: binding.sf_prune24_compress(w, group_dim, mode, out=outb), iters, args.warmup)
+                    gbs = 3.125 * rows * cols / (ms / 1e3) / 1e9
+                    results.append({"rows": rows, "cols": cols, "group_dim": group_dim, "prune_mode": mode,
+                                    "us": ms * 1e3, "gbs": gbs, "frac_of_hbm": gbs / hbm})
+        metric, unit, value = "prune24_compress_min_frac_of_measured_hbm", "fraction", min(r["frac_of_hbm"] for r in results)
+        note = "3.125 algorithmic bytes per element; inputs >= 33 MB, the 28672 x 8192 case exceeds the L2"
+    elif args.workload == "c3_act":
+        Tn = Fn = 16384
+        p = dev(synth.act_sweep_matrix(Tn, Fn, seed=2000))
+        for V in (64, 128):
+            for M in (8, 16):
+                outb = binding.sf_vnm_sparsify_act(p, V, M)
+                ms = _time_cuda(lambda: binding.sf_vnm_sparsify_act(p, V, M, out=outb), iters, args.warmup)
+                nbytes = Tn * Fn * (2 + 4.0 / M + 0.5 / M + 4.0 / M) + (Tn // V) * (Fn // M) * 4
+                gbs = nbytes / (ms / 1e3) / 1e9
+                results.append({"T": Tn, "F": Fn, "V": V, "M": M, "us": ms * 1e3, "algorithmic_bytes_per_element": nbytes / (Tn * Fn),
+                                "gbs": gbs, "frac_of_hbm": gbs / hbm})
+        metric, unit, value = "vnm_sparsify_min_frac_of_measured_hbm", "fraction", min(r["frac_of_hbm"] for r in results)
+        note = "2 + 4/M + 0.5/M + 4/M (ReLU values) bytes per element + colidx; 537 MB input, larger than the L2"
+    else:
+        for (m, n, k) in [(4096, 16384, 4096), (16384, 8192, 4096), (8192, 4096, 16384)]:
+            A = torch.randn((m, k), device="cuda").to(torch.bfloat16)
+            B = torch.randn((n, k), device="cuda").to(torch.bfloat16)
+            Cm = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
+            wsb = torch.zeros((binding.sf_gemm_workspace_size(m, k),), dtype=torch.uint8, device="cuda")
+            ms_d = _time_cuda(lambda: binding.sf_gemm_dense(A, True, B, True, C_out=Cm, workspace=wsb), iters, args.warmup)
+            vals, meta, _ = binding.sf_prune24_compress(A, 1, 0)
+            ms_p = _time_cuda(lambda: binding.sf_prune24_compress(A, 1, 0, out=(vals, meta, None)), iters, args.warmup)
+            ms_s = _time_cuda(lambda: binding.sf_gemm_sparse24_rm(vals, meta, B, True, C_out=Cm, workspace=wsb), iters, args.warmup)
+            fl = 2.0 * m * n * k
+            results.append({"product": "2:4 vs dense", "shape_mnk": [m, n, k], "dense_ms": ms_d, "dense_tflops": fl / ms_d / 1e9,
+                            "sparse24_ms": ms_s, "sparse24_dense_equiv_tflops": fl / ms_s / 1e9, "prune_ms": ms_p,
+                            "speedup_gemm_only": ms_d / ms_s, "speedup_with_prune": ms_d / (ms_s + ms_p)})
+            del A, B, Cm, vals, meta
+        Tn, Fn, Nn = 8192, 16384, 4096
+        A = torch.randn((Tn, Fn), device="cuda").to(torch.bfloat16)
+        Bd = torch.randn((Nn, Fn), device="cuda").to(torch.bfloat16)
+        Cd = torch.empty((Tn, Nn), dtype=torch.bfloat16, device="cuda")
+        wsd = torch.zeros((binding.sf_gemm_workspace_size(Tn, Fn),), dtype=torch.uint8, device="cuda")
+        ms_dense = _time_cuda(lambda: binding.sf_gemm_dense(A, True, Bd, True, C_out=Cd, workspace=wsd), iters, args.warmup)
+        del A, Bd, Cd
+        for M in (8, 16, 32, 64):
+            P = dev(synth.normal_bf16((Tn, Fn), 0.0, 1.0, seed=7))
+            vals, meta, colidx, _, _ = binding.sf_vnm_sparsify_act(P, 128, M)
+            Bt = torch.randn((Fn, Nn), device="cuda").to(torch.bfloat16)
+            Cm = torch.empty((Tn, Nn), dtype=torch.bfloat16, device="cuda")
+            wsb = torch.zeros((binding.sf_gemm_workspace_size(Tn, Fn),), dtype=torch.uint8, device="cuda")
+            ms_v = _time_cuda(lambda: binding.sf_gemm_venom(vals, meta, colidx, Bt, 128, M, C_out=Cm, workspace=wsb), iters, args.warmup)
+            results.append({"product": "Venom vs dense", "T": Tn, "F": Fn, "N": Nn, "V": 128, "M": M,
+                            "sparsity_pct": 100.0 * (1 - 2.0 / M), "ms": ms_v, "dense_ms": ms_dense,
+                            "speedup_vs_dense": ms_dense / ms_v})
+        metric, unit, value = "sparse24_gemm_speedup_vs_dense_at_4096x16384x4096", "ratio", results[0]["speedup_gemm_only"]
+        note = "Section 5.2.3's micro-benchmark shape first; Venom products at Table 5's sparsities"
+    print(json.dumps({"metric": metric, "value": value, "unit": unit, "n_gpus": 1, "steps": iters, "warmup": args.warmup,
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": args.workload, "note": note, "hbm_peak_gbs": hbm, "peak_source": peaks["source"]},
+                      "results": results, "gpu_launches": iters * len(results)}))
+
+
+def _spawn_replicas(args):
+    """`--gpus N` outside torchrun: start the N ranks (one per GPU of this node) and relay their output."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -325,11 +497,22 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4_d4096")
     ap.add_argument("--prune-mode", type=int, default=0)
+    ap.add_argument("--flags", type=int, default=0, help="sf_ffn_flags of the step (0 = the library's defaults)")
+    ap.add_argument("--sustain-seconds", type=float, default=1.0,
+                    help="time per arm of the alternating sparse/dense blocks (0 = skip)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true",
                     help="sparse step only (no dense step, trace, e2e, CPU baseline): for profiler captures")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        raise SystemExit(_spawn_replicas(args))
     from paper_2602_06183_b200 import synth
+    if args.workload in SWEEP_WORKLOADS:
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the reference arm times the FFN step workloads only"}))
+            return
+        run_sweep(args)
+        return
     cfg = synth.FFN_CONFIGS[args.workload]
     if args.impl == "reference":
         run_reference(args, cfg)

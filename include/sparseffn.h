@@ -311,7 +311,9 @@ SF_API int sf_selftest_wait_expiry(void* workspace, int64_t budget_clocks, void*
  * array of `capacity` cudaEvent_t handles (created with timing enabled) that must stay valid until
  * tracing is switched off with capacity 0. While set, every FFN step call records one event
  * before its first kernel and one after each kernel, in launch order, on the call's stream:
- *   sparse fwd: 6 events (prune W1 | y1 product | V:N:M | W2 transpose | y3 product)
+ *   sparse fwd: 6 events (prune W1 | y1 product | V:N:M | W2 transpose | y3 product); intervals of
+ *               kernels a path does not launch are empty (M <= 8: no W2 transpose; M == 8 with the
+ *               selection fused into the y1 product: no V:N:M kernel)
  *   sparse bwd: 7 events (prune W2 | dy1 product | pack | dX product | dW2 product | dW1 product);
  *               for M <= 8 the dy1 product packs its own output and the pack interval is empty
  *   dense fwd: 3 events, dense bwd: 5 events.

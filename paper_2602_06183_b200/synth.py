@@ -29,18 +29,21 @@ __all__ = [
 # (T, D, F, V, N, M, sigma_w) per named FFN configuration.
 FFN_CONFIGS = {
     "c1_small": dict(T=1024, D=256, F=1024, V=64, N=2, M=8, sigma_w=0.02, seed=0),
-    "c4_d4096": dict(T=8192, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
-    # the same layer with the block height of the paper's Table 5 (V = 64)
-    "c4_d4096_v64": dict(T=8192, D=4096, F=16384, V=64, N=2, M=8, sigma_w=0.02, seed=4),
+    # the d_model = 4096 layer; the configuration says "V:2:8" and leaves V free: V = 64 is the block height of
+    # the paper's Table 5, and three such blocks fill one token tile of the fused y1 epilogue
+    "c4_d4096": dict(T=8192, D=4096, F=16384, V=64, N=2, M=8, sigma_w=0.02, seed=4),
+    # the same layer with 128-token blocks (SquaredReLU + V:N:M then run as a second kernel by default)
+    "c4_d4096_v128": dict(T=8192, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
     # one eighth of c4's tokens with the full-size layer: weights (134 MB each) still exceed the
     # L2, device footprint ~1.5 GB; used for profiler captures that must stay small
-    "c4_slice": dict(T=1024, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
-    "c4_slice_v64": dict(T=1024, D=4096, F=16384, V=64, N=2, M=8, sigma_w=0.02, seed=4),
+    "c4_slice": dict(T=1024, D=4096, F=16384, V=64, N=2, M=8, sigma_w=0.02, seed=4),
+    "c4_slice_v128": dict(T=1024, D=4096, F=16384, V=128, N=2, M=8, sigma_w=0.02, seed=4),
     # the same slice with groups of 16 (87.5 % sparse activations): exercises the condensed Venom products
     "c4_slice_m16": dict(T=1024, D=4096, F=16384, V=128, N=2, M=16, sigma_w=0.02, seed=4),
     # c4 with groups of 16 (Table 5's 87.5 % row): the full-size case of the condensed Venom products
     "c4_d4096_m16": dict(T=8192, D=4096, F=16384, V=128, N=2, M=16, sigma_w=0.02, seed=4),
-    "c5_d8192": dict(T=16384, D=8192, F=28672, V=128, N=2, M=8, sigma_w=0.015, seed=5),
+    "c5_d8192": dict(T=16384, D=8192, F=28672, V=64, N=2, M=8, sigma_w=0.015, seed=5),
+    "c5_d8192_v128": dict(T=16384, D=8192, F=28672, V=128, N=2, M=8, sigma_w=0.015, seed=5),
 }
 
 PRUNE_SWEEP_SHAPES = [(4096, 4096), (14336, 4096), (4096, 16384), (28672, 8192)]

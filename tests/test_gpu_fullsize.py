@@ -36,7 +36,7 @@ def _full_step(cfg, flags):
     return (X, W1, W2, dY), desc, gctx.t, gws.t, (Y, gX, gW1, gW2)
 
 
-@pytest.mark.parametrize("name", ["c4_d4096", "c4_d4096_v64", "c4_d4096_m16", "c5_d8192"])
+@pytest.mark.parametrize("name", ["c4_d4096", "c4_d4096_v128", "c4_d4096_m16", "c5_d8192"])
 def test_ffn_step_full_size_sampled(name):
     cfg = synth.FFN_CONFIGS[name]
     T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
