@@ -297,6 +297,67 @@ SF_API int sf_ffn_bwd_scheduled(const sf_schedule* schedule, int64_t step, const
                          const void* fwd_ctx, size_t fwd_ctx_bytes, void* dX, void* dW1, void* dW2,
                          void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * The routed step: neuron-level experts that produce the V:N:M pattern (Section 3.1, Algorithm 3
+ * "Convert Activation to Venom", Figure 4; Section 3.2.2 steps 1-3; Algorithm 1 line 6 `MoEToVenom`).
+ *
+ * Offline, the hidden features are clustered into E non-overlapping experts of Fe = F / E features
+ * each and renumbered expert-major (rows of W1 and columns of W2 together: a reparametrisation of
+ * the layer), so that expert e owns features [e Fe, (e+1) Fe); `means` holds the E cluster centres
+ * as bf16 [E, D]. V:N:M keeps four of every M columns, hence E = M / 4 (M = 64: sixteen experts).
+ * Per step each token goes to the expert with the largest x . mean (top-1, ties to the lower
+ * expert; float32 accumulation), tokens are grouped by expert, and every product touches only the
+ * token's expert block: y1, y2 = 2:4(ReLU(y1)^2) inside every four features of the block (greedy
+ * magnitude rule of Section 2.3), Y = y2 W2^T, and Algorithm 2 on that mask. Interleaving the
+ * expert blocks four features at a time gives the V:N:M matrix of Section 2.3 with the expert's
+ * columns 4e..4e+3 kept in every group. Each product costs 1 / E of its dense counterpart (the
+ * 2:4 ones half of that again); the token grouping is one gather pass per operand.
+ *
+ * Shape rules: T, D multiples of 256; 1 <= E <= 16; F / E a multiple of 256; T <= 2^20.
+ * flags: SF_FFN_SAVE_Y1 only. Buffers as for the step above (sizes from
+ * sf_routed_ffn_workspace_size; first 256 bytes of the workspace = status word).
+ *
+ * sf_router_route:   expert int32 [T] (and, optionally, logits float32 [T, E]) for X [T, D].
+ * sf_routed_ffn_fwd: `forced_expert` (optional DEVICE int32 [T]) replaces the routing decision, for
+ *                    stage-wise comparison with an implementation that accumulates the logits
+ *                    differently; NULL = route with `means`.
+ * sf_routed_ctx_view: device pointers into the context / workspace. Rows of the row-indexed fields
+ *                    follow the grouped token order: SF_RCTX_SRC_OF_ROW gives the token of a row (-1 on
+ *                    padding rows, which hold zeros), SF_RCTX_ROW_OF_TOKEN the inverse,
+ *                    SF_RCTX_SEGMENTS = int32 [2E + 1]: first row of each expert's segment, total rows,
+ *                    then the token count of each expert.
+ */
+typedef struct sf_router_desc {
+  int64_t T, D, F;
+  int32_t E;
+  int32_t prune_mode;  /* as sf_ffn_desc */
+  int32_t flags;       /* SF_FFN_SAVE_Y1 or 0 */
+  int32_t reserved;
+} sf_router_desc;
+typedef enum sf_routed_ctx_field {
+  SF_RCTX_EXPERT = 0,       /* int32 [T] */
+  SF_RCTX_ROW_OF_TOKEN = 1, /* int32 [T] */
+  SF_RCTX_SRC_OF_ROW = 2,   /* int32 [rows_max], rows_max = T + 256 E rounded up to 256 */
+  SF_RCTX_SEGMENTS = 3,     /* int32 [2E + 1] */
+  SF_RCTX_LOGITS = 4,       /* float32 [T, E] (written when the step routes itself) */
+  SF_RCTX_Y2_VALS = 5,      /* bf16 [rows_max, Fe/2]: kept activations, two per four features of the expert block */
+  SF_RCTX_RELU_VALS = 6,    /* bf16 [rows_max, Fe/2]: ReLU(y1) at the same positions */
+  SF_RCTX_META = 7,         /* uint16 [rows_max, Fe/16]: canonical 2:4 metadata of those positions */
+  SF_RCTX_Y1 = 8,           /* bf16 [rows_max, Fe] (only with SF_FFN_SAVE_Y1) */
+  SF_RCTX_DY1_VALS = 9      /* bf16 [rows_max, Fe/2], in the WORKSPACE after sf_routed_ffn_bwd */
+} sf_routed_ctx_field;
+SF_API int sf_router_route(const void* X, const void* means, int64_t T, int64_t D, int E, void* expert,
+                           void* logits, void* stream);
+SF_API int sf_routed_ffn_workspace_size(const sf_router_desc* desc, size_t* fwd_ctx_bytes, size_t* workspace_bytes);
+SF_API int sf_routed_ffn_fwd(const sf_router_desc* desc, const void* X, const void* W1, const void* W2,
+                             const void* means, const void* forced_expert, void* Y, void* fwd_ctx,
+                             size_t fwd_ctx_bytes, void* workspace, size_t workspace_bytes, void* stream);
+SF_API int sf_routed_ffn_bwd(const sf_router_desc* desc, const void* dY, const void* X, const void* W1,
+                             const void* W2, const void* fwd_ctx, size_t fwd_ctx_bytes, void* dX, void* dW1,
+                             void* dW2, void* workspace, size_t workspace_bytes, void* stream);
+SF_API int sf_routed_ctx_view(const sf_router_desc* desc, const void* fwd_ctx_or_workspace, int field,
+                              const void** ptr, size_t* bytes);
+
 /* Bounded-wait self-test (the paper has no counterpart). Every device-side wait of the tensor-core
  * kernels gives up after a clock budget, raises the status word at the start of the workspace and
  * lets its CTA leave; sf_check_status then reports SF_ERR_TIMEOUT. This call runs that mechanism

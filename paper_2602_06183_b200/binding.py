@@ -31,6 +31,15 @@ class sf_ffn_desc(C.Structure):
                 ("prune_mode", C.c_int32), ("flags", C.c_int32)]
 
 
+class sf_router_desc(C.Structure):
+    _fields_ = [("T", C.c_int64), ("D", C.c_int64), ("F", C.c_int64), ("E", C.c_int32), ("prune_mode", C.c_int32),
+                ("flags", C.c_int32), ("reserved", C.c_int32)]
+
+
+(SF_RCTX_EXPERT, SF_RCTX_ROW_OF_TOKEN, SF_RCTX_SRC_OF_ROW, SF_RCTX_SEGMENTS, SF_RCTX_LOGITS, SF_RCTX_Y2_VALS,
+ SF_RCTX_RELU_VALS, SF_RCTX_META, SF_RCTX_Y1, SF_RCTX_DY1_VALS) = range(10)
+
+
 class sf_schedule(C.Structure):
     _fields_ = [("warmup_steps", C.c_int64), ("sparse_steps", C.c_int64), ("total_steps", C.c_int64)]
 
@@ -77,6 +86,11 @@ _SIGNATURES = {
                                     _sz, _vp, _sz, _vp]),
     "sf_ffn_bwd_scheduled": (_i32, [C.POINTER(sf_schedule), _i64, C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp,
                                     _sz, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "sf_router_route": (_i32, [_vp, _vp, _i64, _i64, _i32, _vp, _vp, _vp]),
+    "sf_routed_ffn_workspace_size": (_i32, [C.POINTER(sf_router_desc), C.POINTER(_sz), C.POINTER(_sz)]),
+    "sf_routed_ffn_fwd": (_i32, [C.POINTER(sf_router_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
+    "sf_routed_ffn_bwd": (_i32, [C.POINTER(sf_router_desc), _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "sf_routed_ctx_view": (_i32, [C.POINTER(sf_router_desc), _vp, _i32, C.POINTER(_vp), C.POINTER(_sz)]),
     "sf_selftest_wait_expiry": (_i32, [_vp, _i64, _vp]),
     "sf_trace_set": (_i32, [C.POINTER(_vp), _i32]),
     "sf_trace_count": (_i32, []),
@@ -329,6 +343,54 @@ def sf_ffn_step_host(desc, dense: bool, hX, hW1, hW2, hdY, hY, hdX, hdW1, hdW2, 
     _check(lib().sf_ffn_step_host(C.byref(desc), int(dense), _ptr(hX), _ptr(hW1), _ptr(hW2), _ptr(hdY), _ptr(hY),
                                   _ptr(hdX), _ptr(hdW1), _ptr(hdW2), _ptr(staging), _ptr(fwd_ctx), _nbytes(fwd_ctx),
                                   _ptr(workspace), _nbytes(workspace), _stream(stream)), "sf_ffn_step_host")
+
+
+# ---- routed step (neuron-level experts) ------------------------------------------------------------
+
+def make_router_desc(T, D, F, E, prune_mode=0, flags=0) -> sf_router_desc:
+    return sf_router_desc(T, D, F, E, prune_mode, flags, 0)
+
+
+def sf_router_route(X: torch.Tensor, means: torch.Tensor, want_logits: bool = True, stream=None):
+    """X [T, D], means [E, D] (16-bit tensors). Returns (expert int32 [T], logits float32 [T, E] or None)."""
+    T, D = X.shape
+    E = means.shape[0]
+    expert = torch.empty((T,), dtype=torch.int32, device=X.device)
+    logits = torch.empty((T, E), dtype=torch.float32, device=X.device) if want_logits else None
+    _check(lib().sf_router_route(_ptr(X), _ptr(means), T, D, E, _ptr(expert), _ptr(logits), _stream(stream)),
+           "sf_router_route")
+    return expert, logits
+
+
+def sf_routed_ffn_workspace_size(desc: sf_router_desc):
+    a, b = _sz(), _sz()
+    _check(lib().sf_routed_ffn_workspace_size(C.byref(desc), C.byref(a), C.byref(b)), "sf_routed_ffn_workspace_size")
+    return a.value, b.value
+
+
+def sf_routed_ffn_fwd(desc, X, W1, W2, means, Y, fwd_ctx, workspace, forced_expert=None, stream=None):
+    _check(lib().sf_routed_ffn_fwd(C.byref(desc), _ptr(X), _ptr(W1), _ptr(W2), _ptr(means), _ptr(forced_expert), _ptr(Y),
+                                   _ptr(fwd_ctx), _nbytes(fwd_ctx), _ptr(workspace), _nbytes(workspace),
+                                   _stream(stream)), "sf_routed_ffn_fwd")
+
+
+def sf_routed_ffn_bwd(desc, dY, X, W1, W2, fwd_ctx, dX, dW1, dW2, workspace, stream=None):
+    _check(lib().sf_routed_ffn_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(W1), _ptr(W2), _ptr(fwd_ctx),
+                                   _nbytes(fwd_ctx), _ptr(dX), _ptr(dW1), _ptr(dW2), _ptr(workspace),
+                                   _nbytes(workspace), _stream(stream)), "sf_routed_ffn_bwd")
+
+
+_RCTX_DTYPES = {SF_RCTX_EXPERT: torch.int32, SF_RCTX_ROW_OF_TOKEN: torch.int32, SF_RCTX_SRC_OF_ROW: torch.int32,
+                SF_RCTX_SEGMENTS: torch.int32, SF_RCTX_LOGITS: torch.float32, SF_RCTX_Y2_VALS: torch.bfloat16,
+                SF_RCTX_RELU_VALS: torch.bfloat16, SF_RCTX_META: torch.int16, SF_RCTX_Y1: torch.bfloat16,
+                SF_RCTX_DY1_VALS: torch.bfloat16}
+
+
+def sf_routed_ctx_view(desc, buf: torch.Tensor, field: int) -> torch.Tensor:
+    p, n = _vp(), _sz()
+    _check(lib().sf_routed_ctx_view(C.byref(desc), _ptr(buf), field, C.byref(p), C.byref(n)), "sf_routed_ctx_view")
+    off = p.value - buf.data_ptr()
+    return buf[off:off + n.value].view(_RCTX_DTYPES[field])
 
 
 def make_schedule(warmup_steps: int, sparse_steps: int, total_steps: int) -> sf_schedule:

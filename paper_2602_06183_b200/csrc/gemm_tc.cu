@@ -81,14 +81,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __host__ __device__ constexpr bool is_drelu_t(int epi) { return epi == EPI_DRELU_T || epi == EPI_DRELU24_T; }
 
 template <int kEpi, int kTileN = BN>
-__device__ __forceinline__ void epi_prefetch(const GemmArgs& args, int64_t m0, int64_t n0, int q, int lane,
+__device__ __forceinline__ void epi_prefetch(const GemmArgs& args, int64_t m0, int64_t n0, int64_t n_limit, int q, int lane,
                                              uint4 (&ax)[is_drelu_t(kEpi) ? kTileN / 32 : 1][4]) {
   if (kEpi == EPI_DRELU24_T) {
     // ReLU(y1) in the 2:4 layout of the activation mask: four stored values and two position nibbles per
     // eight features; (x, y) = values, z = nibbles
 #pragma unroll
     for (int ch = 0; ch < kTileN / 32; ++ch) {
-      if (n0 + ch * 32 >= args.N) break;
+      if (n0 + ch * 32 >= n_limit) break;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int64_t token = n0 + ch * 32 + i * 8 + (lane >> 2), f = m0 + q * 32 + (lane & 3) * 8;
@@ -102,7 +102,7 @@ __device__ __forceinline__ void epi_prefetch(const GemmArgs& args, int64_t m0, i
   if (kEpi == EPI_DRELU_T) {
 #pragma unroll
     for (int ch = 0; ch < kTileN / 32; ++ch) {
-      if (n0 + ch * 32 >= args.N) break;
+      if (n0 + ch * 32 >= n_limit) break;
 #pragma unroll
       for (int i = 0; i < 4; ++i)
         ax[kEpi == EPI_DRELU_T ? ch : 0][i] = __ldg(reinterpret_cast<const uint4*>(
@@ -113,13 +113,13 @@ __device__ __forceinline__ void epi_prefetch(const GemmArgs& args, int64_t m0, i
 }
 
 template <int kEpi, int kTileN = BN>
-__device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0, int q, int lane,
-                                         uint8_t* my_stage,
+__device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0, int64_t n_limit,
+                                         int q, int lane, uint8_t* my_stage,
                                          const uint4 (&ax)[is_drelu_t(kEpi) ? kTileN / 32 : 1][4]) {
   const int64_t row = m0 + q * 32 + lane;                                  // this thread's D row
   auto chunk = [&](int ch, const uint4 (&a4)[4], const uint32_t (&v)[32]) {
     const int64_t col0 = n0 + ch * 32;
-    if (col0 >= args.N) return;                                            // ragged last tile (warp-uniform)
+    if (col0 >= n_limit) return;                                           // ragged last tile (warp-uniform)
     if (kEpi == EPI_STORE || kEpi == EPI_SQRELU || kEpi == EPI_DRELU) {
       uint16_t* crow = reinterpret_cast<uint16_t*>(args.C) + row * args.ldc + col0;
       if (kEpi == EPI_STORE) {
@@ -209,6 +209,30 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
       for (int i = 0; i < 4; ++i) {
         const int t = i * 8 + (lane >> 2), seg = lane & 3;
         const uint4 o = *reinterpret_cast<const uint4*>(my_stage + t * kEpiStageRow + seg * 16);
+        if (kEpi == EPI_ACT24_T) {
+          // o = y1 of eight neighbouring features of one token: SquaredReLU, then the two larger of every four
+          const int64_t token = col0 + t, fl = m0 + q * 32 + seg * 8, Fe = args.M;
+          const uint32_t r0w = bf2_relu(o.x), r1w = bf2_relu(o.y), r2w = bf2_relu(o.z), r3w = bf2_relu(o.w);
+          uint32_t pa, pb;
+          const uint32_t na = top2of4_packed(bf2_sq(r0w), bf2_sq(r1w), &pa), nb = top2of4_packed(bf2_sq(r2w), bf2_sq(r3w), &pb);
+          const uint32_t ra = __byte_perm(r0w, r1w, 0x1010u + (na & 3u) * 0x22u + (na >> 2) * 0x2200u);
+          const uint32_t rb = __byte_perm(r2w, r3w, 0x1010u + (nb & 3u) * 0x22u + (nb >> 2) * 0x2200u);
+          const int64_t pv = (token * (Fe >> 1) + (fl >> 1)) >> 2;             // 8-byte units
+          reinterpret_cast<uint2*>(args.vn_vals24)[pv] = make_uint2(pa, pb);
+          reinterpret_cast<uint2*>(args.vn_relu24)[pv] = make_uint2(ra, rb);
+          uint32_t mb = na | (nb << 4);
+          reinterpret_cast<uint4*>(args.vn_dense)[(token * Fe + fl) >> 3] = expand24_x8(make_uint2(pa, pb), mb);
+          if (args.vn_y1) reinterpret_cast<uint4*>(args.vn_y1)[(token * Fe + fl) >> 3] = o;
+          // metadata: one byte per lane, four neighbouring lanes hold the warp's 32 features of this token
+          mb |= __shfl_down_sync(0xFFFFFFFFu, mb, 1) << 8;
+          const uint32_t mb32 = (mb & 0xFFFFu) | (__shfl_down_sync(0xFFFFFFFFu, mb, 2) << 16);
+          const int64_t kw = (m0 + q * 32) >> 4;
+          if (seg == 0) reinterpret_cast<uint32_t*>(args.vn_meta24)[(token * (Fe >> 4) + kw) >> 1] = mb32;
+          if ((seg & 1) == 0)
+            *reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(args.vn_meta24_hw) +
+                                         meta_hw_offset(token, kw + (seg >> 1), Fe)) = (uint16_t)mb;
+          continue;
+        }
         if (kEpi != EPI_DRELU24_T || args.C != nullptr)
           *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.C) + (col0 + t) * args.ldc + m0 + q * 32 + seg * 8) = o;
         if (pack) {
@@ -285,8 +309,8 @@ constexpr int kVnmEpiWarps = 8;                                  // two sets of 
 __host__ __device__ constexpr int vnm_epi_bytes(int V) { return kVnmEpiWarps * vnm_warp_bytes(V); }
 
 template <int kTileN, int kV>
-__device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0, int q,
-                                              int lane, uint8_t* wsm, uint64_t* tmem_empty_bar) {
+__device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0,
+                                              int64_t n_limit, int q, int lane, uint8_t* wsm, uint64_t* tmem_empty_bar) {
   uint32_t* stage = reinterpret_cast<uint32_t*>(wsm);                     // [kV / 2][32 features]
   uint8_t* cidx = wsm + vnm_stage_bytes(kV);                              // [4 groups][4]
   uint4* sel_tab = reinterpret_cast<uint4*>(wsm + vnm_stage_bytes(kV) + 16);   // [4 groups][7]
@@ -296,7 +320,7 @@ __device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t tad
   const int jm = lane & 7, gl = lane & 3;
   constexpr int kBlocks = kTileN / kV;
   int nblk = kBlocks;
-  while (nblk > 0 && n0 + (int64_t)(nblk - 1) * kV >= args.N) --nblk;      // ragged last tile: whole blocks only
+  while (nblk > 0 && n0 + (int64_t)(nblk - 1) * kV >= n_limit) --nblk;     // ragged last tile: whole blocks only
   if (nblk == 0) {
     tc_fence_before();
     __syncwarp();
@@ -680,11 +704,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
       // The dy1 epilogue multiplies by a [token, feature] tile of the saved activations; its loads do
       // not depend on the accumulator, so they are issued before the wait and land during the main loop.
       uint4 ax[is_drelu_t(kEpi) ? BN / 32 : 1][4];
-      epi_prefetch<kEpi>(args, m0, n0, q, lane, ax);
+      epi_prefetch<kEpi>(args, m0, n0, args.N, q, lane, ax);
       if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
-      epi_tile<kEpi>(args, taddr, m0, n0, q, lane, my_stage, ax);
+      epi_tile<kEpi>(args, taddr, m0, n0, args.N, q, lane, my_stage, ax);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&ctl->tmem_empty[acc]);
@@ -745,6 +769,19 @@ struct SmemCtl2 {
   int abort_flag;
 };
 
+// The tile a CTA pair works on: from the regular raster, or from a device-built table (grouped products).
+template <int kBN>
+__device__ __forceinline__ GemmTile get_tile(const GemmArgs& args, int tile, int num_m, int num_n, int nkb_full) {
+  if (args.tile_table) {
+    const int4* p = reinterpret_cast<const int4*>(args.tile_table + tile);
+    const int4 a = __ldg(p), b = __ldg(p + 1);
+    return GemmTile{a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+  }
+  int mt, nt;
+  tile_coords(tile, num_m, num_n, mt, nt);
+  return GemmTile{mt * 256, 0, nt * kBN, 0, nkb_full, mt * 256, nt * kBN, (int)args.N};
+}
+
 __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
   return (static_cast<uint64_t>(hi) << 32) | lo;
 }
@@ -784,8 +821,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   const uint32_t rank = cluster_ctarank();               // 0 = leader
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const int num_m_tiles = args.num_m_tiles, num_n_tiles_ = args.num_n_tiles;   // 256-row tiles
-  const int num_tiles = num_m_tiles * num_n_tiles_;
-  const int nkb = (int)(args.K / kBK);
+  const int num_tiles = args.tile_table ? __ldg(args.num_tiles_dev) : num_m_tiles * num_n_tiles_;
+  const int nkb_full = (int)(args.K / kBK);
 
   if (threadIdx.x == 0) {
     prefetch_tmap(&tmapA);
@@ -826,10 +863,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     uint32_t stage = 0, phase = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-      int mt, nt;
-      tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
-      const int m0 = mt * 256 + (int)rank * 128;         // this CTA's rows of A / D
-      const int nb0 = nt * kBN + (int)rank * (kBN / 2);  // this CTA's columns of B
+      const GemmTile tc = get_tile<kBN>(args, tile, num_m_tiles, num_n_tiles_, nkb_full);
+      const int m0 = tc.a_row + (int)rank * 128;         // this CTA's rows of A / D
+      const int nb0 = tc.b_row + (int)rank * (kBN / 2);  // this CTA's columns of B
+      const int nkb = tc.nkb, ak0 = tc.a_k0, bk0 = tc.b_k0;
       for (int kb = 0; kb < nkb; ++kb) {
         if (!mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
         if (lane == 0) {
@@ -848,17 +885,17 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
             if (kExpand == 1) {
               // packed A: this CTA's 128 features of 64 tokens, into the staging ring (own barrier)
             } else if (!kAMN) {
-              tma_load_2d_2cta(sA, &tmapA, bar, kb * 64, m0);
+              tma_load_2d_2cta(sA, &tmapA, bar, ak0 + kb * 64, m0);
             } else {
-              tma_load_2d_2cta(sA, &tmapA, bar, m0, kb * 64);
-              tma_load_2d_2cta(sA + 8192, &tmapA, bar, m0 + 64, kb * 64);
+              tma_load_2d_2cta(sA, &tmapA, bar, m0, ak0 + kb * 64);
+              tma_load_2d_2cta(sA + 8192, &tmapA, bar, m0 + 64, ak0 + kb * 64);
             }
             if (kExpand == 2) {
             } else if (!kBMN) {
-              tma_load_2d_2cta(sB, &tmapB, bar, kb * 64, nb0);                 // box {64 k, 128 n}
+              tma_load_2d_2cta(sB, &tmapB, bar, bk0 + kb * 64, nb0);           // box {64 k, 128 n}
             } else {
-              tma_load_2d_2cta(sB, &tmapB, bar, nb0, kb * 64);                 // box {64 n, 64 k}
-              tma_load_2d_2cta(sB + 8192, &tmapB, bar, nb0 + 64, kb * 64);
+              tma_load_2d_2cta(sB, &tmapB, bar, nb0, bk0 + kb * 64);           // box {64 n, 64 k}
+              tma_load_2d_2cta(sB + 8192, &tmapB, bar, nb0 + 64, bk0 + kb * 64);
             }
             if (kExpand) {
               const int f0 = kExpand == 1 ? m0 : nb0;                          // first feature of this CTA's half
@@ -868,16 +905,16 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
               tma_load_2d(sP + 8192, &tmapMeta, &ctl->pk_full[stage], f0 >> 4, kb * 64); // metadata: box {8, 64}
             }
           } else {
-            tma_load_2d_2cta(sA, &tmapA, bar, kb * 64, m0);                    // stored values: box {64, 128}
+            tma_load_2d_2cta(sA, &tmapA, bar, (ak0 >> 1) + kb * 64, m0);       // stored values: box {64, 128}
             // metadata atoms are rows of 2 x 1 KB in a [2 * atoms, 256] uint32 view
-            const int atom = (m0 >> 7) * nkb + kb;
+            const int atom = (m0 >> 7) * nkb_full + (ak0 >> 7) + kb;
             tma_load_2d_2cta(sM, &tmapMeta, bar, 0, 2 * atom);
             if (!kBMN) {
-              tma_load_2d_2cta(sB, &tmapB, bar, kb * 128, nb0);                // two 64-wide K slabs
-              tma_load_2d_2cta(sB + kBSlabBytes, &tmapB, bar, kb * 128 + 64, nb0);
+              tma_load_2d_2cta(sB, &tmapB, bar, bk0 + kb * 128, nb0);          // two 64-wide K slabs
+              tma_load_2d_2cta(sB + kBSlabBytes, &tmapB, bar, bk0 + kb * 128 + 64, nb0);
             } else {
-              tma_load_2d_2cta(sB, &tmapB, bar, nb0, kb * 128);                // two chunks {64 n, 128 k}
-              tma_load_2d_2cta(sB + 16384, &tmapB, bar, nb0 + 64, kb * 128);
+              tma_load_2d_2cta(sB, &tmapB, bar, nb0, bk0 + kb * 128);          // two chunks {64 n, 128 k}
+              tma_load_2d_2cta(sB + 16384, &tmapB, bar, nb0 + 64, bk0 + kb * 128);
             }
           }
         }
@@ -906,6 +943,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
       uint32_t acc = 0, acc_phase = 0;
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        const int nkb = args.tile_table ? __ldg(&args.tile_table[tile].nkb) : nkb_full;
         if (!mbar_wait(&ctl->tmem_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * kBN;
@@ -949,7 +987,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     uint32_t stage = 0, phase = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-      for (int kb = 0; kb < nkb; ++kb) {
+      for (int kb = 0; kb < nkb_full; ++kb) {
         if (!mbar_wait(&ctl->pk_full[stage], phase, abort_flag)) { ok = false; break; }
         const uint8_t* sP = pk_stage + stage * kPkStageBytes;
         uint8_t* dst = smem + stage * kStageBytes + (kExpand == 1 ? 0 : kAStageBytes) + (seg >> 3) * 8192;
@@ -992,7 +1030,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
       if (!mbar_wait(&ctl->tmem_full[set], acc_phase, abort_flag)) break;
       tc_fence_after();
       // releases the accumulator itself, as soon as its last column has been read
-      epi_vnm8_tile<kBN, kV>(args, taddr, m0, n0, q, lane, wsm, &ctl->tmem_empty[set]);
+      epi_vnm8_tile<kBN, kV>(args, taddr, m0, n0, args.N, q, lane, wsm, &ctl->tmem_empty[set]);
       acc_phase ^= 1;
     }
   } else {
@@ -1002,15 +1040,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-      int mt, nt;
-      tile_coords(tile, num_m_tiles, num_n_tiles_, mt, nt);
-      const int64_t m0 = (int64_t)mt * 256 + (int64_t)rank * 128, n0 = (int64_t)nt * kBN;
+      const GemmTile tc = get_tile<kBN>(args, tile, num_m_tiles, num_n_tiles_, nkb_full);
+      const int64_t m0 = (int64_t)tc.out_m + (int64_t)rank * 128, n0 = tc.out_n, n_limit = tc.n_limit;
       const uint32_t taddr = tmem_base + acc * kBN + ((uint32_t)(q * 32) << 16);
       uint4 ax[is_drelu_t(kEpi) ? kBN / 32 : 1][4];
-      epi_prefetch<kEpi, kBN>(args, m0, n0, q, lane, ax);
+      epi_prefetch<kEpi, kBN>(args, m0, n0, n_limit, q, lane, ax);
       if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      epi_tile<kEpi, kBN>(args, taddr, m0, n0, q, lane, my_stage, ax);
+      epi_tile<kEpi, kBN>(args, taddr, m0, n0, n_limit, q, lane, my_stage, ax);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(&ctl->tmem_empty[acc]);
@@ -1115,7 +1152,9 @@ int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
   }
   a.num_m_tiles = (int)(a.M / 256);
   a.num_n_tiles = (int)((a.N + kBN - 1) / kBN);
-  const int tiles = a.num_m_tiles * a.num_n_tiles;
+  // table-driven products: the table's length is on the device; launch for its upper bound
+  const int tiles = a.tile_table ? a.num_k_blocks /* upper bound, see the grouped launchers */
+                                 : a.num_m_tiles * a.num_n_tiles;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
   kern<<<2 * pairs, threads2(kEpi, kExpand), smem, s>>>(ta, tb, tm, tpk ? *tpk : ta, a);
@@ -1242,6 +1281,84 @@ int gemm_sparse24_vnm8(const void* a_vals, const uint8_t* meta_hw, const void* X
   a.vn_y1 = out.y1; a.vn_dense = out.dense;
   if (V == 64) return launch_two<MODE_SPARSE24, false, false, EPI_VNM8, 192>(ta, tb, tm, a, s);
   return launch_two<MODE_SPARSE24, false, false, EPI_VNM8, 128>(ta, tb, tm, a, s);
+}
+
+// ---- grouped (table-driven) products of the routed step --------------------------------------------------
+// All of them run on CTA pairs; the caller's tables hold one entry per output tile and `max_tiles` bounds
+// their length (it sizes the grid; GemmArgs::num_k_blocks carries it to the launcher).
+
+int gemm_grouped_act24(const void* a_vals, const uint8_t* meta_hw, const void* Xp, int64_t rows, int64_t F, int64_t Fe,
+                       int64_t D, const Act24Out& out, const GemmTile* tiles, const int* num_tiles, int max_tiles,
+                       int* status, cudaStream_t s) {
+  if (F % 256 || Fe % 256 || D % 128 || rows % 32 || max_tiles <= 0) return SF_ERR_SHAPE;
+  CUtensorMap ta, tb, tm;
+  int st = make_tmap(&ta, a_vals, F, D / 2, D / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tb, Xp, rows, D, D, 64, kNarrowBN / 2, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tm, meta_hw, 2 * (F / 128) * (D / 128), 256, 256, 256, 2, CU_TENSOR_MAP_SWIZZLE_NONE, 1);
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = Fe; a.N = rows; a.K = D;                           // M: width of the outputs (features per expert)
+  a.status = status;
+  a.vn_vals24 = out.vals; a.vn_relu24 = out.relu; a.vn_meta24 = out.meta; a.vn_meta24_hw = out.meta_hw;
+  a.vn_dense = out.dense; a.vn_y1 = out.y1;
+  a.tile_table = tiles; a.num_tiles_dev = num_tiles; a.num_k_blocks = max_tiles;
+  return launch_two<MODE_SPARSE24, false, false, EPI_ACT24_T, kNarrowBN>(ta, tb, tm, a, s);
+}
+
+int gemm_grouped_drelu24(const void* a_vals, const uint8_t* meta_hw, const void* dYp, int64_t rows, int64_t F,
+                         int64_t Fe, int64_t D, const void* relu_vals, const void* meta, void* pack_vals, void* dense,
+                         const GemmTile* tiles, const int* num_tiles, int max_tiles, int* status, cudaStream_t s) {
+  if (F % 256 || Fe % 256 || D % 128 || rows % 32 || max_tiles <= 0) return SF_ERR_SHAPE;
+  CUtensorMap ta, tb, tm;
+  int st = make_tmap(&ta, a_vals, F, D / 2, D / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tb, dYp, rows, D, D, 64, kNarrowBN / 2, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tm, meta_hw, 2 * (F / 128) * (D / 128), 256, 256, 256, 2, CU_TENSOR_MAP_SWIZZLE_NONE, 1);
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = Fe; a.N = rows; a.K = D;
+  a.C = dense; a.ldc = Fe; a.aux = relu_vals; a.pack_meta = meta; a.pack_vals = pack_vals;
+  a.status = status;
+  a.tile_table = tiles; a.num_tiles_dev = num_tiles; a.num_k_blocks = max_tiles;
+  return launch_two<MODE_SPARSE24, false, false, EPI_DRELU24_T, kNarrowBN>(ta, tb, tm, a, s);
+}
+
+int gemm_grouped_sparse24_rm(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t rows,
+                             int64_t N, int64_t Fe, int64_t Ktot, void* C, const GemmTile* tiles, const int* num_tiles,
+                             int max_tiles, int* status, cudaStream_t s) {
+  if (rows % 256 || N % 256 || Fe % 128 || Ktot % Fe || max_tiles <= 0) return SF_ERR_SHAPE;
+  CUtensorMap ta, tb, tm;
+  int st = make_tmap(&ta, a_vals, rows, Fe / 2, Fe / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  if (b_kmajor) st = make_tmap(&tb, B, N, Ktot, Ktot, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  else          st = make_tmap(&tb, B, Ktot, N, N, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tm, meta_hw, 2 * (rows / 128) * (Fe / 128), 256, 256, 256, 2, CU_TENSOR_MAP_SWIZZLE_NONE, 1);
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = rows; a.N = N; a.K = Fe;                           // K of the packed operand: its metadata atoms follow it
+  a.C = C; a.ldc = N; a.status = status;
+  a.tile_table = tiles; a.num_tiles_dev = num_tiles; a.num_k_blocks = max_tiles;
+  if (b_kmajor) return launch_two<MODE_SPARSE24, false, false, EPI_STORE>(ta, tb, tm, a, s);
+  return launch_two<MODE_SPARSE24, false, true, EPI_STORE>(ta, tb, tm, a, s);
+}
+
+int gemm_grouped_dense_tn(const void* A, int64_t Ma, const void* B, int64_t Nb, int64_t rows, void* C, int64_t ldc,
+                          const GemmTile* tiles, const int* num_tiles, int max_tiles, int* status, cudaStream_t s) {
+  if (Ma % 256 || Nb % 256 || rows % 64 || max_tiles <= 0) return SF_ERR_SHAPE;
+  CUtensorMap ta, tb;
+  int st = make_tmap(&ta, A, rows, Ma, Ma, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tb, B, rows, Nb, Nb, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = Ma; a.N = ldc; a.K = rows;                         // N bounds the stored columns: the whole output row
+  a.C = C; a.ldc = ldc; a.status = status;
+  a.tile_table = tiles; a.num_tiles_dev = num_tiles; a.num_k_blocks = max_tiles;
+  return launch_two<MODE_DENSE, true, true, EPI_STORE>(ta, tb, ta, a, s);
 }
 
 int gemm_dense_expand(const void* dense_op, int packed_operand, const void* pk_vals, const void* pk_meta, int64_t M,

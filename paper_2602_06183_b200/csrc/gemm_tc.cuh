@@ -16,8 +16,21 @@ enum GemmEpilogue {
   EPI_DRELU_T = 4,  // C[n, m] = bf16(2 * acc * aux[n, m]), +0 where aux is zero       (Eq. 6 on the mask)
   EPI_VNM8 = 5,     // SquaredReLU + V:N:M selection (groups of eight) on the accumulator tile itself: rows are
                     // features, columns are tokens; writes the packed activation, never the dense y1  (Eq. 2, Section 2.3)
-  EPI_DRELU24_T = 6 // as EPI_DRELU_T with aux given in the 2:4 layout of the mask (values [n, m/2] + pack_meta) and
+  EPI_DRELU24_T = 6,// as EPI_DRELU_T with aux given in the 2:4 layout of the mask (values [n, m/2] + pack_meta) and
                     // only the packed output written
+  EPI_ACT24_T = 7   // transposed output with SquaredReLU and a 2:4 selection inside every four features of a token
+                    // (the routed step's activation, Section 3.1 step 3): packed values, packed ReLU values, both
+                    // metadata orders and the masked dense copy; never the pre-activation unless asked for
+};
+
+// One output tile of a table-driven (grouped) product on CTA pairs. Offsets are in elements of the
+// operand's own coordinates: a_row / b_row select the 256 (A) or tile-width (B) rows or columns the tile
+// reads, a_k0 / b_k0 where its reduction range starts in either operand, nkb how many k-blocks (of 128
+// logical K for 2:4 products, 64 for dense ones) it spans; out_m / out_n are the output coordinates the
+// epilogue uses (they differ from a_row / b_row when an operand is a slice of a larger matrix), n_limit
+// the first output column that does not belong to the tile's group any more.
+struct GemmTile {
+  int a_row, a_k0, b_row, b_k0, nkb, out_m, out_n, n_limit;
 };
 
 struct GemmArgs {
@@ -49,6 +62,9 @@ struct GemmArgs {
   void* vn_meta24_hw;       // the same words in tensor-core order
   void* vn_y1;              // optional bf16 [T, F]: the pre-activation itself
   void* vn_dense;           // optional bf16 [T, F]: the activation on its mask, +0 elsewhere
+  // table-driven tiles (grouped products of the routed step); null = the regular tile raster
+  const GemmTile* tile_table;
+  const int* num_tiles_dev;  // device word holding the number of valid entries of tile_table
 };
 
 // Outputs of the fused y1 product (see GemmArgs::vn_*).
@@ -71,6 +87,31 @@ int gemm_dense_expand(const void* dense_op, int packed_operand, const void* pk_v
 int gemm_sparse24_vnm8(const void* a_vals, const uint8_t* meta_hw, const void* X, int64_t F, int64_t T, int64_t D,
                        int V, const Vnm8Out& out, int* status, cudaStream_t s);
 bool gemm_sparse24_vnm8_supported(int64_t F, int64_t T, int64_t D, int V);
+
+// ---- grouped products of the routed step (tile tables built on the device, see router.cu) ------------------
+// Outputs of the routed y1 product's epilogue, all indexed [row of the permuted token order, local feature]
+// with Fe = features per expert: values / ReLU values [rows, Fe/2], canonical metadata [rows, Fe/16] and its
+// tensor-core order, masked dense copy [rows, Fe], optional pre-activation [rows, Fe].
+struct Act24Out {
+  void *vals, *relu, *meta, *meta_hw, *dense, *y1;
+};
+// y1c = Xp W1s[expert block]^T with the epilogue above. a_vals/meta_hw: W1s [F, D] packed; Xp [rows, D].
+int gemm_grouped_act24(const void* a_vals, const uint8_t* meta_hw, const void* Xp, int64_t rows, int64_t F, int64_t Fe,
+                       int64_t D, const Act24Out& out, const GemmTile* tiles, const int* num_tiles, int max_tiles,
+                       int* status, cudaStream_t s);
+// dy1c = 2 (dYp W2s[expert block]) ReLU(y1c) on the mask: packed (pack_vals) and masked dense (C) copies.
+int gemm_grouped_drelu24(const void* a_vals, const uint8_t* meta_hw, const void* dYp, int64_t rows, int64_t F,
+                         int64_t Fe, int64_t D, const void* relu_vals, const void* meta, void* pack_vals, void* dense,
+                         const GemmTile* tiles, const int* num_tiles, int max_tiles, int* status, cudaStream_t s);
+// C[rows, N] = A_s[rows, Fe] (2:4-packed activations) times the expert's slice of a weight matrix:
+// b_kmajor: B = W [N, Ktot] row-major (slice of columns); else B = W [Ktot, N] row-major (slice of rows).
+int gemm_grouped_sparse24_rm(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t rows,
+                             int64_t N, int64_t Fe, int64_t Ktot, void* C, const GemmTile* tiles, const int* num_tiles,
+                             int max_tiles, int* status, cudaStream_t s);
+// C[M, N] (leading dimension ldc) accumulates A^T B over each tile's own range of rows: A [rows, Ma], B [rows, Nb]
+// row-major (both reduced over rows).
+int gemm_grouped_dense_tn(const void* A, int64_t Ma, const void* B, int64_t Nb, int64_t rows, void* C, int64_t ldc,
+                          const GemmTile* tiles, const int* num_tiles, int max_tiles, int* status, cudaStream_t s);
 // A_s[M,K] 2:4-packed times B (b_kmajor: [N,K] row-major, else [K,N] row-major).
 // epi EPI_STORE_T / EPI_DRELU_T: transposed output Ct[N,M] (b_kmajor only); EPI_STORE: C[M,N]
 // (two-CTA kernel, M % 256 == 0).
