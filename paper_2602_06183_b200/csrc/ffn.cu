@@ -20,10 +20,6 @@ inline size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 cudaEvent_t* g_trace_events = nullptr;
 int g_trace_cap = 0, g_trace_n = 0;
 
-inline void trace_mark(cudaStream_t s) {
-  if (g_trace_events && g_trace_n < g_trace_cap) cudaEventRecord(g_trace_events[g_trace_n++], s);
-}
-
 // Copy/compute overlap of the host-buffer step: while sf_ffn_step_host runs, the step functions wait
 // for an operand's upload right before its first use and signal a result as soon as its product is
 // enqueued. Null outside sf_ffn_step_host.
@@ -209,6 +205,10 @@ inline uint8_t* at(void* base, size_t off) { return reinterpret_cast<uint8_t*>(b
 inline const uint8_t* at(const void* base, size_t off) { return reinterpret_cast<const uint8_t*>(base) + off; }
 
 }  // namespace
+
+void trace_mark(cudaStream_t s) {
+  if (g_trace_events && g_trace_n < g_trace_cap) cudaEventRecord(g_trace_events[g_trace_n++], s);
+}
 
 int launch_meta_reorder(const void* meta, void* meta_hw, int64_t R, int64_t K, cudaStream_t s) {
   const int64_t n = R * (K >> 4);

@@ -6,7 +6,7 @@
 //   step 1  route_kernel        logits = x . ExpertMeans, top-1 expert per token (ties to the lower expert)
 //   step 2  group_kernel        tokens grouped by expert, stable, every segment padded to 256 rows of zeros;
 //           tile_tables_kernel  one table entry per output tile of each grouped product (no host round trip)
-//           permute_rows_kernel gathers X (and dY) into that order
+//           gather_rows_kernel  gathers X (and dY) into that order, and scatters Y / dX back
 //   step 3  grouped tensor-core products over the tables: every product touches only the expert's Fe features
 //           of a token, so each costs 1 / E of its dense counterpart (and the 2:4 ones half of that again).
 // Interleaving the expert blocks four features at a time turns a segment into V:N:M blocks with M = 4 E whose
@@ -336,14 +336,17 @@ int sf_routed_ffn_fwd(const sf_router_desc* desc, const void* X, const void* W1,
   int* src = (int*)at(fwd_ctx, L.src_of_row);
 
   // Algorithm 1 line 4: W1s = sparsify24(W1) along d_model
+  trace_mark(s);
   SF_TRY(launch_prune24(W1, d.F, d.D, d.D, 1, d.prune_mode, at(workspace, L.w1_vals), at(workspace, L.w1_meta),
                         at(workspace, L.w1_meta_hw), nullptr, s));
+  trace_mark(s);
   // Section 3.1 step 1: expert of every token (or the caller's, for stage-wise comparison)
   if (forced_expert) {
     SF_CUDA_TRY(cudaMemcpyAsync(expert, forced_expert, (size_t)d.T * 4, cudaMemcpyDeviceToDevice, s));
   } else {
     SF_TRY(launch_route(X, means, d.T, d.D, d.E, expert, at(fwd_ctx, L.logits), s));
   }
+  trace_mark(s);
   // step 2: token order, tile tables, gathered X
   static bool attr_done[64] = {false};
   int dev = 0;
@@ -361,16 +364,20 @@ int sf_routed_ffn_fwd(const sf_router_desc* desc, const void* X, const void* W1,
                                        (GemmTile*)at(fwd_ctx, L.tabD), counts);
   SF_LAUNCH_CHECK();
   SF_TRY(launch_gather_rows(X, src, at(fwd_ctx, L.xp), L.rows_max, d.D, s));
+  trace_mark(s);
   // step 3: y1 = Xp W1s[expert]^T with SquaredReLU and the 2:4 selection in the epilogue
   Act24Out out{at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.relu_vals), at(fwd_ctx, L.meta), at(fwd_ctx, L.meta_hw),
                at(fwd_ctx, L.y2_dense), (d.flags & SF_FFN_SAVE_Y1) ? (void*)at(fwd_ctx, L.y1) : nullptr};
   SF_TRY(gemm_grouped_act24(at(workspace, L.w1_vals), at(workspace, L.w1_meta_hw), at(fwd_ctx, L.xp), L.rows_max, d.F,
                             L.Fe, d.D, out, (const GemmTile*)at(fwd_ctx, L.tabA), counts + 0, L.max_tiles[0], status, s));
+  trace_mark(s);
   // Algorithm 1 line 7: y3 = y2 W2^T over the expert's features only (W2 dense), then back to token order
   SF_TRY(gemm_grouped_sparse24_rm(at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta_hw), W2, true, L.rows_max, d.D, L.Fe, d.F,
                                   at(workspace, L.y3p), (const GemmTile*)at(fwd_ctx, L.tabB), counts + 1,
                                   L.max_tiles[1], status, s));
+  trace_mark(s);
   SF_TRY(launch_gather_rows(at(workspace, L.y3p), (const int*)at(fwd_ctx, L.row_of_token), Y, d.T, d.D, s));
+  trace_mark(s);
   return SF_OK;
 }
 
@@ -389,24 +396,32 @@ int sf_routed_ffn_bwd(const sf_router_desc* desc, const void* dY, const void* X,
   const int* src = (const int*)at(fwd_ctx, L.src_of_row);
 
   // Algorithm 2 line 2: W2s = sparsify24(W2^T) along d_model (strided groups of W2 [D, F])
+  trace_mark(s);
   SF_TRY(launch_prune24(W2, d.D, d.F, d.F, 0, d.prune_mode, at(workspace, L.w2_vals), at(workspace, L.w2_meta),
                         at(workspace, L.w2_meta_hw), nullptr, s));
+  trace_mark(s);
   SF_TRY(launch_gather_rows(dY, src, at(workspace, L.dyp), L.rows_max, d.D, s));
+  trace_mark(s);
   // dy2 = dYp W2s[expert];  line 4: dy1 = 2 dy2 ReLU(y1) on y2's mask, in the product's epilogue
   SF_TRY(gemm_grouped_drelu24(at(workspace, L.w2_vals), at(workspace, L.w2_meta_hw), at(workspace, L.dyp), L.rows_max,
                               d.F, L.Fe, d.D, at(fwd_ctx, L.relu_vals), at(fwd_ctx, L.meta), at(workspace, L.dy1_vals),
                               at(workspace, L.dy1_dense), (const GemmTile*)at(fwd_ctx, L.tabA), counts + 0,
                               L.max_tiles[0], status, s));
+  trace_mark(s);
   // line 5: dX = dy1 W1 over the expert's features (W1 dense), back to token order
   SF_TRY(gemm_grouped_sparse24_rm(at(workspace, L.dy1_vals), at(fwd_ctx, L.meta_hw), W1, false, L.rows_max, d.D, L.Fe,
                                   d.F, at(workspace, L.dxp), (const GemmTile*)at(fwd_ctx, L.tabB), counts + 1,
                                   L.max_tiles[1], status, s));
+  trace_mark(s);
   SF_TRY(launch_gather_rows(at(workspace, L.dxp), (const int*)at(fwd_ctx, L.row_of_token), dX, d.T, d.D, s));
+  trace_mark(s);
   // line 3: dW2[:, expert block] = dY_e^T y2_e;  line 6: dW1[expert block, :] = dy1_e^T X_e
   SF_TRY(gemm_grouped_dense_tn(at(workspace, L.dyp), d.D, at(fwd_ctx, L.y2_dense), L.Fe, L.rows_max, dW2, d.F,
                                (const GemmTile*)at(fwd_ctx, L.tabC), counts + 2, L.max_tiles[2], status, s));
+  trace_mark(s);
   SF_TRY(gemm_grouped_dense_tn(at(workspace, L.dy1_dense), L.Fe, at(fwd_ctx, L.xp), d.D, L.rows_max, dW1, d.D,
                                (const GemmTile*)at(fwd_ctx, L.tabD), counts + 3, L.max_tiles[3], status, s));
+  trace_mark(s);
   return SF_OK;
 }
 

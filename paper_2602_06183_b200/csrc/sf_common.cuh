@@ -96,6 +96,8 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
                void* relu_dense_out, void* vals24, void* meta24, void* meta24_hw, void* relu24, cudaStream_t s);
 bool vnm_has_24_view(int64_t F, int V, int M);
 int launch_transpose(const void* in, void* out, int64_t rows, int64_t cols, cudaStream_t s);
+// Records the next caller-owned trace event on `s` while stage tracing is on (sf_trace_set); else a no-op.
+void trace_mark(cudaStream_t s);
 
 // Byte offset of the metadata word (row m, 16-column word kw) inside the hardware-ordered
 // metadata tensor of a [R, K] 2:4 operand: 2 KB atoms of 128 rows x 128 columns, atoms of one
