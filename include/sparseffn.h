@@ -346,6 +346,14 @@ typedef enum sf_routed_ctx_field {
   SF_RCTX_Y1 = 8,           /* bf16 [rows_max, Fe] (only with SF_FFN_SAVE_Y1) */
   SF_RCTX_DY1_VALS = 9      /* bf16 [rows_max, Fe/2], in the WORKSPACE after sf_routed_ffn_bwd */
 } sf_routed_ctx_field;
+/* Offline clustering (HOST routine, all pointers are HOST pointers; no GPU is touched): balanced k-means
+ * with L2 distance over the F feature vectors of W1 [F, D] (Figure 4a), at most `iters` Lloyd iterations.
+ * Outputs: host_expert int32 [F] (expert of each feature, exactly F / E per expert), host_perm int32 [F]
+ * (feature perm[i] of the old numbering becomes feature i of the expert-major one: apply it to the rows of
+ * W1 and the columns of W2 once), host_means bf16 [E, D] (cluster centres = the router's ExpertMeans).
+ * Deterministic. F % E == 0, 1 <= E <= 16. */
+SF_API int sf_router_fit_host(const void* host_W1, int64_t F, int64_t D, int E, int iters, void* host_expert,
+                              void* host_perm, void* host_means);
 SF_API int sf_router_route(const void* X, const void* means, int64_t T, int64_t D, int E, void* expert,
                            void* logits, void* stream);
 SF_API int sf_routed_ffn_workspace_size(const sf_router_desc* desc, size_t* fwd_ctx_bytes, size_t* workspace_bytes);

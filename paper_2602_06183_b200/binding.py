@@ -86,6 +86,7 @@ _SIGNATURES = {
                                     _sz, _vp, _sz, _vp]),
     "sf_ffn_bwd_scheduled": (_i32, [C.POINTER(sf_schedule), _i64, C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp,
                                     _sz, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "sf_router_fit_host": (_i32, [_vp, _i64, _i64, _i32, _i32, _vp, _vp, _vp]),
     "sf_router_route": (_i32, [_vp, _vp, _i64, _i64, _i32, _vp, _vp, _vp]),
     "sf_routed_ffn_workspace_size": (_i32, [C.POINTER(sf_router_desc), C.POINTER(_sz), C.POINTER(_sz)]),
     "sf_routed_ffn_fwd": (_i32, [C.POINTER(sf_router_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
@@ -349,6 +350,19 @@ def sf_ffn_step_host(desc, dense: bool, hX, hW1, hW2, hdY, hY, hdX, hdW1, hdW2, 
 
 def make_router_desc(T, D, F, E, prune_mode=0, flags=0) -> sf_router_desc:
     return sf_router_desc(T, D, F, E, prune_mode, flags, 0)
+
+
+def sf_router_fit_host(W1_bits, E: int, iters: int = 8):
+    """Offline balanced clustering on the host. W1_bits: numpy uint16 [F, D] (bf16 patterns).
+    Returns numpy arrays (expert int32 [F], perm int32 [F], means uint16 [E, D])."""
+    import numpy as np
+    W = np.ascontiguousarray(W1_bits, dtype=np.uint16)
+    F, D = W.shape
+    expert, perm = np.empty(F, dtype=np.int32), np.empty(F, dtype=np.int32)
+    means = np.empty((E, D), dtype=np.uint16)
+    _check(lib().sf_router_fit_host(W.ctypes.data_as(_vp), F, D, E, iters, expert.ctypes.data_as(_vp),
+                                    perm.ctypes.data_as(_vp), means.ctypes.data_as(_vp)), "sf_router_fit_host")
+    return expert, perm, means
 
 
 def sf_router_route(X: torch.Tensor, means: torch.Tensor, want_logits: bool = True, stream=None):

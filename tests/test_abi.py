@@ -129,3 +129,37 @@ def test_context_size_of_the_d4096_layer(lib):
     lean = binding.make_desc(8192, 4096, 16384, 128, 8, flags=binding.SF_FFN_PACKED_GRAD_OPERANDS)
     lctx, lws = binding.sf_ffn_workspace_size(lean)
     assert lctx < 0.6e9 and lws < ws
+
+
+def test_router_fit_matches_the_oracle(lib):
+    """The offline clustering is host code, so it is compared with the oracle here: planted clusters
+    come back whole, the partition is balanced, the permutation is expert-major and stable, the means
+    are the centroids, and on unstructured weights the assignment agrees with the oracle's."""
+    import numpy as np
+    from oracle import router as R
+    from oracle import f32_to_bf16, bf16_to_f32
+    from paper_2602_06183_b200 import synth
+    rng = np.random.default_rng(0)
+    E, cap, D = 4, 24, 16
+    centres = rng.integers(-4, 5, size=(E, D)).astype(np.float32) * 8.0
+    label = rng.permutation(np.repeat(np.arange(E), cap))
+    W = f32_to_bf16(centres[label] + rng.integers(-1, 2, size=(E * cap, D)).astype(np.float32)).reshape(E * cap, D)
+    expert, perm, means = binding.sf_router_fit_host(W, E)
+    o_expert, o_means = R.fit_experts(W, E)
+    assert np.array_equal(expert, o_expert) and np.array_equal(means, o_means)
+    assert np.array_equal(perm, R.expert_major_permutation(o_expert))
+    for e in range(E):
+        assert len(set(label[expert == e])) == 1
+    W1 = synth.normal_bf16((512, 64), 0.0, 0.02, seed=3)
+    for E in (2, 16):
+        expert, perm, means = binding.sf_router_fit_host(W1, E, iters=1)
+        o_expert, o_means = R.fit_experts(W1, E, iters=1)
+        assert np.array_equal(np.bincount(expert, minlength=E), np.full(E, 512 // E))
+        assert np.array_equal(expert[perm], np.repeat(np.arange(E), 512 // E))
+        assert (expert == o_expert).mean() > 0.99
+        for e in range(E):
+            c = bf16_to_f32(W1[expert == e]).astype(np.float64).mean(axis=0).astype(np.float32)
+            assert np.array_equal(means[e], f32_to_bf16(c))
+    a, b = C.c_void_p(0x1000), None
+    assert lib.sf_router_fit_host(a, 10, 4, 3, 1, a, a, a) == binding.SF_ERR_SHAPE
+    assert lib.sf_router_fit_host(b, 12, 4, 3, 1, a, a, a) == binding.SF_ERR_NULL

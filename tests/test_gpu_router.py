@@ -24,9 +24,12 @@ def _nibbles(meta):
     return np.stack([(meta >> np.uint16(4 * i)) & np.uint16(0xF) for i in range(4)], axis=-1).reshape(meta.shape[0], -1)
 
 
-def _run(T, D, F, E, seed, prune_mode=0, forced=None, skew=None):
+def _run(T, D, F, E, seed, prune_mode=0, forced=None, skew=None, fit=False):
     X, W1, W2, dY = synth.ffn_inputs(T, D, F, 0.05, seed)
     means = synth.normal_bf16((E, D), 0.0, 1.0, seed, 9)
+    if fit:                                    # the whole offline recipe: cluster, renumber the hidden features
+        _, perm, means = binding.sf_router_fit_host(W1, E, iters=2)
+        W1, W2 = np.ascontiguousarray(W1[perm]), np.ascontiguousarray(W2[:, perm])
     if skew is not None:                       # a shared component in the tokens that one expert's mean picks up
         m, x = oracle.bf16_to_f32(means).copy(), oracle.bf16_to_f32(X).copy()
         x[:, 0] = 2.0
@@ -150,6 +153,14 @@ def test_routed_step_soft_threshold_and_skewed_routing():
     Fe = F // E
     for e in (1, 2, 3, 4, 6, 7):
         assert not g["dW1"][e * Fe:(e + 1) * Fe].any() and not g["dW2"][:, e * Fe:(e + 1) * Fe].any()
+
+
+def test_routed_step_with_fitted_experts():
+    """Offline fit on the host (balanced clusters, expert-major renumbering of W1's rows and W2's
+    columns, means as the router's operand), then the step: the composition a user runs."""
+    T, D, F, E = 512, 256, 1024, 4
+    inputs, g = _run(T, D, F, E, seed=77, fit=True)
+    _check(inputs, g, T, D, F, E)
 
 
 def test_router_entry_point_alone():
