@@ -221,6 +221,18 @@ def run_ours(args, cfg):
         raise SystemExit("device status: a bounded wait expired during warm-up")
 
     flop_step = 12.0 * T * D * F
+    if args.quick and args.quick_arm == "routed":
+        E = M // 4
+        rdesc = binding.make_router_desc(T, D, F, E, prune_mode=args.prune_mode)
+        rc, rw = binding.sf_routed_ffn_workspace_size(rdesc)
+        rctx, rws = torch.zeros((rc,), dtype=torch.uint8, device="cuda"), torch.zeros((rw,), dtype=torch.uint8, device="cuda")
+        means = torch.from_numpy(synth.normal_bf16((E, D), 0.0, 1.0, cfg["seed"], 9).view(np.int16)).cuda().view(torch.bfloat16)
+
+        def sparse_step():                     # the quick path below times whatever this name holds
+            binding.sf_routed_ffn_fwd(rdesc, dX_, dW1_, dW2_, means, Y, rctx, rws)
+            binding.sf_routed_ffn_bwd(rdesc, ddY, dX_, dW1_, dW2_, rctx, gX, gW1, gW2, rws)
+        for _ in range(W):
+            sparse_step()
     if args.quick:
         ms = timed(sparse_step, K)
         if rank == 0:
@@ -544,6 +556,8 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true",
                     help="sparse step only (no dense step, trace, e2e, CPU baseline): for profiler captures")
+    ap.add_argument("--quick-arm", default="sparse", choices=["sparse", "routed"],
+                    help="with --quick: the magnitude-selection step or the routed step")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         raise SystemExit(_spawn_replicas(args))
