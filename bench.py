@@ -282,22 +282,22 @@ def run_ours(args, cfg):
 
         for _ in range(3):
             routed_step()
-        with binding.StageTrace(15 * K) as rtr:
+        with binding.StageTrace(13 * K) as rtr:
             ms_r = timed(routed_step, K)
         if binding.sf_check_status(rws) != binding.SF_OK:
             raise SystemExit("device status: a bounded wait expired in the routed step")
         rd = rtr.durations_ms()
-        rnames = ["prune24_W1", "route", "group_tables_gather_X", "gemm_y1", "gemm_y3", "scatter_Y", None,
-                  "prune24_W2", "gather_dY", "gemm_dy1", "gemm_dX", "scatter_dX", "gemm_dW2", "gemm_dW1"]
+        rnames = ["prune24_W1", "route", "group_tables_gather_X", "gemm_y1", "gemm_y3", None,
+                  "prune24_W2", "gather_dY", "gemm_dy1", "gemm_dX", "gemm_dW2", "gemm_dW1"]
         rper = {}
         for st in range(K):
-            for n, v in zip(rnames, rd[15 * st: 15 * st + 14]):
+            for n, v in zip(rnames, rd[13 * st: 13 * st + 12]):
                 if n:
                     rper.setdefault(n, []).append(v)
         seg = binding.sf_routed_ctx_view(rdesc, rctx, binding.SF_RCTX_SEGMENTS).cpu().numpy()
         routed = {"experts": E, "ms_per_step": ms_r / K, "value": replicas.aggregate_tflops(flop_step, K, ms_r),
                   "speedup_vs_dense_step": ms_dense / ms_r, "kernel_ms": {n: float(np.mean(v)) for n, v in rper.items()},
-                  "tokens_per_expert": seg[E + 1:].tolist(), "rows_with_padding": int(seg[E]), "gpu_launches": 17 * K,
+                  "tokens_per_expert": seg[E + 1:].tolist(), "rows_with_padding": int(seg[E]), "gpu_launches": 15 * K,
                   "routing": "synthetic expert means ~ N(0,1): near-uniform top-1 routing",
                   "note": "Algorithm 1 line 6 as the paper words it (MoEToVenom): every product touches one expert's "
                           "F/E features per token; reported beside the magnitude-selection step, not instead of it"}

@@ -386,8 +386,8 @@ SF_API int sf_selftest_wait_expiry(void* workspace, int64_t budget_clocks, void*
  *   sparse bwd: 7 events (prune W2 | dy1 product | pack | dX product | dW2 product | dW1 product);
  *               for M <= 8 the dy1 product packs its own output and the pack interval is empty
  *   dense fwd: 3 events, dense bwd: 5 events.
- *   routed fwd: 7 events (prune W1 | route | group + tile tables + gather X | y1 product | y3 product | gather Y)
- *   routed bwd: 8 events (prune W2 | gather dY | dy1 product | dX product | gather dX | dW2 product | dW1 product).
+ *   routed fwd: 6 events (prune W1 | route | group + tile tables + gather X | y1 product | y3 product)
+ *   routed bwd: 7 events (prune W2 | gather dY | dy1 product | dX product | dW2 product | dW1 product).
  * sf_trace_count returns how many events have been recorded since sf_trace_set. Not thread-safe. */
 SF_API int sf_trace_set(void** events, int capacity);
 SF_API int sf_trace_count(void);

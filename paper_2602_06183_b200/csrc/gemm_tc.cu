@@ -116,13 +116,20 @@ template <int kEpi, int kTileN = BN>
 __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, int64_t m0, int64_t n0, int64_t n_limit,
                                          int q, int lane, uint8_t* my_stage,
                                          const uint4 (&ax)[is_drelu_t(kEpi) ? kTileN / 32 : 1][4]) {
-  const int64_t row = m0 + q * 32 + lane;                                  // this thread's D row
+  int64_t row = m0 + q * 32 + lane;                                        // this thread's D row
+  bool row_live = true;
+  if (kEpi == EPI_STORE && args.row_map) {                                 // scattered output rows
+    const int r = __ldg(args.row_map + row);
+    row_live = r >= 0;
+    row = r;
+  }
   auto chunk = [&](int ch, const uint4 (&a4)[4], const uint32_t (&v)[32]) {
     const int64_t col0 = n0 + ch * 32;
     if (col0 >= n_limit) return;                                           // ragged last tile (warp-uniform)
     if (kEpi == EPI_STORE || kEpi == EPI_SQRELU || kEpi == EPI_DRELU) {
       uint16_t* crow = reinterpret_cast<uint16_t*>(args.C) + row * args.ldc + col0;
       if (kEpi == EPI_STORE) {
+        if (!row_live) return;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           uint4 o;
@@ -1327,8 +1334,8 @@ int gemm_grouped_drelu24(const void* a_vals, const uint8_t* meta_hw, const void*
 }
 
 int gemm_grouped_sparse24_rm(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t rows,
-                             int64_t N, int64_t Fe, int64_t Ktot, void* C, const GemmTile* tiles, const int* num_tiles,
-                             int max_tiles, int* status, cudaStream_t s) {
+                             int64_t N, int64_t Fe, int64_t Ktot, void* C, const int* row_map, const GemmTile* tiles,
+                             const int* num_tiles, int max_tiles, int* status, cudaStream_t s) {
   if (rows % 256 || N % 256 || Fe % 128 || Ktot % Fe || max_tiles <= 0) return SF_ERR_SHAPE;
   CUtensorMap ta, tb, tm;
   int st = make_tmap(&ta, a_vals, rows, Fe / 2, Fe / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -1340,7 +1347,7 @@ int gemm_grouped_sparse24_rm(const void* a_vals, const uint8_t* meta_hw, const v
   if (st != SF_OK) return st;
   GemmArgs a{};
   a.M = rows; a.N = N; a.K = Fe;                           // K of the packed operand: its metadata atoms follow it
-  a.C = C; a.ldc = N; a.status = status;
+  a.C = C; a.ldc = N; a.status = status; a.row_map = row_map;
   a.tile_table = tiles; a.num_tiles_dev = num_tiles; a.num_k_blocks = max_tiles;
   if (b_kmajor) return launch_two<MODE_SPARSE24, false, false, EPI_STORE>(ta, tb, tm, a, s);
   return launch_two<MODE_SPARSE24, false, true, EPI_STORE>(ta, tb, tm, a, s);

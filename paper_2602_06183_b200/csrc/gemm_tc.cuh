@@ -65,6 +65,8 @@ struct GemmArgs {
   // table-driven tiles (grouped products of the routed step); null = the regular tile raster
   const GemmTile* tile_table;
   const int* num_tiles_dev;  // device word holding the number of valid entries of tile_table
+  // EPI_STORE only, optional: output row r of the product is written to row row_map[r] of C (skipped when < 0)
+  const int* row_map;
 };
 
 // Outputs of the fused y1 product (see GemmArgs::vn_*).
@@ -105,9 +107,11 @@ int gemm_grouped_drelu24(const void* a_vals, const uint8_t* meta_hw, const void*
                          const GemmTile* tiles, const int* num_tiles, int max_tiles, int* status, cudaStream_t s);
 // C[rows, N] = A_s[rows, Fe] (2:4-packed activations) times the expert's slice of a weight matrix:
 // b_kmajor: B = W [N, Ktot] row-major (slice of columns); else B = W [Ktot, N] row-major (slice of rows).
+// row_map (optional): row r of the product lands in row row_map[r] of C, rows mapped to -1 are dropped (the
+// un-grouping of the routed step's outputs, done by the epilogue's own stores).
 int gemm_grouped_sparse24_rm(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t rows,
-                             int64_t N, int64_t Fe, int64_t Ktot, void* C, const GemmTile* tiles, const int* num_tiles,
-                             int max_tiles, int* status, cudaStream_t s);
+                             int64_t N, int64_t Fe, int64_t Ktot, void* C, const int* row_map, const GemmTile* tiles,
+                             const int* num_tiles, int max_tiles, int* status, cudaStream_t s);
 // C[M, N] (leading dimension ldc) accumulates A^T B over each tile's own range of rows: A [rows, Ma], B [rows, Nb]
 // row-major (both reduced over rows).
 int gemm_grouped_dense_tn(const void* A, int64_t Ma, const void* B, int64_t Nb, int64_t rows, void* C, int64_t ldc,

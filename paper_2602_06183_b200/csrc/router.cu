@@ -6,7 +6,8 @@
 //   step 1  route_kernel        logits = x . ExpertMeans, top-1 expert per token (ties to the lower expert)
 //   step 2  group_kernel        tokens grouped by expert, stable, every segment padded to 256 rows of zeros;
 //           tile_tables_kernel  one table entry per output tile of each grouped product (no host round trip)
-//           gather_rows_kernel  gathers X (and dY) into that order, and scatters Y / dX back
+//           gather_rows_kernel  gathers X (and dY) into that order (Y and dX go back to token order through
+//                               the row map of the product's own epilogue)
 //   step 3  grouped tensor-core products over the tables: every product touches only the expert's Fe features
 //           of a token, so each costs 1 / E of its dense counterpart (and the 2:4 ones half of that again).
 // Interleaving the expert blocks four features at a time turns a segment into V:N:M blocks with M = 4 E whose
@@ -201,7 +202,7 @@ struct RoutedLayout {
   size_t expert, row_of_token, src_of_row, seg, counts, tabA, tabB, tabC, tabD, logits, xp, y2_vals, relu_vals, meta,
       meta_hw, y2_dense, y1, ctx_total;
   // workspace
-  size_t w1_vals, w1_meta, w1_meta_hw, w2_vals, w2_meta, w2_meta_hw, y3p, dyp, dy1_vals, dy1_dense, dxp, ws_total;
+  size_t w1_vals, w1_meta, w1_meta_hw, w2_vals, w2_meta, w2_meta_hw, dyp, dy1_vals, dy1_dense, ws_total;
 };
 
 RoutedLayout routed_layout(const sf_router_desc& d) {
@@ -240,11 +241,9 @@ RoutedLayout routed_layout(const sf_router_desc& d) {
   L.w2_vals = take(F * D);
   L.w2_meta = take(F * D / 8);
   L.w2_meta_hw = take(F * D / 8);
-  L.y3p = take(R * D * 2);
   L.dyp = take(R * D * 2);
   L.dy1_vals = take(R * Fe);
   L.dy1_dense = take(R * Fe * 2);
-  L.dxp = take(R * D * 2);
   L.ws_total = o;
   return L;
 }
@@ -372,11 +371,9 @@ int sf_routed_ffn_fwd(const sf_router_desc* desc, const void* X, const void* W1,
                             L.Fe, d.D, out, (const GemmTile*)at(fwd_ctx, L.tabA), counts + 0, L.max_tiles[0], status, s));
   trace_mark(s);
   // Algorithm 1 line 7: y3 = y2 W2^T over the expert's features only (W2 dense), then back to token order
+  // (the epilogue stores every row at its token's place: src_of_row is the row map, padding rows are dropped)
   SF_TRY(gemm_grouped_sparse24_rm(at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta_hw), W2, true, L.rows_max, d.D, L.Fe, d.F,
-                                  at(workspace, L.y3p), (const GemmTile*)at(fwd_ctx, L.tabB), counts + 1,
-                                  L.max_tiles[1], status, s));
-  trace_mark(s);
-  SF_TRY(launch_gather_rows(at(workspace, L.y3p), (const int*)at(fwd_ctx, L.row_of_token), Y, d.T, d.D, s));
+                                  Y, src, (const GemmTile*)at(fwd_ctx, L.tabB), counts + 1, L.max_tiles[1], status, s));
   trace_mark(s);
   return SF_OK;
 }
@@ -410,10 +407,8 @@ int sf_routed_ffn_bwd(const sf_router_desc* desc, const void* dY, const void* X,
   trace_mark(s);
   // line 5: dX = dy1 W1 over the expert's features (W1 dense), back to token order
   SF_TRY(gemm_grouped_sparse24_rm(at(workspace, L.dy1_vals), at(fwd_ctx, L.meta_hw), W1, false, L.rows_max, d.D, L.Fe,
-                                  d.F, at(workspace, L.dxp), (const GemmTile*)at(fwd_ctx, L.tabB), counts + 1,
-                                  L.max_tiles[1], status, s));
-  trace_mark(s);
-  SF_TRY(launch_gather_rows(at(workspace, L.dxp), (const int*)at(fwd_ctx, L.row_of_token), dX, d.T, d.D, s));
+                                  d.F, dX, src, (const GemmTile*)at(fwd_ctx, L.tabB), counts + 1, L.max_tiles[1],
+                                  status, s));
   trace_mark(s);
   // line 3: dW2[:, expert block] = dY_e^T y2_e;  line 6: dW1[expert block, :] = dy1_e^T X_e
   SF_TRY(gemm_grouped_dense_tn(at(workspace, L.dyp), d.D, at(fwd_ctx, L.y2_dense), L.Fe, L.rows_max, dW2, d.F,
