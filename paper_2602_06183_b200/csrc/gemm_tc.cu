@@ -454,9 +454,13 @@ __device__ __forceinline__ void epi_vnm8_tile(const GemmArgs& args, uint32_t tad
         *reinterpret_cast<uint16_t*>(hw_atom + (mi >> 4) * 256u + (mi & 7u) * 16u + ((mi >> 3) & 1u) * 2u) = (uint16_t)mb;
       }
     };
+    // A quarter-warp reads two token pairs x four groups; pairs alternate which 16-byte half they fetch
+    // first, so each of the two loads touches every bank exactly once.
+    const int swap = (lane >> 2) & 1;
 #pragma unroll 1
     for (int it = 0; it < kV / 16; ++it) {
-      const uint4 qa = *reinterpret_cast<const uint4*>(sp), qb = *reinterpret_cast<const uint4*>(sp + 4);
+      const uint4 q0 = *reinterpret_cast<const uint4*>(sp + 4 * swap), q1 = *reinterpret_cast<const uint4*>(sp + 4 - 4 * swap);
+      const uint4 qa = swap ? q1 : q0, qb = swap ? q0 : q1;
       // de-interleave the token pair: low halves = even token, high halves = odd token
       const uint32_t r0[4] = {__byte_perm(qa.x, qa.y, 0x5410), __byte_perm(qa.z, qa.w, 0x5410),
                               __byte_perm(qb.x, qb.y, 0x5410), __byte_perm(qb.z, qb.w, 0x5410)};
