@@ -29,21 +29,30 @@ constexpr size_t kStatusBytes = 256;
 inline size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // ---- step 1: routing ----------------------------------------------------------------------------------
-// One warp per token. A lane owns eight consecutive elements of every 256-element chunk and keeps one float32
-// partial sum per expert; the partial sums are combined by a fixed xor-shuffle tree, so the result does not
-// depend on the launch.
+// One warp per four tokens (the expert means are read once per four tokens). A lane owns eight consecutive
+// elements of every 256-element chunk and keeps one float32 partial sum per (token, expert); the partial
+// sums are combined by a fixed xor-shuffle tree, so the result does not depend on the launch.
+constexpr int kRouteTokens = 4;
+
 __global__ void __launch_bounds__(256)
 route_kernel(const uint16_t* __restrict__ X, const uint16_t* __restrict__ means, int T, int D, int E,
              int* __restrict__ expert, float* __restrict__ logits) {
   const int lane = threadIdx.x & 31;
-  const int t = (int)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (t >= T) return;
-  float acc[kMaxExperts];
+  const int t0 = ((int)blockIdx.x * 8 + (threadIdx.x >> 5)) * kRouteTokens;
+  if (t0 >= T) return;
+  float acc[kRouteTokens][kMaxExperts];
 #pragma unroll
-  for (int e = 0; e < kMaxExperts; ++e) acc[e] = 0.f;
+  for (int i = 0; i < kRouteTokens; ++i)
+#pragma unroll
+    for (int e = 0; e < kMaxExperts; ++e) acc[i][e] = 0.f;
   for (int c = lane * 8; c < D; c += 256) {
-    const uint4 xv = __ldg(reinterpret_cast<const uint4*>(X + (int64_t)t * D + c));
-    const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+    uint32_t xw[kRouteTokens][4];
+#pragma unroll
+    for (int i = 0; i < kRouteTokens; ++i) {
+      const int t = min(t0 + i, T - 1);                                     // a ragged last group re-reads the last token
+      const uint4 xv = __ldg(reinterpret_cast<const uint4*>(X + (int64_t)t * D + c));
+      xw[i][0] = xv.x; xw[i][1] = xv.y; xw[i][2] = xv.z; xw[i][3] = xv.w;
+    }
 #pragma unroll
     for (int e = 0; e < kMaxExperts; ++e) {
       if (e < E) {
@@ -51,25 +60,33 @@ route_kernel(const uint16_t* __restrict__ X, const uint16_t* __restrict__ means,
         const uint32_t mw[4] = {mv.x, mv.y, mv.z, mv.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          acc[e] = __fmaf_rn(bf16_bits_to_float(xw[j] & 0xFFFFu), bf16_bits_to_float(mw[j] & 0xFFFFu), acc[e]);
-          acc[e] = __fmaf_rn(bf16_bits_to_float(xw[j] >> 16), bf16_bits_to_float(mw[j] >> 16), acc[e]);
+          const float m0 = bf16_bits_to_float(mw[j] & 0xFFFFu), m1 = bf16_bits_to_float(mw[j] >> 16);
+#pragma unroll
+          for (int i = 0; i < kRouteTokens; ++i) {
+            acc[i][e] = __fmaf_rn(bf16_bits_to_float(xw[i][j] & 0xFFFFu), m0, acc[i][e]);
+            acc[i][e] = __fmaf_rn(bf16_bits_to_float(xw[i][j] >> 16), m1, acc[i][e]);
+          }
         }
       }
     }
   }
-  int best = 0;
-  float bestv = 0.f;
 #pragma unroll
-  for (int e = 0; e < kMaxExperts; ++e) {
-    if (e < E) {
-      float v = acc[e];
+  for (int i = 0; i < kRouteTokens; ++i) {
+    const int t = t0 + i;
+    int best = 0;
+    float bestv = 0.f;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-      if (lane == 0 && logits) logits[(int64_t)t * E + e] = v;
-      if (e == 0 || v > bestv) { bestv = v; best = e; }        // strict: ties stay with the lower expert
+    for (int e = 0; e < kMaxExperts; ++e) {
+      if (e < E) {
+        float v = acc[i][e];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        if (lane == 0 && logits && t < T) logits[(int64_t)t * E + e] = v;
+        if (e == 0 || v > bestv) { bestv = v; best = e; }        // strict: ties stay with the lower expert
+      }
     }
+    if (lane == 0 && t < T) expert[t] = best;
   }
-  if (lane == 0) expert[t] = best;
 }
 
 // ---- step 2: grouping ---------------------------------------------------------------------------------------
@@ -271,7 +288,7 @@ int check_ptrs(std::initializer_list<const void*> ps) {
 
 int launch_route(const void* X, const void* means, int64_t T, int64_t D, int E, void* expert, void* logits,
                  cudaStream_t s) {
-  route_kernel<<<(unsigned)((T + 7) / 8), 256, 0, s>>>((const uint16_t*)X, (const uint16_t*)means, (int)T, (int)D, E,
+  route_kernel<<<(unsigned)((T + 8 * kRouteTokens - 1) / (8 * kRouteTokens)), 256, 0, s>>>((const uint16_t*)X, (const uint16_t*)means, (int)T, (int)D, E,
                                                        (int*)expert, (float*)logits);
   SF_LAUNCH_CHECK();
   return SF_OK;
