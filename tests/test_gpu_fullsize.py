@@ -148,3 +148,88 @@ def test_act_sweep_full_size_sampled_blocks(V, M):
     # the sparsity the paper quotes for trained models: about 90 % zeros before the format's own pruning
     zero_frac = float((oracle.bf16_to_f32(p[:1024]) <= 0).mean())
     assert 0.88 < zero_frac < 0.93
+
+
+@pytest.mark.parametrize("E", [2, 16])
+def test_routed_step_full_size_sampled(E):
+    """The routed step at the d_model = 4096 layer's full size (the shape bench.py times). Sampled
+    tokens give exact restrictions for Y, dy1 and dX (a token only needs its own row and its expert's
+    block); sampled groups of four features give exact restrictions for dW2 / dW1 (a feature's
+    gradient sums over the tokens of its expert, whose activations only need the four features)."""
+    from oracle import router as R
+    T, D, F = 8192, 4096, 16384
+    Fe = F // E
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, 0.02, 4)
+    means = synth.normal_bf16((E, D), 0.0, 1.0, 4, 9)
+    desc = binding.make_router_desc(T, D, F, E, flags=binding.SF_FFN_SAVE_Y1)
+    nctx, nws = binding.sf_routed_ffn_workspace_size(desc)
+    gctx, gws = Guarded(nctx, zero=True), Guarded(nws, zero=True)
+    dX_, dW1_, dW2_, ddY, dM = (to_dev(a) for a in (X, W1, W2, dY, means))
+    outs = [Guarded((T, D), torch.bfloat16), Guarded((T, D), torch.bfloat16), Guarded((F, D), torch.bfloat16),
+            Guarded((D, F), torch.bfloat16)]
+    Y, gX, gW1, gW2 = (o.t for o in outs)
+    binding.sf_routed_ffn_fwd(desc, dX_, dW1_, dW2_, dM, Y, gctx.t, gws.t)
+    binding.sf_routed_ffn_bwd(desc, ddY, dX_, dW1_, dW2_, gctx.t, gX, gW1, gW2, gws.t)
+    assert binding.sf_check_status(gws.t) == binding.SF_OK
+    for g, nm in zip([gctx, gws] + outs, ["context", "workspace", "Y", "dX", "dW1", "dW2"]):
+        g.check(nm)
+    view = lambda buf, f: binding.sf_routed_ctx_view(desc, buf, f)
+    expert = view(gctx.t, binding.SF_RCTX_EXPERT).cpu().numpy()
+    row = view(gctx.t, binding.SF_RCTX_ROW_OF_TOKEN).cpu().numpy()
+    ref_expert, ref_logits = R.route(X, means)
+    assert (expert == ref_expert).mean() > 0.995                      # near ties may differ (float32 accumulation)
+    rows_max = view(gctx.t, binding.SF_RCTX_SRC_OF_ROW).numel()
+    y1_dev = view(gctx.t, binding.SF_RCTX_Y1).view(rows_max, Fe)
+    vals_dev = view(gctx.t, binding.SF_RCTX_Y2_VALS).view(rows_max, Fe // 2)
+    meta_dev = view(gctx.t, binding.SF_RCTX_META).view(rows_max, Fe // 16)
+    dy1_dev = view(gws.t, binding.SF_RCTX_DY1_VALS).view(rows_max, Fe // 2)
+    f64 = lambda b: oracle.bf16_to_f32(b).astype(np.float64)
+
+    # ---- sample 1: 96 tokens spread over the batch
+    toks = np.sort(np.random.default_rng(E).choice(T, size=96, replace=False))
+    rt = torch.from_numpy(row[toks].astype(np.int64)).cuda()
+    y1_rows = bits(y1_dev[rt])
+    free = R.routed_ffn_fwd(X[toks], W1, W2, means, E, forced_expert=expert[toks])
+    cols = expert[toks][:, None].astype(np.int64) * Fe + np.arange(Fe)[None, :]
+    free_y1 = np.take_along_axis(free.y1b, cols, axis=1)
+    assert rel_fro(oracle.bf16_to_f32(y1_rows), oracle.bf16_to_f32(free_y1)) < TOL
+    assert_close_elementwise(oracle.bf16_to_f32(y1_rows), oracle.bf16_to_f32(free_y1), D, "y1")
+    fwd = R.routed_ffn_fwd(X[toks], W1, W2, means, E, forced_expert=expert[toks], forced_y1b=y1_rows)
+    m_rows = bits(meta_dev[rt])
+    assert np.array_equal(oracle.decompress24(bits(vals_dev[rt]), m_rows), np.take_along_axis(fwd.y2, cols, axis=1))
+    tt = torch.from_numpy(toks).cuda()
+    assert rel_fro(f32(Y[tt]), fwd.y3) < TOL
+    assert_close_elementwise(f32(Y[tt]), fwd.y3, Fe, "Y")
+    bwd = R.routed_ffn_bwd(dY[toks], X[toks], W1, W2, fwd)
+    dy1_rows = oracle.decompress24(bits(dy1_dev[rt]), m_rows)
+    ref_dy1 = np.take_along_axis(bwd.dy1, cols, axis=1)
+    assert rel_fro(oracle.bf16_to_f32(dy1_rows), oracle.bf16_to_f32(ref_dy1)) < TOL
+    assert_close_elementwise(oracle.bf16_to_f32(dy1_rows), oracle.bf16_to_f32(ref_dy1), D, "dy1")
+    dy1_full = np.zeros((len(toks), F), dtype=np.uint16)
+    np.put_along_axis(dy1_full, cols, dy1_rows, axis=1)
+    dX_ref = f64(dy1_full) @ f64(W1)
+    assert rel_fro(f32(gX[tt]), dX_ref) < TOL
+    assert_close_elementwise(f32(gX[tt]), dX_ref, Fe, "dX")
+
+    # ---- sample 2: groups of four features of three experts, all tokens of those experts
+    for e in sorted({0, E // 2, E - 1}):
+        te = np.flatnonzero(expert == e)
+        rte = torch.from_numpy(row[te].astype(np.int64)).cuda()
+        fl = np.concatenate([np.arange(4 * g, 4 * g + 4) for g in (0, Fe // 8, Fe // 4 - 1)])     # local features
+        flt = torch.from_numpy(fl).cuda()
+        y1g = bits(y1_dev[rte][:, flt])
+        hb, relu = oracle.vnm.squared_relu_bf16(y1g)
+        _, keep = R._select_top2_of4((hb & np.uint16(0x7FFF)).reshape(len(te), -1, 4))
+        keep = keep.reshape(len(te), -1)
+        y2g = np.where(keep, hb, np.uint16(0))
+        gf = e * Fe + fl                                                            # global features
+        gft = torch.from_numpy(gf).cuda()
+        dW2_ref = f64(dY[te]).T @ f64(y2g)
+        assert rel_fro(f32(gW2[:, gft]), dW2_ref) < TOL
+        assert_close_elementwise(f32(gW2[:, gft]), dW2_ref, len(te), "dW2")
+        w2s = oracle.prune24(np.ascontiguousarray(W2[:, gf]), group_dim=0).dense
+        dy2 = (f64(dY[te]) @ f64(w2s)).astype(np.float32)
+        dy1g = oracle.f32_to_bf16((np.float32(2.0) * dy2 * oracle.bf16_to_f32(relu)).astype(np.float32)).reshape(dy2.shape)
+        dy1g = np.where(keep, dy1g, np.uint16(0))
+        dW1_ref = f64(dy1g).T @ f64(X[te])
+        assert rel_fro(f32(gW1[gft]), dW1_ref) < TOL
