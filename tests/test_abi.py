@@ -163,3 +163,23 @@ def test_router_fit_matches_the_oracle(lib):
     a, b = C.c_void_p(0x1000), None
     assert lib.sf_router_fit_host(a, 10, 4, 3, 1, a, a, a) == binding.SF_ERR_SHAPE
     assert lib.sf_router_fit_host(b, 12, 4, 3, 1, a, a, a) == binding.SF_ERR_NULL
+
+
+def test_routed_step_argument_checks_on_the_host(lib):
+    desc = binding.make_router_desc(1024, 256, 1024, 4)
+    need_ctx, need_ws = binding.sf_routed_ffn_workspace_size(desc)
+    assert need_ctx > 0 and need_ws > 256
+    ok = C.c_void_p(0x10000)
+    d = C.byref(desc)
+    assert lib.sf_routed_ffn_fwd(d, ok, ok, ok, ok, None, ok, ok, need_ctx - 1, ok, need_ws, None) == binding.SF_ERR_WORKSPACE
+    assert lib.sf_routed_ffn_bwd(d, ok, ok, ok, ok, ok, need_ctx, ok, ok, ok, ok, need_ws - 1, None) == binding.SF_ERR_WORKSPACE
+    assert lib.sf_routed_ffn_fwd(d, None, ok, ok, ok, None, ok, ok, need_ctx, ok, need_ws, None) == binding.SF_ERR_NULL
+    assert lib.sf_routed_ffn_fwd(d, C.c_void_p(0x10008), ok, ok, ok, None, ok, ok, need_ctx, ok, need_ws, None) == binding.SF_ERR_ALIGN
+    bad = binding.make_router_desc(1024, 256, 1024, 4, flags=binding.SF_FFN_UNFUSED_ACT)
+    a, b = C.c_size_t(), C.c_size_t()
+    assert lib.sf_routed_ffn_workspace_size(C.byref(bad), C.byref(a), C.byref(b)) == binding.SF_ERR_UNSUPPORTED
+    assert lib.sf_router_route(ok, ok, 128, 100, 4, ok, None, None) == binding.SF_ERR_SHAPE
+    assert lib.sf_router_route(ok, ok, 0, 256, 4, ok, None, None) == binding.SF_OK
+    p, n = C.c_void_p(), C.c_size_t()
+    assert lib.sf_routed_ctx_view(d, ok, binding.SF_RCTX_Y1, C.byref(p), C.byref(n)) == binding.SF_ERR_UNSUPPORTED
+    assert lib.sf_routed_ctx_view(d, ok, 99, C.byref(p), C.byref(n)) == binding.SF_ERR_SHAPE

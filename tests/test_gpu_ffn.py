@@ -146,6 +146,35 @@ def test_fused_activation_epilogue_equals_the_two_kernel_path(V, act_shift):
         assert np.array_equal(fused[k], packed[k]), k
 
 
+@pytest.mark.parametrize("flags", [0, binding.SF_FFN_UNFUSED_ACT], ids=["fused", "two_kernel"])
+def test_all_zero_activation_takes_the_default_pattern(flags):
+    """Degenerate input: X = 0 makes every pre-activation +0, so every column score ties at zero. The
+    block keeps columns 0-3 (ties to the lower column), every row positions (0, 1), all values are zero
+    and every output of the step is exactly zero."""
+    cfg = dict(T=512, D=256, F=512, V=64, N=2, M=8, sigma_w=0.05, seed=5)
+    T, D, F, V, M = cfg["T"], cfg["D"], cfg["F"], cfg["V"], cfg["M"]
+    _, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
+    X = np.zeros((T, D), dtype=np.uint16)
+    desc = binding.make_desc(T, D, F, V, M, flags=flags | binding.SF_FFN_SAVE_Y1)
+    ctx, ws = binding.alloc_ffn_buffers(desc)
+    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
+    Y = torch.full((T, D), 7.0, dtype=torch.bfloat16, device="cuda")
+    gX, gW1, gW2 = torch.full_like(dX_, 7.0), torch.full_like(dW1_, 7.0), torch.full_like(dW2_, 7.0)
+    binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
+    binding.sf_sparse_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    G = F // M
+    colidx = binding.sf_ctx_view(desc, ctx, binding.SF_CTX_COLIDX).cpu().numpy().reshape(T // V, G, 4)
+    assert np.all(colidx == np.arange(4))
+    assert np.all(bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_META)) == 0x4444)
+    assert not bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y2_VALS)).any()
+    assert not bits(binding.sf_ctx_view(desc, ctx, binding.SF_CTX_Y1)).any()
+    ref = oracle.sparse_ffn_fwd(X, W1, W2, V=V, M=M)
+    assert np.array_equal(colidx, ref.act.colidx) and np.all(ref.act.meta == 0x4444)
+    for t in (Y, gX, gW1, gW2):
+        assert not bits(t).any()
+
+
 def test_plain_24_view_of_m4_activations_is_exact():
     """M = 4 is 2:4 activation sparsity: the packed V:N:M form is itself the 2:4 operand the products
     consume. Decompressed with its own metadata it must be the oracle's masked dense y2 bit for bit,

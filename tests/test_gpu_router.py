@@ -163,6 +163,57 @@ def test_routed_step_with_fitted_experts():
     _check(inputs, g, T, D, F, E)
 
 
+def test_routed_step_without_saved_y1_and_repeated_is_bit_identical():
+    """The benchmarked layout keeps no y1; two runs in a row on the same buffers and the run that saves
+    y1 must produce the same bits everywhere (no atomics, no order-dependent accumulation)."""
+    T, D, F, E = 768, 256, 1024, 4
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, 0.05, 55)
+    means = synth.normal_bf16((E, D), 0.0, 1.0, 55, 9)
+    dX_, dW1_, dW2_, dY_, dM = (to_dev(a) for a in (X, W1, W2, dY, means))
+    results = []
+    for flags in (0, 0, binding.SF_FFN_SAVE_Y1):
+        desc = binding.make_router_desc(T, D, F, E, flags=flags)
+        nctx, nws = binding.sf_routed_ffn_workspace_size(desc)
+        if flags == 0 and results:
+            pass                                   # second run re-uses the first run's dirty buffers
+        else:
+            ctx = torch.zeros((nctx,), dtype=torch.uint8, device="cuda")
+            ws = torch.zeros((nws,), dtype=torch.uint8, device="cuda")
+        Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+        gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
+        binding.sf_routed_ffn_fwd(desc, dX_, dW1_, dW2_, dM, Y, ctx, ws)
+        binding.sf_routed_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+        assert binding.sf_check_status(ws) == binding.SF_OK
+        results.append((Y, gX, gW1, gW2, binding.sf_routed_ctx_view(desc, ctx, binding.SF_RCTX_Y2_VALS).clone(),
+                        binding.sf_routed_ctx_view(desc, ctx, binding.SF_RCTX_EXPERT).clone()))
+    for other in results[1:]:
+        for a, b in zip(results[0], other):
+            assert torch.equal(a, b)
+
+
+def test_routed_step_all_zero_tokens():
+    """X = 0: every logit ties at zero, so every token goes to expert 0 (ties to the lower expert), the
+    other experts keep one zero tile each, and all outputs are exactly zero."""
+    T, D, F, E = 512, 256, 1024, 4
+    _, W1, W2, dY = synth.ffn_inputs(T, D, F, 0.05, 9)
+    X = np.zeros((T, D), dtype=np.uint16)
+    means = synth.normal_bf16((E, D), 0.0, 1.0, 9, 9)
+    desc = binding.make_router_desc(T, D, F, E)
+    nctx, nws = binding.sf_routed_ffn_workspace_size(desc)
+    ctx, ws = torch.zeros((nctx,), dtype=torch.uint8, device="cuda"), torch.zeros((nws,), dtype=torch.uint8, device="cuda")
+    dX_, dW1_, dW2_, dY_, dM = (to_dev(a) for a in (X, W1, W2, dY, means))
+    Y = torch.full((T, D), 3.0, dtype=torch.bfloat16, device="cuda")
+    gX, gW1, gW2 = torch.full_like(dX_, 3.0), torch.full_like(dW1_, 3.0), torch.full_like(dW2_, 3.0)
+    binding.sf_routed_ffn_fwd(desc, dX_, dW1_, dW2_, dM, Y, ctx, ws)
+    binding.sf_routed_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    assert not binding.sf_routed_ctx_view(desc, ctx, binding.SF_RCTX_EXPERT).any()
+    seg = binding.sf_routed_ctx_view(desc, ctx, binding.SF_RCTX_SEGMENTS).cpu().numpy()
+    assert seg.tolist() == [0, 512, 768, 1024, 1280, 512, 0, 0, 0]
+    for t in (Y, gX, gW1, gW2):
+        assert not bits(t).any()
+
+
 def test_router_entry_point_alone():
     T, D, E = 2048, 512, 16
     X = synth.normal_bf16((T, D), 0, 1, seed=1)
