@@ -1185,6 +1185,12 @@ bool use_two_cta(int64_t M) { return M % 256 == 0; }
 
 }  // namespace
 
+int make_tmap_2d(void* map, const void* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
+                 uint32_t box_rows, bool swizzle128) {
+  return make_tmap(reinterpret_cast<CUtensorMap*>(map), base, rows, cols, ld, box_cols, box_rows,
+                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE);
+}
+
 int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64_t M, int64_t N, int64_t K, int epi,
                void* C, int64_t ldc, void* C2, int64_t ldc2, const void* aux, int64_t ldaux, int* status,
                cudaStream_t s) {

@@ -128,6 +128,11 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
 int gemm_venom(const void* a_vals, const uint8_t* meta_hw, const uint8_t* colidx, const void* Bt, int64_t T,
                int64_t F, int64_t N, int V, int Mv, void* C, int64_t ldc, int* status, cudaStream_t s);
 
+// 2D TMA descriptor (a CUtensorMap, 128 bytes, 64-byte aligned) over a row-major [rows, cols] matrix of 2-byte
+// elements with leading dimension ld; box = {box_cols, box_rows}.
+int make_tmap_2d(void* map, const void* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
+                 uint32_t box_rows, bool swizzle128);
+
 // canonical [R, K/16] metadata words -> hardware-ordered atoms (R % 128 == 0, K % 128 == 0)
 int launch_meta_reorder(const void* meta, void* meta_hw, int64_t R, int64_t K, cudaStream_t s);
 // dy1 packing: gather a dense [T, F] matrix at the positions recorded by (colidx, meta)

@@ -67,7 +67,7 @@ __device__ __forceinline__ uint32_t top2of4(uint32_t k0, uint32_t k1, uint32_t k
 // Returns the nibble; *packed = kept values (pos0 low half, pos1 high half); *third_idx = index of
 // the third-ranked element.
 __device__ __forceinline__ uint32_t top2of4_packed(uint32_t lo, uint32_t hi, uint32_t* packed,
-                                                   uint32_t* third_idx = nullptr) {
+                                                   uint32_t* third_idx = nullptr, uint32_t* perm_sel = nullptr) {
   const uint32_t c0 = ((lo << 2) & 0x1FFFCu) | 3u, c1 = ((lo >> 14) & 0x1FFFCu) | 2u;
   const uint32_t c2 = ((hi << 2) & 0x1FFFCu) | 1u, c3 = ((hi >> 14) & 0x1FFFCu);
   const uint32_t h01 = max(c0, c1), l01 = min(c0, c1), h23 = max(c2, c3), l23 = min(c2, c3);
@@ -78,7 +78,9 @@ __device__ __forceinline__ uint32_t top2of4_packed(uint32_t lo, uint32_t hi, uin
   const uint32_t ia = 3u - (top1 & 3u), ib = 3u - (top2 & 3u);
   const uint32_t p0 = min(ia, ib), p1 = max(ia, ib);
   // byte permute: bytes (2p0, 2p0+1) then (2p1, 2p1+1) out of the 8 bytes {lo, hi}
-  *packed = __byte_perm(lo, hi, 0x1010u + p0 * 0x22u + p1 * 0x2200u);
+  const uint32_t sel = 0x1010u + p0 * 0x22u + p1 * 0x2200u;
+  *packed = __byte_perm(lo, hi, sel);
+  if (perm_sel) *perm_sel = sel;             // the same selector picks the pair out of any other {lo, hi}
   if (third_idx) {
     const uint32_t other_low = first_pair_wins ? l23 : l01;
     *third_idx = 3u - (max(min(mid, under), other_low) & 3u);
@@ -95,6 +97,10 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
                void* vals, void* meta, void* meta_hw, void* colidx, void* relu_vals, void* dense_out,
                void* relu_dense_out, void* vals24, void* meta24, void* meta24_hw, void* relu24, cudaStream_t s);
 bool vnm_has_24_view(int64_t F, int V, int M);
+// Streaming form of the M = 8 sparsifier (values, ReLU values, canonical metadata and colidx only).
+bool vnm_stream_supported(int64_t F, int64_t ld, int V, int M, const void* P);
+int launch_vnm_stream(const void* P, int64_t T, int64_t F, int64_t ld, int V, int apply_sqrelu, void* vals, void* meta,
+                      void* colidx, void* relu_vals, cudaStream_t s);
 int launch_transpose(const void* in, void* out, int64_t rows, int64_t cols, cudaStream_t s);
 // Records the next caller-owned trace event on `s` while stage tracing is on (sf_trace_set); else a no-op.
 void trace_mark(cudaStream_t s);
