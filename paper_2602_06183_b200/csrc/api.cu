@@ -96,7 +96,7 @@ int sf_vnm_sparsify_act(const void* preact, int64_t T, int64_t F, int64_t ld, in
   st = check_arch();
   if (st != SF_OK) return st;
   if (!dense_out && vnm_stream_supported(F, ld, V, M, preact))
-    return launch_vnm_stream(preact, T, F, ld, V, apply_sqrelu, vals, meta, colidx, relu_vals, (cudaStream_t)stream);
+    return launch_vnm_stream(preact, T, F, ld, V, M, apply_sqrelu, vals, meta, colidx, relu_vals, (cudaStream_t)stream);
   return launch_vnm(preact, T, F, ld, V, M, apply_sqrelu, vals, meta, nullptr, colidx, relu_vals, dense_out,
                     nullptr, nullptr, nullptr, nullptr, nullptr, (cudaStream_t)stream);
 }

@@ -97,10 +97,10 @@ int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, in
                void* vals, void* meta, void* meta_hw, void* colidx, void* relu_vals, void* dense_out,
                void* relu_dense_out, void* vals24, void* meta24, void* meta24_hw, void* relu24, cudaStream_t s);
 bool vnm_has_24_view(int64_t F, int V, int M);
-// Streaming form of the M = 8 sparsifier (values, ReLU values, canonical metadata and colidx only).
+// Streaming form of the sparsifier (values, ReLU values, canonical metadata and colidx only).
 bool vnm_stream_supported(int64_t F, int64_t ld, int V, int M, const void* P);
-int launch_vnm_stream(const void* P, int64_t T, int64_t F, int64_t ld, int V, int apply_sqrelu, void* vals, void* meta,
-                      void* colidx, void* relu_vals, cudaStream_t s);
+int launch_vnm_stream(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu, void* vals,
+                      void* meta, void* colidx, void* relu_vals, cudaStream_t s);
 int launch_transpose(const void* in, void* out, int64_t rows, int64_t cols, cudaStream_t s);
 // Records the next caller-owned trace event on `s` while stage tracing is on (sf_trace_set); else a no-op.
 void trace_mark(cudaStream_t s);

@@ -1,6 +1,6 @@
-// SquaredReLU + V:N:M sparsification with groups of eight columns, streaming form (Eq. 2, Section 2.3).
+// SquaredReLU + V:N:M sparsification, streaming form (Eq. 2, Section 2.3), for M in {8, 16, 32, 64}.
 //
-// Same selection rule and outputs as vnm8_kernel (values, ReLU values, canonical metadata, colidx), organised
+// Same selection rule and outputs as the kernels of vnm.cu (values, ReLU values, canonical metadata, colidx), organised
 // as a pipeline so that loading, scoring and emitting overlap inside one CTA instead of alternating:
 //   warp 0        TMA producer: one bulk tensor load per V x 256 strip into a three-slot ring
 //   warps 1..4    column scores (sequential float32 sums, two columns per thread), ranking of the eight columns
@@ -26,7 +26,7 @@ template <int kSW>
 struct StripAux {
   uint32_t score[kSW];
   uint8_t keep[kSW];
-  uint8_t cidx[kSW / 8 * 4];
+  uint8_t cidx[kSW / 8 * 4];             // [groups of the strip][4]; sized for the narrowest group
 };
 
 struct StreamCtl {
@@ -38,9 +38,9 @@ __device__ __forceinline__ void named_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
-template <int kSW>
+template <int kSW, int kM>
 __global__ void __launch_bounds__(kThreadsS)
-vnm8_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t F, int V, int apply,
+vnm_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t F, int V, int apply,
                    uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ colidx,
                    uint16_t* __restrict__ relu_vals) {
   extern __shared__ uint8_t smem_dyn[];
@@ -53,7 +53,7 @@ vnm8_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nsx = (int)((F + kSW - 1) / kSW);
   const int64_t nstrips = (T / V) * nsx;
-  const int64_t G = F >> 3;
+  const int64_t G = F / kM;
 
   if (tid == 0) {
     prefetch_tmap(&tmapP);
@@ -112,12 +112,12 @@ vnm8_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t
       named_sync(1, 128);
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
-        const int j = 2 * ts + c, jm = j & 7, base = j - jm;
+        const int j = 2 * ts + c, jm = j & (kM - 1), base = j - jm;
         if (j >= kSW) break;
         const uint32_t s = a.score[j];
         int rank = 0;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
+#pragma unroll 8
+        for (int k = 0; k < kM; ++k) {
           const uint32_t sk = a.score[base + k];
           rank += (sk > s) || (sk == s && k < jm);
         }
@@ -126,18 +126,18 @@ vnm8_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t
       named_sync(1, 128);
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
-        const int j = 2 * ts + c, jm = j & 7, base = j - jm;
+        const int j = 2 * ts + c, jm = j & (kM - 1), base = j - jm;
         if (j >= kSW) break;
         if (a.keep[j]) {
           int pos = 0;
           for (int k = 0; k < jm; ++k) pos += a.keep[base + k];
-          a.cidx[(j >> 3) * 4 + pos] = (uint8_t)jm;
+          a.cidx[(j / kM) * 4 + pos] = (uint8_t)jm;
         }
       }
       named_sync(1, 128);
-      const int ng = cvalid >> 3;
+      const int ng = cvalid / kM;
       if (ts < ng)
-        *reinterpret_cast<uint32_t*>(colidx + (blk * G + cx * (kSW / 8) + ts) * 4) =
+        *reinterpret_cast<uint32_t*>(colidx + (blk * G + cx * (kSW / kM) + ts) * 4) =
             *reinterpret_cast<const uint32_t*>(a.cidx + ts * 4);
       __syncwarp();
       if (lane == 0) mbar_arrive(&ctl->scored[slot]);
@@ -145,14 +145,14 @@ vnm8_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t
     }
   } else {
     // =========================== emit (256 threads) ===========================
-    constexpr int kGS = kSW / 8, kRows = 256 / kGS;          // groups per strip row, rows in flight
+    constexpr int kGS = kSW / kM, kRows = 256 / kGS;         // groups per strip row, rows in flight
     const int te = tid - 160, g = te & (kGS - 1), r0 = te / kGS;
     const bool want_relu = relu_vals != nullptr && apply;
     uint32_t slot = 0, phase = 0;
     for (int64_t i = blockIdx.x; i < nstrips; i += gridDim.x) {
       const int64_t blk = i / nsx, cx = i - blk * nsx;
       const int cvalid = (int)min((int64_t)kSW, F - cx * kSW);
-      const bool live = g < (cvalid >> 3);
+      const bool live = g < cvalid / kM;
       const Aux& a = aux[slot];
       if (!mbar_wait(&ctl->scored[slot], phase, abort_flag)) break;
       const uint32_t c4 = *reinterpret_cast<const uint32_t*>(a.cidx + g * 4);
@@ -164,19 +164,30 @@ vnm8_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t
         selp[pr] = sa | ((sa + 1u) << 4) | (sb << 8) | ((sb + 1u) << 12);
         mhi[pr] = ((ca & 4u) ? 0x0000FFFFu : 0u) | ((cb & 4u) ? 0xFFFF0000u : 0u);
       }
-      const int64_t gg = cx * (kSW / 8) + g, trow = blk * V + r0;
-      const uint8_t* tp = smem + slot * strip_bytes + r0 * (kSW * 2) + g * 16;
+      const int64_t gg = cx * (kSW / kM) + g, trow = blk * V + r0;
+      const uint8_t* tp = smem + slot * strip_bytes + r0 * (kSW * 2) + g * (kM * 2);
+      const int o0 = 2 * (int)(c4 & 0xFFu), o1 = 2 * (int)((c4 >> 8) & 0xFFu), o2 = 2 * (int)((c4 >> 16) & 0xFFu),
+                o3 = 2 * (int)(c4 >> 24);                      // byte offsets of the kept columns inside the group
       uint32_t* p_vals = reinterpret_cast<uint32_t*>(vals) + trow * G + gg;
       uint32_t* p_relu = want_relu ? reinterpret_cast<uint32_t*>(relu_vals) + trow * G + gg : nullptr;
       uint16_t* p_meta = meta + trow * (G >> 2) + (gg >> 2);
       const int64_t s_vals = kRows * G, s_meta = kRows * (G >> 2);
       const bool lead4 = (g & 3) == 0;
       for (int r = r0; r < V; r += kRows) {
-        const uint4 q = *reinterpret_cast<const uint4*>(tp);
         // the four kept columns as two packed pairs, then the activation on those only
-        const uint32_t a0 = __byte_perm(q.x, q.y, selp[0]), b0 = __byte_perm(q.z, q.w, selp[0]);
-        const uint32_t a1 = __byte_perm(q.x, q.y, selp[1]), b1 = __byte_perm(q.z, q.w, selp[1]);
-        uint32_t rk0 = (a0 & ~mhi[0]) | (b0 & mhi[0]), rk1 = (a1 & ~mhi[1]) | (b1 & mhi[1]);
+        uint32_t rk0, rk1;
+        if constexpr (kM == 8) {                              // one 16-byte load, picked apart by byte permutes
+          const uint4 q = *reinterpret_cast<const uint4*>(tp);
+          const uint32_t a0 = __byte_perm(q.x, q.y, selp[0]), b0 = __byte_perm(q.z, q.w, selp[0]);
+          const uint32_t a1 = __byte_perm(q.x, q.y, selp[1]), b1 = __byte_perm(q.z, q.w, selp[1]);
+          rk0 = (a0 & ~mhi[0]) | (b0 & mhi[0]);
+          rk1 = (a1 & ~mhi[1]) | (b1 & mhi[1]);
+        } else {                                              // wide groups: four 16-bit loads
+          rk0 = (uint32_t)*reinterpret_cast<const uint16_t*>(tp + o0) |
+                ((uint32_t)*reinterpret_cast<const uint16_t*>(tp + o1) << 16);
+          rk1 = (uint32_t)*reinterpret_cast<const uint16_t*>(tp + o2) |
+                ((uint32_t)*reinterpret_cast<const uint16_t*>(tp + o3) << 16);
+        }
         uint32_t hk0 = rk0, hk1 = rk1;
         if (apply) {
           rk0 = bf2_relu(rk0); rk1 = bf2_relu(rk1);
@@ -207,11 +218,15 @@ vnm8_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t
 }  // namespace
 
 bool vnm_stream_supported(int64_t F, int64_t ld, int V, int M, const void* P) {
-  // TMA: 16-byte aligned base and row pitch; box rows = V; the emit threads take rows in steps of 8 or 16
-  return M == 8 && V % 16 == 0 && V >= 16 && V <= 128 && F % 32 == 0 && ld % 8 == 0 && aligned16(P);
+  // TMA: 16-byte aligned base and row pitch; box rows = V; emit threads take rows in steps of 256 * M / strip width
+  if (!(M == 8 || M == 16 || M == 32 || M == 64)) return false;
+  // 256 emit threads over (strip width / M) groups; M = 64 always takes 256-column strips (a metadata word
+  // spans four groups)
+  const int rows_in_flight = (V <= 64 || M == 64) ? M : 2 * M;
+  return V >= 16 && V <= 128 && V % 16 == 0 && V % rows_in_flight == 0 && F % (4 * M) == 0 && ld % 8 == 0 && aligned16(P);
 }
 
-template <int kSW>
+template <int kSW, int kM>
 static int launch_stream_t(const void* P, int64_t T, int64_t F, int64_t ld, int V, int apply_sqrelu, void* vals, void* meta,
                            void* colidx, void* relu_vals, cudaStream_t s) {
   alignas(64) CUtensorMap tm;
@@ -224,7 +239,7 @@ static int launch_stream_t(const void* P, int64_t T, int64_t F, int64_t ld, int 
   SF_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return SF_ERR_UNSUPPORTED;
   if (!attr_done[dev]) {
-    SF_CUDA_TRY(cudaFuncSetAttribute(vnm8_stream_kernel<kSW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    SF_CUDA_TRY(cudaFuncSetAttribute(vnm_stream_kernel<kSW, kM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      128 + kSlots * 128 * kSW * 2 + kSlots * (int)sizeof(StripAux<kSW>) +
                                          (int)sizeof(StreamCtl)));
     SF_CUDA_TRY(cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev));
@@ -234,17 +249,25 @@ static int launch_stream_t(const void* P, int64_t T, int64_t F, int64_t ld, int 
   const int per_sm = smem <= 110 * 1024 ? 2 : 1;
   const int64_t resident = (int64_t)sms[dev] * per_sm;
   const unsigned grid = (unsigned)(nstrips < resident ? nstrips : resident);
-  vnm8_stream_kernel<kSW><<<grid, kThreadsS, smem, s>>>(tm, T, F, V, apply_sqrelu, (uint16_t*)vals, (uint16_t*)meta,
-                                                        (uint8_t*)colidx, (uint16_t*)relu_vals);
+  vnm_stream_kernel<kSW, kM><<<grid, kThreadsS, smem, s>>>(tm, T, F, V, apply_sqrelu, (uint16_t*)vals, (uint16_t*)meta,
+                                                           (uint8_t*)colidx, (uint16_t*)relu_vals);
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
 
-int launch_vnm_stream(const void* P, int64_t T, int64_t F, int64_t ld, int V, int apply_sqrelu, void* vals, void* meta,
-                      void* colidx, void* relu_vals, cudaStream_t s) {
+int launch_vnm_stream(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu, void* vals,
+                      void* meta, void* colidx, void* relu_vals, cudaStream_t s) {
   if (T == 0 || F == 0) return SF_OK;
-  if (V <= 64) return launch_stream_t<256>(P, T, F, ld, V, apply_sqrelu, vals, meta, colidx, relu_vals, s);
-  return launch_stream_t<128>(P, T, F, ld, V, apply_sqrelu, vals, meta, colidx, relu_vals, s);
+#define SF_STREAM_CASE(MM)                                                                                      \
+  if (M == MM)                                                                                                  \
+    return V <= 64 ? launch_stream_t<256, MM>(P, T, F, ld, V, apply_sqrelu, vals, meta, colidx, relu_vals, s)   \
+                   : launch_stream_t<128, MM>(P, T, F, ld, V, apply_sqrelu, vals, meta, colidx, relu_vals, s);
+  SF_STREAM_CASE(8)
+  SF_STREAM_CASE(16)
+  SF_STREAM_CASE(32)
+#undef SF_STREAM_CASE
+  if (M == 64) return launch_stream_t<256, 64>(P, T, F, ld, V, apply_sqrelu, vals, meta, colidx, relu_vals, s);
+  return SF_ERR_UNSUPPORTED;
 }
 
 }  // namespace sf

@@ -61,6 +61,29 @@ def test_vnm_bit_exact(T, F, V, M):
     assert np.array_equal(bits(dense), ref.dense)
 
 
+@pytest.mark.parametrize("T,F,V,M,apply", [
+    (128, 512, 64, 8, True), (256, 1024, 128, 8, True), (192, 832, 64, 8, True),       # ragged last strip (832 = 3 x 256 + 64)
+    (96, 1088, 32, 8, False), (256, 1024, 128, 16, True), (128, 1600, 64, 16, True),   # 1600 = 6 x 256 + 64
+    (128, 1152, 32, 32, True), (256, 1152, 128, 32, False), (128, 1280, 64, 64, True), (256, 768, 128, 64, True),
+    (48, 576, 16, 8, True), (4096, 2048, 64, 8, True)])                                 # many strips per persistent CTA
+def test_vnm_streaming_kernel_bit_exact(T, F, V, M, apply):
+    """Without a dense copy the call runs the streaming kernel (TMA-fed strip ring, overlapped scoring and
+    emitting warps); every output must equal the oracle's bit for bit, also through a strided view."""
+    p = synth.act_sweep_matrix(T, F, seed=4000 + T + F + M)
+    ref = oracle.vnm_sparsify(p, V=V, M=M, apply_sqrelu=apply)
+    wide = torch.zeros((T, F + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :F] = to_dev(p)
+    for src in (to_dev(p), wide[:, :F]):
+        vals, meta, colidx, relu, dense = binding.sf_vnm_sparsify_act(src, V, M, apply_sqrelu=apply)
+        torch.cuda.synchronize()
+        assert dense is None
+        assert np.array_equal(colidx.cpu().numpy(), ref.colidx)
+        assert np.array_equal(bits(meta), ref.meta)
+        assert np.array_equal(bits(vals), ref.vals)
+        if apply:
+            assert np.array_equal(bits(relu), ref.relu_vals)
+
+
 def test_vnm_no_activation_and_ties():
     # raw magnitudes with many exact ties, negative values, apply_sqrelu = 0
     p = synth.prune_sweep_matrix(128, 512, seed=9, tie_frac=0.5)
