@@ -6,7 +6,8 @@ format (Section 2.3), SquaredReLU (Eq. 2) and the masked FFN forward/backward pr
 (Eqs. 1-8 with the operand colouring of Algorithms 1 and 2), and the sparse/dense step
 schedule with the paper's speed-up arithmetic (Sections 3.1, 5.1, 5.3.2; `oracle.schedule`), and
 the neuron-level router that produces the V:N:M pattern from experts (Section 3.1, Algorithm 3;
-`oracle.router`).
+`oracle.router`), and E4M3 operands whose quantisation rides on the pruning pass (Section 3.2.2, last
+paragraph; `oracle.fp8`: format, scaling and order of operations are this oracle's readings, stated there).
 
 Nothing in here is shared with, imported by, or derived from the CUDA path. Only the tests,
 the smoke check and the benchmark's CPU-baseline leg may import this package; the product
