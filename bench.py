@@ -506,7 +506,24 @@ def run_sweep(args):
             results.append({"product": "2:4 vs dense", "shape_mnk": [m, n, k], "dense_ms": ms_d, "dense_tflops": fl / ms_d / 1e9,
                             "sparse24_ms": ms_s, "sparse24_dense_equiv_tflops": fl / ms_s / 1e9, "prune_ms": ms_p,
                             "speedup_gemm_only": ms_d / ms_s, "speedup_with_prune": ms_d / (ms_s + ms_p)})
-            del A, B, Cm, vals, meta
+            # the same product on E4M3 operands (Section 3.2.2, last paragraph): quantisation rides on the pruning pass
+            sa, sb = 64.0, 64.0
+            Aq, Bq = binding.sf_fp8_quantize(A, sa), binding.sf_fp8_quantize(B, sb)
+            ws8 = torch.zeros((binding.sf_gemm_fp8_workspace_size(m, k),), dtype=torch.uint8, device="cuda")
+            ms_q = _time_cuda(lambda: binding.sf_fp8_quantize(B, sb, out=Bq), iters, args.warmup)
+            ms_d8 = _time_cuda(lambda: binding.sf_gemm_fp8_dense(Aq, Bq, 1.0 / (sa * sb), C_out=Cm, workspace=ws8), iters, args.warmup)
+            o8 = binding.sf_prune24_compress_fp8(A, 0, sa)
+            ms_p8 = _time_cuda(lambda: binding.sf_prune24_compress_fp8(A, 0, sa, out=o8), iters, args.warmup)
+            ms_s8 = _time_cuda(lambda: binding.sf_gemm_fp8_sparse24(o8[0], o8[1], Bq, 1.0 / (sa * sb), C_out=Cm, workspace=ws8),
+                               iters, args.warmup)
+            results.append({"product": "fp8 (E4M3) 2:4 vs dense", "shape_mnk": [m, n, k], "dense_fp8_ms": ms_d8,
+                            "dense_fp8_tflops": fl / ms_d8 / 1e9, "sparse24_fp8_ms": ms_s8,
+                            "sparse24_fp8_dense_equiv_tflops": fl / ms_s8 / 1e9, "prune_quantise_ms": ms_p8,
+                            "prune_quantise_gbs": 2.625 * m * k / ms_p8 / 1e6, "quantise_B_ms": ms_q,
+                            "quantise_B_gbs": 3.0 * n * k / ms_q / 1e6,
+                            "speedup_gemm_only": ms_d8 / ms_s8, "speedup_with_prune": ms_d8 / (ms_s8 + ms_p8),
+                            "speedup_vs_bf16_dense": ms_d / ms_s8})
+            del A, B, Cm, vals, meta, Aq, Bq, o8
         Tn, Fn, Nn = 8192, 16384, 4096
         A = torch.randn((Tn, Fn), device="cuda").to(torch.bfloat16)
         Bd = torch.randn((Nn, Fn), device="cuda").to(torch.bfloat16)

@@ -179,6 +179,38 @@ SF_API int sf_gemm_sparse24_noalloc(const void* a_vals, const void* a_meta, cons
                                     int64_t Mr, int64_t Nc, int64_t K, void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * FP8 (E4M3) operands with the quantisation folded into the pass that already scans the matrix
+ * (Section 3.2.2, last paragraph; the paper names the idea and fixes no format or scaling).
+ * As built: E4M3 codes (1-4-3 bits, bias 7, no infinities, |max| = 448), one float32 scale per
+ * tensor supplied by the caller; code = e4m3(float(x) * scale) with one float32 product and one
+ * conversion (round to nearest even, magnitudes above 448 and infinities clamp to 448, a NaN gives
+ * a NaN code). Device pointers; `ld` in elements.
+ *
+ * sf_fp8_quantize: Xq[r, c] = code of X[r, c]. X bf16 [rows, cols] (ld >= cols, ld % 8 == 0),
+ *     Xq uint8 [rows, cols] contiguous. cols % 16 == 0.
+ * sf_prune24_compress_fp8: the 2:4 pass of sf_prune24_compress with group_dim = 1 (groups of four
+ *     along a row; same selection, same soft-threshold shrinkage rounded to bf16) whose kept values
+ *     leave as codes: vals uint8 [rows, cols/2], meta uint16 [rows, cols/16] (canonical, identical to
+ *     the bf16 pass), optional dense_out uint8 [rows, cols] (codes on the mask, +0 elsewhere).
+ *     cols % 32 == 0. 2 B read + 0.625 B written per element.
+ * sf_gemm_fp8_dense:    C[Mr,Nc] = bf16(alpha * A B^T), A uint8 [Mr,K], B uint8 [Nc,K] (codes).
+ * sf_gemm_fp8_sparse24: the same with A given 2:4-packed: a_vals uint8 [Mr,K/2], a_meta canonical
+ *     uint16 [Mr,K/16]. alpha is normally 1 / (scale_A * scale_B).
+ *     Mr % 256 == 0, Nc % 256 == 0, K % 128 == 0 (dense) or K % 256 == 0 (2:4). fp32 accumulation.
+ * `workspace`: sf_gemm_fp8_workspace_size(Mr, K) bytes (status word + metadata in the order the
+ *     8-bit 2:4 instruction reads it); read its status with sf_check_status.
+ * Errors as everywhere: SF_ERR_SHAPE / NULL / ALIGN / ARCH before anything is launched. */
+SF_API int sf_fp8_quantize(const void* X, int64_t rows, int64_t cols, int64_t ld, float scale, void* Xq, void* stream);
+SF_API int sf_prune24_fp8_sizes(int64_t rows, int64_t cols, size_t* vals_bytes, size_t* meta_bytes);
+SF_API int sf_prune24_compress_fp8(const void* W, int64_t rows, int64_t cols, int64_t ld, int prune_mode, float scale,
+                                   void* vals, void* meta, void* dense_out, void* stream);
+SF_API int sf_gemm_fp8_workspace_size(int64_t Mr, int64_t K, size_t* bytes);
+SF_API int sf_gemm_fp8_dense(const void* A, const void* B, void* C, int64_t Mr, int64_t Nc, int64_t K, float alpha,
+                             void* workspace, void* stream);
+SF_API int sf_gemm_fp8_sparse24(const void* a_vals, const void* a_meta, const void* B, void* C, int64_t Mr, int64_t Nc,
+                                int64_t K, float alpha, void* workspace, void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * The FFN step (Algorithm 1 = forward, Algorithm 2 = backward; Eqs. 1-8 for the dense phase).
  *
  * sf_ffn_workspace_size: bytes of the forward context (saved for backward) and of the scratch

@@ -68,6 +68,12 @@ _SIGNATURES = {
     "sf_gemm_sparse24": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
     "sf_gemm_sparse24_rm": (_i32, [_vp, _vp, _vp, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "sf_gemm_sparse24_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
+    "sf_fp8_quantize": (_i32, [_vp, _i64, _i64, _i64, C.c_float, _vp, _vp]),
+    "sf_prune24_fp8_sizes": (_i32, [_i64, _i64, C.POINTER(_sz), C.POINTER(_sz)]),
+    "sf_prune24_compress_fp8": (_i32, [_vp, _i64, _i64, _i64, _i32, C.c_float, _vp, _vp, _vp, _vp]),
+    "sf_gemm_fp8_workspace_size": (_i32, [_i64, _i64, C.POINTER(_sz)]),
+    "sf_gemm_fp8_dense": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, C.c_float, _vp, _vp]),
+    "sf_gemm_fp8_sparse24": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, C.c_float, _vp, _vp]),
     "sf_gemm_venom": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp, _vp]),
     "sf_ffn_workspace_size": (_i32, [C.POINTER(sf_ffn_desc), C.POINTER(_sz), C.POINTER(_sz)]),
     "sf_sparse_ffn_fwd": (_i32, [C.POINTER(sf_ffn_desc), _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
@@ -248,6 +254,67 @@ def sf_gemm_sparse24_rm(a_vals, a_meta, B, b_kmajor: bool, C_out=None, workspace
     st = lib().sf_gemm_sparse24_rm(_ptr(a_vals), _ptr(a_meta), _ptr(B), int(b_kmajor), _ptr(C_out), Mr, Nc, K,
                                    _ptr(workspace), _stream(stream))
     _check(st, "sf_gemm_sparse24_rm")
+    return C_out, workspace
+
+
+def sf_fp8_quantize(X, scale: float, out=None, stream=None):
+    """E4M3 codes (uint8 [rows, cols]) of float(X) * scale; X bf16, may be a strided row view."""
+    rows, cols = X.shape
+    if out is None:
+        out = torch.empty((rows, cols), dtype=torch.uint8, device=X.device)
+    _check(lib().sf_fp8_quantize(_ptr(X), rows, cols, X.stride(0) if rows > 1 else cols, float(scale), _ptr(out),
+                                 _stream(stream)), "sf_fp8_quantize")
+    return out
+
+
+def sf_prune24_compress_fp8(W, prune_mode: int, scale: float, want_dense: bool = False, out=None, stream=None):
+    """2:4 along the rows with the kept values quantised to E4M3 in the same pass.
+    Returns (vals uint8 [rows, cols/2], meta int16 [rows, cols/16], dense uint8 [rows, cols] or None);
+    ``out`` = a previous result to write into."""
+    rows, cols = W.shape
+    vb, mb = _sz(), _sz()
+    _check(lib().sf_prune24_fp8_sizes(rows, cols, C.byref(vb), C.byref(mb)), "sf_prune24_fp8_sizes")
+    if out is not None:
+        vals, meta, dense = out
+    else:
+        vals = torch.empty((rows, cols // 2), dtype=torch.uint8, device=W.device)
+        meta = torch.empty((rows, cols // 16), dtype=torch.int16, device=W.device)
+        dense = torch.empty((rows, cols), dtype=torch.uint8, device=W.device) if want_dense else None
+    _check(lib().sf_prune24_compress_fp8(_ptr(W), rows, cols, W.stride(0) if rows > 1 else cols, prune_mode,
+                                         float(scale), _ptr(vals), _ptr(meta), _ptr(dense), _stream(stream)),
+           "sf_prune24_compress_fp8")
+    return vals, meta, dense
+
+
+def sf_gemm_fp8_workspace_size(Mr: int, K: int) -> int:
+    b = _sz()
+    _check(lib().sf_gemm_fp8_workspace_size(Mr, K, C.byref(b)), "sf_gemm_fp8_workspace_size")
+    return b.value
+
+
+def sf_gemm_fp8_dense(A, B, alpha: float, C_out=None, workspace=None, stream=None):
+    """C[Mr,Nc] = bf16(alpha * A B^T) on E4M3 codes A [Mr,K], B [Nc,K] (uint8)."""
+    Mr, K = A.shape
+    Nc = B.shape[0]
+    if C_out is None:
+        C_out = torch.empty((Mr, Nc), dtype=torch.bfloat16, device=B.device)
+    if workspace is None:
+        workspace = _workspace(sf_gemm_fp8_workspace_size(Mr, K), B.device)
+    _check(lib().sf_gemm_fp8_dense(_ptr(A), _ptr(B), _ptr(C_out), Mr, Nc, K, float(alpha), _ptr(workspace),
+                                   _stream(stream)), "sf_gemm_fp8_dense")
+    return C_out, workspace
+
+
+def sf_gemm_fp8_sparse24(a_vals, a_meta, B, alpha: float, C_out=None, workspace=None, stream=None):
+    """The same product with A 2:4-packed: a_vals uint8 [Mr,K/2], a_meta canonical [Mr,K/16]."""
+    Mr, K = a_vals.shape[0], a_vals.shape[1] * 2
+    Nc = B.shape[0]
+    if C_out is None:
+        C_out = torch.empty((Mr, Nc), dtype=torch.bfloat16, device=B.device)
+    if workspace is None:
+        workspace = _workspace(sf_gemm_fp8_workspace_size(Mr, K), B.device)
+    _check(lib().sf_gemm_fp8_sparse24(_ptr(a_vals), _ptr(a_meta), _ptr(B), _ptr(C_out), Mr, Nc, K, float(alpha),
+                                      _ptr(workspace), _stream(stream)), "sf_gemm_fp8_sparse24")
     return C_out, workspace
 
 

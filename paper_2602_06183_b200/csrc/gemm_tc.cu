@@ -130,13 +130,14 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
       uint16_t* crow = reinterpret_cast<uint16_t*>(args.C) + row * args.ldc + col0;
       if (kEpi == EPI_STORE) {
         if (!row_live) return;
+        const float al = args.out_scale != 0.f ? args.out_scale : 1.f;      // x 1 is exact: bf16 products unchanged
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           uint4 o;
-          o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
-          o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
-          o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
-          o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+          o.x = pack_bf16x2(__fmul_rn(__uint_as_float(v[8 * j + 0]), al), __fmul_rn(__uint_as_float(v[8 * j + 1]), al));
+          o.y = pack_bf16x2(__fmul_rn(__uint_as_float(v[8 * j + 2]), al), __fmul_rn(__uint_as_float(v[8 * j + 3]), al));
+          o.z = pack_bf16x2(__fmul_rn(__uint_as_float(v[8 * j + 4]), al), __fmul_rn(__uint_as_float(v[8 * j + 5]), al));
+          o.w = pack_bf16x2(__fmul_rn(__uint_as_float(v[8 * j + 6]), al), __fmul_rn(__uint_as_float(v[8 * j + 7]), al));
           reinterpret_cast<uint4*>(crow)[j] = o;
         }
       } else if (kEpi == EPI_SQRELU) {
@@ -753,8 +754,11 @@ __host__ __device__ constexpr int threads2(int epi, int expand) {
   return expand ? kThreads2Expand : (epi == EPI_VNM8 ? kThreads2Vnm : kThreads2);
 }
 constexpr int kPkStageBytes = 8192 + 1024;               // packed values [64 tokens][64] + metadata bytes [64][16]
-__host__ __device__ constexpr int stage_bytes2(bool sparse, int bn = BN) {
-  return sparse ? (16384 + 2 * (bn / 2) * 128 + 2048) : (16384 + 16384);
+// 8-bit operands (fp8 = true) keep the byte geometry of a stage (128-byte rows now hold 128 elements, so a
+// 2:4 stage spans 256 logical K) and double its metadata: two 2 KB atoms.
+__host__ __device__ constexpr int meta_stage_bytes2(bool fp8) { return fp8 ? 4096 : 2048; }
+__host__ __device__ constexpr int stage_bytes2(bool sparse, int bn = BN, bool fp8 = false) {
+  return sparse ? (16384 + 2 * (bn / 2) * 128 + meta_stage_bytes2(fp8)) : (16384 + 16384);
 }
 __host__ __device__ constexpr int num_stages2(bool sparse, int bn = BN, bool expand = false) {
   return sparse ? 4 : (expand ? 5 : 6);
@@ -764,8 +768,9 @@ __host__ __device__ constexpr int vnm_block(int bn) { return bn == 192 ? 64 : 12
 __host__ __device__ constexpr int epi_bytes2(int epi, int bn = BN) {
   return epi == EPI_VNM8 ? vnm_epi_bytes(vnm_block(bn)) : kEpiStageBytes;
 }
-__host__ __device__ constexpr int smem_bytes2(bool sparse, int bn = BN, int epi = EPI_STORE, bool expand = false) {
-  return 1024 + num_stages2(sparse, bn, expand) * (stage_bytes2(sparse, bn) + (expand ? kPkStageBytes : 0)) +
+__host__ __device__ constexpr int smem_bytes2(bool sparse, int bn = BN, int epi = EPI_STORE, bool expand = false,
+                                              bool fp8 = false) {
+  return 1024 + num_stages2(sparse, bn, expand) * (stage_bytes2(sparse, bn, fp8) + (expand ? kPkStageBytes : 0)) +
          epi_bytes2(epi, bn) + 1024;
 }
 
@@ -800,7 +805,10 @@ __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
 // kExpand (dense mode with both operands MN-major only): 1 = operand A, 2 = operand B is not loaded as a
 // dense tile; its 2:4-packed form (tmapPk: values, tmapMeta: metadata bytes) is staged by TMA and four
 // extra warps expand it, zero-filled, into the swizzled layout the MMA reads.
-template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN, int kExpand = 0>
+// kFp8: E4M3 operands (both K-major). The kernel is unchanged in bytes: K, k-block counts and operand
+// coordinates are given in 2-byte units (two codes each); only the instruction kind, the descriptor's formats
+// and the amount of metadata per stage differ.
+template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN, int kExpand = 0, bool kFp8 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(threads2(kEpi, kExpand), 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                 const __grid_constant__ CUtensorMap tmapMeta, const __grid_constant__ CUtensorMap tmapPk,
@@ -811,10 +819,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   constexpr int kStages = num_stages2(kSparse, kBN, kExpand != 0);
   constexpr int kBK = kSparse ? 128 : 64;                // logical K per stage
   static_assert(kExpand == 0 || (kMode == MODE_DENSE && kAMN && kBMN), "packed operands: weight-gradient products only");
+  static_assert(!kFp8 || (!kAMN && !kBMN && kExpand == 0 && kMode != MODE_VENOM), "8-bit operands are K-major");
+  constexpr int kMetaBytes = meta_stage_bytes2(kFp8);
+  constexpr uint32_t kMetaCols = kFp8 ? 8u : 4u;          // TMEM columns of one stage's metadata
   constexpr int kAStageBytes = 16384;
   constexpr int kBSlabBytes = (kBN / 2) * 128;            // this CTA's half of B for one 64-wide K slab
   constexpr int kBHalfBytes = kSparse ? 2 * kBSlabBytes : kBSlabBytes;
-  constexpr int kStageBytes = stage_bytes2(kSparse, kBN);
+  constexpr int kStageBytes = stage_bytes2(kSparse, kBN, kFp8);
   // 2:4 mode: TMEM holds the metadata next to the accumulators, so 256-column tiles leave room for one
   // accumulator only; 224-column tiles fit two (448 columns + 8 of metadata) and the epilogue of a tile
   // then overlaps the main loop of the next.
@@ -890,7 +901,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
             // shared-memory stores, not by TMA)
             mbar_arrive_expect_tx(bar, 2u * ((kExpand == 1 ? 0u : (uint32_t)kAStageBytes) +
                                              (kExpand == 2 ? 0u : (uint32_t)kBHalfBytes) +
-                                             (kSparse ? (uint32_t)kMetaStageBytes : 0u)));
+                                             (kSparse ? (uint32_t)kMetaBytes : 0u)));
           }
           if (kMode == MODE_DENSE) {
             if (kExpand == 1) {
@@ -917,9 +928,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
             }
           } else {
             tma_load_2d_2cta(sA, &tmapA, bar, (ak0 >> 1) + kb * 64, m0);       // stored values: box {64, 128}
-            // metadata atoms are rows of 2 x 1 KB in a [2 * atoms, 256] uint32 view
+            // metadata atoms are rows of 2 x 1 KB in a [2 * atoms, 256] uint32 view (8-bit operands: a pair of
+            // atoms per stage, 4 rows)
             const int atom = (m0 >> 7) * nkb_full + (ak0 >> 7) + kb;
-            tma_load_2d_2cta(sM, &tmapMeta, bar, 0, 2 * atom);
+            tma_load_2d_2cta(sM, &tmapMeta, bar, 0, (kFp8 ? 4 : 2) * atom);
             if (!kBMN) {
               tma_load_2d_2cta(sB, &tmapB, bar, bk0 + kb * 128, nb0);          // two 64-wide K slabs
               tma_load_2d_2cta(sB + kBSlabBytes, &tmapB, bar, bk0 + kb * 128 + 64, nb0);
@@ -935,7 +947,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
   } else if (warp == 1) {
     // =========================== MMA issuer (leader CTA only) ===========================
     if (rank == 0 && lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(256, kBN, kAMN, kBMN, kSparse);
+      constexpr uint32_t idesc = kFp8 ? idesc_e4m3(256, kBN, kSparse) : idesc_bf16(256, kBN, kAMN, kBMN, kSparse);
       // Descriptor halves that never change: high word = stride offset, version, swizzle; the low
       // word is (address >> 4) | leading offset, advanced by plain 32-bit adds.
       const uint32_t smem0 = smem_u32(smem);
@@ -963,8 +975,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
           tc_fence_after();
           const uint32_t soff = stage * (uint32_t)(kStageBytes >> 4);
           const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
-          const uint32_t mbuf = tmem_base + kMetaCol + 4u * ((uint32_t)kb & 1u);       // metadata double buffer
+          const uint32_t mbuf = tmem_base + kMetaCol + kMetaCols * ((uint32_t)kb & 1u);   // metadata double buffer
           if (kSparse) tmem_cp_128x128b_2cta(mbuf, desc64(m_lo0 + soff, m_hi));
+          if (kSparse && kFp8) tmem_cp_128x128b_2cta(mbuf + 4u, desc64(m_lo0 + soff + (2048u >> 4), m_hi));
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
@@ -972,11 +985,16 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
               // K = 32 per instruction: 32 B of stored A, 64 B of B inside a 64-wide K slab
               const uint32_t bk = kBMN ? (uint32_t)k * (4096 >> 4)      // 32 k rows of 128 B
                                        : (uint32_t)((k >> 1) * (kBSlabBytes >> 4) + (k & 1) * (64 >> 4));
-              mma_sp_f16_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi),
-                              mbuf + (uint32_t)(k & ~1), idesc | (uint32_t)(k & 1), accum);
+              if (kFp8)      // 64 logical K per instruction: two metadata columns each
+                mma_sp_f8_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi), mbuf + 2u * (uint32_t)k,
+                               idesc, accum);
+              else
+                mma_sp_f16_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi),
+                                mbuf + (uint32_t)(k & ~1), idesc | (uint32_t)(k & 1), accum);
             } else {
               const uint32_t bk = (uint32_t)k * (kBMN ? (2048 >> 4) : (32 >> 4));
-              mma_f16_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi), idesc, accum);
+              if (kFp8) mma_f8_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi), idesc, accum);
+              else      mma_f16_2cta(tmem_d, desc64(a_lo + k * a_step, a_hi), desc64(b_lo + bk, b_hi), idesc, accum);
             }
           }
           mma_commit_2cta(&ctl->empty[stage]);             // frees the stage in both CTAs
@@ -1148,11 +1166,11 @@ int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& a, 
   return SF_OK;
 }
 
-template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN, int kExpand = 0>
+template <int kMode, bool kAMN, bool kBMN, int kEpi, int kBN = BN, int kExpand = 0, bool kFp8 = false>
 int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tm, GemmArgs a, cudaStream_t s,
                const CUtensorMap* tpk = nullptr) {
-  auto kern = gemm_tc2_kernel<kMode, kAMN, kBMN, kEpi, kBN, kExpand>;
-  constexpr int smem = smem_bytes2(kMode != MODE_DENSE, kBN, kEpi, kExpand != 0);
+  auto kern = gemm_tc2_kernel<kMode, kAMN, kBMN, kEpi, kBN, kExpand, kFp8>;
+  constexpr int smem = smem_bytes2(kMode != MODE_DENSE, kBN, kEpi, kExpand != 0, kFp8);
   static_assert(smem <= 232448, "shared memory per CTA");
   static bool attr_done[64] = {false};
   int dev = 0;
@@ -1271,6 +1289,33 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
                : launch_one<MODE_SPARSE24, false, false, EPI_DRELU_T>(ta, tb, a, s);
   if (epi == EPI_DRELU24_T) return launch_two<MODE_SPARSE24, false, false, EPI_DRELU24_T, kNarrowBN>(ta, tb, tm, a, s);
   return SF_ERR_UNSUPPORTED;
+}
+
+int gemm_fp8(bool sparse, const void* A, const uint8_t* meta_hw, const void* B, int64_t M, int64_t N, int64_t K,
+             float alpha, void* C, int64_t ldc, int* status, cudaStream_t s) {
+  if (M % 256 || N % 32 || K % (sparse ? 256 : 128) || (sparse && !meta_hw)) return SF_ERR_SHAPE;
+  if (M == 0 || N == 0) return SF_OK;
+  // the operands in 2-byte units: [M, K/2] (dense) or [M, K/4] (2:4 values), [N, K/2]
+  const int64_t K2 = K / 2;
+  CUtensorMap ta, tb, tm;
+  int st = sparse ? make_tmap(&ta, A, M, K2 / 2, K2 / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B, 2)
+                  : make_tmap(&ta, A, M, K2, K2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B, 2);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tb, B, N, K2, K2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B, 2);
+  if (st != SF_OK) return st;
+  tm = ta;
+  if (sparse) {
+    // per 128 rows and 256 logical K: two 2 KB atoms = four rows of the [4 * atom pairs, 256] uint32 view
+    const int64_t pairs = (M / 128) * (K / 256);
+    st = make_tmap(&tm, meta_hw, 4 * pairs, 256, 256, 256, 4, CU_TENSOR_MAP_SWIZZLE_NONE, 1);
+    if (st != SF_OK) return st;
+  }
+  GemmArgs a{};
+  a.M = M; a.N = N; a.K = K2;
+  a.C = C; a.ldc = ldc; a.meta_hw = meta_hw; a.status = status; a.out_scale = alpha;
+  a.num_k_blocks = (int)(K2 / 64);
+  if (sparse) return launch_two<MODE_SPARSE24, false, false, EPI_STORE, BN, 0, true>(ta, tb, tm, a, s);
+  return launch_two<MODE_DENSE, false, false, EPI_STORE, BN, 0, true>(ta, tb, tm, a, s);
 }
 
 bool gemm_sparse24_vnm8_supported(int64_t F, int64_t T, int64_t D, int V) {

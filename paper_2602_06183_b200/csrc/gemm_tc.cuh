@@ -67,6 +67,8 @@ struct GemmArgs {
   const int* num_tiles_dev;  // device word holding the number of valid entries of tile_table
   // EPI_STORE only, optional: output row r of the product is written to row row_map[r] of C (skipped when < 0)
   const int* row_map;
+  // EPI_STORE only: the accumulator is multiplied by this before rounding (0 = no scaling)
+  float out_scale;
 };
 
 // Outputs of the fused y1 product (see GemmArgs::vn_*).
@@ -124,6 +126,11 @@ int gemm_grouped_dense_tn(const void* A, int64_t Ma, const void* B, int64_t Nb, 
 int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t M, int64_t N,
                   int64_t K, int epi, void* C, int64_t ldc, const void* aux, int64_t ldaux, int* status,
                   cudaStream_t s, const void* pack_meta = nullptr, void* pack_vals = nullptr);
+// E4M3 operands, both K-major: C[M, N] = bf16(alpha * A B^T). sparse: A = 2:4 values [M, K/2] (codes) with
+// metadata in the 8-bit instruction's order (see meta_hw8_offset); else A [M, K]. B [N, K].
+// M % 256 == 0, N % 32 == 0, K % 256 == 0 (2:4) or K % 128 == 0 (dense).
+int gemm_fp8(bool sparse, const void* A, const uint8_t* meta_hw, const void* B, int64_t M, int64_t N, int64_t K,
+             float alpha, void* C, int64_t ldc, int* status, cudaStream_t s);
 // C[T,N] = A_vnm[T,F] Bt[F,N]; A_vnm packed (vals [T, 2F/Mv], hardware-ordered metadata, colidx).
 int gemm_venom(const void* a_vals, const uint8_t* meta_hw, const uint8_t* colidx, const void* Bt, int64_t T,
                int64_t F, int64_t N, int V, int Mv, void* C, int64_t ldc, int* status, cudaStream_t s);

@@ -116,4 +116,13 @@ __host__ __device__ __forceinline__ size_t meta_hw_offset(int64_t m, int64_t kw,
          (kwi >> 1) * 4 + ((mi >> 3) & 1) * 2;
 }
 
+// The same for an 8-bit (E4M3) 2:4 operand: per 128 rows and 256 columns a pair of 2 KB atoms (128 columns
+// each); inside an atom the rows are plain: 16 bytes per row, the eight 16-column words in order.
+__host__ __device__ __forceinline__ size_t meta_hw8_offset(int64_t m, int64_t kw, int64_t K) {
+  const int64_t pairs_per_rowblock = K >> 8;
+  const int64_t pair = (m >> 7) * pairs_per_rowblock + (kw >> 4);
+  const int mi = static_cast<int>(m & 127), kwi = static_cast<int>(kw & 15);
+  return static_cast<size_t>(pair) * 4096 + (kwi >> 3) * 2048 + mi * 16 + (kwi & 7) * 2;
+}
+
 }  // namespace sf

@@ -246,6 +246,30 @@ __device__ __forceinline__ void mma_sp_f16_2cta(uint32_t tmem_d, uint64_t adesc,
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(tmem_e), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same two instructions for 8-bit floating-point operands (kind::f8f6f4: K = 32 per dense instruction,
+// 64 logical K per 2:4 instruction; the operand formats sit in the instruction descriptor).
+__device__ __forceinline__ void mma_f8_2cta(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t"
+      "}\n"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_sp_f8_2cta(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t tmem_e,
+                                               uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.sp.cta_group::2.kind::f8f6f4 [%0], %1, %2, [%3], %4, p;\n\t"
+      "}\n"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(tmem_e), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // Arrive on the barrier at this offset in both CTAs of the pair once all prior MMAs are done.
 __device__ __forceinline__ void mma_commit_2cta(uint64_t* bar) {
   asm volatile(
@@ -277,6 +301,11 @@ __host__ __device__ constexpr uint32_t idesc_bf16(uint32_t M, uint32_t N, bool a
                                                   bool sparse) {
   return (sparse ? (1u << 2) : 0u) | (1u << 4) /* D = f32 */ | (1u << 7) /* A = bf16 */ | (1u << 10) /* B = bf16 */ |
          ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+// Instruction descriptor for kind::f8f6f4 with E4M3 A and B (format code 0), both K-major, fp32 D.
+__host__ __device__ constexpr uint32_t idesc_e4m3(uint32_t M, uint32_t N, bool sparse) {
+  return (sparse ? (1u << 2) : 0u) | (1u << 4) /* D = f32 */ | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
 }  // namespace ptx
