@@ -52,8 +52,10 @@ typedef enum sf_status {
 } sf_status;
 
 /* Problem descriptor of one FFN layer step. Ragged shapes are rejected, never padded:
- * T, D, F multiples of 256 (the tile of a CTA pair, which every product of the step runs on),
- * T % V == 0, (4F/M) % 128 == 0, V in {64,128}, N == 2, M in {4,8,16,32,64}. */
+ * T, D, F multiples of 128 and at least 256 (every product runs on 256-row tiles of a CTA pair; the
+ * last pair of a product may be half empty), T % V == 0, F % (4 M) == 0, V in {64,128}, N == 2,
+ * M in {4,8,16,32,64}. With M >= 16 (products on the gathered Venom kernel) or with
+ * SF_FFN_PACKED_GRAD_OPERANDS: multiples of 256, and (4F/M) % 128 == 0 for M >= 16. */
 typedef enum sf_ffn_flags {
   SF_FFN_SAVE_Y1 = 1,     /* also store the full bf16 pre-activation y1 in the context (SF_CTX_Y1) */
   SF_FFN_UNFUSED_ACT = 2, /* M == 8: run SquaredReLU + V:N:M as its own kernel on a stored y1, never inside the

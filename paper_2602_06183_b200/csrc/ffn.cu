@@ -195,8 +195,12 @@ int check_desc(const sf_ffn_desc* d) {
   if ((d->flags & SF_FFN_UNFUSED_ACT) && (d->flags & SF_FFN_FUSED_ACT)) return SF_ERR_UNSUPPORTED;
   if (d->V != 64 && d->V != 128) return SF_ERR_SHAPE;
   if (d->T <= 0 || d->D <= 0 || d->F <= 0) return SF_ERR_SHAPE;
-  if (d->T % 256 || d->D % 256 || d->F % 256 || d->T % d->V) return SF_ERR_SHAPE;
-  if ((4 * d->F / d->M) % 128) return SF_ERR_SHAPE;
+  // every product runs on 256-row CTA-pair tiles whose last pair may be half empty: multiples of 128, at least 256.
+  // The gathered Venom products (M >= 16) and the operand expander keep whole 256-wide tiles.
+  const int64_t q = (d->M >= 16 || (d->flags & SF_FFN_PACKED_GRAD_OPERANDS)) ? 256 : 128;
+  if (d->T % q || d->D % q || d->F % q || d->T < 256 || d->D < 256 || d->F < 256 || d->T % d->V) return SF_ERR_SHAPE;
+  if (d->F % (4 * d->M)) return SF_ERR_SHAPE;                            // whole metadata words
+  if (d->M >= 16 && (4 * d->F / d->M) % 128) return SF_ERR_SHAPE;         // condensed reduction in whole stages
   if (d->prune_mode != 0 && d->prune_mode != 1) return SF_ERR_SHAPE;
   return SF_OK;
 }

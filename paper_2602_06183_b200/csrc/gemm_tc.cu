@@ -1058,8 +1058,16 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
       const uint32_t taddr = tmem_base + set * kBN + ((uint32_t)(q * 32) << 16);
       if (!mbar_wait(&ctl->tmem_full[set], acc_phase, abort_flag)) break;
       tc_fence_after();
-      // releases the accumulator itself, as soon as its last column has been read
-      epi_vnm8_tile<kBN, kV>(args, taddr, m0, n0, args.N, q, lane, wsm, &ctl->tmem_empty[set]);
+      if (m0 >= args.M) {
+        // M % 256 == 128: the second CTA of the last row of pairs holds no rows (its operand loads were
+        // zero-filled); it only hands the accumulator back
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_leader(&ctl->tmem_empty[set]);
+      } else {
+        // releases the accumulator itself, as soon as its last column has been read
+        epi_vnm8_tile<kBN, kV>(args, taddr, m0, n0, args.N, q, lane, wsm, &ctl->tmem_empty[set]);
+      }
       acc_phase ^= 1;
     }
   } else {
@@ -1073,10 +1081,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
       const int64_t m0 = (int64_t)tc.out_m + (int64_t)rank * 128, n0 = tc.out_n, n_limit = tc.n_limit;
       const uint32_t taddr = tmem_base + acc * kBN + ((uint32_t)(q * 32) << 16);
       uint4 ax[is_drelu_t(kEpi) ? kBN / 32 : 1][4];
-      epi_prefetch<kEpi, kBN>(args, m0, n0, n_limit, q, lane, ax);
+      // M % 256 == 128 (regular raster only): the second CTA of the last row of pairs holds no rows
+      const bool live = args.tile_table != nullptr || m0 < args.M;
+      if (live) epi_prefetch<kEpi, kBN>(args, m0, n0, n_limit, q, lane, ax);
       if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      epi_tile<kEpi, kBN>(args, taddr, m0, n0, n_limit, q, lane, my_stage, ax);
+      if (live) epi_tile<kEpi, kBN>(args, taddr, m0, n0, n_limit, q, lane, my_stage, ax);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(&ctl->tmem_empty[acc]);
@@ -1179,7 +1189,7 @@ int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
     SF_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     if (dev >= 0 && dev < 64) attr_done[dev] = true;
   }
-  a.num_m_tiles = (int)(a.M / 256);
+  a.num_m_tiles = (int)((a.M + 255) / 256);
   a.num_n_tiles = (int)((a.N + kBN - 1) / kBN);
   // table-driven products: the table's length is on the device; launch for its upper bound
   const int tiles = a.tile_table ? a.num_k_blocks /* upper bound, see the grouped launchers */
@@ -1198,8 +1208,9 @@ int launch_two(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
 #endif
 constexpr int kNarrowBN = SF_NARROW_BN;
 
-// The two-CTA kernels need M % 256 == 0; other shapes run the one-CTA kernels.
-bool use_two_cta(int64_t M) { return M % 256 == 0; }
+// CTA pairs work on 256-row tiles; with M % 256 == 128 the second CTA of the last row of pairs runs on
+// zero-filled operand rows and stores nothing. A single 128-row block runs the one-CTA kernels.
+bool use_two_cta(int64_t M) { return M >= 256; }
 
 }  // namespace
 
@@ -1212,9 +1223,9 @@ int make_tmap_2d(void* map, const void* base, int64_t rows, int64_t cols, int64_
 int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64_t M, int64_t N, int64_t K, int epi,
                void* C, int64_t ldc, void* C2, int64_t ldc2, const void* aux, int64_t ldaux, int* status,
                cudaStream_t s) {
-  if (M % BM || N % BN || K % 64) return SF_ERR_SHAPE;
-  if (M == 0 || N == 0) return SF_OK;
   const bool two = use_two_cta(M);
+  if (M % BM || N % (two ? 128 : BN) || K % 64) return SF_ERR_SHAPE;     // pairs: a ragged last tile of whole 32-column chunks
+  if (M == 0 || N == 0) return SF_OK;
   CUtensorMap ta, tb;
   int st;
   if (a_kmajor) st = make_tmap(&ta, A, M, K, K, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -1250,10 +1261,10 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
                   int64_t K, int epi, void* C, int64_t ldc, const void* aux, int64_t ldaux, int* status,
                   cudaStream_t s, const void* pack_meta, void* pack_vals) {
   if ((pack_meta != nullptr) != (pack_vals != nullptr) || (pack_vals && !is_drelu_t(epi))) return SF_ERR_UNSUPPORTED;
-  if (epi == EPI_DRELU24_T && (!pack_vals || !aux || M % 256)) return SF_ERR_UNSUPPORTED;   // C (dense copy) optional
-  if (M % BM || N % BN || K % 128) return SF_ERR_SHAPE;
-  if (M == 0 || N == 0) return SF_OK;
   const bool two = use_two_cta(M);
+  if (epi == EPI_DRELU24_T && (!pack_vals || !aux || !two)) return SF_ERR_UNSUPPORTED;   // C (dense copy) optional
+  if (M % BM || N % (two ? 128 : BN) || K % 128) return SF_ERR_SHAPE;
+  if (M == 0 || N == 0) return SF_OK;
   const bool plain = (epi == EPI_STORE);                 // row-major output, either B layout: two-CTA kernel only
   if ((plain || !b_kmajor) && !two) return SF_ERR_UNSUPPORTED;
   CUtensorMap ta, tb, tm;
@@ -1319,7 +1330,7 @@ int gemm_fp8(bool sparse, const void* A, const uint8_t* meta_hw, const void* B, 
 }
 
 bool gemm_sparse24_vnm8_supported(int64_t F, int64_t T, int64_t D, int V) {
-  return F > 0 && T > 0 && F % 256 == 0 && D % 128 == 0 && (V == 64 || V == 128) && T % V == 0;
+  return F >= 256 && T > 0 && F % 128 == 0 && D % 128 == 0 && (V == 64 || V == 128) && T % V == 0;
 }
 
 int gemm_sparse24_vnm8(const void* a_vals, const uint8_t* meta_hw, const void* X, int64_t F, int64_t T, int64_t D,

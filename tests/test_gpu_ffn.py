@@ -210,8 +210,22 @@ def test_sparse_ffn_smallest_and_odd_tile_counts(T, D, F, V, M):
     _check_against_oracle(inputs, g, cfg)
 
 
-def test_dense_ffn_c1():
-    cfg = synth.FFN_CONFIGS["c1_small"]
+@pytest.mark.parametrize("T,D,F,V,M", [(384, 384, 640, 64, 8), (640, 384, 384, 128, 8), (896, 640, 384, 64, 8),
+                                       (384, 640, 896, 64, 4), (384, 384, 1152, 128, 8)])
+@pytest.mark.parametrize("flags", [binding.SF_FFN_SAVE_Y1, binding.SF_FFN_SAVE_Y1 | binding.SF_FFN_UNFUSED_ACT],
+                         ids=["default", "two_kernel"])
+def test_sparse_ffn_odd_multiples_of_128(T, D, F, V, M, flags):
+    """T, D or F = 128 (mod 256): the last row of CTA pairs of a product is half empty (its second CTA works
+    on zero-filled rows and must store nothing: the guard zones around every buffer check that too)."""
+    cfg = dict(T=T, D=D, F=F, V=V, N=2, M=M, sigma_w=0.05, seed=T + 2 * D + 3 * F)
+    for prune_mode in (0, 1):
+        inputs, g = _run_sparse(cfg, prune_mode, flags=flags)
+        _check_against_oracle(inputs, g, cfg, prune_mode)
+
+
+@pytest.mark.parametrize("name", ["c1_small", "odd128"])
+def test_dense_ffn_c1(name):
+    cfg = synth.FFN_CONFIGS["c1_small"] if name == "c1_small" else dict(T=384, D=640, F=896, V=64, M=8, sigma_w=0.05, seed=77)
     T, D, F = cfg["T"], cfg["D"], cfg["F"]
     X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
     desc = binding.make_desc(T, D, F, cfg["V"], cfg["M"])
@@ -319,10 +333,13 @@ def test_sparse_step_replays_from_a_cuda_graph():
 
 
 def test_ffn_rejects_ragged_shapes():
-    desc = binding.make_desc(1000, 256, 1024, 64, 8)
-    with pytest.raises(binding.SparseFFNError) as e:
-        binding.sf_ffn_workspace_size(desc)
-    assert e.value.status == binding.SF_ERR_SHAPE
+    for shape in [(1000, 256, 1024, 64, 8), (128, 256, 1024, 64, 8),      # not a multiple of 128; a single 128-row block
+                  (384, 256, 1024, 128, 16),                                # gathered Venom products keep whole 256-row tiles
+                  (512, 384, 1024, 128, 32)]:
+        desc = binding.make_desc(*shape)
+        with pytest.raises(binding.SparseFFNError) as e:
+            binding.sf_ffn_workspace_size(desc)
+        assert e.value.status == binding.SF_ERR_SHAPE
     desc = binding.make_desc(1024, 256, 1024, 64, 8, N=1)
     with pytest.raises(binding.SparseFFNError) as e:
         binding.sf_ffn_workspace_size(desc)
@@ -363,22 +380,23 @@ def test_scheduled_steps_dispatch_to_the_right_kind():
 
 
 def _legal_random_configs(n, seed):
-    """Seeded draw of legal step shapes: T, D, F multiples of 256, V in {64, 128}, M in {4..32},
-    condensed reduction 4F/M a multiple of 128, both prune modes, symmetric or ~90 %-negative
-    pre-activations."""
+    """Seeded draw of legal step shapes: T, D, F multiples of 128 from 256 up (of 256 for M >= 16, whose gathered
+    products keep whole tiles), V in {64, 128}, M in {4..32}, whole metadata words, condensed reduction 4F/M a
+    multiple of 128 for M >= 16, both prune modes, symmetric or ~90 %-negative pre-activations."""
     rng = np.random.default_rng(seed)
     out = []
     while len(out) < n:
-        T, D, F = (int(rng.integers(1, 4)) * 256 for _ in range(3))
-        F *= int(rng.integers(1, 3))
         V, M = int(rng.choice([64, 128])), int(rng.choice([4, 8, 16, 32]))
-        if (4 * F // M) % 128:
+        q = 256 if M >= 16 else 128
+        T, D, F = (int(rng.integers(256 // q, 1024 // q + 1)) * q for _ in range(3))
+        F *= int(rng.integers(1, 3))
+        if T % V or F % (4 * M) or (M >= 16 and (4 * F // M) % 128):
             continue
         out.append((T, D, F, V, M, int(rng.integers(0, 2)), float(rng.choice([0.0, -1.3])), int(rng.integers(1, 1 << 20))))
     return out
 
 
-@pytest.mark.parametrize("T,D,F,V,M,prune_mode,act_shift,seed", _legal_random_configs(10, seed=20260206))
+@pytest.mark.parametrize("T,D,F,V,M,prune_mode,act_shift,seed", _legal_random_configs(12, seed=20260206))
 def test_sparse_ffn_random_legal_shapes(T, D, F, V, M, prune_mode, act_shift, seed):
     cfg = dict(T=T, D=D, F=F, V=V, N=2, M=M, sigma_w=0.05, seed=seed)
     inputs, g = _run_sparse(cfg, prune_mode, act_shift)
