@@ -39,7 +39,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "sparse_ffn_fwd_bwd_dense_equiv_tflops"
 UNIT = "TFLOP/s"
-SWEEP_WORKLOADS = ("c2_prune", "c3_act", "gemm_micro")
+SWEEP_WORKLOADS = ("c2_prune", "c3_act", "gemm_micro", "fp8_micro")
 
 
 def _peaks():
@@ -493,7 +493,8 @@ def run_sweep(args):
         metric, unit, value = "vnm_sparsify_min_frac_of_measured_hbm", "fraction", min(r["frac_of_hbm"] for r in results)
         note = "2 + 4/M + 0.5/M + 4/M (ReLU values) bytes per element + colidx; 537 MB input, larger than the L2"
     else:
-        for (m, n, k) in [(4096, 16384, 4096), (16384, 8192, 4096), (8192, 4096, 16384)]:
+        shapes = [(4096, 16384, 4096)] if args.workload == "fp8_micro" else [(4096, 16384, 4096), (16384, 8192, 4096), (8192, 4096, 16384)]
+        for (m, n, k) in shapes:
             A = torch.randn((m, k), device="cuda").to(torch.bfloat16)
             B = torch.randn((n, k), device="cuda").to(torch.bfloat16)
             Cm = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
@@ -524,23 +525,24 @@ def run_sweep(args):
                             "speedup_gemm_only": ms_d8 / ms_s8, "speedup_with_prune": ms_d8 / (ms_s8 + ms_p8),
                             "speedup_vs_bf16_dense": ms_d / ms_s8})
             del A, B, Cm, vals, meta, Aq, Bq, o8
-        Tn, Fn, Nn = 8192, 16384, 4096
-        A = torch.randn((Tn, Fn), device="cuda").to(torch.bfloat16)
-        Bd = torch.randn((Nn, Fn), device="cuda").to(torch.bfloat16)
-        Cd = torch.empty((Tn, Nn), dtype=torch.bfloat16, device="cuda")
-        wsd = torch.zeros((binding.sf_gemm_workspace_size(Tn, Fn),), dtype=torch.uint8, device="cuda")
-        ms_dense = _time_cuda(lambda: binding.sf_gemm_dense(A, True, Bd, True, C_out=Cd, workspace=wsd), iters, args.warmup)
-        del A, Bd, Cd
-        for M in (8, 16, 32, 64):
-            P = dev(synth.normal_bf16((Tn, Fn), 0.0, 1.0, seed=7))
-            vals, meta, colidx, _, _ = binding.sf_vnm_sparsify_act(P, 128, M)
-            Bt = torch.randn((Fn, Nn), device="cuda").to(torch.bfloat16)
-            Cm = torch.empty((Tn, Nn), dtype=torch.bfloat16, device="cuda")
-            wsb = torch.zeros((binding.sf_gemm_workspace_size(Tn, Fn),), dtype=torch.uint8, device="cuda")
-            ms_v = _time_cuda(lambda: binding.sf_gemm_venom(vals, meta, colidx, Bt, 128, M, C_out=Cm, workspace=wsb), iters, args.warmup)
-            results.append({"product": "Venom vs dense", "T": Tn, "F": Fn, "N": Nn, "V": 128, "M": M,
-                            "sparsity_pct": 100.0 * (1 - 2.0 / M), "ms": ms_v, "dense_ms": ms_dense,
-                            "speedup_vs_dense": ms_dense / ms_v})
+        if args.workload == "gemm_micro":
+            Tn, Fn, Nn = 8192, 16384, 4096
+            A = torch.randn((Tn, Fn), device="cuda").to(torch.bfloat16)
+            Bd = torch.randn((Nn, Fn), device="cuda").to(torch.bfloat16)
+            Cd = torch.empty((Tn, Nn), dtype=torch.bfloat16, device="cuda")
+            wsd = torch.zeros((binding.sf_gemm_workspace_size(Tn, Fn),), dtype=torch.uint8, device="cuda")
+            ms_dense = _time_cuda(lambda: binding.sf_gemm_dense(A, True, Bd, True, C_out=Cd, workspace=wsd), iters, args.warmup)
+            del A, Bd, Cd
+            for M in (8, 16, 32, 64):
+                P = dev(synth.normal_bf16((Tn, Fn), 0.0, 1.0, seed=7))
+                vals, meta, colidx, _, _ = binding.sf_vnm_sparsify_act(P, 128, M)
+                Bt = torch.randn((Fn, Nn), device="cuda").to(torch.bfloat16)
+                Cm = torch.empty((Tn, Nn), dtype=torch.bfloat16, device="cuda")
+                wsb = torch.zeros((binding.sf_gemm_workspace_size(Tn, Fn),), dtype=torch.uint8, device="cuda")
+                ms_v = _time_cuda(lambda: binding.sf_gemm_venom(vals, meta, colidx, Bt, 128, M, C_out=Cm, workspace=wsb), iters, args.warmup)
+                results.append({"product": "Venom vs dense", "T": Tn, "F": Fn, "N": Nn, "V": 128, "M": M,
+                                "sparsity_pct": 100.0 * (1 - 2.0 / M), "ms": ms_v, "dense_ms": ms_dense,
+                                "speedup_vs_dense": ms_dense / ms_v})
         metric, unit, value = "sparse24_gemm_speedup_vs_dense_at_4096x16384x4096", "ratio", results[0]["speedup_gemm_only"]
         note = "Section 5.2.3's micro-benchmark shape first; Venom products at Table 5's sparsities"
     print(json.dumps({"metric": metric, "value": value, "unit": unit, "n_gpus": 1, "steps": iters, "warmup": args.warmup,

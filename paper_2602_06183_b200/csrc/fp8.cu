@@ -205,14 +205,9 @@ int sf_gemm_fp8_sparse24(const void* a_vals, const void* a_meta, const void* B, 
   SF_TRY(check_arch());
   cudaStream_t s = (cudaStream_t)stream;
   uint8_t* hw = reinterpret_cast<uint8_t*>(workspace) + kStatusBytes8;
-#ifdef SF_FP8_PROBE
-  // probe build: a_meta is already in raw hardware order
-  SF_CUDA_TRY(cudaMemcpyAsync(hw, a_meta, (size_t)Mr * K / 8, cudaMemcpyDeviceToDevice, s));
-#else
   const int64_t n = Mr * (K >> 4);
   meta_reorder8_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>((const uint16_t*)a_meta, hw, Mr, K);
   SF_LAUNCH_CHECK();
-#endif
   return gemm_fp8(true, a_vals, hw, B, Mr, Nc, K, alpha, C, Nc, (int*)workspace, s);
 }
 

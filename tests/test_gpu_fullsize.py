@@ -233,3 +233,38 @@ def test_routed_step_full_size_sampled(E):
         dy1g = np.where(keep, dy1g, np.uint16(0))
         dW1_ref = f64(dy1g).T @ f64(X[te])
         assert rel_fro(f32(gW1[gft]), dW1_ref) < TOL
+
+
+@pytest.mark.parametrize("m,n,k", [(4096, 16384, 4096), (8192, 4096, 16384)])
+def test_fp8_products_full_size_sampled(m, n, k):
+    """The E4M3 route at the micro-benchmark's shapes: prune + quantise on the GPU checked bit for bit on sampled
+    rows, the dense and the 2:4 product on sampled rows x sampled columns against float64 products of the
+    oracle's codes."""
+    from oracle import fp8
+    w = synth.prune_sweep_matrix(m, k, seed=31, tie_frac=0.02)
+    x = synth.normal_bf16((n, k), 0, 1, seed=32)
+    sw, sx = 3000.0, 32.0
+    alpha = 1.0 / (sw * sx)
+    wd, xd = to_dev(w), to_dev(x)
+    vals, meta, _ = binding.sf_prune24_compress_fp8(wd, 0, sw)
+    wq, xq = binding.sf_fp8_quantize(wd, sw), binding.sf_fp8_quantize(xd, sx)
+    outs = Guarded((m, n), torch.bfloat16), Guarded((m, n), torch.bfloat16)
+    Cs, ws = binding.sf_gemm_fp8_sparse24(vals, meta, xq, alpha, C_out=outs[0].t)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    Cd, ws = binding.sf_gemm_fp8_dense(wq, xq, alpha, C_out=outs[1].t)
+    assert binding.sf_check_status(ws) == binding.SF_OK
+    for o in outs:
+        o.check("fp8 product")
+    rng = np.random.default_rng(m + n)
+    rows = np.sort(np.concatenate([rng.choice(m, size=93, replace=False), [0, m - 129, m - 1]]))
+    cols = np.sort(np.concatenate([rng.choice(n, size=381, replace=False), [0, n - 225, n - 1]]))
+    rt, ct = torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()
+    p = fp8.prune24_fp8(w[rows], sw)
+    assert np.array_equal(vals[rt].cpu().numpy(), p.vals) and np.array_equal(bits(meta[rt]), p.meta)
+    xq_ref = fp8.quantize_fp8(x[cols], sx)
+    assert np.array_equal(xq[ct].cpu().numpy(), xq_ref)
+    for C, a_codes, what in ((Cs, p.dense, "fp8 2:4 product"), (Cd, fp8.quantize_fp8(w[rows], sw), "fp8 dense product")):
+        got = f32(C[rt][:, ct])
+        ref = fp8.gemm_fp8(a_codes, xq_ref, alpha)
+        assert rel_fro(got, ref) < TOL, what
+        assert_close_elementwise(got, ref, k, what)
