@@ -175,8 +175,8 @@ SF_API int sf_gemm_venom(const void* a_vals, const void* a_meta, const void* col
  *     start-up, outside any stream capture, from one host thread; later calls take no memory.
  *   - All calls share the one array: two calls that may overlap on the GPU (different streams,
  *     or different host threads) race on it. Serialise them on one stream.
- *   - A bounded-wait expiry is recorded in the built-in status word, which no call reads back;
- *     use sf_gemm_sparse24 + sf_check_status where that matters. */
+ *   - A bounded-wait expiry is recorded in the array's own status word, which every call clears
+ *     before its kernels start; sf_check_status(NULL, stream) reads it (and allocates nothing). */
 SF_API int sf_gemm_sparse24_noalloc(const void* a_vals, const void* a_meta, const void* B, void* Ct,
                                     int64_t Mr, int64_t Nc, int64_t K, void* stream);
 
@@ -427,7 +427,9 @@ SF_API int sf_trace_set(void** events, int capacity);
 SF_API int sf_trace_count(void);
 
 /* Synchronises `stream` and reads the device status word kept at the start of `workspace`:
- * SF_OK, or SF_ERR_TIMEOUT if a bounded wait inside a tensor-core kernel expired. */
+ * SF_OK, or SF_ERR_TIMEOUT (once; the word is cleared) if a bounded wait inside a tensor-core
+ * kernel expired. workspace == NULL names the status word of sf_gemm_sparse24_noalloc's built-in
+ * scratch array on the current device. */
 SF_API int sf_check_status(void* workspace, void* stream);
 
 #ifdef __cplusplus

@@ -675,7 +675,11 @@ int sf_trace_set(void** events, int capacity) {
 int sf_trace_count(void) { return g_trace_n; }
 
 int sf_check_status(void* workspace, void* stream) {
-  if (!workspace) return SF_ERR_NULL;
+  if (!workspace) {
+    // the status word of sf_gemm_sparse24_noalloc's built-in scratch array (no allocation here either)
+    SF_TRY(check_arch());
+    SF_TRY(noalloc_status_word(&workspace));
+  }
   cudaStream_t s = (cudaStream_t)stream;
   SF_CUDA_TRY(cudaStreamSynchronize(s));
   int host = 0;

@@ -35,6 +35,15 @@ int noalloc_scratch(unsigned char** out) {
 }
 
 }  // namespace
+
+// Device address of the built-in status word (sf_check_status with a null workspace reads it).
+int noalloc_status_word(void** out) {
+  unsigned char* p = nullptr;
+  const int st = noalloc_scratch(&p);
+  *out = p;
+  return st;
+}
+
 }  // namespace sf
 
 using namespace sf;

@@ -102,6 +102,8 @@ bool vnm_stream_supported(int64_t F, int64_t ld, int V, int M, const void* P);
 int launch_vnm_stream(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu, void* vals,
                       void* meta, void* colidx, void* relu_vals, cudaStream_t s);
 int launch_transpose(const void* in, void* out, int64_t rows, int64_t cols, cudaStream_t s);
+// Device address of the status word of the built-in scratch array (sf_gemm_sparse24_noalloc).
+int noalloc_status_word(void** out);
 // Records the next caller-owned trace event on `s` while stage tracing is on (sf_trace_set); else a no-op.
 void trace_mark(cudaStream_t s);
 

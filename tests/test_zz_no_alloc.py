@@ -40,6 +40,8 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row():
         torch.cuda.synchronize()
         assert allocs() == before                                              # nothing through torch's allocator
         assert torch.cuda.mem_get_info()[0] == free_before                     # and nothing from the driver either
+        assert binding.sf_check_status(None) == binding.SF_OK                  # the built-in status word: no expired wait
+        assert torch.cuda.mem_get_info()[0] == free_before
         # against the float64 product of the oracle's pruned matrix, then against the regular entry point
         assert rel_fro(f32(out), oracle_ref) < 1e-2
         assert_close_elementwise(f32(out), oracle_ref, K, "no-allocation 2:4 product")
