@@ -88,32 +88,45 @@ vnm_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t 
       const int cvalid = (int)min((int64_t)kSW, F - cx * kSW);
       Aux& a = aux[slot];
       if (!mbar_wait(&ctl->full[slot], phase, abort_flag)) break;
-      // columns 2 ts and 2 ts + 1, rows first to last, one float32 add per element
-      const uint32_t* col = reinterpret_cast<const uint32_t*>(smem + slot * strip_bytes) + ts;
-      float s0 = 0.f, s1 = 0.f;
-      if (2 * ts < kSW)
-      for (int r = 0; r < V; r += 8) {
-        uint32_t h[8];
+      // rows first to last, one float32 add per element: two columns per thread (256-column strips) or one
+      if constexpr (kSW == 256) {
+        const uint32_t* col = reinterpret_cast<const uint32_t*>(smem + slot * strip_bytes) + ts;
+        float s0 = 0.f, s1 = 0.f;
+        for (int r = 0; r < V; r += 8) {
+          uint32_t h[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const uint32_t w = col[(r + u) * (kSW / 2)];
-          h[u] = apply ? bf2_sq(bf2_relu(w)) : (w & 0x7FFF7FFFu);
-        }
+          for (int u = 0; u < 8; ++u) {
+            const uint32_t w = col[(r + u) * (kSW / 2)];
+            h[u] = apply ? bf2_sq(bf2_relu(w)) : (w & 0x7FFF7FFFu);
+          }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          s0 = __fadd_rn(s0, __uint_as_float(h[u] << 16));
-          s1 = __fadd_rn(s1, __uint_as_float(h[u] & 0xFFFF0000u));
+          for (int u = 0; u < 8; ++u) {
+            s0 = __fadd_rn(s0, __uint_as_float(h[u] << 16));
+            s1 = __fadd_rn(s1, __uint_as_float(h[u] & 0xFFFF0000u));
+          }
         }
-      }
-      if (2 * ts < kSW) {
         a.score[2 * ts] = __float_as_uint(s0);
         a.score[2 * ts + 1] = __float_as_uint(s1);
+      } else {
+        const uint16_t* col = reinterpret_cast<const uint16_t*>(smem + slot * strip_bytes) + ts;
+        float s0 = 0.f;
+        for (int r = 0; r < V; r += 16) {
+          uint32_t h[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            const uint32_t w = col[(r + u) * kSW];
+            h[u] = apply ? bf2_sq(bf2_relu(w)) : (w & 0x7FFFu);
+          }
+#pragma unroll
+          for (int u = 0; u < 16; ++u) s0 = __fadd_rn(s0, __uint_as_float(h[u] << 16));
+        }
+        a.score[ts] = __float_as_uint(s0);
       }
       named_sync(1, 128);
+      constexpr int kCPT = kSW / 128;                          // columns per scoring thread
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        const int j = 2 * ts + c, jm = j & (kM - 1), base = j - jm;
-        if (j >= kSW) break;
+      for (int c = 0; c < kCPT; ++c) {
+        const int j = kCPT * ts + c, jm = j & (kM - 1), base = j - jm;
         const uint32_t s = a.score[j];
         int rank = 0;
 #pragma unroll 8
@@ -125,9 +138,8 @@ vnm_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t 
       }
       named_sync(1, 128);
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        const int j = 2 * ts + c, jm = j & (kM - 1), base = j - jm;
-        if (j >= kSW) break;
+      for (int c = 0; c < kCPT; ++c) {
+        const int j = kCPT * ts + c, jm = j & (kM - 1), base = j - jm;
         if (a.keep[j]) {
           int pos = 0;
           for (int k = 0; k < jm; ++k) pos += a.keep[base + k];
