@@ -68,24 +68,27 @@ __device__ __forceinline__ uint32_t top2of4(uint32_t k0, uint32_t k1, uint32_t k
 // the third-ranked element.
 __device__ __forceinline__ uint32_t top2of4_packed(uint32_t lo, uint32_t hi, uint32_t* packed,
                                                    uint32_t* third_idx = nullptr, uint32_t* perm_sel = nullptr) {
-  const uint32_t c0 = ((lo << 2) & 0x1FFFCu) | 3u, c1 = ((lo >> 14) & 0x1FFFCu) | 2u;
-  const uint32_t c2 = ((hi << 2) & 0x1FFFCu) | 1u, c3 = ((hi >> 14) & 0x1FFFCu);
+  // The integer-logic pipe is what these kernels run out of, so the widening is written as multiply-adds
+  // (x * 4 + index term; x >> 14 as the high half of x * 2^18), which issue on the FMA pipe.
+  const uint32_t c0 = (lo & 0x7FFFu) * 4u + 3u, c1 = __umulhi(lo & 0x7FFF0000u, 1u << 18) + 2u;
+  const uint32_t c2 = (hi & 0x7FFFu) * 4u + 1u, c3 = __umulhi(hi & 0x7FFF0000u, 1u << 18);
   const uint32_t h01 = max(c0, c1), l01 = min(c0, c1), h23 = max(c2, c3), l23 = min(c2, c3);
   const uint32_t top1 = max(h01, h23), mid = min(h01, h23);
-  const bool first_pair_wins = h01 > h23;
-  const uint32_t under = first_pair_wins ? l01 : l23;        // partner of the winner
-  const uint32_t top2 = max(mid, under);
-  const uint32_t ia = 3u - (top1 & 3u), ib = 3u - (top2 & 3u);
+  // second overall = the larger of the losing pair-winner and the two pair-losers
+  const uint32_t top2 = max(mid, max(l01, l23));
+  const uint32_t ia = ~top1 & 3u, ib = ~top2 & 3u;           // 3 - (key & 3)
   const uint32_t p0 = min(ia, ib), p1 = max(ia, ib);
   // byte permute: bytes (2p0, 2p0+1) then (2p1, 2p1+1) out of the 8 bytes {lo, hi}
   const uint32_t sel = 0x1010u + p0 * 0x22u + p1 * 0x2200u;
   *packed = __byte_perm(lo, hi, sel);
   if (perm_sel) *perm_sel = sel;             // the same selector picks the pair out of any other {lo, hi}
   if (third_idx) {
-    const uint32_t other_low = first_pair_wins ? l23 : l01;
-    *third_idx = 3u - (max(min(mid, under), other_low) & 3u);
+    // third overall = the smaller of the losing pair-winner and the winner's partner, or the other pair's loser
+    const bool first_pair_wins = h01 > h23;
+    const uint32_t under = first_pair_wins ? l01 : l23, other_low = first_pair_wins ? l23 : l01;
+    *third_idx = ~max(min(mid, under), other_low) & 3u;
   }
-  return p0 | (p1 << 2);
+  return p1 * 4u + p0;
 }
 
 // ---- internal launchers (defined in the .cu files) ---------------------------------------
