@@ -75,6 +75,9 @@ template <bool kSoft>
 __global__ void __launch_bounds__(256)
 prune24_fp8_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t ld, float scale,
                    uint32_t* __restrict__ vals, uint32_t* __restrict__ meta, uint2* __restrict__ dense_out) {
+  __shared__ uint32_t lut[16];
+  top2_lut_init(lut, threadIdx.x);
+  __syncthreads();
   const uint32_t upr = (uint32_t)cols >> 3;                       // units per row
   const int64_t total = rows * (int64_t)upr;
   const int64_t base = (int64_t)blockIdx.x * (256 * kUnitsPerThread) + threadIdx.x;
@@ -99,8 +102,20 @@ prune24_fp8_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t 
 #pragma unroll
   for (int j = 0; j < kUnitsPerThread; ++j) {
     const int64_t u = base + j * 256;                             // warp-uniform validity except in the last warp
-    uint32_t pa, pb;
-    const uint32_t na = prune_group<kSoft>(q[j].x, q[j].y, pa), nb = prune_group<kSoft>(q[j].z, q[j].w, pb);
+    uint32_t pa, pb, na, nb;
+    if (!kSoft) {
+      // hard pruning: the unit's two groups share one pass of the 16-bit-halves selection
+      uint32_t ea, eb;
+      top2of4_x2(__byte_perm(q[j].x, q[j].z, 0x5410u), __byte_perm(q[j].x, q[j].z, 0x7632u),
+                 __byte_perm(q[j].y, q[j].w, 0x5410u), __byte_perm(q[j].y, q[j].w, 0x7632u), lut, ea, eb);
+      pa = __byte_perm(q[j].x, q[j].y, ea);
+      pb = __byte_perm(q[j].z, q[j].w, eb);
+      na = (ea >> 16) & 0xFu;
+      nb = (eb >> 16) & 0xFu;
+    } else {
+      na = prune_group<kSoft>(q[j].x, q[j].y, pa);
+      nb = prune_group<kSoft>(q[j].z, q[j].w, pb);
+    }
     const uint32_t ca = quant2(pa, scale), cb = quant2(pb, scale);
     uint32_t mb = na | (nb << 4);
     mb |= __shfl_down_sync(0xFFFFFFFFu, mb, 1) << 8;

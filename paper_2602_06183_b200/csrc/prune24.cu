@@ -8,6 +8,8 @@
 //     shared memory, selects per column, and writes the transposed packed panel with 128-bit
 //     stores through a padded staging buffer.
 #include "sf_common.cuh"
+#include "tc_ptx.cuh"
+#include "gemm_tc.cuh"
 
 namespace sf {
 
@@ -46,6 +48,9 @@ __global__ void __launch_bounds__(256)
 prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t ld,
                     uint4* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
                     uint4* __restrict__ dense_out) {
+  __shared__ uint32_t lut[16];
+  top2_lut_init(lut, threadIdx.x);
+  __syncthreads();
   const int words_per_row = cols >> 4;                           // 16-element chunks per row
   const int kw = (int)blockIdx.x * 32 + (int)(threadIdx.x & 31);
   const int64_t r = ((int64_t)blockIdx.z * gridDim.y + blockIdx.y) * kRowsPerCta + (threadIdx.x >> 5);
@@ -57,13 +62,27 @@ prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t
   const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
 
   uint32_t packed[4], m = 0, dense[8];
+  if (!kSoft) {
+    // hard pruning: two groups per pass through the 16-bit-halves selection
+    uint32_t e[4];
 #pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    const uint32_t nib = prune_group_packed<kSoft>(w[2 * g], w[2 * g + 1], packed[g]);
-    m |= nib << (4 * g);
-    if (dense_out) {
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t a_lo = w[4 * h], a_hi = w[4 * h + 1], b_lo = w[4 * h + 2], b_hi = w[4 * h + 3];
+      top2of4_x2(__byte_perm(a_lo, b_lo, 0x5410u), __byte_perm(a_lo, b_lo, 0x7632u), __byte_perm(a_hi, b_hi, 0x5410u),
+                 __byte_perm(a_hi, b_hi, 0x7632u), lut, e[2 * h], e[2 * h + 1]);
+    }
+#pragma unroll
+    for (int g = 0; g < 4; ++g) packed[g] = __byte_perm(w[2 * g], w[2 * g + 1], e[g]);
+    m = ((e[0] & 0x000F0000u) | (e[1] & 0x00F00000u) | (e[2] & 0x0F000000u) | (e[3] & 0xF0000000u)) >> 16;
+  } else {
+#pragma unroll
+    for (int g = 0; g < 4; ++g) m |= prune_group_packed<kSoft>(w[2 * g], w[2 * g + 1], packed[g]) << (4 * g);
+  }
+  if (dense_out) {
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
       uint32_t d[4];
-      expand_group(nib, packed[g] & 0xFFFFu, packed[g] >> 16, d);
+      expand_group((m >> (4 * g)) & 0xFu, packed[g] & 0xFFFFu, packed[g] >> 16, d);
       dense[2 * g] = d[0] | (d[1] << 16);
       dense[2 * g + 1] = d[2] | (d[3] << 16);
     }
@@ -86,68 +105,75 @@ prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t
 
 // Strided groups. W is [Kd, Rc] row-major (Kd = rows = reduction dim, Rc = cols); outputs are
 // vals [Rc, Kd/2], meta [Rc, Kd/16]. Panel: 128 reduction rows x 64 columns.
-// Persistent CTAs walk the panels; the next panel streams into a second shared-memory tile with
-// cp.async while the current one is selected and stored, so loads, arithmetic and stores overlap.
+// Persistent CTAs walk the panels. One TMA load brings a panel into a three-slot ring two panels ahead
+// (out-of-range rows and columns arrive as zeros), so no thread computes load addresses; selection runs
+// on column pairs; packed values, canonical metadata and the tensor-core-ordered metadata of a panel are
+// assembled in shared memory and leave as 128-bit stores.
 constexpr int kPanelK = 128, kPanelC = 64;
+constexpr int kColsSlots = 3;
 constexpr int kStageRow = (kPanelK / 2) * 2 + 16;   // packed bytes per column + 16 B pad
-constexpr int kColsTileBytes = kPanelK * (kPanelC + 8) * 2, kColsStageBytes = kPanelC * kStageRow;
-constexpr int kColsSmemBytes = 2 * kColsTileBytes + kColsStageBytes + kPanelC * (kPanelK / 16) * 2;
-constexpr int kColsCtasPerSm = 4;
+constexpr int kColsTileBytes = kPanelK * kPanelC * 2, kColsStageBytes = kPanelC * kStageRow;
+constexpr int kColsMetaBytes = kPanelC * (kPanelK / 16) * 2;       // canonical words [column][8]; the same again in hardware order
+constexpr int kColsSmemBytes = 128 + kColsSlots * kColsTileBytes + kColsStageBytes + 2 * kColsMetaBytes + 64;
+constexpr int kColsCtasPerSm = 3;
 static_assert(kPanelK / 16 == 8 && kPanelC == 64, "index shifts in prune24_cols_kernel assume a 128 x 64 panel");
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
-               : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int kPending>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
 
 template <bool kSoft>
 __global__ void __launch_bounds__(256)
-prune24_cols_kernel(const uint16_t* __restrict__ W, int64_t Kd, int64_t Rc, int64_t ld,
+prune24_cols_kernel(const __grid_constant__ CUtensorMap tmapW, int64_t Kd, int64_t Rc,
                     uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
                     uint16_t* __restrict__ dense_out, int panels_x, int num_panels) {
-  extern __shared__ __align__(16) uint8_t cols_smem[];
-  typedef uint16_t TileRow[kPanelC + 8];                                 // +8: 16 B pad per row
+  using namespace ptx;
+  extern __shared__ uint8_t cols_smem_raw[];
+  uint8_t* cols_smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(cols_smem_raw) + 127) & ~uintptr_t(127));
+  typedef uint16_t TileRow[kPanelC];
   typedef uint8_t StageRow[kStageRow];
   typedef uint16_t MetaRow[kPanelK / 16];
-  StageRow* stage = reinterpret_cast<StageRow*>(cols_smem + 2 * kColsTileBytes);                       // [kPanelC]
-  MetaRow* mstage = reinterpret_cast<MetaRow*>(cols_smem + 2 * kColsTileBytes + kColsStageBytes);      // [kPanelC]
+  StageRow* stage = reinterpret_cast<StageRow*>(cols_smem + kColsSlots * kColsTileBytes);              // [kPanelC]
+  MetaRow* mstage = reinterpret_cast<MetaRow*>(cols_smem + kColsSlots * kColsTileBytes + kColsStageBytes);   // [kPanelC]
+  uint8_t* mhw = reinterpret_cast<uint8_t*>(mstage) + kColsMetaBytes;                                   // four 256-byte row blocks
+  uint64_t* full = reinterpret_cast<uint64_t*>(mhw + kColsMetaBytes);                                   // [kColsSlots]
+  int* abort_flag = reinterpret_cast<int*>(full + kColsSlots);
   const int tid = threadIdx.x;
 
-  // 8 threads x 16 B per row of 64 columns
-  auto prefetch = [&](int panel, int buf) {
+  auto issue = [&](int it) {                    // thread 0: load panel number `it` of this CTA into its slot
+    const int panel = (int)blockIdx.x + it * (int)gridDim.x;
+    if (panel >= num_panels) return;
     const int py = panel / panels_x, px = panel - py * panels_x;
-    const int64_t c0 = (int64_t)px * kPanelC, k0 = (int64_t)py * kPanelK;
-    const int kvalid = (int)min((int64_t)kPanelK, Kd - k0), cvalid = (int)min((int64_t)kPanelC, Rc - c0);
-    TileRow* tile = reinterpret_cast<TileRow*>(cols_smem + buf * kColsTileBytes);
-#pragma unroll
-    for (int u = 0; u < kPanelK * (kPanelC / 8) / 256; ++u) {
-      const int i = tid + u * 256;
-      const int kr = i >> 3, cc = (i & 7) << 3;
-      if (kr < kvalid && cc < cvalid) cp_async16(&tile[kr][cc], W + (k0 + kr) * ld + c0 + cc);
-    }
-    cp_async_commit();
+    const int slot = it % kColsSlots;
+    mbar_arrive_expect_tx(&full[slot], (uint32_t)kColsTileBytes);
+    tma_load_2d(cols_smem + slot * kColsTileBytes, &tmapW, &full[slot], px * kPanelC, py * kPanelK);
   };
+  __shared__ uint32_t lut[16];
+  top2_lut_init(lut, tid);
+  if (tid == 0) {
+    prefetch_tmap(&tmapW);
+    for (int sl = 0; sl < kColsSlots; ++sl) mbar_init(&full[sl], 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+    issue(0);
+    issue(1);
+  }
+  __syncthreads();
 
-  int buf = 0;
-  if ((int)blockIdx.x < num_panels) prefetch(blockIdx.x, 0);
-  for (int panel = blockIdx.x; panel < num_panels; panel += gridDim.x, buf ^= 1) {
-    const int next = panel + (int)gridDim.x;
-    if (next < num_panels) {
-      prefetch(next, buf ^ 1);
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
+  int it = 0;
+  for (int panel = blockIdx.x; panel < num_panels; panel += gridDim.x, ++it) {
+    const int slot = it % kColsSlots;
+    __syncthreads();            // the previous panel is stored: its stage buffers and the slot of the panel before are free
+    if (tid == 0) {
+      fence_proxy_async_smem(); // earlier generic writes to that slot (masked copy) before the TMA write
+      issue(it + 2);
     }
-    __syncthreads();            // this panel's tile is complete; the previous panel's stage has been drained
+    // one warp waits for the load (bounded), the block follows through the barrier
+    bool ok = true;
+    if (tid < 32) ok = mbar_wait(&full[slot], (uint32_t)(it / kColsSlots) & 1u, abort_flag);
+    if (__syncthreads_or(!ok)) break;
 
     const int py = panel / panels_x, px = panel - py * panels_x;
     const int64_t c0 = (int64_t)px * kPanelC, k0 = (int64_t)py * kPanelK;
     const int kvalid = (int)min((int64_t)kPanelK, Kd - k0);               // multiple of 16
     const int cvalid = (int)min((int64_t)kPanelC, Rc - c0);               // multiple of 8
-    TileRow* tile = reinterpret_cast<TileRow*>(cols_smem + buf * kColsTileBytes);
+    TileRow* tile = reinterpret_cast<TileRow*>(cols_smem + slot * kColsTileBytes);
 
     // select: one thread per (column pair, 16-row chunk); lanes run along column pairs, so the 32-bit
     // loads of a warp are conflict-free, and two byte permutes turn two rows into the two columns' pairs
@@ -162,11 +188,20 @@ prune24_cols_kernel(const uint16_t* __restrict__ W, int64_t Kd, int64_t Rc, int6
         uint32_t rw[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) rw[j] = *reinterpret_cast<const uint32_t*>(&tile[kr + j][c]);
+        // hard pruning: the two columns of the pair share one pass of the 16-bit-halves selection
+        uint32_t ent[2] = {0u, 0u};
+        if (!kSoft) top2of4_x2(rw[0], rw[1], rw[2], rw[3], lut, ent[0], ent[1]);
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const uint32_t sel = e ? 0x7632u : 0x5410u;
           const uint32_t lo = __byte_perm(rw[0], rw[1], sel), hi = __byte_perm(rw[2], rw[3], sel);
-          const uint32_t nib = prune_group_packed<kSoft>(lo, hi, packed[e][g]);
+          uint32_t nib;
+          if (!kSoft) {
+            packed[e][g] = __byte_perm(lo, hi, ent[e]);
+            nib = (ent[e] >> 16) & 0xFu;
+          } else {
+            nib = prune_group_packed<kSoft>(lo, hi, packed[e][g]);
+          }
           m[e] |= nib << (4 * g);
           if (dense_out) {
             uint32_t d[4];
@@ -180,27 +215,44 @@ prune24_cols_kernel(const uint16_t* __restrict__ W, int64_t Kd, int64_t Rc, int6
       for (int e = 0; e < 2; ++e) {
         *reinterpret_cast<uint4*>(&stage[c + e][ch * 16]) = make_uint4(packed[e][0], packed[e][1], packed[e][2], packed[e][3]);
         mstage[c + e][ch] = (uint16_t)m[e];
+        // tensor-core order (see meta_hw_offset): the panel's 64 output rows are four 16-row blocks of one atom
+        const int mi = c + e;
+        *reinterpret_cast<uint16_t*>(mhw + (mi >> 4) * 256 + (ch & 1) * 128 + (mi & 7) * 16 + (ch >> 1) * 4 +
+                                     ((mi >> 3) & 1) * 2) = (uint16_t)m[e];
       }
     }
     __syncthreads();
 
     // store packed values: per column kvalid/2 elements = kvalid bytes, 16 B per thread
     const int chunks = kvalid >> 4;
-    const bool full = chunks == kPanelK / 16;
+    const bool full_k = chunks == kPanelK / 16;
     for (int i = tid; i < kPanelC * chunks; i += 256) {
-      const int c = full ? (i >> 3) : (i / chunks), ch = i - c * chunks;
+      const int c = full_k ? (i >> 3) : (i / chunks), ch = i - c * chunks;
       if (c >= cvalid) continue;
       const uint4 q = *reinterpret_cast<const uint4*>(&stage[c][ch * 16]);
       const int64_t orow = c0 + c;
       *reinterpret_cast<uint4*>(vals + orow * (Kd >> 1) + (k0 >> 1) + ch * 8) = q;
-      const uint16_t mw = mstage[c][ch];
-      const int64_t kw = (k0 >> 4) + ch;
-      meta[orow * (Kd >> 4) + kw] = mw;
-      if (meta_hw) {
-        const uint32_t mi = (uint32_t)orow & 127u, kwi = (uint32_t)kw & 7u;
-        const int64_t atom = (orow >> 7) * (Kd >> 7) + (kw >> 3);
-        const uint32_t in_atom = (mi >> 4) * 256u + (kwi & 1u) * 128u + (mi & 7u) * 16u + (kwi >> 1) * 4u + ((mi >> 3) & 1u) * 2u;
-        *reinterpret_cast<uint16_t*>(meta_hw + atom * 2048 + in_atom) = mw;
+    }
+    if (full_k && (Kd & 127) == 0) {
+      // whole panels: a column's eight metadata words are 16 contiguous, aligned bytes in either order
+      if (tid < kPanelC) {
+        if (tid < cvalid)
+          *reinterpret_cast<uint4*>(meta + (c0 + tid) * (Kd >> 4) + (k0 >> 4)) = *reinterpret_cast<const uint4*>(&mstage[tid][0]);
+      } else if (tid < 2 * kPanelC && meta_hw) {
+        const int t = tid - kPanelC;                                        // 16-byte piece of the panel's 1 KB
+        // (the hardware order exists for whole 128-row blocks only, so all 64 columns are valid here)
+        const int64_t atom = (c0 >> 7) * (Kd >> 7) + (k0 >> 7);
+        *reinterpret_cast<uint4*>(meta_hw + atom * 2048 + ((c0 & 127) >> 4) * 256 + t * 16) =
+            *reinterpret_cast<const uint4*>(mhw + t * 16);
+      }
+    } else {
+      for (int i = tid; i < kPanelC * chunks; i += 256) {
+        const int c = i / chunks, ch = i - c * chunks;
+        if (c >= cvalid) continue;
+        const int64_t orow = c0 + c, kw = (k0 >> 4) + ch;
+        const uint16_t mw = mstage[c][ch];
+        meta[orow * (Kd >> 4) + kw] = mw;
+        if (meta_hw) *reinterpret_cast<uint16_t*>(meta_hw + meta_hw_offset(orow, kw, Kd)) = mw;
       }
     }
     if (dense_out) {
@@ -209,7 +261,6 @@ prune24_cols_kernel(const uint16_t* __restrict__ W, int64_t Kd, int64_t Rc, int6
         if (kr < kvalid && cc < cvalid)
           *reinterpret_cast<uint4*>(dense_out + (k0 + kr) * Rc + c0 + cc) = *reinterpret_cast<const uint4*>(&tile[kr][cc]);
       }
-      __syncthreads();          // this tile is overwritten by the prefetch two panels ahead
     }
   }
 }
@@ -313,16 +364,17 @@ int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int gr
       SF_CUDA_TRY(cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev));
       attr_done[dev] = true;
     }
+    alignas(64) CUtensorMap tm;
+    int st = make_tmap_2d(&tm, W, rows, cols, ld, kPanelC, kPanelK, false);
+    if (st != SF_OK) return st;
     const int resident = sms[dev] * kColsCtasPerSm;
     const unsigned grid = (unsigned)(num_panels < resident ? num_panels : resident);
     if (prune_mode == 0)
-      prune24_cols_kernel<false><<<grid, 256, kColsSmemBytes, s>>>((const uint16_t*)W, rows, cols, ld, (uint16_t*)vals,
-                                                                   (uint16_t*)meta, (uint8_t*)meta_hw,
-                                                                   (uint16_t*)dense_out, (int)px, num_panels);
+      prune24_cols_kernel<false><<<grid, 256, kColsSmemBytes, s>>>(tm, rows, cols, (uint16_t*)vals, (uint16_t*)meta,
+                                                                   (uint8_t*)meta_hw, (uint16_t*)dense_out, (int)px, num_panels);
     else
-      prune24_cols_kernel<true><<<grid, 256, kColsSmemBytes, s>>>((const uint16_t*)W, rows, cols, ld, (uint16_t*)vals,
-                                                                  (uint16_t*)meta, (uint8_t*)meta_hw,
-                                                                  (uint16_t*)dense_out, (int)px, num_panels);
+      prune24_cols_kernel<true><<<grid, 256, kColsSmemBytes, s>>>(tm, rows, cols, (uint16_t*)vals, (uint16_t*)meta,
+                                                                  (uint8_t*)meta_hw, (uint16_t*)dense_out, (int)px, num_panels);
   }
   SF_LAUNCH_CHECK();
   return SF_OK;

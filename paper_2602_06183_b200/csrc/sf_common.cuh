@@ -91,6 +91,40 @@ __device__ __forceinline__ uint32_t top2of4_packed(uint32_t lo, uint32_t hi, uin
   return p1 * 4u + p0;
 }
 
+// The same selection for TWO groups at once, in the 16-bit halves of 32-bit words: x_i holds element i of
+// group A in its low half and of group B in its high half (bf16 patterns). With magnitudes below 0x8000,
+// (a | 0x8000) - b has bit 15 set exactly when a >= b and never borrows from the other half, so one
+// subtraction compares both groups; "element i is kept" (fewer than two elements precede it in the order
+// magnitude descending, index ascending) is a majority of three such flags, one logic operation each.
+// The four keep flags of a group index a 16-entry table (top2_lut_init) whose entry holds the byte-permute
+// selector that gathers the kept pair out of {lo, hi} in its low half and the metadata nibble,
+// replicated into all four nibbles, in its high half. Returns the entries of group A and group B.
+__device__ __forceinline__ uint32_t top2_lut_entry(uint32_t keep_mask) {
+  const uint32_t p0 = __ffs(keep_mask) - 1u, p1 = 31u - __clz(keep_mask);
+  return (0x1010u + p0 * 0x22u + p1 * 0x2200u) | ((p0 | (p1 << 2)) * 0x11110000u);
+}
+// lut: 16 words of shared memory; call from at least 16 threads, then synchronise.
+__device__ __forceinline__ void top2_lut_init(uint32_t* lut, int tid) {
+  if (tid < 16) lut[tid] = (__popc(tid) == 2) ? top2_lut_entry((uint32_t)tid) : 0u;
+}
+__device__ __forceinline__ void top2of4_x2(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3, const uint32_t* lut,
+                                           uint32_t& entry_a, uint32_t& entry_b) {
+  constexpr uint32_t kMag = 0x7FFF7FFFu, kTop = 0x80008000u;
+  const uint32_t m1 = x1 & kMag, m2 = x2 & kMag, m3 = x3 & kMag;
+  const uint32_t o0 = x0 | kTop, o1 = x1 | kTop, o2 = x2 | kTop;
+  const uint32_t g01 = o0 - m1, g02 = o0 - m2, g03 = o0 - m3, g12 = o1 - m2, g13 = o1 - m3, g23 = o2 - m3;
+  // element j < i precedes i when m_j >= m_i; element j > i precedes i when not (m_i >= m_j)
+  const uint32_t k0 = (g01 & g02) | (g01 & g03) | (g02 & g03);
+  const uint32_t k1 = (~g01 & g12) | (~g01 & g13) | (g12 & g13);
+  const uint32_t k2 = (~g02 & ~g12) | (~g02 & g23) | (~g12 & g23);
+  const uint32_t k3 = ~((g03 & g13) | (g03 & g23) | (g13 & g23));
+  // flags (bits 15 and 31) -> byte offsets into the table (bits 2..5 of either half)
+  const uint32_t t = ((k0 >> 13) & 0x00040004u) | ((k1 >> 12) & 0x00080008u) | ((k2 >> 11) & 0x00100010u) |
+                     ((k3 >> 10) & 0x00200020u);
+  entry_a = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(lut) + (t & 0xFFFFu));
+  entry_b = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(lut) + (t >> 16));
+}
+
 // ---- internal launchers (defined in the .cu files) ---------------------------------------
 // meta_hw (optional) receives the same metadata words in the order the sparse tensor-core
 // instruction reads them (see meta_hw_offset below); requires R % 128 == 0 and K % 128 == 0.

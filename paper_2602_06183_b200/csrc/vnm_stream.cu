@@ -55,6 +55,8 @@ vnm_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t 
   const int64_t nstrips = (T / V) * nsx;
   const int64_t G = F / kM;
 
+  __shared__ uint32_t lut[16];
+  top2_lut_init(lut, tid);
   if (tid == 0) {
     prefetch_tmap(&tmapP);
     for (int s = 0; s < kSlots; ++s) {
@@ -185,40 +187,59 @@ vnm_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t 
       uint16_t* p_meta = meta + trow * (G >> 2) + (gg >> 2);
       const int64_t s_vals = kRows * G, s_meta = kRows * (G >> 2);
       const bool lead4 = (g & 3) == 0;
-      for (int r = r0; r < V; r += kRows) {
-        // the four kept columns as two packed pairs, then the activation on those only
-        uint32_t rk0, rk1;
+      // the four kept columns of a row as two packed pairs, then the activation on those only
+      auto kept = [&](const uint8_t* rowp, uint32_t& rk0, uint32_t& rk1, uint32_t& hk0, uint32_t& hk1) {
         if constexpr (kM == 8) {                              // one 16-byte load, picked apart by byte permutes
-          const uint4 q = *reinterpret_cast<const uint4*>(tp);
+          const uint4 q = *reinterpret_cast<const uint4*>(rowp);
           const uint32_t a0 = __byte_perm(q.x, q.y, selp[0]), b0 = __byte_perm(q.z, q.w, selp[0]);
           const uint32_t a1 = __byte_perm(q.x, q.y, selp[1]), b1 = __byte_perm(q.z, q.w, selp[1]);
           rk0 = (a0 & ~mhi[0]) | (b0 & mhi[0]);
           rk1 = (a1 & ~mhi[1]) | (b1 & mhi[1]);
         } else {                                              // wide groups: four 16-bit loads
-          rk0 = (uint32_t)*reinterpret_cast<const uint16_t*>(tp + o0) |
-                ((uint32_t)*reinterpret_cast<const uint16_t*>(tp + o1) << 16);
-          rk1 = (uint32_t)*reinterpret_cast<const uint16_t*>(tp + o2) |
-                ((uint32_t)*reinterpret_cast<const uint16_t*>(tp + o3) << 16);
+          rk0 = (uint32_t)*reinterpret_cast<const uint16_t*>(rowp + o0) |
+                ((uint32_t)*reinterpret_cast<const uint16_t*>(rowp + o1) << 16);
+          rk1 = (uint32_t)*reinterpret_cast<const uint16_t*>(rowp + o2) |
+                ((uint32_t)*reinterpret_cast<const uint16_t*>(rowp + o3) << 16);
         }
-        uint32_t hk0 = rk0, hk1 = rk1;
+        hk0 = rk0; hk1 = rk1;
         if (apply) {
           rk0 = bf2_relu(rk0); rk1 = bf2_relu(rk1);
           hk0 = bf2_sq(rk0); hk1 = bf2_sq(rk1);
         }
-        uint32_t packed, psel;
-        const uint32_t nib = top2of4_packed(hk0, hk1, &packed, nullptr, &psel);
+      };
+      auto put = [&](uint32_t packed, uint32_t rpair, uint32_t nib) {
         if (live) *p_vals = packed;
         if (want_relu) {
-          if (live) *p_relu = __byte_perm(rk0, rk1, psel);
+          if (live) *p_relu = rpair;
           p_relu += s_vals;
         }
         uint32_t word = nib;
         word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 4;
         word |= __shfl_down_sync(0xFFFFFFFFu, word, 2) << 8;
         if (lead4 && live) *p_meta = (uint16_t)word;
-        tp += kRows * kSW * 2;
         p_vals += s_vals;
         p_meta += s_meta;
+      };
+      int r = r0;
+      // groups of eight (the emit-heavy case): two rows per pass, their 2:4 choices share one run of the
+      // 16-bit-halves selection; wider groups measured faster one row at a time
+      if constexpr (kM == 8)
+      for (; r + kRows < V; r += 2 * kRows) {
+        uint32_t ra0, ra1, ha0, ha1, rb0, rb1, hb0, hb1, ea, eb;
+        kept(tp, ra0, ra1, ha0, ha1);
+        kept(tp + kRows * kSW * 2, rb0, rb1, hb0, hb1);
+        top2of4_x2(__byte_perm(ha0, hb0, 0x5410u), __byte_perm(ha0, hb0, 0x7632u), __byte_perm(ha1, hb1, 0x5410u),
+                   __byte_perm(ha1, hb1, 0x7632u), lut, ea, eb);
+        put(__byte_perm(ha0, ha1, ea), __byte_perm(ra0, ra1, ea), (ea >> 16) & 0xFu);
+        put(__byte_perm(hb0, hb1, eb), __byte_perm(rb0, rb1, eb), (eb >> 16) & 0xFu);
+        tp += 2 * kRows * kSW * 2;
+      }
+      for (; r < V; r += kRows) {                             // single rows: wide groups, or an odd last pass
+        uint32_t rk0, rk1, hk0, hk1, packed, psel;
+        kept(tp, rk0, rk1, hk0, hk1);
+        const uint32_t nib = top2of4_packed(hk0, hk1, &packed, nullptr, &psel);
+        put(packed, __byte_perm(rk0, rk1, psel), nib);
+        tp += kRows * kSW * 2;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&ctl->empty[slot]);
