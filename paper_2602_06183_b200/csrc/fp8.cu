@@ -48,23 +48,6 @@ quantize_fp8_kernel(const uint4* __restrict__ X, int64_t rows, int cols, int64_t
   out[idx] = o;
 }
 
-// 2:4 selection of a group (lo, hi = its four bf16 patterns), optional soft-threshold shrinkage rounded to
-// bf16 as in the bf16 pass; returns the nibble, *packed = the two kept bf16 values.
-template <bool kSoft>
-__device__ __forceinline__ uint32_t prune_group(uint32_t lo, uint32_t hi, uint32_t& packed) {
-  uint32_t third;
-  const uint32_t nib = top2of4_packed(lo, hi, &packed, kSoft ? &third : nullptr);
-  if (kSoft) {
-    const uint32_t tw = (third & 2u) ? hi : lo;
-    const float t = bf16_bits_to_float(((third & 1u) ? (tw >> 16) : tw) & 0x7FFFu);
-    const float f0 = bf16_bits_to_float(packed & 0xFFFFu), f1 = bf16_bits_to_float(packed >> 16);
-    const float s0 = f0 > 0.f ? __fsub_rn(f0, t) : (f0 < 0.f ? __fadd_rn(f0, t) : 0.f);
-    const float s1 = f1 > 0.f ? __fsub_rn(f1, t) : (f1 < 0.f ? __fadd_rn(f1, t) : 0.f);
-    packed = float_to_bf16_bits(s0) | (float_to_bf16_bits(s1) << 16);
-  }
-  return nib;
-}
-
 // Work unit = eight consecutive elements of a row (two groups, one 128-bit load): four codes, one metadata
 // byte. All outputs are contiguous by unit, so a thread takes kUnitsPerThread units a whole CTA apart: every
 // load and store instruction of a warp covers one contiguous range. The four metadata bytes of four
@@ -75,7 +58,7 @@ template <bool kSoft>
 __global__ void __launch_bounds__(256)
 prune24_fp8_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t ld, float scale,
                    uint32_t* __restrict__ vals, uint32_t* __restrict__ meta, uint2* __restrict__ dense_out) {
-  __shared__ uint32_t lut[16];
+  __shared__ Top2Entry lut[16];
   top2_lut_init(lut, threadIdx.x);
   __syncthreads();
   const uint32_t upr = (uint32_t)cols >> 3;                       // units per row
@@ -102,20 +85,13 @@ prune24_fp8_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t 
 #pragma unroll
   for (int j = 0; j < kUnitsPerThread; ++j) {
     const int64_t u = base + j * 256;                             // warp-uniform validity except in the last warp
-    uint32_t pa, pb, na, nb;
-    if (!kSoft) {
-      // hard pruning: the unit's two groups share one pass of the 16-bit-halves selection
-      uint32_t ea, eb;
-      top2of4_x2(__byte_perm(q[j].x, q[j].z, 0x5410u), __byte_perm(q[j].x, q[j].z, 0x7632u),
-                 __byte_perm(q[j].y, q[j].w, 0x5410u), __byte_perm(q[j].y, q[j].w, 0x7632u), lut, ea, eb);
-      pa = __byte_perm(q[j].x, q[j].y, ea);
-      pb = __byte_perm(q[j].z, q[j].w, eb);
-      na = (ea >> 16) & 0xFu;
-      nb = (eb >> 16) & 0xFu;
-    } else {
-      na = prune_group<kSoft>(q[j].x, q[j].y, pa);
-      nb = prune_group<kSoft>(q[j].z, q[j].w, pb);
-    }
+    // the unit's two groups share one pass of the 16-bit-halves selection
+    Top2Entry ea, eb;
+    top2of4_x2<kSoft>(__byte_perm(q[j].x, q[j].z, 0x5410u), __byte_perm(q[j].x, q[j].z, 0x7632u),
+                      __byte_perm(q[j].y, q[j].w, 0x5410u), __byte_perm(q[j].y, q[j].w, 0x7632u), lut, ea, eb);
+    const uint32_t pa = kSoft ? soft_threshold_pair(q[j].x, q[j].y, ea) : __byte_perm(q[j].x, q[j].y, ea.kept);
+    const uint32_t pb = kSoft ? soft_threshold_pair(q[j].z, q[j].w, eb) : __byte_perm(q[j].z, q[j].w, eb.kept);
+    const uint32_t na = (ea.kept >> 16) & 0xFu, nb = (eb.kept >> 16) & 0xFu;
     const uint32_t ca = quant2(pa, scale), cb = quant2(pb, scale);
     uint32_t mb = na | (nb << 4);
     mb |= __shfl_down_sync(0xFFFFFFFFu, mb, 1) << 8;

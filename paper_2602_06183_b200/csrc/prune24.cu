@@ -15,23 +15,6 @@ namespace sf {
 
 namespace {
 
-// Selection for one group: lo/hi hold the group's four bf16 patterns; returns the nibble and the two
-// kept (hard) or shrunk by the third-ranked magnitude (soft) values packed into one word.
-template <bool kSoft>
-__device__ __forceinline__ uint32_t prune_group_packed(uint32_t lo, uint32_t hi, uint32_t& packed) {
-  uint32_t third;
-  const uint32_t nib = top2of4_packed(lo, hi, &packed, kSoft ? &third : nullptr);
-  if (kSoft) {
-    const uint32_t tw = (third & 2u) ? hi : lo;
-    const float t = bf16_bits_to_float(((third & 1u) ? (tw >> 16) : tw) & 0x7FFFu);
-    const float f0 = bf16_bits_to_float(packed & 0xFFFFu), f1 = bf16_bits_to_float(packed >> 16);
-    const float s0 = f0 > 0.f ? __fsub_rn(f0, t) : (f0 < 0.f ? __fadd_rn(f0, t) : 0.f);
-    const float s1 = f1 > 0.f ? __fsub_rn(f1, t) : (f1 < 0.f ? __fadd_rn(f1, t) : 0.f);
-    packed = float_to_bf16_bits(s0) | (float_to_bf16_bits(s1) << 16);
-  }
-  return nib;
-}
-
 // Expand (nibble, two values) to the four dense patterns of a group.
 __device__ __forceinline__ void expand_group(uint32_t nib, uint32_t v0, uint32_t v1, uint32_t d[4]) {
   const uint32_t p0 = nib & 3u, p1 = nib >> 2;
@@ -48,7 +31,7 @@ __global__ void __launch_bounds__(256)
 prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t ld,
                     uint4* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
                     uint4* __restrict__ dense_out) {
-  __shared__ uint32_t lut[16];
+  __shared__ Top2Entry lut[16];
   top2_lut_init(lut, threadIdx.x);
   __syncthreads();
   const int words_per_row = cols >> 4;                           // 16-element chunks per row
@@ -62,21 +45,19 @@ prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t
   const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
 
   uint32_t packed[4], m = 0, dense[8];
-  if (!kSoft) {
-    // hard pruning: two groups per pass through the 16-bit-halves selection
-    uint32_t e[4];
+  {
+    // two groups per pass through the 16-bit-halves selection
+    Top2Entry e[4];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const uint32_t a_lo = w[4 * h], a_hi = w[4 * h + 1], b_lo = w[4 * h + 2], b_hi = w[4 * h + 3];
-      top2of4_x2(__byte_perm(a_lo, b_lo, 0x5410u), __byte_perm(a_lo, b_lo, 0x7632u), __byte_perm(a_hi, b_hi, 0x5410u),
-                 __byte_perm(a_hi, b_hi, 0x7632u), lut, e[2 * h], e[2 * h + 1]);
+      top2of4_x2<kSoft>(__byte_perm(a_lo, b_lo, 0x5410u), __byte_perm(a_lo, b_lo, 0x7632u),
+                        __byte_perm(a_hi, b_hi, 0x5410u), __byte_perm(a_hi, b_hi, 0x7632u), lut, e[2 * h], e[2 * h + 1]);
     }
 #pragma unroll
-    for (int g = 0; g < 4; ++g) packed[g] = __byte_perm(w[2 * g], w[2 * g + 1], e[g]);
-    m = ((e[0] & 0x000F0000u) | (e[1] & 0x00F00000u) | (e[2] & 0x0F000000u) | (e[3] & 0xF0000000u)) >> 16;
-  } else {
-#pragma unroll
-    for (int g = 0; g < 4; ++g) m |= prune_group_packed<kSoft>(w[2 * g], w[2 * g + 1], packed[g]) << (4 * g);
+    for (int g = 0; g < 4; ++g)
+      packed[g] = kSoft ? soft_threshold_pair(w[2 * g], w[2 * g + 1], e[g]) : __byte_perm(w[2 * g], w[2 * g + 1], e[g].kept);
+    m = ((e[0].kept & 0x000F0000u) | (e[1].kept & 0x00F00000u) | (e[2].kept & 0x0F000000u) | (e[3].kept & 0xF0000000u)) >> 16;
   }
   if (dense_out) {
 #pragma unroll
@@ -144,7 +125,7 @@ prune24_cols_kernel(const __grid_constant__ CUtensorMap tmapW, int64_t Kd, int64
     mbar_arrive_expect_tx(&full[slot], (uint32_t)kColsTileBytes);
     tma_load_2d(cols_smem + slot * kColsTileBytes, &tmapW, &full[slot], px * kPanelC, py * kPanelK);
   };
-  __shared__ uint32_t lut[16];
+  __shared__ Top2Entry lut[16];
   top2_lut_init(lut, tid);
   if (tid == 0) {
     prefetch_tmap(&tmapW);
@@ -188,20 +169,15 @@ prune24_cols_kernel(const __grid_constant__ CUtensorMap tmapW, int64_t Kd, int64
         uint32_t rw[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) rw[j] = *reinterpret_cast<const uint32_t*>(&tile[kr + j][c]);
-        // hard pruning: the two columns of the pair share one pass of the 16-bit-halves selection
-        uint32_t ent[2] = {0u, 0u};
-        if (!kSoft) top2of4_x2(rw[0], rw[1], rw[2], rw[3], lut, ent[0], ent[1]);
+        // the two columns of the pair share one pass of the 16-bit-halves selection
+        Top2Entry ent[2];
+        top2of4_x2<kSoft>(rw[0], rw[1], rw[2], rw[3], lut, ent[0], ent[1]);
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const uint32_t sel = e ? 0x7632u : 0x5410u;
           const uint32_t lo = __byte_perm(rw[0], rw[1], sel), hi = __byte_perm(rw[2], rw[3], sel);
-          uint32_t nib;
-          if (!kSoft) {
-            packed[e][g] = __byte_perm(lo, hi, ent[e]);
-            nib = (ent[e] >> 16) & 0xFu;
-          } else {
-            nib = prune_group_packed<kSoft>(lo, hi, packed[e][g]);
-          }
+          packed[e][g] = kSoft ? soft_threshold_pair(lo, hi, ent[e]) : __byte_perm(lo, hi, ent[e].kept);
+          const uint32_t nib = (ent[e].kept >> 16) & 0xFu;
           m[e] |= nib << (4 * g);
           if (dense_out) {
             uint32_t d[4];

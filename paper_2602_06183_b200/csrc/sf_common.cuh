@@ -96,19 +96,26 @@ __device__ __forceinline__ uint32_t top2of4_packed(uint32_t lo, uint32_t hi, uin
 // (a | 0x8000) - b has bit 15 set exactly when a >= b and never borrows from the other half, so one
 // subtraction compares both groups; "element i is kept" (fewer than two elements precede it in the order
 // magnitude descending, index ascending) is a majority of three such flags, one logic operation each.
-// The four keep flags of a group index a 16-entry table (top2_lut_init) whose entry holds the byte-permute
-// selector that gathers the kept pair out of {lo, hi} in its low half and the metadata nibble,
-// replicated into all four nibbles, in its high half. Returns the entries of group A and group B.
-__device__ __forceinline__ uint32_t top2_lut_entry(uint32_t keep_mask) {
+// The four keep flags of a group index a 16-entry table (top2_lut_init). Entry .x: low half = the
+// byte-permute selector that gathers the kept pair out of {lo, hi}, high half = the metadata nibble
+// replicated into all four nibbles; .y = the selector of the two dropped elements.
+// Returns the entries of group A and group B.
+struct Top2Entry { uint32_t kept, dropped; };
+__device__ __forceinline__ Top2Entry top2_lut_entry(uint32_t keep_mask) {
   const uint32_t p0 = __ffs(keep_mask) - 1u, p1 = 31u - __clz(keep_mask);
-  return (0x1010u + p0 * 0x22u + p1 * 0x2200u) | ((p0 | (p1 << 2)) * 0x11110000u);
+  const uint32_t drop = ~keep_mask & 0xFu;
+  const uint32_t q0 = __ffs(drop) - 1u, q1 = 31u - __clz(drop);
+  return Top2Entry{(0x1010u + p0 * 0x22u + p1 * 0x2200u) | ((p0 | (p1 << 2)) * 0x11110000u),
+                   0x1010u + q0 * 0x22u + q1 * 0x2200u};
 }
-// lut: 16 words of shared memory; call from at least 16 threads, then synchronise.
-__device__ __forceinline__ void top2_lut_init(uint32_t* lut, int tid) {
-  if (tid < 16) lut[tid] = (__popc(tid) == 2) ? top2_lut_entry((uint32_t)tid) : 0u;
+// lut: 16 entries of shared memory; call from at least 16 threads, then synchronise.
+__device__ __forceinline__ void top2_lut_init(Top2Entry* lut, int tid) {
+  if (tid < 16) lut[tid] = (__popc(tid) == 2) ? top2_lut_entry((uint32_t)tid) : Top2Entry{0u, 0u};
 }
-__device__ __forceinline__ void top2of4_x2(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3, const uint32_t* lut,
-                                           uint32_t& entry_a, uint32_t& entry_b) {
+// kDropped: the entries' .dropped selectors are loaded too (soft-thresholding needs the dropped pair).
+template <bool kDropped = false>
+__device__ __forceinline__ void top2of4_x2(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3, const Top2Entry* lut,
+                                           Top2Entry& entry_a, Top2Entry& entry_b) {
   constexpr uint32_t kMag = 0x7FFF7FFFu, kTop = 0x80008000u;
   const uint32_t m1 = x1 & kMag, m2 = x2 & kMag, m3 = x3 & kMag;
   const uint32_t o0 = x0 | kTop, o1 = x1 | kTop, o2 = x2 | kTop;
@@ -118,11 +125,33 @@ __device__ __forceinline__ void top2of4_x2(uint32_t x0, uint32_t x1, uint32_t x2
   const uint32_t k1 = (~g01 & g12) | (~g01 & g13) | (g12 & g13);
   const uint32_t k2 = (~g02 & ~g12) | (~g02 & g23) | (~g12 & g23);
   const uint32_t k3 = ~((g03 & g13) | (g03 & g23) | (g13 & g23));
-  // flags (bits 15 and 31) -> byte offsets into the table (bits 2..5 of either half)
-  const uint32_t t = ((k0 >> 13) & 0x00040004u) | ((k1 >> 12) & 0x00080008u) | ((k2 >> 11) & 0x00100010u) |
-                     ((k3 >> 10) & 0x00200020u);
-  entry_a = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(lut) + (t & 0xFFFFu));
-  entry_b = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(lut) + (t >> 16));
+  // flags (bits 15 and 31) -> byte offsets into the table (bits 3..6 of either half)
+  const uint32_t t = ((k0 >> 12) & 0x00080008u) | ((k1 >> 11) & 0x00100010u) | ((k2 >> 10) & 0x00200020u) |
+                     ((k3 >> 9) & 0x00400040u);
+  const uint8_t* base = reinterpret_cast<const uint8_t*>(lut);
+  if (kDropped) {
+    const uint2 a = *reinterpret_cast<const uint2*>(base + (t & 0xFFFFu)), b = *reinterpret_cast<const uint2*>(base + (t >> 16));
+    entry_a = Top2Entry{a.x, a.y};
+    entry_b = Top2Entry{b.x, b.y};
+  } else {
+    entry_a = Top2Entry{*reinterpret_cast<const uint32_t*>(base + (t & 0xFFFFu)), 0u};
+    entry_b = Top2Entry{*reinterpret_cast<const uint32_t*>(base + (t >> 16)), 0u};
+  }
+}
+// Soft-thresholding (Section 2.2) of a group's kept pair, given the group as {lo, hi} and its table entry:
+// the threshold is the larger magnitude of the two dropped elements; every kept value moves towards zero
+// by it (never across: kept magnitudes are at least the threshold). The packed bf16 subtraction rounds
+// the exact difference once, which equals the float32 subtraction followed by rounding to bf16 (the
+// float32 result is exact unless the threshold is below 2^-16 of the value, where both give the value
+// itself). A kept NaN is neither above nor below the threshold and becomes zero.
+__device__ __forceinline__ uint32_t soft_threshold_pair(uint32_t lo, uint32_t hi, const Top2Entry& e) {
+  const uint32_t kept = __byte_perm(lo, hi, e.kept);
+  const uint32_t dm = __byte_perm(lo, hi, e.dropped) & 0x7FFF7FFFu;
+  const uint32_t t = max(dm & 0xFFFFu, dm >> 16);
+  const uint32_t ct = (kept & 0x80008000u) | (t * 0x00010001u);          // the threshold with each value's sign
+  const __nv_bfloat162 d = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&kept), *reinterpret_cast<const __nv_bfloat162*>(&ct));
+  const __nv_bfloat162 kv = *reinterpret_cast<const __nv_bfloat162*>(&kept);
+  return *reinterpret_cast<const uint32_t*>(&d) & ~__hneu2_mask(kv, kv);
 }
 
 // ---- internal launchers (defined in the .cu files) ---------------------------------------

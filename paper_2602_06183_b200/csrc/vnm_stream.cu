@@ -55,7 +55,7 @@ vnm_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t 
   const int64_t nstrips = (T / V) * nsx;
   const int64_t G = F / kM;
 
-  __shared__ uint32_t lut[16];
+  __shared__ Top2Entry lut[16];
   top2_lut_init(lut, tid);
   if (tid == 0) {
     prefetch_tmap(&tmapP);
@@ -225,13 +225,14 @@ vnm_stream_kernel(const __grid_constant__ CUtensorMap tmapP, int64_t T, int64_t 
       // 16-bit-halves selection; wider groups measured faster one row at a time
       if constexpr (kM == 8)
       for (; r + kRows < V; r += 2 * kRows) {
-        uint32_t ra0, ra1, ha0, ha1, rb0, rb1, hb0, hb1, ea, eb;
+        uint32_t ra0, ra1, ha0, ha1, rb0, rb1, hb0, hb1;
+        Top2Entry ea, eb;
         kept(tp, ra0, ra1, ha0, ha1);
         kept(tp + kRows * kSW * 2, rb0, rb1, hb0, hb1);
         top2of4_x2(__byte_perm(ha0, hb0, 0x5410u), __byte_perm(ha0, hb0, 0x7632u), __byte_perm(ha1, hb1, 0x5410u),
                    __byte_perm(ha1, hb1, 0x7632u), lut, ea, eb);
-        put(__byte_perm(ha0, ha1, ea), __byte_perm(ra0, ra1, ea), (ea >> 16) & 0xFu);
-        put(__byte_perm(hb0, hb1, eb), __byte_perm(rb0, rb1, eb), (eb >> 16) & 0xFu);
+        put(__byte_perm(ha0, ha1, ea.kept), __byte_perm(ra0, ra1, ea.kept), (ea.kept >> 16) & 0xFu);
+        put(__byte_perm(hb0, hb1, eb.kept), __byte_perm(rb0, rb1, eb.kept), (eb.kept >> 16) & 0xFu);
         tp += 2 * kRows * kSW * 2;
       }
       for (; r < V; r += kRows) {                             // single rows: wide groups, or an odd last pass

@@ -47,6 +47,30 @@ def test_prune24_strided_input_and_special_values():
     assert np.array_equal(bits(meta), ref.meta) and np.array_equal(bits(vals), ref.vals)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("group_dim", [1, 0])
+def test_prune24_special_values_both_modes(group_dim, mode):
+    """Infinities, NaNs, subnormals, signed zeros and exact ties in every position of a group, hard and soft:
+    the order is the one of the magnitude bit patterns, a NaN that is kept becomes zero under soft-thresholding
+    (it is neither above nor below the threshold), an infinite threshold makes NaN of infinite kept values."""
+    rng = np.random.default_rng(40 + group_dim + 2 * mode)
+    special = np.array([0x0000, 0x8000, 0x0001, 0x8001, 0x007F, 0x0080, 0x7F80, 0xFF80, 0x7FC0, 0xFFC0, 0x7F7F, 0xFF7F,
+                        0x3F80, 0xBF80, 0x3F81, 0x4000], dtype=np.uint16)
+    w = synth.prune_sweep_matrix(128, 256, seed=41, tie_frac=0.3)
+    pick = rng.random(w.shape) < 0.35
+    w[pick] = special[rng.integers(0, len(special), size=int(pick.sum()))]
+    ref = oracle.prune24(w, group_dim, mode)
+    vals, meta, dense = binding.sf_prune24_compress(to_dev(w), group_dim, mode, want_dense=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(meta), ref.meta)
+
+    def same(a, b):                                   # NaN payloads are not part of the contract
+        fa, fb = oracle.bf16_to_f32(a), oracle.bf16_to_f32(b)
+        return np.array_equal(np.isnan(fa), np.isnan(fb)) and np.array_equal(a[~np.isnan(fa)], b[~np.isnan(fb)])
+    assert same(bits(vals), ref.vals)
+    assert same(bits(dense), ref.dense)
+
+
 @pytest.mark.parametrize("T,F,V,M", [(128, 512, 64, 8), (256, 1024, 128, 16), (128, 320, 64, 4),
                                      (64, 256, 32, 32), (128, 256, 64, 64), (192, 832, 64, 8)])
 def test_vnm_bit_exact(T, F, V, M):
