@@ -86,17 +86,17 @@ prune24_rows_kernel(const uint4* __restrict__ W, int64_t rows, int cols, int64_t
 
 // Strided groups. W is [Kd, Rc] row-major (Kd = rows = reduction dim, Rc = cols); outputs are
 // vals [Rc, Kd/2], meta [Rc, Kd/16]. Panel: 128 reduction rows x 64 columns.
-// Persistent CTAs walk the panels. One TMA load brings a panel into a three-slot ring two panels ahead
+// Persistent CTAs walk the panels. One TMA load brings the next panel into a two-slot ring
 // (out-of-range rows and columns arrive as zeros), so no thread computes load addresses; selection runs
 // on column pairs; packed values, canonical metadata and the tensor-core-ordered metadata of a panel are
 // assembled in shared memory and leave as 128-bit stores.
 constexpr int kPanelK = 128, kPanelC = 64;
-constexpr int kColsSlots = 3;
+constexpr int kColsSlots = 2;                       // the next panel loads while this one is worked on
 constexpr int kStageRow = (kPanelK / 2) * 2 + 16;   // packed bytes per column + 16 B pad
 constexpr int kColsTileBytes = kPanelK * kPanelC * 2, kColsStageBytes = kPanelC * kStageRow;
 constexpr int kColsMetaBytes = kPanelC * (kPanelK / 16) * 2;       // canonical words [column][8]; the same again in hardware order
 constexpr int kColsSmemBytes = 128 + kColsSlots * kColsTileBytes + kColsStageBytes + 2 * kColsMetaBytes + 64;
-constexpr int kColsCtasPerSm = 3;
+constexpr int kColsCtasPerSm = 5;                   // 44 KB each; measured best among 3..5 with two or three slots
 static_assert(kPanelK / 16 == 8 && kPanelC == 64, "index shifts in prune24_cols_kernel assume a 128 x 64 panel");
 
 template <bool kSoft>
@@ -132,8 +132,7 @@ prune24_cols_kernel(const __grid_constant__ CUtensorMap tmapW, int64_t Kd, int64
     for (int sl = 0; sl < kColsSlots; ++sl) mbar_init(&full[sl], 1);
     *abort_flag = 0;
     fence_mbar_init();
-    issue(0);
-    issue(1);
+    for (int d = 0; d < kColsSlots - 1; ++d) issue(d);
   }
   __syncthreads();
 
@@ -143,7 +142,7 @@ prune24_cols_kernel(const __grid_constant__ CUtensorMap tmapW, int64_t Kd, int64
     __syncthreads();            // the previous panel is stored: its stage buffers and the slot of the panel before are free
     if (tid == 0) {
       fence_proxy_async_smem(); // earlier generic writes to that slot (masked copy) before the TMA write
-      issue(it + 2);
+      issue(it + kColsSlots - 1);
     }
     // one warp waits for the load (bounded), the block follows through the barrier
     bool ok = true;
