@@ -155,3 +155,65 @@ def test_vnm_special_values_bit_exact():
         assert np.array_equal(bits(vals), ref.vals)
         assert np.array_equal(bits(relu), ref.relu_vals)
         assert np.array_equal(bits(dense), ref.dense)
+
+
+def _random_prune_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        group_dim = int(rng.integers(0, 2))
+        k = int(rng.integers(1, 40)) * 16                      # reduction length: whole metadata words
+        r = int(rng.integers(1, 60)) * 8
+        rows, cols = (r, k) if group_dim == 1 else (k, r)
+        out.append((rows, cols, group_dim, int(rng.integers(0, 2)), int(rng.integers(0, 3)) * 8, int(rng.integers(1, 1 << 20))))
+    return out
+
+
+@pytest.mark.parametrize("rows,cols,group_dim,mode,pad,seed", _random_prune_shapes(24, seed=20260207))
+def test_prune24_random_shapes(rows, cols, group_dim, mode, pad, seed):
+    """Seeded draw of legal shapes (ragged panels, single rows, padded leading dimension), both directions and modes."""
+    w = synth.prune_sweep_matrix(rows, cols, seed=seed, tie_frac=0.2)
+    ref = oracle.prune24(w, group_dim, mode)
+    wide = torch.zeros((rows, cols + pad), dtype=torch.bfloat16, device="cuda")
+    wide[:, :cols] = to_dev(w)
+    vals, meta, dense = binding.sf_prune24_compress(wide[:, :cols], group_dim, mode, want_dense=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(meta), ref.meta)
+    assert np.array_equal(bits(vals), ref.vals)
+    assert np.array_equal(bits(dense), ref.dense)
+    vals2, meta2, _ = binding.sf_prune24_compress(wide[:, :cols], group_dim, mode)
+    assert torch.equal(vals2, vals) and torch.equal(meta2, meta)
+
+
+def _random_vnm_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < n:
+        M = int(rng.choice([4, 8, 16, 32, 64]))
+        V = int(rng.choice([16, 32, 48, 64, 96, 128]))
+        T = V * int(rng.integers(1, 5))
+        F = 64 * int(rng.integers(1, 30))
+        if F % (4 * M):
+            continue
+        out.append((T, F, V, M, bool(rng.integers(0, 2)), int(rng.integers(0, 3)) * 8, int(rng.integers(1, 1 << 20))))
+    return out
+
+
+@pytest.mark.parametrize("T,F,V,M,apply,pad,seed", _random_vnm_shapes(24, seed=20260208))
+def test_vnm_random_shapes(T, F, V, M, apply, pad, seed):
+    """Seeded draw of legal (T, F, V, M): whichever kernel the call picks (streaming or strip-staged) must give the
+    oracle's bits, with and without the dense copy, through a strided view."""
+    p = synth.act_sweep_matrix(T, F, seed=seed)
+    ref = oracle.vnm_sparsify(p, V=V, M=M, apply_sqrelu=apply)
+    wide = torch.zeros((T, F + pad), dtype=torch.bfloat16, device="cuda")
+    wide[:, :F] = to_dev(p)
+    for want_dense in (False, True):
+        vals, meta, colidx, relu, dense = binding.sf_vnm_sparsify_act(wide[:, :F], V, M, apply_sqrelu=apply, want_dense=want_dense)
+        torch.cuda.synchronize()
+        assert np.array_equal(colidx.cpu().numpy(), ref.colidx)
+        assert np.array_equal(bits(meta), ref.meta)
+        assert np.array_equal(bits(vals), ref.vals)
+        if apply:
+            assert np.array_equal(bits(relu), ref.relu_vals)
+        if want_dense:
+            assert np.array_equal(bits(dense), ref.dense)
