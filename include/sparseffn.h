@@ -190,11 +190,12 @@ SF_API int sf_gemm_sparse24_noalloc(const void* a_vals, const void* a_meta, cons
  *
  * sf_fp8_quantize: Xq[r, c] = code of X[r, c]. X bf16 [rows, cols] (ld >= cols, ld % 8 == 0),
  *     Xq uint8 [rows, cols] contiguous. cols % 16 == 0.
- * sf_prune24_compress_fp8: the 2:4 pass of sf_prune24_compress with group_dim = 1 (groups of four
- *     along a row; same selection, same soft-threshold shrinkage rounded to bf16) whose kept values
- *     leave as codes: vals uint8 [rows, cols/2], meta uint16 [rows, cols/16] (canonical, identical to
- *     the bf16 pass), optional dense_out uint8 [rows, cols] (codes on the mask, +0 elsewhere).
- *     cols % 32 == 0. 2 B read + 0.625 B written per element.
+ * sf_prune24_compress_fp8: the 2:4 pass of sf_prune24_compress (same group_dim convention, same
+ *     selection, same soft-threshold shrinkage rounded to bf16) whose kept values leave as codes:
+ *     vals uint8 [R, K/2], meta uint16 [R, K/16] (canonical, identical to the bf16 pass; R, K as
+ *     for sf_prune24_compress). group_dim = 1: cols % 32 == 0, optional dense_out uint8
+ *     [rows, cols] (codes on the mask, +0 elsewhere). group_dim = 0: rows % 16 == 0, cols % 8 == 0,
+ *     dense_out must be NULL (SF_ERR_UNSUPPORTED otherwise). 2 B read + 0.625 B written per element.
  * sf_gemm_fp8_dense:    C[Mr,Nc] = bf16(alpha * A B^T), A uint8 [Mr,K], B uint8 [Nc,K] (codes).
  * sf_gemm_fp8_sparse24: the same with A given 2:4-packed: a_vals uint8 [Mr,K/2], a_meta canonical
  *     uint16 [Mr,K/16]. alpha is normally 1 / (scale_A * scale_B).
@@ -203,9 +204,9 @@ SF_API int sf_gemm_sparse24_noalloc(const void* a_vals, const void* a_meta, cons
  *     8-bit 2:4 instruction reads it); read its status with sf_check_status.
  * Errors as everywhere: SF_ERR_SHAPE / NULL / ALIGN / ARCH before anything is launched. */
 SF_API int sf_fp8_quantize(const void* X, int64_t rows, int64_t cols, int64_t ld, float scale, void* Xq, void* stream);
-SF_API int sf_prune24_fp8_sizes(int64_t rows, int64_t cols, size_t* vals_bytes, size_t* meta_bytes);
-SF_API int sf_prune24_compress_fp8(const void* W, int64_t rows, int64_t cols, int64_t ld, int prune_mode, float scale,
-                                   void* vals, void* meta, void* dense_out, void* stream);
+SF_API int sf_prune24_fp8_sizes(int64_t rows, int64_t cols, int group_dim, size_t* vals_bytes, size_t* meta_bytes);
+SF_API int sf_prune24_compress_fp8(const void* W, int64_t rows, int64_t cols, int64_t ld, int group_dim, int prune_mode,
+                                   float scale, void* vals, void* meta, void* dense_out, void* stream);
 SF_API int sf_gemm_fp8_workspace_size(int64_t Mr, int64_t K, size_t* bytes);
 SF_API int sf_gemm_fp8_dense(const void* A, const void* B, void* C, int64_t Mr, int64_t Nc, int64_t K, float alpha,
                              void* workspace, void* stream);

@@ -72,9 +72,10 @@ class Prune24Fp8Result:
     pos: np.ndarray      # uint8 [R, K/4, 2]
 
 
-def prune24_fp8(w_bits: np.ndarray, scale, mode: int = 0) -> Prune24Fp8Result:
-    """2:4 along the rows (four consecutive elements), then quantisation of what is kept."""
-    p = prune24(w_bits, group_dim=1, mode=mode)
+def prune24_fp8(w_bits: np.ndarray, scale, mode: int = 0, group_dim: int = 1) -> Prune24Fp8Result:
+    """2:4 (groups along a row, or along a column with K-major outputs, as in `prune24`), then
+    quantisation of what is kept. `dense` keeps the orientation of the input."""
+    p = prune24(w_bits, group_dim=group_dim, mode=mode)
     return Prune24Fp8Result(vals=quantize_fp8(p.vals, scale), meta=p.meta, dense=quantize_fp8(p.dense, scale), pos=p.pos)
 
 

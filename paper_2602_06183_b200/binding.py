@@ -69,8 +69,8 @@ _SIGNATURES = {
     "sf_gemm_sparse24_rm": (_i32, [_vp, _vp, _vp, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "sf_gemm_sparse24_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "sf_fp8_quantize": (_i32, [_vp, _i64, _i64, _i64, C.c_float, _vp, _vp]),
-    "sf_prune24_fp8_sizes": (_i32, [_i64, _i64, C.POINTER(_sz), C.POINTER(_sz)]),
-    "sf_prune24_compress_fp8": (_i32, [_vp, _i64, _i64, _i64, _i32, C.c_float, _vp, _vp, _vp, _vp]),
+    "sf_prune24_fp8_sizes": (_i32, [_i64, _i64, _i32, C.POINTER(_sz), C.POINTER(_sz)]),
+    "sf_prune24_compress_fp8": (_i32, [_vp, _i64, _i64, _i64, _i32, _i32, C.c_float, _vp, _vp, _vp, _vp]),
     "sf_gemm_fp8_workspace_size": (_i32, [_i64, _i64, C.POINTER(_sz)]),
     "sf_gemm_fp8_dense": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, C.c_float, _vp, _vp]),
     "sf_gemm_fp8_sparse24": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, C.c_float, _vp, _vp]),
@@ -267,20 +267,22 @@ def sf_fp8_quantize(X, scale: float, out=None, stream=None):
     return out
 
 
-def sf_prune24_compress_fp8(W, prune_mode: int, scale: float, want_dense: bool = False, out=None, stream=None):
-    """2:4 along the rows with the kept values quantised to E4M3 in the same pass.
-    Returns (vals uint8 [rows, cols/2], meta int16 [rows, cols/16], dense uint8 [rows, cols] or None);
-    ``out`` = a previous result to write into."""
+def sf_prune24_compress_fp8(W, prune_mode: int, scale: float, want_dense: bool = False, out=None, stream=None,
+                            group_dim: int = 1):
+    """2:4 with the kept values quantised to E4M3 in the same pass. group_dim as for sf_prune24_compress
+    (1: groups along a row; 0: along a column, outputs K-major). Returns (vals uint8 [R, K/2], meta int16
+    [R, K/16], dense uint8 [rows, cols] or None); ``out`` = a previous result to write into."""
     rows, cols = W.shape
+    R, K = (rows, cols) if group_dim == 1 else (cols, rows)
     vb, mb = _sz(), _sz()
-    _check(lib().sf_prune24_fp8_sizes(rows, cols, C.byref(vb), C.byref(mb)), "sf_prune24_fp8_sizes")
+    _check(lib().sf_prune24_fp8_sizes(rows, cols, group_dim, C.byref(vb), C.byref(mb)), "sf_prune24_fp8_sizes")
     if out is not None:
         vals, meta, dense = out
     else:
-        vals = torch.empty((rows, cols // 2), dtype=torch.uint8, device=W.device)
-        meta = torch.empty((rows, cols // 16), dtype=torch.int16, device=W.device)
+        vals = torch.empty((R, K // 2), dtype=torch.uint8, device=W.device)
+        meta = torch.empty((R, K // 16), dtype=torch.int16, device=W.device)
         dense = torch.empty((rows, cols), dtype=torch.uint8, device=W.device) if want_dense else None
-    _check(lib().sf_prune24_compress_fp8(_ptr(W), rows, cols, W.stride(0) if rows > 1 else cols, prune_mode,
+    _check(lib().sf_prune24_compress_fp8(_ptr(W), rows, cols, W.stride(0) if rows > 1 else cols, group_dim, prune_mode,
                                          float(scale), _ptr(vals), _ptr(meta), _ptr(dense), _stream(stream)),
            "sf_prune24_compress_fp8")
     return vals, meta, dense

@@ -4,8 +4,7 @@
 //
 // q = e4m3(float(x) * scale): one float32 product, one conversion (round to nearest even, magnitudes
 // above 448 clamp to 448). Selection and soft-threshold shrinkage are those of the bf16 pass.
-#include <cuda_fp8.h>
-
+#include "fp8_fmt.cuh"
 #include "gemm_tc.cuh"
 #include "sf_common.cuh"
 
@@ -20,15 +19,6 @@ namespace sf {
 namespace {
 
 constexpr size_t kStatusBytes8 = 256;
-
-// two floats -> two E4M3 codes (low byte = first)
-__device__ __forceinline__ uint32_t e4m3x2(float a, float b) {
-  return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
-}
-// a word of two bf16 patterns -> two codes
-__device__ __forceinline__ uint32_t quant2(uint32_t w, float scale) {
-  return e4m3x2(__fmul_rn(bf16_bits_to_float(w & 0xFFFFu), scale), __fmul_rn(bf16_bits_to_float(w >> 16), scale));
-}
 
 // One thread converts 16 consecutive elements of a row: two 128-bit loads, one 128-bit store.
 __global__ void __launch_bounds__(256)
@@ -136,24 +126,28 @@ int sf_fp8_quantize(const void* X, int64_t rows, int64_t cols, int64_t ld, float
   return SF_OK;
 }
 
-int sf_prune24_fp8_sizes(int64_t rows, int64_t cols, size_t* vals_bytes, size_t* meta_bytes) {
+int sf_prune24_fp8_sizes(int64_t rows, int64_t cols, int group_dim, size_t* vals_bytes, size_t* meta_bytes) {
   if (!vals_bytes || !meta_bytes) return SF_ERR_NULL;
-  if (rows < 0 || cols < 0 || cols % 32 != 0) return SF_ERR_SHAPE;
+  if (rows < 0 || cols < 0 || (group_dim != 0 && group_dim != 1)) return SF_ERR_SHAPE;
+  if (group_dim == 1 ? cols % 32 != 0 : (rows % 16 != 0 || cols % 8 != 0)) return SF_ERR_SHAPE;
   *vals_bytes = (size_t)rows * cols / 2;        // R * K/2 codes
   *meta_bytes = (size_t)rows * cols / 8;        // R * K/16 words * 2 B
   return SF_OK;
 }
 
-int sf_prune24_compress_fp8(const void* W, int64_t rows, int64_t cols, int64_t ld, int prune_mode, float scale,
-                            void* vals, void* meta, void* dense_out, void* stream) {
-  if (rows < 0 || cols < 0 || cols % 32 != 0 || cols > (int64_t)1 << 30 || (prune_mode != 0 && prune_mode != 1))
+int sf_prune24_compress_fp8(const void* W, int64_t rows, int64_t cols, int64_t ld, int group_dim, int prune_mode,
+                            float scale, void* vals, void* meta, void* dense_out, void* stream) {
+  if (rows < 0 || cols < 0 || (group_dim != 0 && group_dim != 1) || (prune_mode != 0 && prune_mode != 1))
     return SF_ERR_SHAPE;
+  if (group_dim == 1 ? (cols % 32 != 0 || cols > (int64_t)1 << 30) : (rows % 16 != 0 || cols % 8 != 0)) return SF_ERR_SHAPE;
+  if (group_dim == 0 && dense_out) return SF_ERR_UNSUPPORTED;      // the masked copy exists for contiguous groups only
   if (rows == 0 || cols == 0) return SF_OK;
   if (!W || !vals || !meta) return SF_ERR_NULL;
   if (ld < cols || ld % 8 != 0 || !aligned16(W) || !aligned16(vals) || !aligned16(meta) ||
       (dense_out && !aligned16(dense_out)))
     return SF_ERR_ALIGN;
   SF_TRY(check_arch());
+  if (group_dim == 0) return launch_prune24_cols_fp8(W, rows, cols, ld, prune_mode, scale, vals, meta, (cudaStream_t)stream);
   const int64_t n = rows * (cols >> 3);
   const int64_t per_cta = 256 * kUnitsPerThread;
   if ((n + per_cta - 1) / per_cta > 0x7FFFFFFF) return SF_ERR_SHAPE;

@@ -8,6 +8,7 @@
 //     shared memory, selects per column, and writes the transposed packed panel with 128-bit
 //     stores through a padded staging buffer.
 #include "sf_common.cuh"
+#include "fp8_fmt.cuh"
 #include "tc_ptx.cuh"
 #include "gemm_tc.cuh"
 
@@ -99,11 +100,12 @@ constexpr int kColsSmemBytes = 128 + kColsSlots * kColsTileBytes + kColsStageByt
 constexpr int kColsCtasPerSm = 5;                   // 44 KB each; measured best among 3..5 with two or three slots
 static_assert(kPanelK / 16 == 8 && kPanelC == 64, "index shifts in prune24_cols_kernel assume a 128 x 64 panel");
 
-template <bool kSoft>
+// kFp8: the kept values leave as E4M3 codes of float(value) * scale (vals = uint8 [Rc, Kd/2]); no masked copy.
+template <bool kSoft, bool kFp8 = false>
 __global__ void __launch_bounds__(256)
 prune24_cols_kernel(const __grid_constant__ CUtensorMap tmapW, int64_t Kd, int64_t Rc,
                     uint16_t* __restrict__ vals, uint16_t* __restrict__ meta, uint8_t* __restrict__ meta_hw,
-                    uint16_t* __restrict__ dense_out, int panels_x, int num_panels) {
+                    uint16_t* __restrict__ dense_out, int panels_x, int num_panels, float scale = 1.f) {
   using namespace ptx;
   extern __shared__ uint8_t cols_smem_raw[];
   uint8_t* cols_smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(cols_smem_raw) + 127) & ~uintptr_t(127));
@@ -188,7 +190,13 @@ prune24_cols_kernel(const __grid_constant__ CUtensorMap tmapW, int64_t Kd, int64
       }
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        *reinterpret_cast<uint4*>(&stage[c + e][ch * 16]) = make_uint4(packed[e][0], packed[e][1], packed[e][2], packed[e][3]);
+        if (kFp8) {
+          const uint32_t q0 = quant2(packed[e][0], scale), q1 = quant2(packed[e][1], scale);
+          const uint32_t q2 = quant2(packed[e][2], scale), q3 = quant2(packed[e][3], scale);
+          *reinterpret_cast<uint2*>(&stage[c + e][ch * 8]) = make_uint2(q0 | (q1 << 16), q2 | (q3 << 16));
+        } else {
+          *reinterpret_cast<uint4*>(&stage[c + e][ch * 16]) = make_uint4(packed[e][0], packed[e][1], packed[e][2], packed[e][3]);
+        }
         mstage[c + e][ch] = (uint16_t)m[e];
         // tensor-core order (see meta_hw_offset): the panel's 64 output rows are four 16-row blocks of one atom
         const int mi = c + e;
@@ -204,9 +212,13 @@ prune24_cols_kernel(const __grid_constant__ CUtensorMap tmapW, int64_t Kd, int64
     for (int i = tid; i < kPanelC * chunks; i += 256) {
       const int c = full_k ? (i >> 3) : (i / chunks), ch = i - c * chunks;
       if (c >= cvalid) continue;
-      const uint4 q = *reinterpret_cast<const uint4*>(&stage[c][ch * 16]);
       const int64_t orow = c0 + c;
-      *reinterpret_cast<uint4*>(vals + orow * (Kd >> 1) + (k0 >> 1) + ch * 8) = q;
+      if (kFp8) {
+        *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(vals) + orow * (Kd >> 1) + (k0 >> 1) + ch * 8) =
+            *reinterpret_cast<const uint2*>(&stage[c][ch * 8]);
+      } else {
+        *reinterpret_cast<uint4*>(vals + orow * (Kd >> 1) + (k0 >> 1) + ch * 8) = *reinterpret_cast<const uint4*>(&stage[c][ch * 16]);
+      }
     }
     if (full_k && (Kd & 127) == 0) {
       // whole panels: a column's eight metadata words are 16 contiguous, aligned bytes in either order
@@ -351,6 +363,38 @@ int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int gr
       prune24_cols_kernel<true><<<grid, 256, kColsSmemBytes, s>>>(tm, rows, cols, (uint16_t*)vals, (uint16_t*)meta,
                                                                   (uint8_t*)meta_hw, (uint16_t*)dense_out, (int)px, num_panels);
   }
+  SF_LAUNCH_CHECK();
+  return SF_OK;
+}
+
+int launch_prune24_cols_fp8(const void* W, int64_t rows, int64_t cols, int64_t ld, int prune_mode, float scale, void* vals,
+                            void* meta, cudaStream_t s) {
+  if (rows == 0 || cols == 0) return SF_OK;
+  const int64_t px = (cols + kPanelC - 1) / kPanelC, py = (rows + kPanelK - 1) / kPanelK;
+  if (px * py > (int64_t)1 << 30) return SF_ERR_SHAPE;
+  const int num_panels = (int)(px * py);
+  static bool attr_done[64] = {false};
+  static int sms[64] = {0};
+  int dev = 0;
+  SF_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return SF_ERR_UNSUPPORTED;
+  if (!attr_done[dev]) {
+    SF_CUDA_TRY(cudaFuncSetAttribute(prune24_cols_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kColsSmemBytes));
+    SF_CUDA_TRY(cudaFuncSetAttribute(prune24_cols_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kColsSmemBytes));
+    SF_CUDA_TRY(cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev));
+    attr_done[dev] = true;
+  }
+  alignas(64) CUtensorMap tm;
+  int st = make_tmap_2d(&tm, W, rows, cols, ld, kPanelC, kPanelK, false);
+  if (st != SF_OK) return st;
+  const int resident = sms[dev] * kColsCtasPerSm;
+  const unsigned grid = (unsigned)(num_panels < resident ? num_panels : resident);
+  if (prune_mode == 0)
+    prune24_cols_kernel<false, true><<<grid, 256, kColsSmemBytes, s>>>(tm, rows, cols, (uint16_t*)vals, (uint16_t*)meta, nullptr,
+                                                                       nullptr, (int)px, num_panels, scale);
+  else
+    prune24_cols_kernel<true, true><<<grid, 256, kColsSmemBytes, s>>>(tm, rows, cols, (uint16_t*)vals, (uint16_t*)meta, nullptr,
+                                                                      nullptr, (int)px, num_panels, scale);
   SF_LAUNCH_CHECK();
   return SF_OK;
 }

@@ -162,6 +162,9 @@ int launch_prune24(const void* W, int64_t rows, int64_t cols, int64_t ld, int gr
 int launch_vnm(const void* P, int64_t T, int64_t F, int64_t ld, int V, int M, int apply_sqrelu,
                void* vals, void* meta, void* meta_hw, void* colidx, void* relu_vals, void* dense_out,
                void* relu_dense_out, void* vals24, void* meta24, void* meta24_hw, void* relu24, cudaStream_t s);
+// Strided groups with the kept values quantised to E4M3 codes in the same pass (vals uint8 [cols, rows/2]).
+int launch_prune24_cols_fp8(const void* W, int64_t rows, int64_t cols, int64_t ld, int prune_mode, float scale, void* vals,
+                            void* meta, cudaStream_t s);
 bool vnm_has_24_view(int64_t F, int V, int M);
 // Streaming form of the sparsifier (values, ReLU values, canonical metadata and colidx only).
 bool vnm_stream_supported(int64_t F, int64_t ld, int V, int M, const void* P);

@@ -57,6 +57,24 @@ def test_prune24_fp8_bit_exact(rows, cols, scale, mode):
     assert none is None and torch.equal(vals2, vals) and torch.equal(meta2, meta)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("rows,cols,scale", [(16, 8, 1.0), (128, 64, 30.0), (400, 136, 500.0), (1024, 512, 2.0), (272, 1000, 64.0)])
+def test_prune24_fp8_strided_groups_bit_exact(rows, cols, scale, mode):
+    """Groups along a column, outputs K-major (the W2 direction): ragged panels, strided source."""
+    w = synth.prune_sweep_matrix(rows, cols, seed=3 * rows + cols + mode, tie_frac=0.15)
+    ref = fp8.prune24_fp8(w, scale, mode=mode, group_dim=0)
+    wide = torch.zeros((rows, cols + 16), dtype=torch.bfloat16, device="cuda")
+    wide[:, :cols] = to_dev(w)
+    for src in (to_dev(w), wide[:, :cols]):
+        vals, meta, none = binding.sf_prune24_compress_fp8(src, mode, scale, group_dim=0)
+        torch.cuda.synchronize()
+        assert none is None
+        assert np.array_equal(bits(meta), ref.meta)
+        assert np.array_equal(_u8(vals), ref.vals)
+    with pytest.raises(binding.SparseFFNError):
+        binding.sf_prune24_compress_fp8(to_dev(w), mode, scale, want_dense=True, group_dim=0)
+
+
 def test_prune24_fp8_saturates_and_keeps_signed_zero():
     w = synth.f32_to_bf16_bits(np.array([[1000.0, -2000.0, 1.0, 2.0, -0.0, 0.0, -1e-30, 1e-30] * 4], dtype=np.float32))
     ref = fp8.prune24_fp8(w.reshape(1, 32), 1.0)

@@ -122,3 +122,13 @@ def test_gemm_fp8_small_by_hand():
     b = fp8.f32_to_e4m3(np.array([[3.0, 1.0], [-1.0, 0.25]], dtype=np.float32))
     c = fp8.gemm_fp8(a, b, 0.5)
     assert np.array_equal(c, np.array([[2.5, -0.25], [-1.25, -0.75]], dtype=np.float32))
+
+
+def test_prune24_fp8_strided_groups_are_the_transposed_problem():
+    rng = np.random.default_rng(12)
+    w = f32_to_bf16((rng.standard_normal((32, 24)) * 0.05).astype(np.float32)).reshape(32, 24)
+    for mode in (0, 1):
+        a = fp8.prune24_fp8(w, 100.0, mode=mode, group_dim=0)
+        b = fp8.prune24_fp8(np.ascontiguousarray(w.T), 100.0, mode=mode, group_dim=1)
+        assert np.array_equal(a.vals, b.vals) and np.array_equal(a.meta, b.meta)
+        assert np.array_equal(a.dense, b.dense.T)
