@@ -45,14 +45,23 @@ route_kernel(const uint16_t* __restrict__ X, const uint16_t* __restrict__ means,
   for (int i = 0; i < kRouteTokens; ++i)
 #pragma unroll
     for (int e = 0; e < kMaxExperts; ++e) acc[i][e] = 0.f;
+  // the next chunk of the four tokens is requested before this one is multiplied
+  uint4 nxt[kRouteTokens];
+  auto fetch = [&](int c) {
+#pragma unroll
+    for (int i = 0; i < kRouteTokens; ++i) {
+      const int t = min(t0 + i, T - 1);                                     // a ragged last group re-reads the last token
+      nxt[i] = __ldg(reinterpret_cast<const uint4*>(X + (int64_t)t * D + c));
+    }
+  };
+  fetch(lane * 8);
   for (int c = lane * 8; c < D; c += 256) {
     uint32_t xw[kRouteTokens][4];
 #pragma unroll
     for (int i = 0; i < kRouteTokens; ++i) {
-      const int t = min(t0 + i, T - 1);                                     // a ragged last group re-reads the last token
-      const uint4 xv = __ldg(reinterpret_cast<const uint4*>(X + (int64_t)t * D + c));
-      xw[i][0] = xv.x; xw[i][1] = xv.y; xw[i][2] = xv.z; xw[i][3] = xv.w;
+      xw[i][0] = nxt[i].x; xw[i][1] = nxt[i].y; xw[i][2] = nxt[i].z; xw[i][3] = nxt[i].w;
     }
+    if (c + 256 < D) fetch(c + 256);
 #pragma unroll
     for (int e = 0; e < kMaxExperts; ++e) {
       if (e < E) {
@@ -200,15 +209,26 @@ tile_tables_kernel(const int* __restrict__ seg, int E, int D, int F, GemmTile* _
   }
 }
 
-// out[r, :] = src[r] >= 0 ? in[src[r], :] : 0   (16 bytes per thread)
+// out[r, :] = src[r] >= 0 ? in[src[r], :] : 0. One warp per output row; a lane keeps four 16-byte loads in
+// flight, every instruction of the warp covers 512 contiguous bytes.
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint4* __restrict__ in, const int* __restrict__ src, uint4* __restrict__ out, int rows,
                    int row_u4) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)rows * row_u4) return;
-  const int r = (int)(idx / row_u4), c = (int)(idx - (int64_t)r * row_u4);
+  const int r = (int)blockIdx.x * 8 + (int)(threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (r >= rows) return;
   const int s = __ldg(src + r);
-  out[idx] = s >= 0 ? __ldg(in + (int64_t)s * row_u4 + c) : make_uint4(0u, 0u, 0u, 0u);
+  const uint4* ip = in + (int64_t)(s >= 0 ? s : 0) * row_u4;
+  uint4* op = out + (int64_t)r * row_u4;
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  int c = lane;
+  for (; c + 96 < row_u4; c += 128) {
+    uint4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = s >= 0 ? __ldg(ip + c + 32 * j) : zero;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) op[c + 32 * j] = v[j];
+  }
+  for (; c < row_u4; c += 32) op[c] = s >= 0 ? __ldg(ip + c) : zero;
 }
 
 // ---- buffers ---------------------------------------------------------------------------------------------------
@@ -295,10 +315,9 @@ int launch_route(const void* X, const void* means, int64_t T, int64_t D, int E, 
 }
 
 int launch_gather_rows(const void* in, const int* src, void* out, int64_t rows, int64_t cols, cudaStream_t s) {
-  const int64_t n = rows * (cols / 8);
-  if (n == 0) return SF_OK;
-  gather_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>((const uint4*)in, src, (uint4*)out, (int)rows,
-                                                                (int)(cols / 8));
+  if (rows == 0 || cols == 0) return SF_OK;
+  gather_rows_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, s>>>((const uint4*)in, src, (uint4*)out, (int)rows,
+                                                               (int)(cols / 8));
   SF_LAUNCH_CHECK();
   return SF_OK;
 }
