@@ -117,6 +117,27 @@ __device__ __forceinline__ void epi_tile(const GemmArgs& args, uint32_t taddr, i
                                          int q, int lane, uint8_t* my_stage,
                                          const uint4 (&ax)[is_drelu_t(kEpi) ? kTileN / 32 : 1][4]) {
   int64_t row = m0 + q * 32 + lane;                                        // this thread's D row
+  if constexpr (kEpi == EPI_ROUTE) {
+    // the row is a token, the first route_E columns its logits
+    uint32_t v[32];
+    tmem_ld_32x32b_x32(taddr, v);
+    tmem_ld_wait_on(v);
+    const int E = args.route_E;
+    int best = 0;
+    float bestv = __uint_as_float(v[0]);
+#pragma unroll
+    for (int e = 1; e < 16; ++e) {
+      const float x = __uint_as_float(v[e]);
+      if (e < E && x > bestv) { bestv = x; best = e; }                     // strict: ties stay with the lower expert
+    }
+    args.route_expert[row] = best;
+    if (args.route_logits) {
+#pragma unroll
+      for (int e = 0; e < 16; ++e)
+        if (e < E) args.route_logits[row * E + e] = __uint_as_float(v[e]);
+    }
+    return;
+  }
   bool row_live = true;
   if (kEpi == EPI_STORE && args.row_map) {                                 // scattered output rows
     const int r = __ldg(args.row_map + row);
@@ -1300,6 +1321,23 @@ int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, boo
                : launch_one<MODE_SPARSE24, false, false, EPI_DRELU_T>(ta, tb, a, s);
   if (epi == EPI_DRELU24_T) return launch_two<MODE_SPARSE24, false, false, EPI_DRELU24_T, kNarrowBN>(ta, tb, tm, a, s);
   return SF_ERR_UNSUPPORTED;
+}
+
+int gemm_route(const void* X, const void* means, int64_t T, int64_t D, int E, int* expert, float* logits, int* status,
+               cudaStream_t s) {
+  if (T % 256 || D % 64 || E < 1 || E > 16) return SF_ERR_SHAPE;
+  if (T == 0) return SF_OK;
+  CUtensorMap ta, tb;
+  int st = make_tmap(&ta, X, T, D, D, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st != SF_OK) return st;
+  st = make_tmap(&tb, means, E, D, D, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);     // rows beyond E arrive as zeros
+  if (st != SF_OK) return st;
+  GemmArgs a{};
+  a.M = T; a.N = 256; a.K = D;
+  a.status = status;
+  a.route_expert = expert; a.route_logits = logits; a.route_E = E;
+  a.num_k_blocks = (int)(D / 64);
+  return launch_two<MODE_DENSE, false, false, EPI_ROUTE>(ta, tb, ta, a, s);
 }
 
 int gemm_fp8(bool sparse, const void* A, const uint8_t* meta_hw, const void* B, int64_t M, int64_t N, int64_t K,

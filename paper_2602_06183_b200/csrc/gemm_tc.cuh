@@ -18,9 +18,11 @@ enum GemmEpilogue {
                     // features, columns are tokens; writes the packed activation, never the dense y1  (Eq. 2, Section 2.3)
   EPI_DRELU24_T = 6,// as EPI_DRELU_T with aux given in the 2:4 layout of the mask (values [n, m/2] + pack_meta) and
                     // only the packed output written
-  EPI_ACT24_T = 7   // transposed output with SquaredReLU and a 2:4 selection inside every four features of a token
+  EPI_ACT24_T = 7,  // transposed output with SquaredReLU and a 2:4 selection inside every four features of a token
                     // (the routed step's activation, Section 3.1 step 3): packed values, packed ReLU values, both
                     // metadata orders and the masked dense copy; never the pre-activation unless asked for
+  EPI_ROUTE = 8     // accumulator rows are tokens, its first route_E columns the experts' logits: each row writes its
+                    // arg-max (ties to the lower expert) and, optionally, the float32 logits   (Section 3.1 step 1)
 };
 
 // One output tile of a table-driven (grouped) product on CTA pairs. Offsets are in elements of the
@@ -69,6 +71,10 @@ struct GemmArgs {
   const int* row_map;
   // EPI_STORE only: the accumulator is multiplied by this before rounding (0 = no scaling)
   float out_scale;
+  // EPI_ROUTE
+  int* route_expert;         // int32 [M]
+  float* route_logits;       // optional float32 [M, route_E]
+  int route_E;               // 1..16
 };
 
 // Outputs of the fused y1 product (see GemmArgs::vn_*).
@@ -126,6 +132,11 @@ int gemm_grouped_dense_tn(const void* A, int64_t Ma, const void* B, int64_t Nb, 
 int gemm_sparse24(const void* a_vals, const uint8_t* meta_hw, const void* B, bool b_kmajor, int64_t M, int64_t N,
                   int64_t K, int epi, void* C, int64_t ldc, const void* aux, int64_t ldaux, int* status,
                   cudaStream_t s, const void* pack_meta = nullptr, void* pack_vals = nullptr);
+// Routing on the tensor cores: logits[T, E] = X[T, D] means[E, D]^T in float32 accumulators, the arg-max per token
+// taken in the epilogue (ties to the lower expert). T % 256 == 0, D % 64 == 0, 1 <= E <= 16; the means need no
+// padding (rows beyond E are read as zeros by the tensor map).
+int gemm_route(const void* X, const void* means, int64_t T, int64_t D, int E, int* expert, float* logits, int* status,
+               cudaStream_t s);
 // E4M3 operands, both K-major: C[M, N] = bf16(alpha * A B^T). sparse: A = 2:4 values [M, K/2] (codes) with
 // metadata in the 8-bit instruction's order (see meta_hw8_offset); else A [M, K]. B [N, K].
 // M % 256 == 0, N % 32 == 0, K % 256 == 0 (2:4) or K % 128 == 0 (dense).

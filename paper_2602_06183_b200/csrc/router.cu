@@ -29,12 +29,12 @@ constexpr size_t kStatusBytes = 256;
 inline size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // ---- step 1: routing ----------------------------------------------------------------------------------
-// One warp per four tokens (the expert means are read once per four tokens). A lane owns eight consecutive
+// One warp per two tokens (the expert means, small enough for the L1, are read once per pair). A lane owns eight consecutive
 // elements of every 256-element chunk and keeps one float32 partial sum per (token, expert); the partial
 // sums are combined by a fixed xor-shuffle tree, so the result does not depend on the launch.
-constexpr int kRouteTokens = 4;
+constexpr int kRouteTokens = 2;
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 route_kernel(const uint16_t* __restrict__ X, const uint16_t* __restrict__ means, int T, int D, int E,
              int* __restrict__ expert, float* __restrict__ logits) {
   const int lane = threadIdx.x & 31;
@@ -45,35 +45,59 @@ route_kernel(const uint16_t* __restrict__ X, const uint16_t* __restrict__ means,
   for (int i = 0; i < kRouteTokens; ++i)
 #pragma unroll
     for (int e = 0; e < kMaxExperts; ++e) acc[i][e] = 0.f;
-  // the next chunk of the four tokens is requested before this one is multiplied
+  // The kernel waits on memory, not arithmetic. The tokens stream past the L1 (no allocation there), so the
+  // expert means stay in it; the next chunk of the tokens is requested before this one is multiplied, and
+  // the means of eight experts are requested together before any of them is used.
+  auto load_stream = [](const uint16_t* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+  };
   uint4 nxt[kRouteTokens];
   auto fetch = [&](int c) {
 #pragma unroll
     for (int i = 0; i < kRouteTokens; ++i) {
       const int t = min(t0 + i, T - 1);                                     // a ragged last group re-reads the last token
-      nxt[i] = __ldg(reinterpret_cast<const uint4*>(X + (int64_t)t * D + c));
+      nxt[i] = load_stream(X + (int64_t)t * D + c);
     }
   };
   fetch(lane * 8);
   for (int c = lane * 8; c < D; c += 256) {
-    uint32_t xw[kRouteTokens][4];
+    // widen the chunk once (eight values per token), then one multiply-add per (token, expert, element) in
+    // element order
+    float xf[kRouteTokens][8];
 #pragma unroll
     for (int i = 0; i < kRouteTokens; ++i) {
-      xw[i][0] = nxt[i].x; xw[i][1] = nxt[i].y; xw[i][2] = nxt[i].z; xw[i][3] = nxt[i].w;
+      const uint32_t xw[4] = {nxt[i].x, nxt[i].y, nxt[i].z, nxt[i].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        xf[i][2 * j] = bf16_bits_to_float(xw[j] & 0xFFFFu);
+        xf[i][2 * j + 1] = bf16_bits_to_float(xw[j] >> 16);
+      }
     }
     if (c + 256 < D) fetch(c + 256);
 #pragma unroll
-    for (int e = 0; e < kMaxExperts; ++e) {
-      if (e < E) {
-        const uint4 mv = __ldg(reinterpret_cast<const uint4*>(means + (int64_t)e * D + c));
-        const uint32_t mw[4] = {mv.x, mv.y, mv.z, mv.w};
+    for (int e0 = 0; e0 < kMaxExperts; e0 += 8) {
+      if (e0 < E) {
+        uint4 mv[8];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float m0 = bf16_bits_to_float(mw[j] & 0xFFFFu), m1 = bf16_bits_to_float(mw[j] >> 16);
+        for (int k = 0; k < 8; ++k)
+          mv[k] = __ldg(reinterpret_cast<const uint4*>(means + (int64_t)min(e0 + k, E - 1) * D + c));
 #pragma unroll
-          for (int i = 0; i < kRouteTokens; ++i) {
-            acc[i][e] = __fmaf_rn(bf16_bits_to_float(xw[i][j] & 0xFFFFu), m0, acc[i][e]);
-            acc[i][e] = __fmaf_rn(bf16_bits_to_float(xw[i][j] >> 16), m1, acc[i][e]);
+        for (int k = 0; k < 8; ++k) {
+          if (e0 + k < E) {
+            const uint32_t mw[4] = {mv[k].x, mv[k].y, mv[k].z, mv[k].w};
+            float mf[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              mf[2 * j] = bf16_bits_to_float(mw[j] & 0xFFFFu);
+              mf[2 * j + 1] = bf16_bits_to_float(mw[j] >> 16);
+            }
+#pragma unroll
+            for (int i = 0; i < kRouteTokens; ++i)
+#pragma unroll
+              for (int j = 0; j < 8; ++j) acc[i][e0 + k] = __fmaf_rn(xf[i][j], mf[j], acc[i][e0 + k]);
           }
         }
       }
@@ -379,7 +403,8 @@ int sf_routed_ffn_fwd(const sf_router_desc* desc, const void* X, const void* W1,
   if (forced_expert) {
     SF_CUDA_TRY(cudaMemcpyAsync(expert, forced_expert, (size_t)d.T * 4, cudaMemcpyDeviceToDevice, s));
   } else {
-    SF_TRY(launch_route(X, means, d.T, d.D, d.E, expert, at(fwd_ctx, L.logits), s));
+    // T % 256 == 0 here: the logits are one tensor-core product with the arg-max in its epilogue
+    SF_TRY(gemm_route(X, means, d.T, d.D, d.E, (int*)expert, (float*)at(fwd_ctx, L.logits), (int*)workspace, s));
   }
   trace_mark(s);
   // step 2: token order, tile tables, gathered X
