@@ -191,6 +191,50 @@ def test_routed_step_without_saved_y1_and_repeated_is_bit_identical():
             assert torch.equal(a, b)
 
 
+def test_routed_step_replays_from_a_cuda_graph():
+    """Routing, grouping and the tile tables all stay on the device (no host round trip, no allocation), so the
+    routed step can be captured once and replayed; a replay on different tokens must follow their routing."""
+    T, D, F, E = 768, 256, 1024, 4
+    X, W1, W2, dY = synth.ffn_inputs(T, D, F, 0.05, 56)
+    X2 = synth.ffn_inputs(T, D, F, 0.05, 57)[0]
+    means = synth.normal_bf16((E, D), 0.0, 1.0, 56, 9)
+    dXa, dXb, dW1_, dW2_, dY_, dM = (to_dev(a) for a in (X, X2, W1, W2, dY, means))
+    desc = binding.make_router_desc(T, D, F, E)
+    nctx, nws = binding.sf_routed_ffn_workspace_size(desc)
+    ctx = torch.zeros((nctx,), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros((nws,), dtype=torch.uint8, device="cuda")
+    Xin = dXa.clone()
+    Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+    gX, gW1, gW2 = torch.empty_like(Xin), torch.empty_like(dW1_), torch.empty_like(dW2_)
+
+    def step():
+        binding.sf_routed_ffn_fwd(desc, Xin, dW1_, dW2_, dM, Y, ctx, ws)
+        binding.sf_routed_ffn_bwd(desc, dY_, Xin, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
+
+    eager = {}
+    for name, src in (("a", dXa), ("b", dXb)):
+        Xin.copy_(src)
+        step()
+        torch.cuda.synchronize()
+        eager[name] = [t.clone() for t in (Y, gX, gW1, gW2)]
+    assert not torch.equal(eager["a"][0], eager["b"][0])
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    for name, src in (("a", dXa), ("b", dXb), ("a", dXa)):
+        Xin.copy_(src)
+        for t in (Y, gX, gW1, gW2):
+            t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert binding.sf_check_status(ws) == binding.SF_OK
+        for a, b in zip(eager[name], (Y, gX, gW1, gW2)):
+            assert torch.equal(a, b)
+
+
 def test_routed_step_all_zero_tokens():
     """X = 0: every logit ties at zero, so every token goes to expert 0 (ties to the lower expert), the
     other experts keep one zero tile each, and all outputs are exactly zero."""
