@@ -67,7 +67,11 @@ typedef enum sf_ffn_flags {
   SF_FFN_PACKED_GRAD_OPERANDS = 8 /* M == 8: keep no masked [T, F] copy of y2 and dy1; the two weight-gradient
                              products expand their operand from its packed form inside the kernel. Saves
                              4*T*F bytes of context + workspace, costs about a third more time in those two
-                             products. Same results, bit for bit. */
+                             products. Same results, bit for bit. */,
+  SF_FFN_W2_FD = 16 /* W2 is given, and dW2 is returned, as [F, D] row-major (the transposed storage) in every
+                       step call of this descriptor, the dense step included. The 2:4 groups of W2 along d_model
+                       are then contiguous (the faster pruning pass), and the M >= 16 step needs no transposed
+                       copy of W2. Without the flag W2 and dW2 are [D, F]. */
 } sf_ffn_flags;
 typedef struct sf_ffn_desc {
   int64_t T, D, F;

@@ -22,7 +22,7 @@ SF_ERR_ARCH, SF_ERR_CUDA, SF_ERR_TIMEOUT, SF_ERR_UNSUPPORTED = -5, -6, -7, -8
 
 SF_CTX_Y2_VALS, SF_CTX_RELU_VALS, SF_CTX_META, SF_CTX_COLIDX, SF_CTX_Y1, SF_CTX_DY1_VALS = range(6)
 SF_CTX_Y2_VALS24, SF_CTX_Y2_META24, SF_CTX_DY1_VALS24, SF_CTX_RELU_VALS24 = 6, 7, 8, 9
-SF_FFN_SAVE_Y1, SF_FFN_UNFUSED_ACT, SF_FFN_FUSED_ACT, SF_FFN_PACKED_GRAD_OPERANDS = 1, 2, 4, 8
+SF_FFN_SAVE_Y1, SF_FFN_UNFUSED_ACT, SF_FFN_FUSED_ACT, SF_FFN_PACKED_GRAD_OPERANDS, SF_FFN_W2_FD = 1, 2, 4, 8, 16
 
 
 class sf_ffn_desc(C.Structure):

@@ -190,7 +190,7 @@ int check_desc(const sf_ffn_desc* d) {
   if (!d) return SF_ERR_NULL;
   if (d->N != 2) return SF_ERR_UNSUPPORTED;
   if (d->M != 4 && d->M != 8 && d->M != 16 && d->M != 32 && d->M != 64) return SF_ERR_SHAPE;
-  if (d->flags & ~(SF_FFN_SAVE_Y1 | SF_FFN_UNFUSED_ACT | SF_FFN_FUSED_ACT | SF_FFN_PACKED_GRAD_OPERANDS))
+  if (d->flags & ~(SF_FFN_SAVE_Y1 | SF_FFN_UNFUSED_ACT | SF_FFN_FUSED_ACT | SF_FFN_PACKED_GRAD_OPERANDS | SF_FFN_W2_FD))
     return SF_ERR_UNSUPPORTED;
   if ((d->flags & SF_FFN_UNFUSED_ACT) && (d->flags & SF_FFN_FUSED_ACT)) return SF_ERR_UNSUPPORTED;
   if (d->V != 64 && d->V != 128) return SF_ERR_SHAPE;
@@ -352,7 +352,7 @@ int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, co
   const SparseLayout L = sparse_layout(d);
   cudaStream_t s = (cudaStream_t)stream;
   int* status = (int*)workspace;
-  const bool save_y1 = (d.flags & SF_FFN_SAVE_Y1) != 0;
+  const bool save_y1 = (d.flags & SF_FFN_SAVE_Y1) != 0, w2_fd = (d.flags & SF_FFN_W2_FD) != 0;
 
   // Algorithm 1 line 4: W1s = sparsify24(W1) along d_model, then y1 = X W1s^T
   trace_mark(s);
@@ -392,14 +392,15 @@ int sf_sparse_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, co
   if (L.plain24) {
     // y2 as a 2:4 operand over all F columns against W2 [D, F] as it is stored (no transpose, no gather)
     trace_mark(s);
-    SF_TRY(gemm_sparse24(at(fwd_ctx, L.vals24), at(fwd_ctx, L.meta24_hw), W2, true, d.T, d.D, d.F, EPI_STORE, Y, d.D,
+    // (W2 given as [F, D]: the same product with W2 as the MN-major operand)
+    SF_TRY(gemm_sparse24(at(fwd_ctx, L.vals24), at(fwd_ctx, L.meta24_hw), W2, !w2_fd, d.T, d.D, d.F, EPI_STORE, Y, d.D,
                          nullptr, 0, status, s));
   } else {
-    // condensed V:N:M operand; rows of W2^T are gathered by the kept columns
-    SF_TRY(launch_transpose(W2, at(fwd_ctx, L.w2t), d.D, d.F, s));
+    // condensed V:N:M operand; rows of W2^T are gathered by the kept columns (W2 given as [F, D] is that matrix)
+    if (!w2_fd) SF_TRY(launch_transpose(W2, at(fwd_ctx, L.w2t), d.D, d.F, s));
     trace_mark(s);
-    SF_TRY(gemm_venom(at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx), at(fwd_ctx, L.w2t), d.T,
-                      d.F, d.D, d.V, d.M, Y, d.D, status, s));
+    SF_TRY(gemm_venom(at(fwd_ctx, L.y2_vals), at(fwd_ctx, L.meta_hw), at(fwd_ctx, L.colidx),
+                      w2_fd ? W2 : (const void*)at(fwd_ctx, L.w2t), d.T, d.F, d.D, d.V, d.M, Y, d.D, status, s));
   }
   trace_mark(s);
   return SF_OK;
@@ -416,11 +417,21 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
   const SparseLayout L = sparse_layout(d);
   cudaStream_t s = (cudaStream_t)stream;
   int* status = (int*)workspace;
+  const bool w2_fd = (d.flags & SF_FFN_W2_FD) != 0;
+  // dW2 = dY^T y2 in the layout of W2: [D, F], or [F, D] = y2^T dY when W2 is stored that way
+  auto grad_w2 = [&](const void* y2_dense) -> int {
+    return w2_fd ? gemm_dense(y2_dense, false, dY, false, d.F, d.D, d.T, EPI_STORE, dW2, d.D, nullptr, 0, nullptr, 0, status, s)
+                 : gemm_dense(dY, false, y2_dense, false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0, nullptr, 0, status, s);
+  };
 
   // Algorithm 2 line 2: W2s = sparsify24(W2^T) along d_model (contiguous in the saved W2^T copy),
   // dy2 = dY W2s;  line 4: dy1 = 2 dy2 ReLU(y1) on y2's mask (fused into the product's epilogue)
   trace_mark(s);
-  if (L.plain24) {
+  if (w2_fd) {
+    // W2 stored as [F, D]: the groups along d_model are contiguous
+    SF_TRY(launch_prune24(W2, d.F, d.D, d.D, 1, d.prune_mode, at(workspace, L.w2_vals), at(workspace, L.w2_meta),
+                          at(workspace, L.w2_meta_hw), nullptr, s));
+  } else if (L.plain24) {
     // no W2^T copy exists on this path: prune the strided groups of W2 [D, F] directly
     SF_TRY(launch_prune24(W2, d.D, d.F, d.F, 0, d.prune_mode, at(workspace, L.w2_vals), at(workspace, L.w2_meta),
                           at(workspace, L.w2_meta_hw), nullptr, s));
@@ -446,10 +457,10 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
     // runs over tokens); their masked operand is a stored [T, F] matrix or is expanded from its packed form
     // inside the kernel
     if (L.expand) {
-      SF_TRY(gemm_dense_expand(dY, 2, at(fwd_ctx, L.vals24), at(fwd_ctx, L.meta24), d.D, d.F, d.T, dW2, d.F, status, s));
+      if (w2_fd) SF_TRY(gemm_dense_expand(dY, 1, at(fwd_ctx, L.vals24), at(fwd_ctx, L.meta24), d.F, d.D, d.T, dW2, d.D, status, s));
+      else       SF_TRY(gemm_dense_expand(dY, 2, at(fwd_ctx, L.vals24), at(fwd_ctx, L.meta24), d.D, d.F, d.T, dW2, d.F, status, s));
     } else {
-      SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.y2_dense), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0,
-                        nullptr, 0, status, s));
+      SF_TRY(grad_w2(at(fwd_ctx, L.y2_dense)));
     }
     trace_mark(s);
     hook_dw2_done(s);
@@ -484,8 +495,7 @@ int sf_sparse_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, co
   trace_mark(s);
   hook_dx_done(s);
   // line 3: dW2 = dY^T y2 [D, F];  line 6: dW1 = dy1^T X [F, D]  (reduction over tokens)
-  SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.y2_dense), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0,
-                    nullptr, 0, status, s));
+  SF_TRY(grad_w2(at(fwd_ctx, L.y2_dense)));
   trace_mark(s);
   hook_dw2_done(s);
   SF_TRY(gemm_dense(at(workspace, L.dy1_dense), false, X, false, d.F, d.D, d.T, EPI_STORE, dW1, d.D, nullptr, 0,
@@ -510,8 +520,8 @@ int sf_dense_ffn_fwd(const sf_ffn_desc* desc, const void* X, const void* W1, con
                     nullptr, 0, status, s));
   trace_mark(s);
   hook_wait_w2(s);
-  SF_TRY(gemm_dense(at(fwd_ctx, L.h), true, W2, true, d.T, d.D, d.F, EPI_STORE, Y, d.D, nullptr, 0, nullptr, 0,
-                    status, s));
+  SF_TRY(gemm_dense(at(fwd_ctx, L.h), true, W2, !(d.flags & SF_FFN_W2_FD), d.T, d.D, d.F, EPI_STORE, Y, d.D, nullptr, 0,
+                    nullptr, 0, status, s));
   trace_mark(s);
   return SF_OK;
 }
@@ -530,7 +540,8 @@ int sf_dense_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, con
   void* dy1 = at(workspace, L.dy1);
   // Eq. 4 + 6: dy1 = 2 (dY W2) ReLU(y1)
   trace_mark(s);
-  SF_TRY(gemm_dense(dY, true, W2, false, d.T, d.F, d.D, EPI_DRELU, dy1, d.F, nullptr, 0, at(fwd_ctx, L.y1), d.F,
+  const bool w2_fd = (d.flags & SF_FFN_W2_FD) != 0;                 // W2 [F, D] is the K-major operand of this product
+  SF_TRY(gemm_dense(dY, true, W2, w2_fd, d.T, d.F, d.D, EPI_DRELU, dy1, d.F, nullptr, 0, at(fwd_ctx, L.y1), d.F,
                     status, s));
   trace_mark(s);
   // Eq. 7: dX = dy1 W1
@@ -538,8 +549,12 @@ int sf_dense_ffn_bwd(const sf_ffn_desc* desc, const void* dY, const void* X, con
   trace_mark(s);
   hook_dx_done(s);
   // Eq. 5: dW2 = dY^T h [D, F];  Eq. 8: dW1 = dy1^T X [F, D]
-  SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.h), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0, nullptr, 0,
-                    status, s));
+  if (w2_fd)
+    SF_TRY(gemm_dense(at(fwd_ctx, L.h), false, dY, false, d.F, d.D, d.T, EPI_STORE, dW2, d.D, nullptr, 0, nullptr, 0,
+                      status, s));
+  else
+    SF_TRY(gemm_dense(dY, false, at(fwd_ctx, L.h), false, d.D, d.F, d.T, EPI_STORE, dW2, d.F, nullptr, 0, nullptr, 0,
+                      status, s));
   trace_mark(s);
   hook_dw2_done(s);
   SF_TRY(gemm_dense(dy1, false, X, false, d.F, d.D, d.T, EPI_STORE, dW1, d.D, nullptr, 0, nullptr, 0, status, s));

@@ -1273,6 +1273,7 @@ int gemm_dense(const void* A, bool a_kmajor, const void* B, bool b_kmajor, int64
     if (!amn && !bmn) SF_DENSE_CASE(false, false, EPI_SQRELU);
   } else if (epi == EPI_DRELU) {
     if (!amn && bmn) SF_DENSE_CASE(false, true, EPI_DRELU);
+    if (!amn && !bmn) SF_DENSE_CASE(false, false, EPI_DRELU);
   }
 #undef SF_DENSE_CASE
   return SF_ERR_UNSUPPORTED;

@@ -26,9 +26,10 @@ def _run_sparse(cfg, prune_mode=0, act_shift=0.0, flags=binding.SF_FFN_SAVE_Y1):
     nctx, nws = binding.sf_ffn_workspace_size(desc)
     gctx, gws = Guarded(nctx, zero=True), Guarded(nws, zero=True)
     ctx, ws = gctx.t, gws.t
-    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
+    w2_fd = bool(flags & binding.SF_FFN_W2_FD)                # W2 handed over (and dW2 returned) as [F, D]
+    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, np.ascontiguousarray(W2.T) if w2_fd else W2, dY))
     gY, ggX = Guarded((T, D), torch.bfloat16), Guarded((T, D), torch.bfloat16)
-    ggW1, ggW2 = Guarded((F, D), torch.bfloat16), Guarded((D, F), torch.bfloat16)
+    ggW1, ggW2 = Guarded((F, D), torch.bfloat16), Guarded((F, D) if w2_fd else (D, F), torch.bfloat16)
     Y, gX, gW1, gW2 = gY.t, ggX.t, ggW1.t, ggW2.t
     binding.sf_sparse_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
     assert binding.sf_check_status(ws) == binding.SF_OK
@@ -43,7 +44,7 @@ def _run_sparse(cfg, prune_mode=0, act_shift=0.0, flags=binding.SF_FFN_SAVE_Y1):
         relu_vals=bits(view(ctx, binding.SF_CTX_RELU_VALS)).reshape(T, 2 * G),
         meta=bits(view(ctx, binding.SF_CTX_META)).reshape(T, G // 4),
         colidx=view(ctx, binding.SF_CTX_COLIDX).cpu().numpy().reshape(T // V, G, 4),
-        Y=f32(Y), dX=f32(gX), dW1=f32(gW1), dW2=f32(gW2))
+        Y=f32(Y), dX=f32(gX), dW1=f32(gW1), dW2=f32(gW2).T if w2_fd else f32(gW2))
     if flags & binding.SF_FFN_SAVE_Y1:
         out["y1"] = bits(view(ctx, binding.SF_CTX_Y1)).reshape(T, F)
     if M == 8:
@@ -223,19 +224,39 @@ def test_sparse_ffn_odd_multiples_of_128(T, D, F, V, M, flags):
         _check_against_oracle(inputs, g, cfg, prune_mode)
 
 
+@pytest.mark.parametrize("T,D,F,V,M", [(1024, 256, 1024, 64, 8), (384, 640, 896, 128, 8), (512, 512, 1024, 64, 4),
+                                       (512, 256, 1024, 128, 16), (256, 512, 2048, 64, 32)])
+def test_sparse_ffn_with_w2_stored_as_f_by_d(T, D, F, V, M):
+    """SF_FFN_W2_FD: the same layer with W2 handed over (and dW2 returned) as [F, D]: contiguous pruning of W2,
+    W2 as the MN-major operand of y3, no transposed copy for the gathered products; checked against the oracle
+    like every other step, in both prune modes and with the two-kernel activation path."""
+    cfg = dict(T=T, D=D, F=F, V=V, N=2, M=M, sigma_w=0.05, seed=T + D + F + M)
+    for prune_mode, extra in ((0, 0), (1, binding.SF_FFN_UNFUSED_ACT if M == 8 else 0)):
+        inputs, g = _run_sparse(cfg, prune_mode, flags=binding.SF_FFN_SAVE_Y1 | binding.SF_FFN_W2_FD | extra)
+        _check_against_oracle(inputs, g, cfg, prune_mode)
+    if M == 8:
+        inputs, g = _run_sparse(cfg, 0, flags=binding.SF_FFN_SAVE_Y1 | binding.SF_FFN_W2_FD | binding.SF_FFN_PACKED_GRAD_OPERANDS) \
+            if (T % 256 == 0 and D % 256 == 0 and F % 256 == 0) else (None, None)
+        if g is not None:
+            _check_against_oracle(inputs, g, cfg, 0)
+
+
 @pytest.mark.parametrize("name", ["c1_small", "odd128"])
 def test_dense_ffn_c1(name):
     cfg = synth.FFN_CONFIGS["c1_small"] if name == "c1_small" else dict(T=384, D=640, F=896, V=64, M=8, sigma_w=0.05, seed=77)
     T, D, F = cfg["T"], cfg["D"], cfg["F"]
     X, W1, W2, dY = synth.ffn_inputs(T, D, F, cfg["sigma_w"], cfg["seed"])
-    desc = binding.make_desc(T, D, F, cfg["V"], cfg["M"])
+    w2_fd = name == "odd128"                                   # this case also hands W2 over as [F, D]
+    desc = binding.make_desc(T, D, F, cfg["V"], cfg["M"], flags=binding.SF_FFN_W2_FD if w2_fd else 0)
     ctx, ws = binding.alloc_ffn_buffers(desc)
-    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, W2, dY))
+    dX_, dW1_, dW2_, dY_ = (to_dev(a) for a in (X, W1, np.ascontiguousarray(W2.T) if w2_fd else W2, dY))
     Y = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
     gX, gW1, gW2 = torch.empty_like(dX_), torch.empty_like(dW1_), torch.empty_like(dW2_)
     binding.sf_dense_ffn_fwd(desc, dX_, dW1_, dW2_, Y, ctx, ws)
     binding.sf_dense_ffn_bwd(desc, dY_, dX_, dW1_, dW2_, ctx, gX, gW1, gW2, ws)
     assert binding.sf_check_status(ws) == binding.SF_OK
+    if w2_fd:
+        gW2 = gW2.T
     y1 = bits(ctx[: T * F * 2].view(torch.bfloat16)).reshape(T, F)
     free = oracle.dense_ffn_fwd(X, W1, W2)
     assert rel_fro(oracle.bf16_to_f32(y1), oracle.bf16_to_f32(free.y1b)) < TOL
