@@ -113,7 +113,7 @@ def test_step_calls_reject_short_buffers_before_launching(lib):
     # NULL and alignment still come first
     assert lib.sf_sparse_ffn_fwd(d, None, ok, ok, ok, ok, need_ctx, ok, need_ws, None) == binding.SF_ERR_NULL
     # unknown flag bits are refused
-    bad = binding.make_desc(1024, 256, 1024, 64, 8, flags=16)
+    bad = binding.make_desc(1024, 256, 1024, 64, 8, flags=32)
     a, b = C.c_size_t(), C.c_size_t()
     assert lib.sf_ffn_workspace_size(C.byref(bad), C.byref(a), C.byref(b)) == binding.SF_ERR_UNSUPPORTED
 
