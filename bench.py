@@ -260,8 +260,15 @@ def run_ours(args, cfg):
     kern_ms = {n: float(np.mean(v)) for n, v in per.items() if n not in not_launched}
     kern_sum = float(sum(kern_ms.values()))
 
-    for _ in range(2):
-        dense_step()
+    def rested_warmup(fn):
+        """Every arm starts like the first one: after an idle gap (the part drops back to its idle power state)
+        and W warm-up steps, so that no arm inherits the heat of the arm before it."""
+        barrier()
+        time.sleep(args.rest_seconds)
+        for _ in range(W):
+            fn()
+
+    rested_warmup(dense_step)
     ms_dense = timed(dense_step, K)
     if binding.sf_check_status(ws) != binding.SF_OK:
         raise SystemExit("device status: a bounded wait expired")
@@ -280,8 +287,7 @@ def run_ours(args, cfg):
             binding.sf_routed_ffn_fwd(rdesc, dX_, dW1_, dW2_, means, Y, rctx, rws)
             binding.sf_routed_ffn_bwd(rdesc, ddY, dX_, dW1_, dW2_, rctx, gX, gW1, gW2, rws)
 
-        for _ in range(3):
-            routed_step()
+        rested_warmup(routed_step)
         with binding.StageTrace(13 * K) as rtr:
             ms_r = timed(routed_step, K)
         if binding.sf_check_status(rws) != binding.SF_OK:
@@ -407,6 +413,7 @@ def run_ours(args, cfg):
         "config": {"workload": args.workload, "T": T, "D": D, "F": F, "V": V, "N": 2, "M": M,
                    "prune_mode": args.prune_mode, "flags": args.flags, "path": path,
                    "parallelism": f"replicas x{world}",
+                   "arms": f"each arm (sparse, dense, routed) is timed after an idle gap of {args.rest_seconds} s and {W} warm-up steps",
                    "l2": f"per-step operands ({(2 * T * D + 2 * F * D) * 2 / 1e6:.0f} MB) and intermediates exceed the 126 MB L2"},
         "dense_step_ms": ms_dense / K, "speedup_vs_dense_step": ms_dense / ms,
         "dense_step_tflops": replicas.aggregate_tflops(flop_step, K, ms_dense),
@@ -572,6 +579,8 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="sf_ffn_flags of the step (0 = the library's defaults)")
     ap.add_argument("--sustain-seconds", type=float, default=1.0,
                     help="time per arm of the alternating sparse/dense blocks (0 = skip)")
+    ap.add_argument("--rest-seconds", type=float, default=0.5,
+                    help="idle gap before the warm-up of the dense and the routed arm (the sparse arm starts from idle too)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true",
                     help="sparse step only (no dense step, trace, e2e, CPU baseline): for profiler captures")
