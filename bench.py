@@ -493,6 +493,8 @@ def run_sweep(args):
     dev = lambda b: torch.from_numpy(np.ascontiguousarray(b).view(np.int16)).cuda().view(torch.bfloat16)
     iters = max(args.steps, 5)
     results = []
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    roofline = None
     if args.workload == "c2_prune":
         flush = torch.empty((256 << 20,), dtype=torch.uint8, device="cuda")      # twice the L2
         for i, (rows, cols) in enumerate(synth.PRUNE_SWEEP_SHAPES):
@@ -506,6 +508,11 @@ def run_sweep(args):
                     results.append({"rows": rows, "cols": cols, "group_dim": group_dim, "prune_mode": mode,
                                     "us": ms * 1e3, "gbs": gbs, "frac_of_hbm": gbs / hbm})
         metric, unit, value = "prune24_compress_min_frac_of_measured_hbm", "fraction", min(r["frac_of_hbm"] for r in results)
+        big = [r for r in results if r["rows"] * r["cols"] == max(x["rows"] * x["cols"] for x in results) and r["prune_mode"] == 0]
+        roofline = {"bound": "hbm", "kernel": "prune24_rows_kernel / prune24_cols_kernel at the largest shape, hard pruning",
+                    "achieved": min(r["gbs"] for r in big), "peak": hbm, "unit": "GB/s",
+                    "frac": min(r["frac_of_hbm"] for r in big), "traffic": None,
+                    "peak_source": f"{peaks['source']} copy bandwidth", "work": "3.125 algorithmic bytes per element"}
         note = ("3.125 algorithmic bytes per element; three of the four inputs would fit the 126 MB L2, so a 256 MB buffer "
                 "is overwritten before every timed launch (each launch timed by its own event pair, input cold)")
     elif args.workload == "c3_act":
@@ -520,6 +527,9 @@ def run_sweep(args):
                 results.append({"T": Tn, "F": Fn, "V": V, "M": M, "us": ms * 1e3, "algorithmic_bytes_per_element": nbytes / (Tn * Fn),
                                 "gbs": gbs, "frac_of_hbm": gbs / hbm})
         metric, unit, value = "vnm_sparsify_min_frac_of_measured_hbm", "fraction", min(r["frac_of_hbm"] for r in results)
+        roofline = {"bound": "hbm", "kernel": "vnm_stream_kernel", "achieved": min(r["gbs"] for r in results), "peak": hbm,
+                    "unit": "GB/s", "frac": value, "traffic": None, "peak_source": f"{peaks['source']} copy bandwidth",
+                    "work": "2 + 4/M + 0.5/M + 4/M algorithmic bytes per element + colidx"}
         note = "2 + 4/M + 0.5/M + 4/M (ReLU values) bytes per element + colidx; 537 MB input, larger than the L2"
     else:
         shapes = [(4096, 16384, 4096)] if args.workload == "fp8_micro" else [(4096, 16384, 4096), (16384, 8192, 4096), (8192, 4096, 16384)]
@@ -574,10 +584,13 @@ def run_sweep(args):
                                 "speedup_vs_dense": ms_dense / ms_v})
         metric, unit, value = "sparse24_gemm_speedup_vs_dense_at_4096x16384x4096", "ratio", results[0]["speedup_gemm_only"]
         note = "Section 5.2.3's micro-benchmark shape first; Venom products at Table 5's sparsities"
-    print(json.dumps({"metric": metric, "value": value, "unit": unit, "n_gpus": 1, "steps": iters, "warmup": args.warmup,
-                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                      "config": {"workload": args.workload, "note": note, "hbm_peak_gbs": hbm, "peak_source": peaks["source"]},
-                      "results": results, "gpu_launches": iters * len(results)}))
+    line = {"metric": metric, "value": value, "unit": unit, "n_gpus": 1, "steps": iters, "warmup": args.warmup,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "note": note, "hbm_peak_gbs": hbm, "peak_source": peaks["source"]},
+            "results": results, "gpu_launches": iters * len(results), "clocks": sampler.stop()}
+    if roofline:
+        line["roofline"] = roofline
+    print(json.dumps(line))
 
 
 def _spawn_replicas(args):
